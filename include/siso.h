@@ -1,0 +1,192 @@
+/*
+ * siso.h - C ABI of the B200 semantic-cache hot path (SISO, arXiv 2508.18736).
+ *
+ * A cache is a slot-indexed array of unit-norm centroid vectors with, per slot, the
+ * paper's two replacement fields cluster_size and access_count (Sec. 4.2, "Caching:
+ * Centroids Replacement") plus a last_access stamp and a valid flag.  Every entry
+ * point below runs hand-written sm_100a kernels; there is no CPU path.
+ *
+ * Conventions
+ *   - d_* arguments are DEVICE pointers owned by the caller; the library never frees
+ *     them and never keeps them after the call returns.  h_* are HOST pointers.
+ *   - stream is a cudaStream_t passed as void*.  Calls are asynchronous on it unless
+ *     stated otherwise; calls on one handle must be issued on one stream (or be
+ *     ordered by the caller).  A handle is not thread-safe; handles are independent.
+ *   - Argument errors are detected on the host, return at once and modify nothing.
+ *     Conditions only the device can see (capacity exhausted, candidate buffer
+ *     overflow, a bounded wait that ran out) are written to a device status word that
+ *     siso_sync_status() returns; the call that hit them modifies nothing.
+ *   - Vectors are row-major [rows, dim], fp32 or bfloat16 (raw 16-bit patterns), and
+ *     MUST be L2-normalised by the caller: similarity = dot product = cosine.
+ *     dim % 8 == 0 and 16-byte aligned base pointers are required (else
+ *     SISO_ERR_UNSUPPORTED / SISO_ERR_INVALID_ARG).
+ *   - Ties in similarity go to the lower slot; the hit and merge tests are strict
+ *     ('>' as printed in Algorithm 1, MergeCentroids).
+ *   - access_count "infinity" (Algorithm 1, else-branch of MergeCentroids) is
+ *     0xFFFFFFFF; additions saturate there.
+ */
+#ifndef SISO_H_
+#define SISO_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct siso_cache siso_cache_t; /* opaque host-side handle */
+
+typedef enum {
+    SISO_OK = 0,
+    SISO_ERR_INVALID_ARG = 1,
+    SISO_ERR_UNSUPPORTED = 2,
+    SISO_ERR_OOM = 3,
+    SISO_ERR_CAPACITY = 4, /* insert: fewer free slots than rows to insert; nothing modified */
+    SISO_ERR_OVERFLOW = 5, /* merge: candidate buffer too small; nothing modified           */
+    SISO_ERR_TIMEOUT = 6,  /* a bounded device-side wait gave up                            */
+    SISO_ERR_CUDA = 7
+} siso_status_t;
+
+typedef enum { SISO_F32 = 0, SISO_BF16 = 1 } siso_dtype_t;
+
+#define SISO_ACCESS_INF 0xFFFFFFFFu
+
+/* merge flags */
+#define SISO_MERGE_SIZES_ONLY 0u    /* Algorithm 1 as printed: only cluster_size moves             */
+#define SISO_MERGE_WEIGHTED_MEAN 1u /* survivors become the cluster_size-weighted mean, renormalised */
+/* evict flags */
+#define SISO_EVICT_DECAY 1u /* afterwards cluster_size /= decay, access_count = 0 (Algorithm 1, FilteringCentroids) */
+
+/* lookup kernel selection (siso_set_option key SISO_OPT_LOOKUP_PATH) */
+#define SISO_OPT_LOOKUP_PATH 1
+#define SISO_OPT_MERGE_MAX_CANDIDATES 2 /* capacity of the merge candidate buffer, in pairs */
+#define SISO_PATH_AUTO 0
+#define SISO_PATH_SIMT 1   /* CUDA-core tiled sweep (fp32 accumulate of exact products)        */
+#define SISO_PATH_TENSOR 2 /* tcgen05 tensor-core sweep, bf16 caches only                      */
+#define SISO_PATH_STREAM 3 /* small-batch streaming sweep, one pass over the centroid matrix   */
+
+/* Device memory for the cache's own state and scratch comes from here.  alloc returns a
+ * device pointer aligned to 256 bytes or NULL; both may be NULL to use cudaMalloc/cudaFree. */
+typedef struct {
+    void *(*alloc)(size_t bytes, void *stream, void *ctx);
+    void (*free)(void *ptr, void *ctx);
+    void *ctx;
+} siso_allocator_t;
+
+typedef struct {
+    int64_t capacity; /* number of slots M ("maximum memory capacity", Algorithm 1), counted in entries */
+    int32_t dim;      /* embedding dimension, multiple of 8                                            */
+    int32_t dtype;    /* siso_dtype_t: storage type of cached vectors AND of query/insert arguments    */
+    int32_t device;   /* CUDA device ordinal                                                           */
+    int32_t reserved;
+    double decay; /* divisor of cluster_size in FilteringCentroids (Algorithm 1: 1.1); 0 selects 1.1 */
+    siso_allocator_t allocator;
+} siso_config_t;
+
+/* Create an empty cache (all slots invalid, clock 0).  Synchronous. */
+siso_status_t siso_cache_create(siso_cache_t **out, const siso_config_t *cfg);
+/* Synchronises the device, then releases everything obtained through the allocator. */
+siso_status_t siso_cache_destroy(siso_cache_t *c);
+
+/* Set a tuning option (SISO_OPT_*).  Host-side only. */
+siso_status_t siso_set_option(siso_cache_t *c, int32_t key, int64_t value);
+
+/* Bulk promotion of n centroids into the cache (the else-branch of MergeCentroids, Algorithm 1:
+ * a new entry gets access_count = infinity).  Rows take the free slots in ascending slot order.
+ * d_vecs [n, dim] in the cache dtype; d_sizes [n] cluster_size per row or NULL (= 1);
+ * d_slots_out [n] receives the slot of each row, or NULL.  Too few free slots:
+ * SISO_ERR_CAPACITY in the status word and nothing is modified. */
+siso_status_t siso_insert(siso_cache_t *c, const void *d_vecs, const double *d_sizes, int64_t n,
+                          int32_t *d_slots_out, void *stream);
+
+/* FindClosestCentroid + CosineSimilarity for a batch (Algorithm 1; Sec. 4.3 "searches the semantic
+ * cache"), exact, and the hit test against the retrieval threshold theta_R (Sec. 3.1), which is
+ * an input because it is adjusted at run time (Sec. 4.3, "Adjusting theta_R to meet SLO").
+ *   d_queries [n_queries, dim] in the cache dtype, unit-norm
+ *   d_theta   [n_queries] per-query thresholds, or NULL to use theta_scalar for all
+ *   k         in [1, 8]: number of best entries returned per query
+ *   d_idx     [n_queries, k] slots by (similarity desc, slot asc); -1 where fewer than k entries exist
+ *   d_sim     [n_queries, k] fp32 similarities (-inf beside idx = -1)
+ *   d_hit     [n_queries] 1 if d_sim[.,0] > theta, else 0 (empty cache: all 0)
+ * Reads the cache, modifies only its lookup/hit statistics. */
+siso_status_t siso_lookup(siso_cache_t *c, const void *d_queries, int64_t n_queries, const float *d_theta,
+                          float theta_scalar, int32_t k, int32_t *d_idx, float *d_sim, uint8_t *d_hit,
+                          void *stream);
+
+/* Same as siso_lookup with HOST buffers (pinned memory recommended): copies queries and
+ * thresholds to the device, runs the lookup, copies the three results back, all on `stream`. */
+siso_status_t siso_lookup_host(siso_cache_t *c, const void *h_queries, int64_t n_queries, const float *h_theta,
+                               float theta_scalar, int32_t k, int32_t *h_idx, float *h_sim, uint8_t *h_hit,
+                               void *stream);
+
+/* Hit update: a centroid is "the central or average point of a group of vectors" (Sec. 3.1), kept as a
+ * running mean.  For every slot j hit by the set H_j of this batch (ascending query order):
+ *     c_j <- normalise(cluster_size_j * c_j + sum_{b in H_j} q_b),  cluster_size_j += |H_j|,
+ *     access_count_j += |H_j| (saturating; Sec. 4.2: "how many times the centroid is referenced while in
+ *     the semantic cache"),  last_access_j <- clock.
+ * The cache clock advances by one per call.  d_idx is read with stride idx_stride (column 0 of a
+ * lookup result: pass k).  Rows with d_hit == 0 are ignored.  bf16 caches keep an fp32 master copy and
+ * re-round the lookup copy. */
+siso_status_t siso_update(siso_cache_t *c, const void *d_queries, int64_t n_queries, const int32_t *d_idx,
+                          int32_t idx_stride, const uint8_t *d_hit, void *stream);
+
+/* MergeCentroids (Algorithm 1) over the cache itself: entries are taken in ascending slot order, each
+ * is compared with the survivors before it (vectors as they were when the call began), and joins the
+ * most similar one if that similarity is > theta_c (cluster_size added, slot freed), else survives.
+ * d_repo must be NULL (merging an external repository array is not implemented: SISO_ERR_UNSUPPORTED).
+ *   flags        SISO_MERGE_SIZES_ONLY or SISO_MERGE_WEIGHTED_MEAN
+ *   d_merge_map  [capacity] slot -> surviving slot (own slot for survivors, -1 for empty slots), or NULL
+ *   h_n_merged   host pointer receiving the number of entries merged away, or NULL.  When not NULL the
+ *                call synchronises `stream` and returns the device status (SISO_ERR_OVERFLOW if the
+ *                pairs above theta_c did not fit the candidate buffer; then nothing was modified). */
+siso_status_t siso_merge(siso_cache_t *c, const void *d_repo, const double *d_repo_sizes, int64_t n_repo,
+                         float theta_c, uint32_t flags, int32_t *d_merge_map, int64_t *h_n_merged, void *stream);
+
+/* FilteringCentroids (Algorithm 1): remove the n_evict entries that come first in ascending
+ * (cluster_size, access_count, last_access, slot) order; with SISO_EVICT_DECAY every remaining entry then
+ * gets cluster_size /= decay and access_count = 0.  d_victims [n_evict] receives the removed slots in that
+ * order (-1 padding if the cache held fewer entries), or NULL. */
+siso_status_t siso_evict(siso_cache_t *c, int64_t n_evict, uint32_t flags, int32_t *d_victims, void *stream);
+
+/* Spare-space caching of individual query vectors (Sec. 5.2.5: "if free space remains, SISO caches
+ * individual vectors and manages them using LRU").  siso_make_room evicts exactly as many entries as the
+ * misses of this batch lack free slots for (max(0, #miss - #free), decided on the device);
+ * d_victims [n] receives them (-1 padding) or NULL.  siso_insert_misses then stores every row with
+ * d_hit == 0, in ascending row order into ascending free slots, as a new entry (cluster_size 1,
+ * access_count infinity, last_access = clock); d_slots_out [n] receives the slot or -1 for hits. */
+siso_status_t siso_make_room(siso_cache_t *c, const uint8_t *d_hit, int64_t n, uint32_t flags,
+                             int32_t *d_victims, void *stream);
+siso_status_t siso_insert_misses(siso_cache_t *c, const void *d_queries, int64_t n, const uint8_t *d_hit,
+                                 int32_t *d_slots_out, void *stream);
+
+/* One micro-batch of the streaming cache: lookup (k = 1), update, make_room, insert_misses, in this
+ * order on `stream`.  Output arrays as in the four calls; d_victims / d_slots_out may be NULL. */
+siso_status_t siso_stream_step(siso_cache_t *c, const void *d_queries, int64_t n, const float *d_theta,
+                               float theta_scalar, int32_t *d_idx, float *d_sim, uint8_t *d_hit,
+                               int32_t *d_victims, int32_t *d_slots_out, void *stream);
+
+/* Copy the state out (checkpoint, parity checks).  Any pointer may be NULL.
+ *   d_vecs   [capacity, dim] lookup copy in the cache dtype     d_master [capacity, dim] fp32 master
+ *   d_sizes  [capacity] fp64   d_access [capacity] u32   d_last [capacity] u64   d_valid [capacity] u8 */
+siso_status_t siso_export(siso_cache_t *c, void *d_vecs, float *d_master, double *d_sizes, uint32_t *d_access,
+                          uint64_t *d_last, uint8_t *d_valid, void *stream);
+/* Replace the whole state (restore a checkpoint).  d_master (fp32) is required; the lookup copy is
+ * re-derived from it.  clock becomes `clock`. */
+siso_status_t siso_import(siso_cache_t *c, const float *d_master, const double *d_sizes, const uint32_t *d_access,
+                          const uint64_t *d_last, const uint8_t *d_valid, uint64_t clock, void *stream);
+
+/* h_counts[8] = occupancy, lookups, hits, inserts, evictions, merges, clock, 0.  Synchronises `stream`. */
+siso_status_t siso_get_stats(siso_cache_t *c, int64_t *h_counts, void *stream);
+/* Synchronise `stream`, return the device status word (SISO_OK if clear) and clear it. */
+siso_status_t siso_sync_status(siso_cache_t *c, void *stream);
+/* Number of kernels this handle has launched so far (host-side count). */
+int64_t siso_launch_count(const siso_cache_t *c);
+const char *siso_status_string(siso_status_t s);
+/* Text of the last CUDA error seen by this library in the calling process ("" if none). */
+const char *siso_last_cuda_error(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SISO_H_ */
