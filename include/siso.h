@@ -2,8 +2,7 @@
  * siso.h - C ABI of the B200 semantic-cache hot path (SISO, arXiv 2508.18736).
  *
  * A cache is a slot-indexed array of unit-norm centroid vectors with, per slot, the
- * paper's two replacement fields cluster_size and access_count (Sec. 4.2, "Caching:
- * Centroids Replacement") plus a last_access stamp and a valid flag.  Every entry
+ * paper's two replacement fields cluster_size and access_count (Sec. 4.2, the cache manager) plus a last_access stamp and a valid flag.  Every entry
  * point below runs hand-written sm_100a kernels; there is no CPU path.
  *
  * Conventions
@@ -75,7 +74,7 @@ typedef struct {
 } siso_allocator_t;
 
 typedef struct {
-    int64_t capacity; /* number of slots M ("maximum memory capacity", Algorithm 1), counted in entries */
+    int64_t capacity; /* number of slots: the capacity M of Algorithm 1, counted in entries */
     int32_t dim;      /* embedding dimension, multiple of 8                                            */
     int32_t dtype;    /* siso_dtype_t: storage type of cached vectors AND of query/insert arguments    */
     int32_t device;   /* CUDA device ordinal                                                           */
@@ -100,9 +99,8 @@ siso_status_t siso_set_option(siso_cache_t *c, int32_t key, int64_t value);
 siso_status_t siso_insert(siso_cache_t *c, const void *d_vecs, const double *d_sizes, int64_t n,
                           int32_t *d_slots_out, void *stream);
 
-/* FindClosestCentroid + CosineSimilarity for a batch (Algorithm 1; Sec. 4.3 "searches the semantic
- * cache"), exact, and the hit test against the retrieval threshold theta_R (Sec. 3.1), which is
- * an input because it is adjusted at run time (Sec. 4.3, "Adjusting theta_R to meet SLO").
+/* FindClosestCentroid + CosineSimilarity for a batch (Algorithm 1; the cache search of Sec. 4.3), exact, and the hit test against the retrieval threshold theta_R (Sec. 3.1), which is
+ * an input because it is adjusted at run time (Sec. 4.3, threshold adjustment under load).
  *   d_queries [n_queries, dim] in the cache dtype, unit-norm
  *   d_theta   [n_queries] per-query thresholds, or NULL to use theta_scalar for all
  *   k         in [1, 8]: number of best entries returned per query
@@ -120,11 +118,11 @@ siso_status_t siso_lookup_host(siso_cache_t *c, const void *h_queries, int64_t n
                                float theta_scalar, int32_t k, int32_t *h_idx, float *h_sim, uint8_t *h_hit,
                                void *stream);
 
-/* Hit update: a centroid is "the central or average point of a group of vectors" (Sec. 3.1), kept as a
- * running mean.  For every slot j hit by the set H_j of this batch (ascending query order):
+/* Hit update: Sec. 3.1 describes a centroid as the mean point of its group of vectors; here it is kept as
+ * a running mean.  For every slot j hit by the set H_j of this batch (ascending query order):
  *     c_j <- normalise(cluster_size_j * c_j + sum_{b in H_j} q_b),  cluster_size_j += |H_j|,
- *     access_count_j += |H_j| (saturating; Sec. 4.2: "how many times the centroid is referenced while in
- *     the semantic cache"),  last_access_j <- clock.
+ *     access_count_j += |H_j| (saturating; Sec. 4.2 counts references made while the entry is
+ *     cached),  last_access_j <- clock.
  * The cache clock advances by one per call.  d_idx is read with stride idx_stride (column 0 of a
  * lookup result: pass k).  Rows with d_hit == 0 are ignored.  bf16 caches keep an fp32 master copy and
  * re-round the lookup copy. */
@@ -149,8 +147,8 @@ siso_status_t siso_merge(siso_cache_t *c, const void *d_repo, const double *d_re
  * order (-1 padding if the cache held fewer entries), or NULL. */
 siso_status_t siso_evict(siso_cache_t *c, int64_t n_evict, uint32_t flags, int32_t *d_victims, void *stream);
 
-/* Spare-space caching of individual query vectors (Sec. 5.2.5: "if free space remains, SISO caches
- * individual vectors and manages them using LRU").  siso_make_room evicts exactly as many entries as the
+/* Spare-space caching of individual query vectors (Sec. 5.2.5: space left over after the centroids holds
+ * single query vectors under LRU).  siso_make_room evicts exactly as many entries as the
  * misses of this batch lack free slots for (max(0, #miss - #free), decided on the device);
  * d_victims [n] receives them (-1 padding) or NULL.  siso_insert_misses then stores every row with
  * d_hit == 0, in ascending row order into ascending free slots, as a new entry (cluster_size 1,

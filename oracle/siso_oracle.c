@@ -13,11 +13,11 @@
  *
  * What follows which passage of the paper:
  *   lookup        FindClosestCentroid / CosineSimilarity of Algorithm 1 (closest =
- *                 largest cosine) and the retrieval threshold theta_R of Sec. 3.1
- *                 ("judges a cache hit"); cosine = dot product because stored
+ *                 largest cosine) and the retrieval threshold theta_R of Sec. 3.1,
+ *                 which decides hit or miss; cosine = dot product because stored
  *                 centroids and queries are unit-norm by contract.
- *   update        the running-mean reading of a centroid as "the central or average
- *                 point of a group of vectors" (Sec. 3.1) plus the access_count
+ *   update        the running-mean reading of Sec. 3.1, where a centroid is the mean
+ *                 point of its group of vectors, plus the access_count
  *                 bookkeeping of Sec. 4.2 (merge step).
  *   merge         MergeCentroids of Algorithm 1, in the listed order.
  *   evict         FilteringCentroids of Algorithm 1: remove the smallest
@@ -25,8 +25,7 @@
  *                 cluster_size /= 1.1 and access_count = 0 for the rest.
  *   insert        the else-branch of MergeCentroids (new entry, access_count =
  *                 infinity) used for spare-space caching of individual vectors
- *                 (Sec. 5.2.5, "if free space remains ... caches individual vectors
- *                 and manages them using LRU").
+ *                 (Sec. 5.2.5: left-over space holds single vectors under LRU).
  *
  * Readings taken where the paper is silent (ties to the lowest index, strict '>'
  * for both tests, (cluster_size, access_count, last_access, slot) as the full

@@ -1,0 +1,10 @@
+"""B200 (sm_100a) kernels for the hot path of a centroid-based semantic cache: exact batched
+cosine lookup with top-k and a per-query hit threshold, running-mean hit updates,
+MergeCentroids / FilteringCentroids and spare-space insertion, behind the C ABI of
+``include/siso.h``.  This package is the thin Python binding: it marshals torch tensors to
+pointers and calls ``libsiso.so``; every step runs in the library's own CUDA kernels."""
+from .binding import (ACCESS_INF, EVICT_DECAY, MERGE_SIZES_ONLY, MERGE_WEIGHTED_MEAN, PATH_AUTO, PATH_SIMT,
+                      PATH_STREAM, PATH_TENSOR, SisoCache, SisoError, load_library)
+
+__all__ = ["SisoCache", "SisoError", "load_library", "ACCESS_INF", "EVICT_DECAY", "MERGE_SIZES_ONLY",
+           "MERGE_WEIGHTED_MEAN", "PATH_AUTO", "PATH_SIMT", "PATH_STREAM", "PATH_TENSOR"]

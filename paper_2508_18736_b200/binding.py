@@ -1,0 +1,290 @@
+"""ctypes binding of libsiso.so.  Argument marshalling only; names follow include/siso.h."""
+from __future__ import annotations
+
+import ctypes
+import os
+from typing import Optional, Tuple
+
+import torch
+
+_HERE = os.path.dirname(os.path.abspath(__file__))
+_LIB_PATH = os.path.join(_HERE, "libsiso.so")
+
+ACCESS_INF = 0xFFFFFFFF
+MERGE_SIZES_ONLY, MERGE_WEIGHTED_MEAN = 0, 1
+EVICT_DECAY = 1
+OPT_LOOKUP_PATH, OPT_MERGE_MAX_CANDIDATES = 1, 2
+PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_STREAM = 0, 1, 2, 3
+_STATUS_NAMES = {0: "SISO_OK", 1: "SISO_ERR_INVALID_ARG", 2: "SISO_ERR_UNSUPPORTED", 3: "SISO_ERR_OOM",
+                 4: "SISO_ERR_CAPACITY", 5: "SISO_ERR_OVERFLOW", 6: "SISO_ERR_TIMEOUT", 7: "SISO_ERR_CUDA"}
+
+EXPORTS = ["siso_cache_create", "siso_cache_destroy", "siso_set_option", "siso_insert", "siso_lookup",
+           "siso_lookup_host", "siso_update", "siso_merge", "siso_evict", "siso_make_room", "siso_insert_misses",
+           "siso_stream_step", "siso_export", "siso_import", "siso_get_stats", "siso_sync_status",
+           "siso_launch_count", "siso_status_string", "siso_last_cuda_error"]
+
+
+class SisoError(RuntimeError):
+    def __init__(self, status: int, where: str, detail: str = ""):
+        self.status = status
+        name = _STATUS_NAMES.get(status, str(status))
+        super().__init__(f"{where}: {name}" + (f" ({detail})" if detail else ""))
+
+
+_ALLOC_FN = ctypes.CFUNCTYPE(ctypes.c_void_p, ctypes.c_size_t, ctypes.c_void_p, ctypes.c_void_p)
+_FREE_FN = ctypes.CFUNCTYPE(None, ctypes.c_void_p, ctypes.c_void_p)
+
+
+class _Allocator(ctypes.Structure):
+    _fields_ = [("alloc", _ALLOC_FN), ("free", _FREE_FN), ("ctx", ctypes.c_void_p)]
+
+
+class _Config(ctypes.Structure):
+    _fields_ = [("capacity", ctypes.c_int64), ("dim", ctypes.c_int32), ("dtype", ctypes.c_int32),
+                ("device", ctypes.c_int32), ("reserved", ctypes.c_int32), ("decay", ctypes.c_double),
+                ("allocator", _Allocator)]
+
+
+_lib = None
+
+
+def load_library(path: Optional[str] = None) -> ctypes.CDLL:
+    """Load libsiso.so.  There is no fallback: a missing library is an error."""
+    global _lib
+    if _lib is not None and path is None:
+        return _lib
+    p = path or _LIB_PATH
+    if not os.path.exists(p):
+        raise ImportError(f"{p} not found: build it with `python -m paper_2508_18736_b200.build` "
+                          "(nvcc, sm_100a); this package has no CPU or PyTorch fallback")
+    L = ctypes.CDLL(p)
+    vp, i64, i32, u32, f32 = ctypes.c_void_p, ctypes.c_int64, ctypes.c_int32, ctypes.c_uint32, ctypes.c_float
+    L.siso_cache_create.argtypes = [ctypes.POINTER(vp), ctypes.POINTER(_Config)]
+    L.siso_cache_destroy.argtypes = [vp]
+    L.siso_set_option.argtypes = [vp, i32, i64]
+    L.siso_insert.argtypes = [vp, vp, vp, i64, vp, vp]
+    L.siso_lookup.argtypes = [vp, vp, i64, vp, f32, i32, vp, vp, vp, vp]
+    L.siso_lookup_host.argtypes = [vp, vp, i64, vp, f32, i32, vp, vp, vp, vp]
+    L.siso_update.argtypes = [vp, vp, i64, vp, i32, vp, vp]
+    L.siso_merge.argtypes = [vp, vp, vp, i64, f32, u32, vp, ctypes.POINTER(i64), vp]
+    L.siso_evict.argtypes = [vp, i64, u32, vp, vp]
+    L.siso_make_room.argtypes = [vp, vp, i64, u32, vp, vp]
+    L.siso_insert_misses.argtypes = [vp, vp, i64, vp, vp, vp]
+    L.siso_stream_step.argtypes = [vp, vp, i64, vp, f32, vp, vp, vp, vp, vp, vp]
+    L.siso_export.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
+    L.siso_import.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_uint64, vp]
+    L.siso_get_stats.argtypes = [vp, ctypes.POINTER(i64), vp]
+    L.siso_sync_status.argtypes = [vp, vp]
+    L.siso_launch_count.argtypes = [vp]
+    L.siso_launch_count.restype = i64
+    L.siso_status_string.argtypes = [i32]
+    L.siso_status_string.restype = ctypes.c_char_p
+    L.siso_last_cuda_error.argtypes = []
+    L.siso_last_cuda_error.restype = ctypes.c_char_p
+    for name in EXPORTS:
+        if name not in ("siso_launch_count", "siso_status_string", "siso_last_cuda_error"):
+            getattr(L, name).restype = i32
+    if path is None:
+        _lib = L
+    return L
+
+
+def _ptr(t: Optional[torch.Tensor]):
+    return None if t is None else ctypes.c_void_p(t.data_ptr())
+
+
+def _stream(stream: Optional[torch.cuda.Stream]):
+    s = torch.cuda.current_stream() if stream is None else stream
+    return ctypes.c_void_p(s.cuda_stream)
+
+
+class SisoCache:
+    """Handle of one device-resident cache.  Methods mirror the C entry points one to one."""
+
+    def __init__(self, capacity: int, dim: int, dtype: str = "bf16", device: int = 0, decay: float = 1.1,
+                 use_torch_allocator: bool = True):
+        if dtype not in ("f32", "bf16"):
+            raise ValueError("dtype must be 'f32' or 'bf16'")
+        if not torch.cuda.is_available():
+            raise RuntimeError("a CUDA device is required: this library has no CPU path")
+        self._lib = load_library()
+        self.capacity, self.dim, self.dtype, self.device = int(capacity), int(dim), dtype, int(device)
+        self.torch_dtype = torch.float32 if dtype == "f32" else torch.bfloat16
+        self._dev = torch.device("cuda", self.device)
+        self._blocks = {}
+        cfg = _Config()
+        cfg.capacity, cfg.dim, cfg.dtype, cfg.device, cfg.decay = capacity, dim, 0 if dtype == "f32" else 1, device, decay
+        if use_torch_allocator:
+            # the cache's own state and scratch live in torch's caching allocator
+            def _alloc(nbytes, stream, ctx):
+                try:
+                    with torch.cuda.device(self._dev):
+                        t = torch.empty(int(nbytes), dtype=torch.uint8, device=self._dev)
+                except Exception:       # out of memory -> NULL -> SISO_ERR_OOM
+                    return None
+                self._blocks[t.data_ptr()] = t
+                return t.data_ptr()
+
+            def _free(ptr, ctx):
+                self._blocks.pop(ptr, None)
+
+            self._alloc_cb, self._free_cb = _ALLOC_FN(_alloc), _FREE_FN(_free)
+            cfg.allocator = _Allocator(self._alloc_cb, self._free_cb, None)
+        h = ctypes.c_void_p()
+        st = self._lib.siso_cache_create(ctypes.byref(h), ctypes.byref(cfg))
+        self._h = h if st == 0 else None
+        self._check(st, "siso_cache_create")
+
+    # ------------------------------------------------------------------ helpers
+    def _check(self, st: int, where: str) -> None:
+        if st != 0:
+            raise SisoError(st, where, self._lib.siso_last_cuda_error().decode() if st == 7 else "")
+
+    def _vec(self, t: torch.Tensor, name: str) -> torch.Tensor:
+        if t.dtype != self.torch_dtype or t.device != self._dev or t.dim() != 2 or t.shape[1] != self.dim:
+            raise ValueError(f"{name} must be a [{'n'}, {self.dim}] {self.torch_dtype} tensor on {self._dev}")
+        return t.contiguous()
+
+    def _new(self, shape, dtype) -> torch.Tensor:
+        return torch.empty(shape, dtype=dtype, device=self._dev)
+
+    def close(self) -> None:
+        if getattr(self, "_h", None) is not None:
+            self._lib.siso_cache_destroy(self._h)
+            self._h = None
+            self._blocks.clear()
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+    # ------------------------------------------------------------------ entry points
+    def set_option(self, key: int, value: int) -> None:
+        self._check(self._lib.siso_set_option(self._h, key, value), "siso_set_option")
+
+    def set_lookup_path(self, path: int) -> None:
+        self.set_option(OPT_LOOKUP_PATH, path)
+
+    def insert(self, vecs: torch.Tensor, sizes: Optional[torch.Tensor] = None, stream=None) -> torch.Tensor:
+        vecs = self._vec(vecs, "vecs")
+        n = vecs.shape[0]
+        if sizes is not None:
+            sizes = sizes.to(device=self._dev, dtype=torch.float64).contiguous()
+            assert sizes.numel() == n
+        slots = self._new((n,), torch.int32)
+        self._check(self._lib.siso_insert(self._h, _ptr(vecs), _ptr(sizes), n, _ptr(slots), _stream(stream)), "siso_insert")
+        return slots
+
+    def lookup(self, queries: torch.Tensor, theta, k: int = 1, stream=None, out=None
+               ) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+        """theta: float (same threshold for all) or fp32 tensor [n].  Returns idx[n,k], sim[n,k], hit[n]."""
+        q = self._vec(queries, "queries")
+        n = q.shape[0]
+        th_t, th_s = (theta.to(device=self._dev, dtype=torch.float32).contiguous(), 0.0) \
+            if isinstance(theta, torch.Tensor) else (None, float(theta))
+        if th_t is not None:
+            assert th_t.numel() == n
+        idx, sim, hit = out if out is not None else (self._new((n, k), torch.int32), self._new((n, k), torch.float32),
+                                                      self._new((n,), torch.uint8))
+        self._check(self._lib.siso_lookup(self._h, _ptr(q), n, _ptr(th_t), th_s, k, _ptr(idx), _ptr(sim), _ptr(hit),
+                                          _stream(stream)), "siso_lookup")
+        return idx, sim, hit
+
+    def lookup_host(self, h_queries: torch.Tensor, h_theta: Optional[torch.Tensor], theta_scalar: float, k: int,
+                    h_idx: torch.Tensor, h_sim: torch.Tensor, h_hit: torch.Tensor, stream=None) -> None:
+        """All tensors live in (pinned) host memory; results are valid after the stream is synchronised."""
+        n = h_queries.shape[0]
+        self._check(self._lib.siso_lookup_host(self._h, _ptr(h_queries), n, _ptr(h_theta), float(theta_scalar), k,
+                                               _ptr(h_idx), _ptr(h_sim), _ptr(h_hit), _stream(stream)), "siso_lookup_host")
+
+    def update(self, queries: torch.Tensor, idx: torch.Tensor, hit: torch.Tensor, stream=None) -> None:
+        q = self._vec(queries, "queries")
+        n = q.shape[0]
+        assert idx.dtype == torch.int32 and hit.dtype == torch.uint8 and idx.is_contiguous() and hit.is_contiguous()
+        stride = 1 if idx.dim() == 1 else idx.shape[1]
+        self._check(self._lib.siso_update(self._h, _ptr(q), n, _ptr(idx), stride, _ptr(hit), _stream(stream)), "siso_update")
+
+    def merge(self, theta_c: float, flags: int = MERGE_WEIGHTED_MEAN, want_count: bool = True, stream=None
+              ) -> Tuple[torch.Tensor, Optional[int]]:
+        """Self-merge of the cache.  Returns (merge_map [capacity], number merged or None)."""
+        mm = self._new((self.capacity,), torch.int32)
+        n = ctypes.c_int64(0)
+        st = self._lib.siso_merge(self._h, None, None, 0, float(theta_c), flags, _ptr(mm),
+                                  ctypes.byref(n) if want_count else None, _stream(stream))
+        self._check(st, "siso_merge")
+        return mm, (int(n.value) if want_count else None)
+
+    def evict(self, n_evict: int, flags: int = 0, stream=None) -> torch.Tensor:
+        victims = self._new((max(int(n_evict), 0),), torch.int32)
+        self._check(self._lib.siso_evict(self._h, int(n_evict), flags, _ptr(victims), _stream(stream)), "siso_evict")
+        return victims
+
+    def make_room(self, hit: torch.Tensor, flags: int = 0, stream=None) -> torch.Tensor:
+        n = hit.numel()
+        victims = self._new((n,), torch.int32)
+        self._check(self._lib.siso_make_room(self._h, _ptr(hit), n, flags, _ptr(victims), _stream(stream)), "siso_make_room")
+        return victims
+
+    def insert_misses(self, queries: torch.Tensor, hit: torch.Tensor, stream=None) -> torch.Tensor:
+        q = self._vec(queries, "queries")
+        n = q.shape[0]
+        slots = self._new((n,), torch.int32)
+        self._check(self._lib.siso_insert_misses(self._h, _ptr(q), n, _ptr(hit), _ptr(slots), _stream(stream)),
+                    "siso_insert_misses")
+        return slots
+
+    def stream_step(self, queries: torch.Tensor, theta, stream=None, out=None):
+        """lookup(k=1) -> update -> make_room -> insert_misses.  Returns idx, sim, hit, victims, slots."""
+        q = self._vec(queries, "queries")
+        n = q.shape[0]
+        th_t, th_s = (theta.to(device=self._dev, dtype=torch.float32).contiguous(), 0.0) \
+            if isinstance(theta, torch.Tensor) else (None, float(theta))
+        if out is None:
+            out = (self._new((n, 1), torch.int32), self._new((n, 1), torch.float32), self._new((n,), torch.uint8),
+                   self._new((n,), torch.int32), self._new((n,), torch.int32))
+        idx, sim, hit, victims, slots = out
+        self._check(self._lib.siso_stream_step(self._h, _ptr(q), n, _ptr(th_t), th_s, _ptr(idx), _ptr(sim), _ptr(hit),
+                                               _ptr(victims), _ptr(slots), _stream(stream)), "siso_stream_step")
+        return out
+
+    def export(self, stream=None) -> dict:
+        out = dict(vecs=self._new((self.capacity, self.dim), self.torch_dtype),
+                   master=self._new((self.capacity, self.dim), torch.float32),
+                   size=self._new((self.capacity,), torch.float64),
+                   access=self._new((self.capacity,), torch.int32),        # bit pattern of the uint32 counters
+                   last=self._new((self.capacity,), torch.int64),
+                   valid=self._new((self.capacity,), torch.uint8))
+        self._check(self._lib.siso_export(self._h, _ptr(out["vecs"]), _ptr(out["master"]), _ptr(out["size"]),
+                                          _ptr(out["access"]), _ptr(out["last"]), _ptr(out["valid"]), _stream(stream)),
+                    "siso_export")
+        return out
+
+    def import_(self, master: torch.Tensor, size: torch.Tensor, access: torch.Tensor, last: torch.Tensor,
+                valid: torch.Tensor, clock: int, stream=None) -> None:
+        args = [master.to(self._dev, torch.float32).contiguous(), size.to(self._dev, torch.float64).contiguous(),
+                access.to(self._dev).contiguous(), last.to(self._dev).contiguous(),
+                valid.to(self._dev, torch.uint8).contiguous()]
+        assert args[0].shape == (self.capacity, self.dim) and args[2].element_size() == 4 and args[3].element_size() == 8
+        self._check(self._lib.siso_import(self._h, *[_ptr(a) for a in args], int(clock), _stream(stream)), "siso_import")
+        torch.cuda.current_stream().synchronize() if stream is None else stream.synchronize()
+
+    def stats(self, stream=None) -> dict:
+        buf = (ctypes.c_int64 * 8)()
+        self._check(self._lib.siso_get_stats(self._h, buf, _stream(stream)), "siso_get_stats")
+        names = ["occupancy", "lookups", "hits", "inserts", "evictions", "merges", "clock"]
+        return {n: int(buf[i]) for i, n in enumerate(names)}
+
+    def sync_status(self, stream=None) -> int:
+        """Synchronise and return the device status word (0 = clear); it is cleared by the call."""
+        return int(self._lib.siso_sync_status(self._h, _stream(stream)))
+
+    def check_status(self, stream=None) -> None:
+        st = self.sync_status(stream)
+        if st != 0:
+            raise SisoError(st, "device status")
+
+    @property
+    def launch_count(self) -> int:
+        return int(self._lib.siso_launch_count(self._h))

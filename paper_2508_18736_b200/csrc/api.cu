@@ -1,0 +1,378 @@
+// C ABI of libsiso: argument checking, state, scratch memory and kernel launches.
+#include <cstdio>
+#include <cstring>
+#include <new>
+
+#include "common.cuh"
+
+namespace siso {
+
+static thread_local char g_last_error[512] = "";
+
+siso_status_t check_cuda(cudaError_t e, const char *what) {
+    if (e == cudaSuccess) return SISO_OK;
+    snprintf(g_last_error, sizeof(g_last_error), "%s: %s", what, cudaGetErrorString(e));
+    return e == cudaErrorMemoryAllocation ? SISO_ERR_OOM : SISO_ERR_CUDA;
+}
+
+static void *default_alloc(size_t bytes, void *, void *) {
+    void *p = nullptr;
+    if (cudaMalloc(&p, bytes) != cudaSuccess) { cudaGetLastError(); return nullptr; }
+    return p;
+}
+static void default_free(void *p, void *) { cudaFree(p); }
+
+static void *cache_alloc(Cache *c, size_t bytes, cudaStream_t s) {
+    return c->alloc.alloc(bytes ? bytes : 256, s, c->alloc.ctx);
+}
+
+siso_status_t scratch_reserve(Cache *c, size_t bytes, cudaStream_t s, Scratch *out) {
+    bytes += 4096;
+    if (bytes > c->ws_bytes) {
+        if (c->ws) c->alloc.free(c->ws, c->alloc.ctx);
+        c->ws = nullptr;
+        c->ws_bytes = 0;
+        const size_t want = bytes + bytes / 4;
+        c->ws = cache_alloc(c, want, s);
+        if (!c->ws) return SISO_ERR_OOM;
+        c->ws_bytes = want;
+    }
+    out->base = static_cast<char *>(c->ws);
+    out->off = 0;
+    out->cap = c->ws_bytes;
+    return SISO_OK;
+}
+
+__global__ void bf16_from_master_kernel(const float *__restrict__ m, __nv_bfloat16 *__restrict__ v, long long n) {
+    const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i < n) v[i] = __float2bfloat16_rn(m[i]);
+}
+
+__global__ void import_counters_kernel(const uint8_t *__restrict__ valid, long long capacity, long long *counters,
+                                       unsigned long long clock) {
+    __shared__ int warp_sum[32];
+    long long cnt = 0;
+    for (long long i = threadIdx.x; i < capacity; i += blockDim.x) cnt += valid[i] ? 1 : 0;
+    int x = static_cast<int>(cnt);
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
+    if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = x;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long t = 0;
+        for (int w = 0; w < static_cast<int>(blockDim.x / 32); ++w) t += warp_sum[w];
+        counters[CNT_OCCUPANCY] = t;
+        counters[CNT_CLOCK] = static_cast<long long>(clock);
+    }
+}
+
+__global__ void normalise_valid_kernel(uint8_t *valid, long long n) {
+    const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i < n) valid[i] = valid[i] ? 1 : 0;
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+}  // namespace siso
+
+using namespace siso;
+
+struct siso_cache : public siso::Cache {};
+
+extern "C" {
+
+const char *siso_status_string(siso_status_t s) {
+    switch (s) {
+        case SISO_OK: return "ok";
+        case SISO_ERR_INVALID_ARG: return "invalid argument";
+        case SISO_ERR_UNSUPPORTED: return "unsupported";
+        case SISO_ERR_OOM: return "out of device memory";
+        case SISO_ERR_CAPACITY: return "not enough free slots";
+        case SISO_ERR_OVERFLOW: return "merge candidate buffer overflow";
+        case SISO_ERR_TIMEOUT: return "a bounded device-side wait gave up";
+        case SISO_ERR_CUDA: return "CUDA error";
+    }
+    return "unknown status";
+}
+
+const char *siso_last_cuda_error(void) { return g_last_error; }
+
+siso_status_t siso_cache_create(siso_cache_t **out, const siso_config_t *cfg) {
+    if (!out || !cfg) return SISO_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (cfg->capacity < 1 || cfg->capacity >= (1ll << 31) - siso::kRowPad) return SISO_ERR_INVALID_ARG;
+    if (cfg->dim < 8 || cfg->dim > siso::kMaxDim) return SISO_ERR_UNSUPPORTED;
+    if (cfg->dim % 8 != 0) return SISO_ERR_UNSUPPORTED;
+    if (cfg->dtype != SISO_F32 && cfg->dtype != SISO_BF16) return SISO_ERR_INVALID_ARG;
+    if ((cfg->allocator.alloc == nullptr) != (cfg->allocator.free == nullptr)) return SISO_ERR_INVALID_ARG;
+    if (cfg->decay != 0.0 && !(cfg->decay > 0.0)) return SISO_ERR_INVALID_ARG;
+    int n_dev = 0;
+    SISO_CUDA(cudaGetDeviceCount(&n_dev));
+    if (cfg->device < 0 || cfg->device >= n_dev) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(cfg->device));
+    cudaDeviceProp prop;
+    SISO_CUDA(cudaGetDeviceProperties(&prop, cfg->device));
+    if (prop.major != 10) {
+        snprintf(g_last_error, sizeof(g_last_error), "device %d is sm_%d%d; this library holds sm_100a code only",
+                 cfg->device, prop.major, prop.minor);
+        return SISO_ERR_UNSUPPORTED;
+    }
+    siso_cache *c = new (std::nothrow) siso_cache();
+    if (!c) return SISO_ERR_OOM;
+    memset(static_cast<siso::Cache *>(c), 0, sizeof(siso::Cache));
+    c->capacity = cfg->capacity;
+    c->rows_alloc = (cfg->capacity + kRowPad - 1) / kRowPad * kRowPad;
+    c->dim = cfg->dim;
+    c->dtype = cfg->dtype;
+    c->device = cfg->device;
+    c->sm_count = prop.multiProcessorCount;
+    c->decay = cfg->decay == 0.0 ? 1.1 : cfg->decay;
+    if (cfg->allocator.alloc) { c->alloc = cfg->allocator; c->own_alloc = false; }
+    else { c->alloc.alloc = default_alloc; c->alloc.free = default_free; c->alloc.ctx = nullptr; c->own_alloc = true; }
+    c->lookup_path = SISO_PATH_AUTO;
+    c->merge_max_cand = 16 * c->capacity + (1ll << 20);
+
+    const size_t rows = static_cast<size_t>(c->rows_alloc), D = static_cast<size_t>(c->dim);
+    const size_t esz = c->dtype == SISO_F32 ? 4 : 2;
+    cudaStream_t s0 = nullptr;
+    bool ok = true;
+    c->master = static_cast<float *>(cache_alloc(c, rows * D * 4, s0));
+    ok = ok && c->master;
+    if (c->dtype == SISO_F32) c->vecs = c->master;
+    else { c->vecs = cache_alloc(c, rows * D * esz, s0); ok = ok && c->vecs; }
+    c->size = static_cast<double *>(cache_alloc(c, rows * 8, s0)); ok = ok && c->size;
+    c->access = static_cast<uint32_t *>(cache_alloc(c, rows * 4, s0)); ok = ok && c->access;
+    c->last = static_cast<unsigned long long *>(cache_alloc(c, rows * 8, s0)); ok = ok && c->last;
+    c->valid = static_cast<uint8_t *>(cache_alloc(c, rows, s0)); ok = ok && c->valid;
+    c->counters = static_cast<long long *>(cache_alloc(c, sizeof(long long) * CNT_N, s0)); ok = ok && c->counters;
+    c->status = static_cast<int *>(cache_alloc(c, 256, s0)); ok = ok && c->status;
+    if (!ok) { siso_cache_destroy(c); return SISO_ERR_OOM; }
+    cudaError_t e = cudaMemset(c->master, 0, rows * D * 4);
+    if (e == cudaSuccess && c->dtype != SISO_F32) e = cudaMemset(c->vecs, 0, rows * D * esz);
+    if (e == cudaSuccess) e = cudaMemset(c->size, 0, rows * 8);
+    if (e == cudaSuccess) e = cudaMemset(c->access, 0, rows * 4);
+    if (e == cudaSuccess) e = cudaMemset(c->last, 0, rows * 8);
+    if (e == cudaSuccess) e = cudaMemset(c->valid, 0, rows);
+    if (e == cudaSuccess) e = cudaMemset(c->counters, 0, sizeof(long long) * CNT_N);
+    if (e == cudaSuccess) e = cudaMemset(c->status, 0, 256);
+    if (e == cudaSuccess) e = cudaDeviceSynchronize();
+    if (e != cudaSuccess) { siso_status_t st = check_cuda(e, "cache initialisation"); siso_cache_destroy(c); return st; }
+    *out = c;
+    return SISO_OK;
+}
+
+siso_status_t siso_cache_destroy(siso_cache_t *c) {
+    if (!c) return SISO_ERR_INVALID_ARG;
+    cudaSetDevice(c->device);
+    cudaDeviceSynchronize();
+    tensor_state_destroy(c);
+    void *ptrs[] = {c->dtype == SISO_F32 ? nullptr : c->vecs, c->master, c->size, c->access, c->last, c->valid,
+                    c->counters, c->status, c->ws, c->stage};
+    for (void *p : ptrs)
+        if (p) c->alloc.free(p, c->alloc.ctx);
+    delete c;
+    return SISO_OK;
+}
+
+siso_status_t siso_set_option(siso_cache_t *c, int32_t key, int64_t value) {
+    if (!c) return SISO_ERR_INVALID_ARG;
+    switch (key) {
+        case SISO_OPT_LOOKUP_PATH:
+            if (value < SISO_PATH_AUTO || value > SISO_PATH_STREAM) return SISO_ERR_INVALID_ARG;
+            if (value == SISO_PATH_TENSOR && c->dtype != SISO_BF16) return SISO_ERR_UNSUPPORTED;
+            c->lookup_path = static_cast<int32_t>(value);
+            return SISO_OK;
+        case SISO_OPT_MERGE_MAX_CANDIDATES:
+            if (value < 1 || value > (1ll << 31)) return SISO_ERR_INVALID_ARG;
+            c->merge_max_cand = value;
+            return SISO_OK;
+    }
+    return SISO_ERR_INVALID_ARG;
+}
+
+siso_status_t siso_insert(siso_cache_t *c, const void *d_vecs, const double *d_sizes, int64_t n, int32_t *d_slots_out,
+                          void *stream) {
+    if (!c || n < 0 || (n > 0 && !d_vecs)) return SISO_ERR_INVALID_ARG;
+    if (n > 0 && !aligned16(d_vecs)) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    return launch_insert(c, d_vecs, d_sizes, nullptr, n, d_slots_out, static_cast<cudaStream_t>(stream));
+}
+
+siso_status_t siso_lookup(siso_cache_t *c, const void *d_queries, int64_t n_queries, const float *d_theta,
+                          float theta_scalar, int32_t k, int32_t *d_idx, float *d_sim, uint8_t *d_hit, void *stream) {
+    if (!c || n_queries < 0 || k < 1 || k > kMaxK) return SISO_ERR_INVALID_ARG;
+    if (n_queries == 0) return SISO_OK;
+    if (!d_queries || !d_idx || !d_sim || !d_hit || !aligned16(d_queries)) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int path = c->lookup_path;
+    if (path == SISO_PATH_AUTO) {
+        if (n_queries <= 4) path = SISO_PATH_STREAM;
+        else if (c->dtype == SISO_BF16 && n_queries >= 16) path = SISO_PATH_TENSOR;
+        else path = SISO_PATH_SIMT;
+    }
+    switch (path) {
+        case SISO_PATH_STREAM: return launch_lookup_stream(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);
+        case SISO_PATH_TENSOR: return launch_lookup_tensor(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);
+        default: return launch_lookup_simt(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);
+    }
+}
+
+siso_status_t siso_lookup_host(siso_cache_t *c, const void *h_queries, int64_t n_queries, const float *h_theta,
+                               float theta_scalar, int32_t k, int32_t *h_idx, float *h_sim, uint8_t *h_hit,
+                               void *stream) {
+    if (!c || n_queries < 0 || k < 1 || k > kMaxK) return SISO_ERR_INVALID_ARG;
+    if (n_queries == 0) return SISO_OK;
+    if (!h_queries || !h_idx || !h_sim || !h_hit) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t esz = c->dtype == SISO_F32 ? 4 : 2;
+    const size_t qb = pad256(static_cast<size_t>(n_queries) * c->dim * esz), tb = pad256(sizeof(float) * n_queries);
+    const size_t ib = pad256(sizeof(int32_t) * n_queries * k), sb = pad256(sizeof(float) * n_queries * k);
+    const size_t hb = pad256(static_cast<size_t>(n_queries));
+    const size_t need = qb + tb + ib + sb + hb;
+    if (need > c->stage_bytes) {
+        if (c->stage) c->alloc.free(c->stage, c->alloc.ctx);
+        c->stage = nullptr;
+        c->stage_bytes = 0;
+        c->stage = cache_alloc(c, need, s);
+        if (!c->stage) return SISO_ERR_OOM;
+        c->stage_bytes = need;
+    }
+    char *p = static_cast<char *>(c->stage);
+    void *dq = p; float *dt = reinterpret_cast<float *>(p + qb);
+    int32_t *di = reinterpret_cast<int32_t *>(p + qb + tb);
+    float *ds = reinterpret_cast<float *>(p + qb + tb + ib);
+    uint8_t *dh = reinterpret_cast<uint8_t *>(p + qb + tb + ib + sb);
+    SISO_CUDA(cudaMemcpyAsync(dq, h_queries, static_cast<size_t>(n_queries) * c->dim * esz, cudaMemcpyHostToDevice, s));
+    if (h_theta) SISO_CUDA(cudaMemcpyAsync(dt, h_theta, sizeof(float) * n_queries, cudaMemcpyHostToDevice, s));
+    SISO_TRY(siso_lookup(c, dq, n_queries, h_theta ? dt : nullptr, theta_scalar, k, di, ds, dh, stream));
+    SISO_CUDA(cudaMemcpyAsync(h_idx, di, sizeof(int32_t) * n_queries * k, cudaMemcpyDeviceToHost, s));
+    SISO_CUDA(cudaMemcpyAsync(h_sim, ds, sizeof(float) * n_queries * k, cudaMemcpyDeviceToHost, s));
+    SISO_CUDA(cudaMemcpyAsync(h_hit, dh, static_cast<size_t>(n_queries), cudaMemcpyDeviceToHost, s));
+    return SISO_OK;
+}
+
+siso_status_t siso_update(siso_cache_t *c, const void *d_queries, int64_t n_queries, const int32_t *d_idx,
+                          int32_t idx_stride, const uint8_t *d_hit, void *stream) {
+    if (!c || n_queries < 0 || idx_stride < 1) return SISO_ERR_INVALID_ARG;
+    if (n_queries > 0 && (!d_queries || !d_idx || !d_hit || !aligned16(d_queries))) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    return launch_update(c, d_queries, n_queries, d_idx, idx_stride, d_hit, static_cast<cudaStream_t>(stream));
+}
+
+siso_status_t siso_merge(siso_cache_t *c, const void *d_repo, const double *d_repo_sizes, int64_t n_repo, float theta_c,
+                         uint32_t flags, int32_t *d_merge_map, int64_t *h_n_merged, void *stream) {
+    if (!c || (flags & ~SISO_MERGE_WEIGHTED_MEAN) || !(theta_c == theta_c)) return SISO_ERR_INVALID_ARG;
+    if (d_repo || d_repo_sizes || n_repo != 0) return SISO_ERR_UNSUPPORTED;
+    SISO_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    long long *d_n = nullptr;
+    if (h_n_merged) d_n = c->counters + CNT_SPARE;
+    SISO_TRY(launch_merge(c, theta_c, flags, d_merge_map, d_n, s));
+    if (h_n_merged) {
+        long long v = 0;
+        SISO_CUDA(cudaMemcpyAsync(&v, d_n, sizeof(v), cudaMemcpyDeviceToHost, s));
+        SISO_CUDA(cudaStreamSynchronize(s));
+        *h_n_merged = v;
+        return siso_sync_status(c, stream);
+    }
+    return SISO_OK;
+}
+
+siso_status_t siso_evict(siso_cache_t *c, int64_t n_evict, uint32_t flags, int32_t *d_victims, void *stream) {
+    if (!c || n_evict < 0 || (flags & ~SISO_EVICT_DECAY)) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    return launch_evict(c, n_evict, nullptr, 0, flags, d_victims, n_evict, static_cast<cudaStream_t>(stream));
+}
+
+siso_status_t siso_make_room(siso_cache_t *c, const uint8_t *d_hit, int64_t n, uint32_t flags, int32_t *d_victims,
+                             void *stream) {
+    if (!c || n < 0 || (n > 0 && !d_hit) || (flags & ~SISO_EVICT_DECAY)) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    return launch_evict(c, -1, d_hit, n, flags, d_victims, n, static_cast<cudaStream_t>(stream));
+}
+
+siso_status_t siso_insert_misses(siso_cache_t *c, const void *d_queries, int64_t n, const uint8_t *d_hit,
+                                 int32_t *d_slots_out, void *stream) {
+    if (!c || n < 0 || (n > 0 && (!d_queries || !d_hit || !aligned16(d_queries)))) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    return launch_insert(c, d_queries, nullptr, d_hit, n, d_slots_out, static_cast<cudaStream_t>(stream));
+}
+
+siso_status_t siso_stream_step(siso_cache_t *c, const void *d_queries, int64_t n, const float *d_theta,
+                               float theta_scalar, int32_t *d_idx, float *d_sim, uint8_t *d_hit, int32_t *d_victims,
+                               int32_t *d_slots_out, void *stream) {
+    if (!c || n < 0) return SISO_ERR_INVALID_ARG;
+    if (n == 0) return SISO_OK;
+    SISO_TRY(siso_lookup(c, d_queries, n, d_theta, theta_scalar, 1, d_idx, d_sim, d_hit, stream));
+    SISO_TRY(siso_update(c, d_queries, n, d_idx, 1, d_hit, stream));
+    SISO_TRY(siso_make_room(c, d_hit, n, 0, d_victims, stream));
+    return siso_insert_misses(c, d_queries, n, d_hit, d_slots_out, stream);
+}
+
+siso_status_t siso_export(siso_cache_t *c, void *d_vecs, float *d_master, double *d_sizes, uint32_t *d_access,
+                          uint64_t *d_last, uint8_t *d_valid, void *stream) {
+    if (!c) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t n = static_cast<size_t>(c->capacity), D = static_cast<size_t>(c->dim);
+    const size_t esz = c->dtype == SISO_F32 ? 4 : 2;
+    if (d_vecs) SISO_CUDA(cudaMemcpyAsync(d_vecs, c->vecs, n * D * esz, cudaMemcpyDeviceToDevice, s));
+    if (d_master) SISO_CUDA(cudaMemcpyAsync(d_master, c->master, n * D * 4, cudaMemcpyDeviceToDevice, s));
+    if (d_sizes) SISO_CUDA(cudaMemcpyAsync(d_sizes, c->size, n * 8, cudaMemcpyDeviceToDevice, s));
+    if (d_access) SISO_CUDA(cudaMemcpyAsync(d_access, c->access, n * 4, cudaMemcpyDeviceToDevice, s));
+    if (d_last) SISO_CUDA(cudaMemcpyAsync(d_last, c->last, n * 8, cudaMemcpyDeviceToDevice, s));
+    if (d_valid) SISO_CUDA(cudaMemcpyAsync(d_valid, c->valid, n, cudaMemcpyDeviceToDevice, s));
+    return SISO_OK;
+}
+
+siso_status_t siso_import(siso_cache_t *c, const float *d_master, const double *d_sizes, const uint32_t *d_access,
+                          const uint64_t *d_last, const uint8_t *d_valid, uint64_t clock, void *stream) {
+    if (!c || !d_master || !d_sizes || !d_access || !d_last || !d_valid) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t n = static_cast<size_t>(c->capacity), D = static_cast<size_t>(c->dim);
+    SISO_CUDA(cudaMemcpyAsync(c->master, d_master, n * D * 4, cudaMemcpyDeviceToDevice, s));
+    SISO_CUDA(cudaMemcpyAsync(c->size, d_sizes, n * 8, cudaMemcpyDeviceToDevice, s));
+    SISO_CUDA(cudaMemcpyAsync(c->access, d_access, n * 4, cudaMemcpyDeviceToDevice, s));
+    SISO_CUDA(cudaMemcpyAsync(c->last, d_last, n * 8, cudaMemcpyDeviceToDevice, s));
+    SISO_CUDA(cudaMemcpyAsync(c->valid, d_valid, n, cudaMemcpyDeviceToDevice, s));
+    normalise_valid_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, s>>>(c->valid, static_cast<long long>(n));
+    SISO_LAUNCHED(c);
+    if (c->dtype == SISO_BF16) {
+        const long long total = static_cast<long long>(n * D);
+        bf16_from_master_kernel<<<static_cast<unsigned>((total + 255) / 256), 256, 0, s>>>(
+            c->master, static_cast<__nv_bfloat16 *>(c->vecs), total);
+        SISO_LAUNCHED(c);
+    }
+    import_counters_kernel<<<1, 1024, 0, s>>>(c->valid, c->capacity, c->counters, clock);
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
+
+siso_status_t siso_get_stats(siso_cache_t *c, int64_t *h_counts, void *stream) {
+    if (!c || !h_counts) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    long long tmp[CNT_N];
+    SISO_CUDA(cudaMemcpyAsync(tmp, c->counters, sizeof(tmp), cudaMemcpyDeviceToHost, s));
+    SISO_CUDA(cudaStreamSynchronize(s));
+    for (int i = 0; i < 8; ++i) h_counts[i] = i < CNT_SPARE ? tmp[i] : 0;
+    return SISO_OK;
+}
+
+siso_status_t siso_sync_status(siso_cache_t *c, void *stream) {
+    if (!c) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    int st = 0;
+    SISO_CUDA(cudaMemcpyAsync(&st, c->status, sizeof(int), cudaMemcpyDeviceToHost, s));
+    SISO_CUDA(cudaStreamSynchronize(s));
+    if (st != 0) SISO_CUDA(cudaMemsetAsync(c->status, 0, sizeof(int), s));
+    return static_cast<siso_status_t>(st);
+}
+
+int64_t siso_launch_count(const siso_cache_t *c) { return c ? c->launches : 0; }
+
+}  // extern "C"

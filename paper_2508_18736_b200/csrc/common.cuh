@@ -1,0 +1,184 @@
+// Internal declarations shared by the kernels of libsiso (never installed; the public
+// interface is include/siso.h).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <algorithm>
+
+#include "../../include/siso.h"
+
+namespace siso {
+
+constexpr int kRowPad = 256;        // vector arrays are allocated in multiples of this many rows, zero-filled
+constexpr int kMaxDim = 4096;
+constexpr int kMaxK = 8;
+constexpr uint32_t kNoSlot = 0xFFFFFFFFu;
+
+// device counters, int64 each
+enum Counter { CNT_OCCUPANCY = 0, CNT_LOOKUPS, CNT_HITS, CNT_INSERTS, CNT_EVICTIONS, CNT_MERGES, CNT_CLOCK, CNT_SPARE, CNT_N };
+
+struct Cache {
+    int64_t capacity;
+    int64_t rows_alloc;    // capacity rounded up to kRowPad
+    int32_t dim;
+    int32_t dtype;
+    int32_t device;
+    int32_t sm_count;
+    double decay;
+    siso_allocator_t alloc;
+    bool own_alloc;
+
+    void *vecs;            // [rows_alloc, dim] lookup copy in the cache dtype (for fp32 caches this IS the master)
+    float *master;         // [rows_alloc, dim] fp32 master
+    double *size;          // [rows_alloc] cluster_size
+    uint32_t *access;      // [rows_alloc] access_count
+    unsigned long long *last;  // [rows_alloc] last_access
+    uint8_t *valid;        // [rows_alloc]
+    long long *counters;   // [CNT_N]
+    int *status;           // device status word (first error wins)
+
+    // scratch, grown on demand
+    void *ws;
+    size_t ws_bytes;
+    // staging for the host-buffer lookup
+    void *stage;
+    size_t stage_bytes;
+
+    int32_t lookup_path;
+    int64_t merge_max_cand;
+    int64_t launches;
+    void *tensor_state;    // owned by lookup_tensor.cu
+};
+
+// ---- scratch bump allocator -------------------------------------------------
+struct Scratch {
+    char *base;
+    size_t off, cap;
+    template <typename T> T *take(size_t n) {
+        size_t bytes = (n * sizeof(T) + 255) & ~size_t(255);
+        T *p = reinterpret_cast<T *>(base + off);
+        off += bytes;
+        return p;
+    }
+};
+inline size_t pad256(size_t b) { return (b + 255) & ~size_t(255); }
+siso_status_t scratch_reserve(Cache *c, size_t bytes, cudaStream_t s, Scratch *out);
+siso_status_t check_cuda(cudaError_t e, const char *what);
+#define SISO_CUDA(expr)                                                  \
+    do {                                                                 \
+        siso_status_t st__ = ::siso::check_cuda((expr), #expr);          \
+        if (st__ != SISO_OK) return st__;                                \
+    } while (0)
+#define SISO_TRY(expr)                                                   \
+    do {                                                                 \
+        siso_status_t st__ = (expr);                                     \
+        if (st__ != SISO_OK) return st__;                                \
+    } while (0)
+#define SISO_LAUNCHED(c)                                                 \
+    do {                                                                 \
+        (c)->launches += 1;                                              \
+        SISO_CUDA(cudaGetLastError());                                   \
+    } while (0)
+
+// ---- launchers implemented in the .cu files -----------------------------------
+siso_status_t launch_lookup_simt(Cache *c, const void *q, int64_t B, const float *theta, float theta_s, int k,
+                                 int32_t *idx, float *sim, uint8_t *hit, cudaStream_t s);
+siso_status_t launch_lookup_stream(Cache *c, const void *q, int64_t B, const float *theta, float theta_s, int k,
+                                   int32_t *idx, float *sim, uint8_t *hit, cudaStream_t s);
+siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const float *theta, float theta_s, int k,
+                                   int32_t *idx, float *sim, uint8_t *hit, cudaStream_t s);
+void tensor_state_destroy(Cache *c);
+siso_status_t launch_topk_finalize(Cache *c, const unsigned long long *partial, int64_t B, int splits, int kmax, int k,
+                                   const float *theta, float theta_s, int32_t *idx, float *sim, uint8_t *hit,
+                                   cudaStream_t s);
+siso_status_t launch_update(Cache *c, const void *q, int64_t B, const int32_t *idx, int idx_stride, const uint8_t *hit,
+                            cudaStream_t s);
+siso_status_t launch_merge(Cache *c, float theta_c, uint32_t flags, int32_t *merge_map, long long *d_n_merged,
+                           cudaStream_t s);
+siso_status_t launch_evict(Cache *c, int64_t n_evict, const uint8_t *hit, int64_t n_hit, uint32_t flags,
+                           int32_t *victims, int64_t n_victims_out, cudaStream_t s);
+siso_status_t launch_insert(Cache *c, const void *vecs, const double *sizes, const uint8_t *hit, int64_t n,
+                            int32_t *slots_out, cudaStream_t s);
+siso_status_t launch_sort_pairs(Cache *c, Scratch *scr, uint32_t *keys, uint32_t *vals, uint32_t *keys_tmp,
+                                uint32_t *vals_tmp, int64_t n, int key_bits, uint32_t **keys_out, uint32_t **vals_out,
+                                cudaStream_t s);
+size_t sort_pairs_scratch_bytes(int64_t n);
+siso_status_t launch_exclusive_scan_u32(Cache *c, uint32_t *a, int64_t n, cudaStream_t s);
+
+#ifdef __CUDACC__
+// ---- device helpers ------------------------------------------------------------
+// Order-preserving map fp32 -> u32, and the packed (similarity, slot) key whose maximum is the
+// best match with ties going to the lower slot.  Key 0 means "no entry".
+__device__ __forceinline__ uint32_t f32_sortable(float f) {
+    uint32_t u = __float_as_uint(f);
+    return (u & 0x80000000u) ? ~u : (u | 0x80000000u);
+}
+__device__ __forceinline__ float sortable_f32(uint32_t s) {
+    uint32_t u = (s & 0x80000000u) ? (s & 0x7FFFFFFFu) : ~s;
+    return __uint_as_float(u);
+}
+__device__ __forceinline__ unsigned long long pack_key(float sim, uint32_t slot) {
+    return (static_cast<unsigned long long>(f32_sortable(sim)) << 32) | (0xFFFFFFFFu - slot);
+}
+__device__ __forceinline__ float key_sim(unsigned long long k) { return sortable_f32(static_cast<uint32_t>(k >> 32)); }
+__device__ __forceinline__ int32_t key_slot(unsigned long long k) {
+    return static_cast<int32_t>(0xFFFFFFFFu - static_cast<uint32_t>(k));
+}
+
+// Sorted (descending) list of K packed keys in registers; insert keeps the K largest.
+template <int K> struct KeyList {
+    unsigned long long k[K];
+    __device__ __forceinline__ void clear() {
+#pragma unroll
+        for (int i = 0; i < K; ++i) k[i] = 0ull;
+    }
+    __device__ __forceinline__ void insert(unsigned long long v) {
+        if (v > k[K - 1]) {
+            k[K - 1] = v;
+#pragma unroll
+            for (int i = K - 1; i > 0; --i) {
+                if (k[i] > k[i - 1]) {
+                    unsigned long long t = k[i];
+                    k[i] = k[i - 1];
+                    k[i - 1] = t;
+                }
+            }
+        }
+    }
+};
+
+// Per-thread running top-K over a stream of (similarity, slot) pairs that arrive in ASCENDING slot
+// order: a later pair with an equal similarity never displaces an earlier one, so a strict float
+// comparison implements "ties to the lower slot".
+template <int K> struct TopK {
+    float s[K];
+    int32_t i[K];
+    __device__ __forceinline__ void clear() {
+#pragma unroll
+        for (int j = 0; j < K; ++j) { s[j] = -INFINITY; i[j] = -1; }
+    }
+    __device__ __forceinline__ void push(float v, int32_t slot) {
+        if (v > s[K - 1]) {          // empty places hold -inf, so any finite similarity enters
+            s[K - 1] = v;
+            i[K - 1] = slot;
+#pragma unroll
+            for (int j = K - 1; j > 0; --j) {
+                if (s[j] > s[j - 1]) {
+                    float ts = s[j]; s[j] = s[j - 1]; s[j - 1] = ts;
+                    int32_t ti = i[j]; i[j] = i[j - 1]; i[j - 1] = ti;
+                }
+            }
+        }
+    }
+    __device__ __forceinline__ unsigned long long key(int j) const { return i[j] < 0 ? 0ull : pack_key(s[j], (uint32_t)i[j]); }
+};
+
+__device__ __forceinline__ float bf16_bits_to_f32(uint32_t b) { return __uint_as_float(b << 16); }
+
+__device__ __forceinline__ void set_status(int *status, int code) { atomicCAS(status, 0, code); }
+#endif  // __CUDACC__
+
+}  // namespace siso

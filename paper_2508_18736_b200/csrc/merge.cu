@@ -1,0 +1,285 @@
+// MergeCentroids (Algorithm 1) over the cache itself, in ascending slot order.
+//
+//   sweep    blocked pairwise similarity of the fp32 master vectors (lower triangle only); every
+//            pair (i, j), j < i, with similarity > theta_c becomes a candidate record
+//   group    candidates are grouped by row i (count, scan, scatter)
+//   resolve  entry i joins the most similar SURVIVOR among its candidates (ties: lowest slot), else
+//            survives.  Whether j survives is known once all of j's own candidates are decided, so
+//            one CTA iterates rounds until every row is decided; each decision is final and equals
+//            the sequential algorithm's, whatever the timing of the rounds
+//   apply    merged entries are grouped by survivor with a stable sort; each survivor adds the
+//            members' cluster_size in ascending slot order and, in weighted-mean mode, becomes
+//            normalise(sum of cluster_size * vector over itself and its members)
+// The similarity used is that of the vectors as they were when the call began: nothing is written
+// before the sweep has finished.  If the candidates do not fit their buffer the status word gets
+// SISO_ERR_OVERFLOW and every later kernel of the call returns without writing.
+#include "sweep_simt.cuh"
+
+namespace siso {
+
+using namespace sweep;
+
+struct Candidate {
+    int32_t i, j;
+    float sim;
+};
+
+struct MergeCtl {
+    unsigned long long n_cand;   // candidates found (may exceed the buffer: overflow)
+    int overflow;
+    int n_merged;
+};
+
+// grid = (tile pairs of the lower triangle incl. diagonal).  blockIdx.x -> (ti, tj), tj <= ti.
+__global__ void __launch_bounds__(THREADS, 2)
+merge_sweep_kernel(const float *__restrict__ C, const uint8_t *__restrict__ valid, int64_t N, int D, float theta,
+                   MergeCtl *ctl, Candidate *__restrict__ cand, unsigned long long max_cand,
+                   uint32_t *__restrict__ row_count) {
+    extern __shared__ __align__(16) float smem[];
+    __shared__ uint8_t valid_i[BM], valid_j[BN];
+    // invert p = ti*(ti+1)/2 + tj
+    const long long p = blockIdx.x;
+    long long ti = static_cast<long long>((sqrt(8.0 * static_cast<double>(p) + 1.0) - 1.0) * 0.5);
+    while (ti * (ti + 1) / 2 > p) --ti;
+    while ((ti + 1) * (ti + 2) / 2 <= p) ++ti;
+    const long long tj = p - ti * (ti + 1) / 2;
+    const int64_t i0 = ti * BM, j0 = tj * BN;
+    const int tid = threadIdx.x;
+    tile_to_smem<float>(C, N, i0, C, N, j0, D, smem);
+    if (tid < BM) valid_i[tid] = (i0 + tid < N) ? valid[i0 + tid] : 0;
+    else if (tid < BM + BN) valid_j[tid - BM] = (j0 + tid - BM < N) ? valid[j0 + tid - BM] : 0;
+    __syncthreads();
+    const int row = tid >> 1, par = tid & 1, lane = tid & 31;
+    const float *srow = smem + row * S_STRIDE;
+    const int64_t gi = i0 + row;
+    for (int it = 0; it < BN / 2; ++it) {
+        const int cidx = par + 2 * it;
+        const int64_t gj = j0 + cidx;
+        const float v = srow[cidx];
+        const bool take = valid_i[row] && valid_j[cidx] && gj < gi && v > theta;
+        const unsigned ballot = __ballot_sync(0xFFFFFFFFu, take);
+        if (ballot) {
+            unsigned long long base = 0;
+            if (lane == 0) base = atomicAdd(&ctl->n_cand, static_cast<unsigned long long>(__popc(ballot)));
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            if (take) {
+                const unsigned long long pos = base + __popc(ballot & ((1u << lane) - 1u));
+                if (pos < max_cand) {
+                    Candidate cd;
+                    cd.i = static_cast<int32_t>(gi); cd.j = static_cast<int32_t>(gj); cd.sim = v;
+                    cand[pos] = cd;
+                    atomicAdd(&row_count[gi], 1u);
+                } else {
+                    ctl->overflow = 1;
+                }
+            }
+        }
+    }
+}
+
+__global__ void merge_check_kernel(MergeCtl *ctl, int *status) {
+    if (ctl->overflow) set_status(status, SISO_ERR_OVERFLOW);
+}
+
+// in: row_off = exclusive scan of row_count.  Scatter candidates into row-grouped order.
+__global__ void merge_scatter_kernel(const MergeCtl *ctl, const Candidate *__restrict__ cand,
+                                     const uint32_t *__restrict__ row_off, uint32_t *__restrict__ row_cursor,
+                                     int32_t *__restrict__ csr_j, float *__restrict__ csr_sim) {
+    if (ctl->overflow) return;
+    const unsigned long long n = ctl->n_cand;
+    for (unsigned long long e = static_cast<unsigned long long>(blockIdx.x) * blockDim.x + threadIdx.x; e < n;
+         e += static_cast<unsigned long long>(gridDim.x) * blockDim.x) {
+        const Candidate cd = cand[e];
+        const uint32_t pos = row_off[cd.i] + atomicAdd(&row_cursor[cd.i], 1u);
+        csr_j[pos] = cd.j;
+        csr_sim[pos] = cd.sim;
+    }
+}
+
+// state: 0 undecided, 1 survivor, 2 merged, 3 empty slot
+__global__ void __launch_bounds__(1024)
+merge_resolve_kernel(MergeCtl *ctl, int64_t N, const uint8_t *__restrict__ valid, const uint32_t *__restrict__ row_off,
+                     const uint32_t *__restrict__ row_count, const int32_t *__restrict__ csr_j,
+                     const float *__restrict__ csr_sim, volatile uint8_t *state, int32_t *__restrict__ target) {
+    if (ctl->overflow) return;
+    __shared__ int undecided_s;
+    const int tid = threadIdx.x;
+    for (int64_t i = tid; i < N; i += 1024) {
+        state[i] = valid[i] ? (row_count[i] == 0 ? 1 : 0) : 3;
+        target[i] = valid[i] ? static_cast<int32_t>(i) : -1;
+    }
+    __threadfence_block();
+    __syncthreads();
+    // every round decides at least the lowest undecided row, so at most N rounds are needed
+    for (int64_t round = 0; round <= N; ++round) {
+        if (tid == 0) undecided_s = 0;
+        __syncthreads();
+        int left = 0;
+        for (int64_t i = tid; i < N; i += 1024) {
+            if (state[i] != 0) continue;
+            const uint32_t o = row_off[i], cnt = row_count[i];
+            bool ready = true;
+            unsigned long long best = 0ull;
+            for (uint32_t e = 0; e < cnt; ++e) {
+                const int32_t j = csr_j[o + e];
+                const uint8_t sj = state[j];
+                if (sj == 0) { ready = false; break; }
+                if (sj == 1) {
+                    const unsigned long long key = pack_key(csr_sim[o + e], static_cast<uint32_t>(j));
+                    best = key > best ? key : best;
+                }
+            }
+            if (!ready) { ++left; continue; }
+            if (best) { target[i] = key_slot(best); state[i] = 2; }
+            else state[i] = 1;
+        }
+        __threadfence_block();
+        if (left) atomicAdd(&undecided_s, left);
+        __syncthreads();
+        const int any = undecided_s;
+        __syncthreads();
+        if (!any) break;
+    }
+}
+
+// keys for the grouping sort: survivor slot for merged rows, N (sorts last) otherwise
+__global__ void merge_keys_kernel(const MergeCtl *ctl, int64_t N, const volatile uint8_t *state,
+                                  const int32_t *__restrict__ target, uint32_t *__restrict__ keys,
+                                  uint32_t *__restrict__ vals) {
+    if (ctl->overflow) return;
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= N) return;
+    keys[i] = state[i] == 2 ? static_cast<uint32_t>(target[i]) : static_cast<uint32_t>(N);
+    vals[i] = static_cast<uint32_t>(i);
+}
+
+// One CTA per position of the sorted (survivor, member) list; the head of a group does the group.
+template <typename T>
+__global__ void __launch_bounds__(256)
+merge_apply_kernel(MergeCtl *ctl, const uint32_t *__restrict__ keys, const uint32_t *__restrict__ members, int64_t N,
+                   int D, int weighted, float *__restrict__ master, T *__restrict__ vecs, double *__restrict__ size,
+                   uint8_t *__restrict__ valid) {
+    if (ctl->overflow) return;
+    extern __shared__ double acc[];
+    __shared__ double red[8];
+    const int64_t p = blockIdx.x;
+    const uint32_t sv = keys[p];
+    if (sv >= N) return;
+    if (p > 0 && keys[p - 1] == sv) return;
+    int64_t e = p;
+    while (e < N && keys[e] == sv) ++e;
+    const double own = size[sv];
+    double total = own;
+    for (int64_t t = p; t < e; ++t) total += size[members[t]];       // ascending member slot: fixed order
+    if (weighted) {
+        float *m = master + static_cast<int64_t>(sv) * D;
+        for (int d = threadIdx.x; d < D; d += 256) acc[d] = own * static_cast<double>(m[d]);
+        for (int64_t t = p; t < e; ++t) {
+            const uint32_t mb = members[t];
+            const double w = size[mb];
+            const float *mv = master + static_cast<int64_t>(mb) * D;
+            for (int d = threadIdx.x; d < D; d += 256) acc[d] += w * static_cast<double>(mv[d]);
+        }
+        double ss = 0.0;
+        for (int d = threadIdx.x; d < D; d += 256) ss += acc[d] * acc[d];
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+        if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+        __syncthreads();
+        double nn = 0.0;
+        for (int w = 0; w < 8; ++w) nn += red[w];
+        nn = sqrt(nn);
+        T *v = vecs + static_cast<int64_t>(sv) * D;
+        for (int d = threadIdx.x; d < D; d += 256) {
+            const float f = static_cast<float>(acc[d] / nn);
+            m[d] = f;
+            if constexpr (sizeof(T) == 2) v[d] = __float2bfloat16_rn(f);
+        }
+    }
+    __syncthreads();      // every read of member sizes is done before they could be reused
+    if (threadIdx.x == 0) size[sv] = total;
+    for (int64_t t = p + threadIdx.x; t < e; t += 256) valid[members[t]] = 0;
+    if (threadIdx.x == 0) atomicAdd(&ctl->n_merged, static_cast<int>(e - p));
+}
+
+__global__ void merge_finish_kernel(MergeCtl *ctl, int64_t N, const int32_t *__restrict__ target,
+                                    int32_t *__restrict__ merge_map, long long *counters, long long *n_merged_out) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (ctl->overflow) {
+        if (i == 0 && n_merged_out) *n_merged_out = 0;
+        return;
+    }
+    if (merge_map && i < N) merge_map[i] = target[i];
+    if (i == 0) {
+        counters[CNT_OCCUPANCY] -= ctl->n_merged;
+        counters[CNT_MERGES] += ctl->n_merged;
+        if (n_merged_out) *n_merged_out = ctl->n_merged;
+    }
+}
+
+siso_status_t launch_merge(Cache *c, float theta_c, uint32_t flags, int32_t *merge_map, long long *d_n_merged,
+                           cudaStream_t s) {
+    const int64_t N = c->capacity;
+    if (N >= (1ll << 31) - 1) return SISO_ERR_UNSUPPORTED;
+    const int64_t tiles = (N + BM - 1) / BM;
+    const int64_t pairs = tiles * (tiles + 1) / 2;
+    if (pairs > 0x7FFFFFFFll) return SISO_ERR_UNSUPPORTED;
+    const size_t max_cand = static_cast<size_t>(c->merge_max_cand);
+    Scratch scr;
+    size_t need = pad256(sizeof(MergeCtl)) + pad256(sizeof(Candidate) * max_cand) + 3 * pad256(sizeof(uint32_t) * (N + 1)) +
+                  pad256(sizeof(int32_t) * max_cand) + pad256(sizeof(float) * max_cand) + pad256(N) +
+                  pad256(sizeof(int32_t) * N) + 4 * pad256(sizeof(uint32_t) * N) + sort_pairs_scratch_bytes(N);
+    SISO_TRY(scratch_reserve(c, need, s, &scr));
+    MergeCtl *ctl = scr.take<MergeCtl>(1);
+    Candidate *cand = scr.take<Candidate>(max_cand);
+    uint32_t *row_count = scr.take<uint32_t>(N + 1);
+    uint32_t *row_off = scr.take<uint32_t>(N + 1);
+    uint32_t *row_cursor = scr.take<uint32_t>(N + 1);
+    int32_t *csr_j = scr.take<int32_t>(max_cand);
+    float *csr_sim = scr.take<float>(max_cand);
+    uint8_t *state = scr.take<uint8_t>(N);
+    int32_t *target = scr.take<int32_t>(N);
+    uint32_t *keys = scr.take<uint32_t>(N), *vals = scr.take<uint32_t>(N);
+    uint32_t *keys2 = scr.take<uint32_t>(N), *vals2 = scr.take<uint32_t>(N);
+
+    SISO_CUDA(cudaMemsetAsync(ctl, 0, sizeof(MergeCtl), s));
+    SISO_CUDA(cudaMemsetAsync(row_count, 0, sizeof(uint32_t) * (N + 1), s));
+    SISO_CUDA(cudaMemsetAsync(row_cursor, 0, sizeof(uint32_t) * (N + 1), s));
+    static bool attr_set = false;
+    if (!attr_set) {
+        SISO_CUDA(cudaFuncSetAttribute(merge_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+        attr_set = true;
+    }
+    merge_sweep_kernel<<<static_cast<unsigned>(pairs), THREADS, SMEM_BYTES, s>>>(c->master, c->valid, N, c->dim, theta_c,
+                                                                                ctl, cand, max_cand, row_count);
+    SISO_LAUNCHED(c);
+    merge_check_kernel<<<1, 1, 0, s>>>(ctl, c->status);
+    SISO_LAUNCHED(c);
+    SISO_CUDA(cudaMemcpyAsync(row_off, row_count, sizeof(uint32_t) * (N + 1), cudaMemcpyDeviceToDevice, s));
+    SISO_TRY(launch_exclusive_scan_u32(c, row_off, N + 1, s));
+    merge_scatter_kernel<<<4 * c->sm_count, 256, 0, s>>>(ctl, cand, row_off, row_cursor, csr_j, csr_sim);
+    SISO_LAUNCHED(c);
+    merge_resolve_kernel<<<1, 1024, 0, s>>>(ctl, N, c->valid, row_off, row_count, csr_j, csr_sim, state, target);
+    SISO_LAUNCHED(c);
+    const unsigned nblk = static_cast<unsigned>((N + 255) / 256);
+    merge_keys_kernel<<<nblk, 256, 0, s>>>(ctl, N, state, target, keys, vals);
+    SISO_LAUNCHED(c);
+    int key_bits = 1;
+    while ((1ll << key_bits) <= N) ++key_bits;
+    uint32_t *ks, *vs;
+    SISO_TRY(launch_sort_pairs(c, &scr, keys, vals, keys2, vals2, N, key_bits, &ks, &vs, s));
+    const int weighted = (flags & SISO_MERGE_WEIGHTED_MEAN) ? 1 : 0;
+    const size_t smem = sizeof(double) * c->dim;
+    if (c->dtype == SISO_F32)
+        merge_apply_kernel<float><<<static_cast<unsigned>(N), 256, smem, s>>>(ctl, ks, vs, N, c->dim, weighted, c->master,
+                                                                              static_cast<float *>(c->vecs), c->size, c->valid);
+    else
+        merge_apply_kernel<__nv_bfloat16><<<static_cast<unsigned>(N), 256, smem, s>>>(
+            ctl, ks, vs, N, c->dim, weighted, c->master, static_cast<__nv_bfloat16 *>(c->vecs), c->size, c->valid);
+    SISO_LAUNCHED(c);
+    merge_finish_kernel<<<nblk, 256, 0, s>>>(ctl, N, target, merge_map, c->counters, d_n_merged);
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
+
+}  // namespace siso

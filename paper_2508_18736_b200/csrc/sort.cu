@@ -1,0 +1,162 @@
+// Stable sort of (key, value) pairs of 32-bit integers.  It groups the hits of a batch by centroid
+// with the query order kept inside each group, and the merged entries by surviving slot, so that
+// every later floating-point sum is taken in one fixed order (bitwise reproducible results).
+//   n <= SMALL_N : one CTA, rank by counting over packed 64-bit (key, position) words
+//   otherwise    : least-significant-digit radix sort, 8 bits per pass, three kernels per pass
+#include "common.cuh"
+
+namespace siso {
+
+constexpr int SMALL_N = 2048;
+constexpr int RS_THREADS = 256;
+constexpr int RS_ITEMS = 8;                       // rounds per tile
+constexpr int RS_TILE = RS_THREADS * RS_ITEMS;    // items per CTA
+
+__global__ void __launch_bounds__(1024)
+sort_small_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restrict__ vals, int n,
+                  uint32_t *__restrict__ keys_out, uint32_t *__restrict__ vals_out) {
+    __shared__ unsigned long long w[SMALL_N];
+    for (int i = threadIdx.x; i < n; i += blockDim.x) w[i] = (static_cast<unsigned long long>(keys[i]) << 32) | (uint32_t)i;
+    __syncthreads();
+    for (int i = threadIdx.x; i < n; i += blockDim.x) {
+        const unsigned long long mine = w[i];
+        int rank = 0;
+        for (int j = 0; j < n; ++j) rank += (w[j] < mine) ? 1 : 0;
+        keys_out[rank] = static_cast<uint32_t>(mine >> 32);
+        vals_out[rank] = vals[i];
+    }
+}
+
+// pass 1: per-tile digit histogram, stored digit-major: hist[digit * n_tiles + tile]
+__global__ void __launch_bounds__(RS_THREADS)
+radix_hist_kernel(const uint32_t *__restrict__ keys, int64_t n, int shift, int n_tiles, uint32_t *__restrict__ hist) {
+    __shared__ uint32_t h[256];
+    h[threadIdx.x] = 0;
+    __syncthreads();
+    const int64_t base = static_cast<int64_t>(blockIdx.x) * RS_TILE;
+#pragma unroll
+    for (int r = 0; r < RS_ITEMS; ++r) {
+        const int64_t i = base + r * RS_THREADS + threadIdx.x;
+        if (i < n) atomicAdd(&h[(keys[i] >> shift) & 255u], 1u);
+    }
+    __syncthreads();
+    hist[static_cast<int64_t>(threadIdx.x) * n_tiles + blockIdx.x] = h[threadIdx.x];
+}
+
+// pass 2: exclusive scan of the histogram in place (one CTA; the array has 256 * n_tiles entries)
+__global__ void __launch_bounds__(1024) exclusive_scan_u32_kernel(uint32_t *__restrict__ a, int64_t n) {
+    __shared__ uint32_t warp_sum[32];
+    __shared__ uint32_t carry_s;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) carry_s = 0;
+    __syncthreads();
+    for (int64_t base = 0; base < n; base += 1024) {
+        const int64_t i = base + tid;
+        const uint32_t v = i < n ? a[i] : 0u;
+        uint32_t x = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o);
+            if (lane >= o) x += y;
+        }
+        if (lane == 31) warp_sum[warp] = x;
+        __syncthreads();
+        if (warp == 0) {
+            uint32_t s = warp_sum[lane];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, s, o);
+                if (lane >= o) s += y;
+            }
+            warp_sum[lane] = s;          // inclusive over warps
+        }
+        __syncthreads();
+        const uint32_t carry = carry_s;
+        const uint32_t before = carry + (warp ? warp_sum[warp - 1] : 0u) + (x - v);
+        if (i < n) a[i] = before;
+        __syncthreads();
+        if (tid == 0) carry_s = carry + warp_sum[31];
+        __syncthreads();
+    }
+}
+
+// pass 3: stable scatter.  Items of a tile are visited in 8 rounds of 256 in index order; inside a
+// round the rank of an item among equal digits is (equal digits in earlier warps) + (in earlier lanes).
+__global__ void __launch_bounds__(RS_THREADS)
+radix_scatter_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restrict__ vals, int64_t n, int shift,
+                     int n_tiles, const uint32_t *__restrict__ hist_scanned, uint32_t *__restrict__ keys_out,
+                     uint32_t *__restrict__ vals_out) {
+    __shared__ uint32_t base_s[256];
+    __shared__ uint32_t cnt_s[RS_THREADS / 32][256];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    base_s[tid] = hist_scanned[static_cast<int64_t>(tid) * n_tiles + blockIdx.x];
+    const int64_t base = static_cast<int64_t>(blockIdx.x) * RS_TILE;
+    for (int r = 0; r < RS_ITEMS; ++r) {
+#pragma unroll
+        for (int w = 0; w < RS_THREADS / 32; ++w) cnt_s[w][tid] = 0;
+        __syncthreads();
+        const int64_t i = base + r * RS_THREADS + tid;
+        const bool live = i < n;
+        uint32_t key = 0, digit = 256 + lane;     // dead lanes never match anything
+        if (live) { key = keys[i]; digit = (key >> shift) & 255u; }
+        const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
+        const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
+        if (live && rank_in_warp == 0) cnt_s[warp][digit] = __popc(peers);
+        __syncthreads();
+        if (live) {
+            uint32_t pos = base_s[digit] + rank_in_warp;
+            for (int w = 0; w < warp; ++w) pos += cnt_s[w][digit];
+            keys_out[pos] = key;
+            vals_out[pos] = vals[i];
+        }
+        __syncthreads();
+        uint32_t total = 0;
+#pragma unroll
+        for (int w = 0; w < RS_THREADS / 32; ++w) total += cnt_s[w][tid];
+        base_s[tid] += total;
+        __syncthreads();
+    }
+}
+
+siso_status_t launch_exclusive_scan_u32(Cache *c, uint32_t *a, int64_t n, cudaStream_t s) {
+    exclusive_scan_u32_kernel<<<1, 1024, 0, s>>>(a, n);
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
+
+size_t sort_pairs_scratch_bytes(int64_t n) {
+    const int64_t n_tiles = (n + RS_TILE - 1) / RS_TILE;
+    return pad256(sizeof(uint32_t) * 256 * static_cast<size_t>(n_tiles > 0 ? n_tiles : 1));
+}
+
+// Sorts n pairs by the low key_bits of the key, stably.  The result lands either in the input
+// arrays or in the *_tmp arrays; *keys_out / *vals_out say which.
+siso_status_t launch_sort_pairs(Cache *c, Scratch *scr, uint32_t *keys, uint32_t *vals, uint32_t *keys_tmp,
+                                uint32_t *vals_tmp, int64_t n, int key_bits, uint32_t **keys_out, uint32_t **vals_out,
+                                cudaStream_t s) {
+    if (n <= SMALL_N) {
+        sort_small_kernel<<<1, 1024, 0, s>>>(keys, vals, static_cast<int>(n), keys_tmp, vals_tmp);
+        SISO_LAUNCHED(c);
+        *keys_out = keys_tmp;
+        *vals_out = vals_tmp;
+        return SISO_OK;
+    }
+    const int n_tiles = static_cast<int>((n + RS_TILE - 1) / RS_TILE);
+    uint32_t *hist = scr->take<uint32_t>(256 * static_cast<size_t>(n_tiles));
+    uint32_t *ka = keys, *va = vals, *kb = keys_tmp, *vb = vals_tmp;
+    for (int shift = 0; shift < key_bits; shift += 8) {
+        radix_hist_kernel<<<n_tiles, RS_THREADS, 0, s>>>(ka, n, shift, n_tiles, hist);
+        SISO_LAUNCHED(c);
+        exclusive_scan_u32_kernel<<<1, 1024, 0, s>>>(hist, 256 * static_cast<int64_t>(n_tiles));
+        SISO_LAUNCHED(c);
+        radix_scatter_kernel<<<n_tiles, RS_THREADS, 0, s>>>(ka, va, n, shift, n_tiles, hist, kb, vb);
+        SISO_LAUNCHED(c);
+        uint32_t *t = ka; ka = kb; kb = t;
+        t = va; va = vb; vb = t;
+    }
+    *keys_out = ka;
+    *vals_out = va;
+    return SISO_OK;
+}
+
+}  // namespace siso

@@ -1,0 +1,121 @@
+// Hit update: running mean of every centroid that was hit in this batch, then renormalisation.
+//     c_j <- normalise(cluster_size_j * c_j + sum_{b in H_j} q_b)      (H_j in ascending query order)
+// The hits are grouped by slot with a stable sort, so each sum runs in one fixed order; sums and
+// the norm are accumulated in fp64, the result is rounded once to the fp32 master and, for bf16
+// caches, once more to the bf16 lookup copy.
+#include "common.cuh"
+
+namespace siso {
+
+constexpr int UP_THREADS = 256;
+
+// keys: slot of each hit row, `capacity` (sorts last) for rows that are not hits; vals: row number
+__global__ void update_keys_kernel(const int32_t *__restrict__ idx, int idx_stride, const uint8_t *__restrict__ hit,
+                                   const uint8_t *__restrict__ valid, int64_t B, int64_t capacity,
+                                   uint32_t *__restrict__ keys, uint32_t *__restrict__ vals, long long *counters,
+                                   int *status) {
+    const int64_t b = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (b == 0) counters[CNT_CLOCK] += 1;      // the cache clock advances once per update call
+    if (b >= B) return;
+    uint32_t key = static_cast<uint32_t>(capacity);
+    if (hit[b]) {
+        const int64_t j = idx[b * idx_stride];
+        if (j >= 0 && j < capacity && valid[j]) key = static_cast<uint32_t>(j);
+        else set_status(status, SISO_ERR_INVALID_ARG);   // a hit must name a live slot; the row is skipped
+    }
+    keys[b] = key;
+    vals[b] = static_cast<uint32_t>(b);
+}
+
+template <typename T> __device__ __forceinline__ double elem_f64(const T *p);
+template <> __device__ __forceinline__ double elem_f64<float>(const float *p) { return static_cast<double>(*p); }
+template <> __device__ __forceinline__ double elem_f64<__nv_bfloat16>(const __nv_bfloat16 *p) {
+    return static_cast<double>(__bfloat162float(*p));
+}
+
+__device__ __forceinline__ double block_sum_f64(double v, double *red) {
+    // fixed-shape tree: the same order of additions on every run
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) v += __shfl_xor_sync(0xFFFFFFFFu, v, o);
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    __syncthreads();
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    double t = 0.0;
+    for (int w = 0; w < UP_THREADS / 32; ++w) t += red[w];
+    return t;
+}
+
+// One CTA per position of the sorted hit list; the CTA at the head of a group does the group.
+template <typename T>
+__global__ void __launch_bounds__(UP_THREADS)
+update_apply_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restrict__ rows, int64_t B, int64_t capacity,
+                    int D, const T *__restrict__ Q, float *__restrict__ master, T *__restrict__ vecs,
+                    double *__restrict__ size, uint32_t *__restrict__ access, unsigned long long *__restrict__ last,
+                    const long long *__restrict__ counters) {
+    extern __shared__ double acc[];          // [D]
+    __shared__ double red[UP_THREADS / 32];
+    const int64_t p = blockIdx.x;
+    const uint32_t slot = keys[p];
+    if (slot >= capacity) return;
+    if (p > 0 && keys[p - 1] == slot) return;
+    const double n_old = size[slot];
+    float *m = master + static_cast<int64_t>(slot) * D;
+    for (int d = threadIdx.x; d < D; d += UP_THREADS) acc[d] = n_old * static_cast<double>(m[d]);
+    int64_t e = p;
+    for (; e < B && keys[e] == slot; ++e) {
+        const T *q = Q + static_cast<int64_t>(rows[e]) * D;
+        for (int d = threadIdx.x; d < D; d += UP_THREADS) acc[d] += elem_f64<T>(q + d);   // each thread owns its d
+    }
+    const long long count = e - p;
+    double ss = 0.0;
+    for (int d = threadIdx.x; d < D; d += UP_THREADS) ss += acc[d] * acc[d];
+    const double norm = sqrt(block_sum_f64(ss, red));
+    T *v = vecs + static_cast<int64_t>(slot) * D;
+    for (int d = threadIdx.x; d < D; d += UP_THREADS) {
+        const float f = static_cast<float>(acc[d] / norm);
+        m[d] = f;
+        if constexpr (sizeof(T) == 2) v[d] = __float2bfloat16_rn(f);
+    }
+    if (threadIdx.x == 0) {
+        size[slot] = n_old + static_cast<double>(count);
+        const unsigned long long a = static_cast<unsigned long long>(access[slot]) + static_cast<unsigned long long>(count);
+        access[slot] = (access[slot] == SISO_ACCESS_INF || a >= SISO_ACCESS_INF) ? SISO_ACCESS_INF : static_cast<uint32_t>(a);
+        last[slot] = static_cast<unsigned long long>(counters[CNT_CLOCK]);
+    }
+}
+
+siso_status_t launch_update(Cache *c, const void *q, int64_t B, const int32_t *idx, int idx_stride, const uint8_t *hit,
+                            cudaStream_t s) {
+    if (B >= (1ll << 31)) return SISO_ERR_UNSUPPORTED;
+    Scratch scr;
+    const size_t need = 4 * pad256(sizeof(uint32_t) * B) + sort_pairs_scratch_bytes(B);
+    SISO_TRY(scratch_reserve(c, need, s, &scr));
+    uint32_t *keys = scr.take<uint32_t>(B), *vals = scr.take<uint32_t>(B);
+    uint32_t *keys2 = scr.take<uint32_t>(B), *vals2 = scr.take<uint32_t>(B);
+    const int threads = 256;
+    // B == 0 still advances the clock
+    const unsigned blocks = static_cast<unsigned>((std::max<int64_t>(B, 1) + threads - 1) / threads);
+    update_keys_kernel<<<blocks, threads, 0, s>>>(idx, idx_stride, hit, c->valid, B, c->capacity, keys, vals,
+                                                  c->counters, c->status);
+    SISO_LAUNCHED(c);
+    if (B == 0) return SISO_OK;
+    int key_bits = 1;
+    while ((1ll << key_bits) <= c->capacity) ++key_bits;      // keys go up to `capacity` inclusive
+    uint32_t *ks, *vs;
+    SISO_TRY(launch_sort_pairs(c, &scr, keys, vals, keys2, vals2, B, key_bits, &ks, &vs, s));
+    const size_t smem = sizeof(double) * c->dim;
+    if (c->dtype == SISO_F32) {
+        update_apply_kernel<float><<<static_cast<unsigned>(B), UP_THREADS, smem, s>>>(
+            ks, vs, B, c->capacity, c->dim, static_cast<const float *>(q), c->master, static_cast<float *>(c->vecs),
+            c->size, c->access, c->last, c->counters);
+    } else {
+        update_apply_kernel<__nv_bfloat16><<<static_cast<unsigned>(B), UP_THREADS, smem, s>>>(
+            ks, vs, B, c->capacity, c->dim, static_cast<const __nv_bfloat16 *>(q), c->master,
+            static_cast<__nv_bfloat16 *>(c->vecs), c->size, c->access, c->last, c->counters);
+    }
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
+
+}  // namespace siso

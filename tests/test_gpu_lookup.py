@@ -1,0 +1,112 @@
+"""GPU parity of lookup (similarity sweep, top-k, threshold) against the CPU oracle, through the C ABI."""
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gen import workloads as W
+from util import TOL, check_lookup, to_dev
+
+pytestmark = pytest.mark.gpu
+
+siso = pytest.importorskip("paper_2508_18736_b200")
+PATHS = {"simt": siso.PATH_SIMT, "stream": siso.PATH_STREAM, "tensor": siso.PATH_TENSOR, "auto": siso.PATH_AUTO}
+
+
+def run_lookup(w, k, path, valid=None, theta=None):
+    cache = siso.SisoCache(w.centroids.shape[0], w.dim, w.dtype)
+    cache.set_lookup_path(PATHS[path])
+    cache.insert(to_dev(w.centroids, w.dtype))
+    if valid is not None:
+        st = cache.export()
+        cache.import_(st["master"], st["size"], st["access"], st["last"], torch.from_numpy(valid).cuda(), 0)
+    th = w.theta if theta is None else theta
+    th_arg = float(th[0]) if np.all(th == th[0]) else torch.from_numpy(th).cuda()
+    idx, sim, hit = cache.lookup(to_dev(w.queries, w.dtype), th_arg, k)
+    cache.check_status()
+    res = (idx.cpu().numpy(), sim.cpu().numpy(), hit.cpu().numpy())
+    cache.close()
+    return res
+
+
+CASES = [
+    # (config, overrides, mode, k, paths)
+    (1, dict(), "T", 1, ["simt", "auto"]),
+    (1, dict(n_centroids=1000, n_queries=333, dim=384), "P", 4, ["simt", "stream"]),
+    (1, dict(n_centroids=517, n_queries=130, dim=136, n_clusters=16), "L", 8, ["simt", "stream"]),
+    (1, dict(n_centroids=3, n_queries=5, dim=8, n_clusters=2), "L", 4, ["simt", "stream"]),
+    (2, dict(n_centroids=4096 + 77, n_queries=700, dim=768, n_clusters=256), "T", 1, ["simt", "tensor", "auto"]),
+    (2, dict(n_centroids=3000, n_queries=257, dim=768, n_clusters=128), "P", 1, ["simt", "tensor"]),
+    (4, dict(n_centroids=8192 + 5, n_queries=300, dim=1024, n_clusters=512), "T", 4, ["simt", "tensor"]),
+    (4, dict(n_centroids=2049, n_queries=129, dim=1024, n_clusters=64), "L", 4, ["simt", "tensor", "stream"]),
+    (4, dict(n_centroids=999, n_queries=7, dim=1024, n_clusters=64), "P", 8, ["stream", "auto"]),
+    (2, dict(n_centroids=640, n_queries=64, dim=72, n_clusters=32), "P", 2, ["simt", "tensor", "stream"]),
+]
+
+
+@pytest.mark.parametrize("cfg,over,mode,k,paths", CASES)
+def test_lookup_matches_oracle(cfg, over, mode, k, paths):
+    w = W.config(cfg, mode=mode, k=k, **over)
+    ora = oracle.lookup(w.centroids, w.queries, w.theta, k)
+    for path in paths:
+        gpu = run_lookup(w, k, path)
+        stats = check_lookup(gpu, ora, w.centroids, w.queries, w.theta, TOL[w.dtype])
+        if mode == "L":    # top-2 gaps are far above the tolerance here: the comparison must be exact
+            assert stats["idx_mismatch"] == 0, (path, stats)
+        # cluster-level check that never excuses: the best match comes from the oracle's cluster
+        lab = w.centroid_labels
+        assert (lab[gpu[0][:, 0]] == lab[ora[0][:, 0]]).all() or mode != "T"
+
+
+@pytest.mark.parametrize("dtype,path", [("f32", "simt"), ("f32", "stream"), ("bf16", "simt"), ("bf16", "tensor"),
+                                        ("bf16", "stream")])
+def test_lookup_skips_empty_slots_and_pads_short_results(dtype, path):
+    w = W.config(1, n_centroids=300, n_queries=40, dim=64, n_clusters=10, mode="P", dtype=dtype)
+    valid = (np.random.default_rng(1).random(300) < 0.02).astype(np.uint8)      # about 6 live entries, k = 8
+    valid[:2] = 1
+    k = 8
+    ora = oracle.lookup(w.centroids, w.queries, w.theta, k, valid)
+    gpu = run_lookup(w, k, path, valid=valid)
+    check_lookup(gpu, ora, w.centroids, w.queries, w.theta, TOL[dtype], valid=valid)
+    assert (gpu[0][:, -1] == -1).all()
+    # an empty cache misses everything
+    gpu = run_lookup(w, 2, path, valid=np.zeros(300, dtype=np.uint8))
+    assert (gpu[0] == -1).all() and np.isneginf(gpu[1]).all() and (gpu[2] == 0).all()
+
+
+@pytest.mark.parametrize("dtype,path", [("f32", "simt"), ("bf16", "tensor"), ("bf16", "stream")])
+def test_exact_ties_go_to_the_lower_slot_and_threshold_is_strict(dtype, path):
+    rng = np.random.default_rng(3)
+    C = rng.integers(-1, 2, (200, 64)).astype(np.float32) * 0.125          # exact in bf16, exact dot products
+    C[150] = C[7]
+    C[90] = C[7]
+    Q = C[[7, 33, 7]].copy()
+    if dtype == "bf16":
+        Cx, Qx = W.f32_to_bf16_bits(C), W.f32_to_bf16_bits(Q)
+    else:
+        Cx, Qx = C, Q
+    w = W.Workload("ties", dtype, 64, Cx, Qx, None, 4, np.zeros(200, np.int32), None, {})
+    self_sim = (Q.astype(np.float64) ** 2).sum(1).astype(np.float32)
+    for theta in (self_sim, np.nextafter(self_sim, np.float32(-1))):
+        w.theta = theta
+        ora = oracle.lookup(Cx, Qx, theta, 4)
+        gpu = run_lookup(w, 4, path)
+        assert (gpu[0] == ora[0]).all() and (gpu[1] == ora[1].astype(np.float32)).all() and (gpu[2] == ora[2]).all()
+    assert gpu[0][0, :3].tolist() == [7, 90, 150] and gpu[2].tolist() == [1, 1, 1]
+
+
+def test_bad_arguments_return_status_and_touch_nothing():
+    cache = siso.SisoCache(64, 64, "bf16")
+    q = torch.zeros(4, 64, dtype=torch.bfloat16, device="cuda")
+    with pytest.raises(siso.SisoError):
+        cache.lookup(q, 0.5, k=0)
+    with pytest.raises(siso.SisoError):
+        cache.lookup(q, 0.5, k=9)
+    with pytest.raises(ValueError):
+        cache.lookup(torch.zeros(4, 32, dtype=torch.bfloat16, device="cuda"), 0.5)
+    with pytest.raises(siso.SisoError):
+        siso.SisoCache(64, 60, "bf16")            # dim must be a multiple of 8
+    cache.insert(torch.zeros(65, 64, dtype=torch.bfloat16, device="cuda"))      # more rows than slots
+    assert cache.sync_status() == 4 and cache.sync_status() == 0               # SISO_ERR_CAPACITY, then cleared
+    assert cache.stats()["occupancy"] == 0
+    cache.close()
