@@ -1,0 +1,304 @@
+#!/usr/bin/env python
+"""Throughput of batched exact lookup at 1,048,576 x 1024 bf16 centroids (queries per second).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--rows N --queries B]
+
+A step is one lookup of a batch of 8,192 synthetic queries (top-4 + per-query hit threshold)
+against the device-resident centroid matrix through the C ABI.  `value` times the call with the
+batch already in HBM; `e2e` times the host-buffer entry point (pinned host memory in, results
+back out).  With N > 1 (torchrun) every rank holds a replica of the cache and looks up its own
+batch: weak scaling, no collective on the data path.  `--impl reference` times the CPU oracle
+on a bounded sample of the same workload instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np  # noqa: E402
+
+METRIC = "lookup queries/sec at 1Mx1024 bf16 centroids"
+UNIT = "queries/s"
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+
+
+def parse_args():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--rows", type=int, default=1 << 20, help="cached centroids (default: the full 1,048,576)")
+    ap.add_argument("--queries", type=int, default=8192, help="query batch per step")
+    ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor", "stream"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-e2e", action="store_true")
+    return ap.parse_args()
+
+
+def load_peaks():
+    p = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(p):
+        with open(p) as f:
+            d = json.load(f)
+        return {k: float(d[k]) for k in FALLBACK_PEAKS if k in d}, "measured"
+    return dict(FALLBACK_PEAKS), "fallback"
+
+
+def workload(args, rank: int, threads: int):
+    from gen import workloads as W
+    n_clusters = max(64, args.rows // 16)
+    return W.config(4, seed=0, query_seed=rank, mode="T", threads=threads, n_centroids=args.rows,
+                    n_queries=args.queries, n_clusters=n_clusters)
+
+
+def workload_name(args) -> str:
+    return (f"config 4: {args.rows} x 1024 bf16 centroids ({max(64, args.rows // 16)} clusters, sigma 0.07 as whole-"
+            f"perturbation length), batch {args.queries} (Zipf 1.0, 20% out-of-distribution), top-4, theta in [0.78, 0.93]")
+
+
+# ------------------------------------------------------------------------------ CPU oracle legs
+def time_oracle(w, n_sample: int, repeats: int = 1):
+    """Seconds per call of the oracle on the first n_sample queries of the batch (all host cores)."""
+    import oracle
+    q, th = w.queries[:n_sample], w.theta[:n_sample]
+    times = []
+    for _ in range(repeats):
+        t0 = time.perf_counter()
+        oracle.lookup(w.centroids, q, th, w.k)
+        times.append(time.perf_counter() - t0)
+    return times
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    cores = os.cpu_count() or 1
+    w = workload(args, 0, cores)
+    import oracle
+    oracle.build()
+    n_sample = max(1, min(args.queries, cores))
+    for _ in range(args.warmup):
+        time_oracle(w, n_sample)
+    t = time_oracle(w, n_sample, args.steps)
+    total = sum(t)
+    value = n_sample * args.steps / total
+    sample = f"{n_sample} of {args.queries} queries per step against all {args.rows} centroids"
+    line = {"impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+            "warmup": args.warmup, "ms_per_step": 1e3 * total / args.steps, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+            "config": {"workload": workload_name(args), "sample": sample},
+            "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample},
+            "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+            "gpu_launches": 0}
+    print(json.dumps(line), flush=True)
+    return 0
+
+
+# ------------------------------------------------------------------------------ clocks
+class ClockSampler:
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, index: int):
+        self.proc = None
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            pass
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            out, _ = self.proc.communicate(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+            out, _ = self.proc.communicate()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in out.splitlines():
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 7:
+                continue
+            try:
+                sm.append(float(f[0]))
+                mx.append(float(f[1]))
+            except ValueError:
+                continue
+            for name, v in zip(names, f[3:7]):
+                if v.lower().startswith("active"):
+                    reasons.add(name)
+        hi = sorted(sm)[len(sm) // 2:] if sm else []     # the upper half of the samples: those under load
+        return {"sm_mhz": statistics.median(hi) if hi else None, "sm_max_mhz": max(mx) if mx else None,
+                "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------ GPU arm
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+    from paper_2508_18736_b200 import build as _b
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} needs WORLD_SIZE={args.gpus} (launch with torch.distributed.run); got {world}")
+    if not torch.cuda.is_available():
+        raise SystemExit("no CUDA device: this benchmark has no CPU path (use --impl reference for the oracle)")
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    if local_rank == 0:
+        _b.build()
+    if world > 1:
+        dist.barrier()
+    import paper_2508_18736_b200 as siso
+
+    cores = os.cpu_count() or 1
+    w = workload(args, rank, max(1, cores // world))
+    B, k = args.queries, w.k
+    dev = torch.device("cuda", local_rank)
+
+    def to_dev(a):
+        return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    cache = siso.SisoCache(args.rows, 1024, "bf16", device=local_rank)
+    step_rows = 1 << 16
+    for lo in range(0, args.rows, step_rows):          # promote the centroids in slices: bounded staging
+        cache.insert(to_dev(w.centroids[lo:lo + step_rows]))
+    cache.check_status()
+    cache.set_lookup_path({"auto": siso.PATH_AUTO, "simt": siso.PATH_SIMT, "tensor": siso.PATH_TENSOR,
+                           "stream": siso.PATH_STREAM}[args.path])
+    q_dev = to_dev(w.queries)
+    th_dev = torch.from_numpy(w.theta).to(dev)
+    out = (torch.empty((B, k), dtype=torch.int32, device=dev), torch.empty((B, k), dtype=torch.float32, device=dev),
+           torch.empty(B, dtype=torch.uint8, device=dev))
+    stream = torch.cuda.current_stream()
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def step_device():
+        cache.lookup(q_dev, th_dev, k, out=out)
+
+    # pinned host buffers of the end-to-end leg
+    h_q = torch.from_numpy(w.queries.view(np.int16)).pin_memory()
+    h_th = torch.from_numpy(w.theta).pin_memory()
+    h_idx = torch.empty((B, k), dtype=torch.int32).pin_memory()
+    h_sim = torch.empty((B, k), dtype=torch.float32).pin_memory()
+    h_hit = torch.empty(B, dtype=torch.uint8).pin_memory()
+
+    def step_host():
+        cache.lookup_host(h_q, h_th, 0.0, k, h_idx, h_sim, h_hit)
+
+    def timed(step, steps):
+        """Returns (ms per step, per-step ms list, launches) with CUDA events on the launching stream."""
+        ev = [torch.cuda.Event(enable_timing=True) for _ in range(steps + 1)]
+        barrier()
+        l0 = cache.launch_count
+        ev[0].record(stream)
+        for i in range(steps):
+            step()
+            ev[i + 1].record(stream)
+        barrier()
+        per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
+        total = ev[0].elapsed_time(ev[steps])
+        if world > 1:
+            t = torch.tensor([total], dtype=torch.float64, device=dev)
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            total = float(t.item())
+        return total / steps, per, cache.launch_count - l0
+
+    for _ in range(max(3, args.warmup)):
+        step_device()
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ms, per_step, launches = timed(step_device, args.steps)
+    clocks = sampler.stop() if sampler else None
+    cache.check_status()
+
+    e2e = None
+    if not args.no_e2e:
+        for _ in range(3):
+            step_host()
+        ms_e2e, _, _ = timed(step_host, args.steps)
+        cache.check_status()
+        e2e = {"value": world * B / (ms_e2e * 1e-3), "unit": UNIT,
+               "h2d_bytes_per_step": int(w.queries.nbytes + w.theta.nbytes),
+               "d2h_bytes_per_step": int(h_idx.numel() * 4 + h_sim.numel() * 4 + h_hit.numel()),
+               "ms_per_step": ms_e2e}
+        # the host-buffer call must return what the device call returns
+        assert torch.equal(h_idx, out[0].cpu()) and torch.equal(h_hit, out[2].cpu())
+
+    if rank != 0:
+        if world > 1:
+            dist.destroy_process_group()
+        return 0
+
+    peaks, peak_kind = load_peaks()
+    flops = 2.0 * B * args.rows * 1024
+    kernel_ms = statistics.median(per_step)           # the sweep kernel plus its small finalize kernel
+    achieved = flops / (kernel_ms * 1e-3) / 1e12
+    roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                "frac": achieved / peaks["bf16_tflops"], "traffic": None, "peak_kind": f"{peak_kind}, burst",
+                "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
+                "hbm_floor_ms": (args.rows * 1024 * 2 + B * 1024 * 2) / (peaks["hbm_gbs"] * 1e9) * 1e3,
+                "kernel": {"auto": "tensor-core sweep (auto)", "tensor": "tensor-core sweep", "simt": "CUDA-core sweep",
+                           "stream": "streaming sweep"}[args.path],
+                "flops_per_launch": flops, "median_launch_ms": kernel_ms}
+    line = {"metric": METRIC, "value": world * B / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": workload_name(args), "parallelism": f"replica x{world}, queries sharded",
+                       "l2": "inputs larger than L2: the 2 GiB centroid matrix is swept on every step",
+                       "lookup_path": args.path},
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline}
+
+    if not args.no_cpu_baseline and world == 1:
+        import oracle
+        oracle.build()
+        n_sample = max(1, min(B, 4 * cores))
+        t0 = time.perf_counter()
+        o_idx, o_sim, o_hit = oracle.lookup(w.centroids, w.queries[:n_sample], w.theta[:n_sample], k)
+        t = time.perf_counter() - t0
+        sample = f"first {n_sample} of {B} queries against all {args.rows} centroids, top-{k}"
+        line["cpu_baseline"] = {"value": n_sample / t, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
+                                "seconds": t}
+        # the sampled rows double as a full-size parity check of the timed configuration
+        g_sim = out[1][:n_sample].cpu().numpy().astype(np.float64)
+        line["parity_sample"] = {"rows": n_sample, "max_sim_err": float(np.abs(g_sim - o_sim).max()),
+                                 "top1_equal": int((out[0][:n_sample, 0].cpu().numpy() == o_idx[:, 0]).sum()),
+                                 "hit_equal": int((out[2][:n_sample].cpu().numpy() == o_hit).sum())}
+    print(json.dumps(line), flush=True)
+    cache.close()
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    args = parse_args()
+    if args.impl == "reference":
+        return run_reference(args)
+    return run_ours(args)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

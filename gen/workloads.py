@@ -164,8 +164,12 @@ def clustered_lookup_workload(name: str, *, n_centroids: int, n_queries: int, di
                               sigma: float, dtype: str, seed: int = 0, mode: str = "T",
                               zipf_s: Optional[float] = None, ood_fraction: float = 0.0,
                               theta: Tuple[float, float] = (0.85, 0.85), k: int = 1,
-                              threads: int = 1) -> Workload:
-    """Centroids and queries drawn around shared cluster means (configs 1, 2, 3, 4)."""
+                              threads: int = 1, query_seed: Optional[int] = None) -> Workload:
+    """Centroids and queries drawn around shared cluster means (configs 1, 2, 3, 4).
+
+    ``query_seed`` (default: ``seed``) keys the draws of the query batch only, so that several
+    batches can be drawn against one centroid set."""
+    qseed = seed if query_seed is None else query_seed
     means = unit_gaussian_rows(n_clusters, dim, seed, _TAG_MEANS, threads)
     spread = spread_for_mode(mode, sigma, n_clusters, dim, seed)
     c_lab = _rng(seed, _TAG_LABEL, 0).integers(0, n_clusters, n_centroids).astype(np.int32)
@@ -173,21 +177,21 @@ def clustered_lookup_workload(name: str, *, n_centroids: int, n_queries: int, di
     q = q_lab = th = None
     if n_queries > 0:
         if zipf_s is None:
-            q_lab = _rng(seed, _TAG_LABEL, 1).integers(0, n_clusters, n_queries).astype(np.int32)
+            q_lab = _rng(qseed, _TAG_LABEL, 1).integers(0, n_clusters, n_queries).astype(np.int32)
         else:
             p = zipf_probs(n_clusters, zipf_s, seed)
-            q_lab = _rng(seed, _TAG_LABEL, 1).choice(n_clusters, size=n_queries, p=p).astype(np.int32)
-        q = cluster_members(means, q_lab, spread, seed, _TAG_QUERY, threads)
+            q_lab = _rng(qseed, _TAG_LABEL, 1).choice(n_clusters, size=n_queries, p=p).astype(np.int32)
+        q = cluster_members(means, q_lab, spread, qseed, _TAG_QUERY, threads)
         if ood_fraction > 0.0:
-            is_ood = _rng(seed, _TAG_OOD, 0).random(n_queries) < ood_fraction
+            is_ood = _rng(qseed, _TAG_OOD, 0).random(n_queries) < ood_fraction
             n_ood = int(is_ood.sum())
-            q[is_ood] = unit_gaussian_rows(n_ood, dim, seed, _TAG_OOD + 100, threads)
+            q[is_ood] = unit_gaussian_rows(n_ood, dim, qseed, _TAG_OOD + 100, threads)
             q_lab = q_lab.copy()
             q_lab[is_ood] = -1
         if theta[0] == theta[1]:
             th = np.full(n_queries, theta[0], dtype=np.float32)
         else:
-            th = thresholds(n_queries, theta[0], theta[1], seed)
+            th = thresholds(n_queries, theta[0], theta[1], qseed)
         q = _store(q, dtype)
     params = dict(n_centroids=n_centroids, n_queries=n_queries, dim=dim, n_clusters=n_clusters, sigma=sigma,
                   mode=mode, seed=seed, zipf_s=zipf_s, ood_fraction=ood_fraction, theta=theta, k=k)
