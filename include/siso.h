@@ -164,6 +164,33 @@ siso_status_t siso_stream_step(siso_cache_t *c, const void *d_queries, int64_t n
                                float theta_scalar, int32_t *d_idx, float *d_sim, uint8_t *d_hit,
                                int32_t *d_victims, int32_t *d_slots_out, void *stream);
 
+/* Small-batch lookup for callers that cannot allocate device memory.  The paper has no counterpart: this
+ * entry point exists for integration reasons only.  Some callers of this library run where cudaMalloc
+ * and cudaFree are off limits - a serving loop whose device memory was handed out at start-up, a callback
+ * that may run while another thread holds an allocator lock, a process with a fixed memory budget -
+ * because those calls synchronise the device and can fail at any moment.  This call allocates nothing,
+ * neither through CUDA nor through the cache's allocator, and needs no cache handle: the caller passes
+ * the centroid matrix and every output.
+ *   d_centroids [n_centroids, dim] row-major in `dtype` (siso_dtype_t), unit-norm; 1 <= dim <= 1024
+ *   d_valid     [n_centroids] 1 = live entry, 0 = skip; NULL = all live
+ *   d_queries   [n_queries, dim] in `dtype`; 1 <= n_queries <= SISO_NOALLOC_MAX_QUERIES
+ *   d_theta / theta_scalar, k (1..8), d_idx, d_sim, d_hit: as in siso_lookup
+ * Its scratch (per-CTA partial top-k lists, 512 KiB) is a fixed array inside the library image that
+ * every GPU loading the library holds until the process exits.  That fixes the limits above; sizes
+ * beyond them return SISO_ERR_UNSUPPORTED and launch nothing.  All calls share that array and it keeps
+ * the previous call's contents; each call overwrites every entry it later reads, so calls issued in
+ * order on one stream are independent, but two calls that may run on the GPU at the same time
+ * (different streams, different threads) race on it and must be ordered by the caller.
+ * The first call on each device looks up the array's device address (with that device current, which
+ * is the caller's current device); make that first call before starting any stream capture.
+ * Asynchronous on `stream`; runs on the calling thread's current device. */
+#define SISO_NOALLOC_MAX_QUERIES 8
+#define SISO_NOALLOC_MAX_DIM 1024
+siso_status_t siso_lookup_small_noalloc(const void *d_centroids, const uint8_t *d_valid, int64_t n_centroids,
+                                        int32_t dim, int32_t dtype, const void *d_queries, int64_t n_queries,
+                                        const float *d_theta, float theta_scalar, int32_t k, int32_t *d_idx,
+                                        float *d_sim, uint8_t *d_hit, void *stream);
+
 /* Copy the state out (checkpoint, parity checks).  Any pointer may be NULL.
  *   d_vecs   [capacity, dim] lookup copy in the cache dtype     d_master [capacity, dim] fp32 master
  *   d_sizes  [capacity] fp64   d_access [capacity] u32   d_last [capacity] u64   d_valid [capacity] u8 */

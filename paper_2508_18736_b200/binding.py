@@ -21,7 +21,7 @@ _STATUS_NAMES = {0: "SISO_OK", 1: "SISO_ERR_INVALID_ARG", 2: "SISO_ERR_UNSUPPORT
 EXPORTS = ["siso_cache_create", "siso_cache_destroy", "siso_set_option", "siso_insert", "siso_lookup",
            "siso_lookup_host", "siso_update", "siso_merge", "siso_evict", "siso_make_room", "siso_insert_misses",
            "siso_stream_step", "siso_export", "siso_import", "siso_get_stats", "siso_sync_status",
-           "siso_launch_count", "siso_status_string", "siso_last_cuda_error"]
+           "siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_lookup_small_noalloc"]
 
 
 class SisoError(RuntimeError):
@@ -71,6 +71,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_make_room.argtypes = [vp, vp, i64, u32, vp, vp]
     L.siso_insert_misses.argtypes = [vp, vp, i64, vp, vp, vp]
     L.siso_stream_step.argtypes = [vp, vp, i64, vp, f32, vp, vp, vp, vp, vp, vp]
+    L.siso_lookup_small_noalloc.argtypes = [vp, vp, i64, i32, i32, vp, i64, vp, f32, i32, vp, vp, vp, vp]
     L.siso_export.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     L.siso_import.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_uint64, vp]
     L.siso_get_stats.argtypes = [vp, ctypes.POINTER(i64), vp]
@@ -288,3 +289,21 @@ class SisoCache:
     @property
     def launch_count(self) -> int:
         return int(self._lib.siso_launch_count(self._h))
+
+
+def lookup_small_noalloc(centroids: torch.Tensor, queries: torch.Tensor, theta, k: int, idx: torch.Tensor,
+                         sim: torch.Tensor, hit: torch.Tensor, valid: Optional[torch.Tensor] = None, stream=None) -> None:
+    """Lookup of at most 8 queries that allocates no device memory: the caller owns every buffer, outputs
+    included, and the library's scratch is a fixed array inside its image.  For callers that must not
+    call the CUDA allocator (see include/siso.h).  Calls that can overlap on the GPU must be ordered by
+    the caller.  Raises SisoError for sizes beyond the fixed limits."""
+    L = load_library()
+    dtype = {torch.float32: 0, torch.bfloat16: 1}[centroids.dtype]
+    assert queries.dtype == centroids.dtype and centroids.is_contiguous() and queries.is_contiguous()
+    th_t, th_s = (theta, 0.0) if isinstance(theta, torch.Tensor) else (None, float(theta))
+    with torch.cuda.device(centroids.device):
+        st = L.siso_lookup_small_noalloc(_ptr(centroids), _ptr(valid), centroids.shape[0], centroids.shape[1], dtype,
+                                         _ptr(queries), queries.shape[0], _ptr(th_t), th_s, k, _ptr(idx), _ptr(sim),
+                                         _ptr(hit), _stream(stream))
+    if st != 0:
+        raise SisoError(st, "siso_lookup_small_noalloc", L.siso_last_cuda_error().decode() if st == 7 else "")
