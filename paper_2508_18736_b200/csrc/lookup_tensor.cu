@@ -1,9 +1,354 @@
-// placeholder until the tcgen05 kernel lands
+// Large-batch lookup as a dense contraction on the 5th-generation tensor cores:
+//     S = Q * C^T  (bf16 x bf16 -> fp32), per-row top-k and threshold fused, S never leaves the SM.
+//
+// One CTA owns 128 queries (the 128 TMEM lanes) and a contiguous range of 256-centroid tiles.
+//   warp 0      TMA producer: per 64-element K slab one 128x64 tile of Q and one 256x64 tile of C
+//               (cp.async.bulk.tensor, 128-byte swizzle) into a ring of shared-memory stages
+//   warp 1      MMA issuer: tcgen05.mma (M=128, N=256, K=16) four times per slab into one of two
+//               256-column TMEM accumulators; tcgen05.commit releases the stage / publishes the tile
+//   warps 2-5   epilogue: tcgen05.ld the finished accumulator (thread = query row), drop empty slots,
+//               keep the row's running top-k in registers, release the accumulator
+// so the tensor pipe works on tile t+1 while the CUDA cores scan tile t.  Products of bf16 values are
+// exact in fp32 and the accumulation is fp32, which is what the 2e-3 tolerance is derived from.
+// Every wait is bounded: when one runs out the CTA raises SISO_ERR_TIMEOUT in the status word, all
+// roles leave their loops, in-flight copies get time to land, TMEM is freed and the kernel returns.
+#include <cuda.h>
+
+#include <cstring>
+
 #include "common.cuh"
+
 namespace siso {
-void tensor_state_destroy(Cache *) {}
+namespace tc {
+
+constexpr int TM = 128;             // queries per CTA (TMEM lanes)
+constexpr int TN = 256;             // centroids per MMA tile (TMEM columns per accumulator)
+constexpr int TK = 64;              // K elements per stage: 128 bytes = one swizzle span
+constexpr int STAGES = 4;
+constexpr int ACC_STAGES = 2;
+constexpr int THREADS = 192;
+constexpr uint32_t A_BYTES = TM * TK * 2;     // 16 KiB
+constexpr uint32_t B_BYTES = TN * TK * 2;     // 32 KiB
+constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+constexpr uint32_t TMEM_COLS = ACC_STAGES * TN;   // 512: the whole tensor memory of the SM
+constexpr uint32_t SPIN_LIMIT = 4u << 20;
+
+// ---- PTX wrappers -------------------------------------------------------------------------------
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+// Bounded wait.  Returns false if the limit ran out or another role has already given up.
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+    for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            __nanosleep(64);
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar))
+                 : "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp receives row (lane base + i)
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"     // same statement: no use of the registers can be scheduled before the wait
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+
+// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes and 128-byte swizzled
+// (what the TMA writes): 8-row groups 1024 bytes apart; descriptor version 1; layout type 2 = 128B swizzle.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);          // start address, 16-byte units
+    d |= static_cast<uint64_t>(1) << 16;                         // leading byte offset (unused for swizzled K-major)
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;                 // stride byte offset: 8 rows x 128 B
+    d |= static_cast<uint64_t>(1) << 46;                         // descriptor version
+    d |= static_cast<uint64_t>(2) << 61;                         // SWIZZLE_128B
+    return d;
+}
+// Instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 128.
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(TN >> 3) << 17) |
+                           (static_cast<uint32_t>(TM >> 4) << 24);
+
+struct Barriers {
+    uint64_t full[STAGES], empty[STAGES], acc_full[ACC_STAGES], acc_empty[ACC_STAGES];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+template <int KMAX>
+__global__ void __launch_bounds__(THREADS, 1)
+lookup_tensor_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_c,
+                     const uint8_t *__restrict__ valid, int64_t B, int D, int tiles_per_split, int n_tiles,
+                     unsigned long long *__restrict__ partial, int splits, int *status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    Barriers *bars = reinterpret_cast<Barriers *>(tiles + STAGES * STAGE_BYTES);
+    volatile int *abort_flag = &bars->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int split = blockIdx.x;
+    const int q0 = blockIdx.y * TM;
+    const int t_begin = split * tiles_per_split;
+    const int t_end = min(n_tiles, t_begin + tiles_per_split);
+    const int k_slabs = (D + TK - 1) / TK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+        for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 4); }
+        bars->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {   // one warp allocates all 512 TMEM columns and writes the base address to smem
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&bars->tmem_base)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = bars->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int t = t_begin; t < t_end && ok; ++t) {
+                const int n0 = t * TN;
+                for (int ks = 0; ks < k_slabs; ++ks) {
+                    if (!mbar_wait(&bars->empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+                    uint8_t *a_dst = tiles + stage * STAGE_BYTES;
+                    uint8_t *b_dst = a_dst + A_BYTES;
+                    mbar_arrive_expect_tx(&bars->full[stage], STAGE_BYTES);
+                    tma_load_2d(a_dst, &map_q, ks * TK, q0, &bars->full[stage]);
+                    tma_load_2d(b_dst, &map_c, ks * TK, n0, &bars->full[stage]);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            bool ok = true;
+            for (int t = t_begin; t < t_end && ok; ++t) {
+                if (!mbar_wait(&bars->acc_empty[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * TN;
+                for (int ks = 0; ks < k_slabs; ++ks) {
+                    if (!mbar_wait(&bars->full[stage], phase, abort_flag)) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const uint32_t a_addr = smem_u32(tiles + stage * STAGE_BYTES);
+                    const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(a_addr + A_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < TK / 16; ++kk) {
+                        // 16 bf16 = 32 bytes further along K inside the swizzle span: +2 in 16-byte units
+                        umma_bf16(d_tmem, da + static_cast<uint64_t>(2 * kk), db + static_cast<uint64_t>(2 * kk), IDESC,
+                                  (ks | kk) ? 1u : 0u);
+                    }
+                    umma_commit(&bars->empty[stage]);          // stage reusable once these MMAs have read it
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit(&bars->acc_full[acc]);             // accumulator complete
+                if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5)
+        const int quarter = warp & 3;                         // TMEM lanes [32*quarter, +32) belong to this warp
+        const int row = quarter * 32 + lane;
+        TopK<KMAX> top;
+        top.clear();
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (int t = t_begin; t < t_end && ok; ++t) {
+            const int n0 = t * TN;
+            if (!mbar_wait(&bars->acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+            tcgen05_fence_after();
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * TN;
+#pragma unroll 1
+            for (int ch = 0; ch < TN / 32; ++ch) {
+                uint32_t r[32];
+                tmem_ld_32x32(taddr + ch * 32, r);
+                // live mask of these 32 slots: lane l reads the flag of slot l, the ballot shares them
+                const uint32_t live = __ballot_sync(0xFFFFFFFFu, valid[static_cast<int64_t>(n0) + ch * 32 + lane] != 0);
+                if (live == 0u) continue;
+                float m = -INFINITY;
+                if (live == 0xFFFFFFFFu) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) m = fmaxf(m, __uint_as_float(r[j]));
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if (!((live >> j) & 1u)) r[j] = 0xFF800000u;      // -inf: never enters a list
+                        m = fmaxf(m, __uint_as_float(r[j]));
+                    }
+                }
+                if (m > top.s[KMAX - 1]) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) top.push(__uint_as_float(r[j]), n0 + ch * 32 + j);
+                }
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(&bars->acc_empty[acc]);
+            if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (ok && static_cast<int64_t>(q0) + row < B) {
+            unsigned long long *dst = partial + ((static_cast<int64_t>(q0) + row) * splits + split) * KMAX;
+#pragma unroll
+            for (int j = 0; j < KMAX; ++j) dst[j] = top.key(j);
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (*abort_flag) {
+        // give copies still in flight time to land before the shared memory is handed back
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        if (threadIdx.x == 0) set_status(status, SISO_ERR_TIMEOUT);
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// ---- host side ------------------------------------------------------------------------------------
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+struct TensorState {
+    EncodeTiledFn encode;
+    CUtensorMap map_c;
+    bool attr_set[3];
+};
+
+static siso_status_t encode_map(EncodeTiledFn fn, CUtensorMap *map, const void *base, uint64_t rows, uint64_t dim,
+                                uint32_t box_rows) {
+    cuuint64_t gdim[2] = {dim, rows};
+    cuuint64_t gstride[1] = {dim * 2};
+    cuuint32_t box[2] = {static_cast<cuuint32_t>(TK), box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return check_cuda(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return SISO_OK;
+}
+
+}  // namespace tc
+
+void tensor_state_destroy(Cache *c) {
+    delete static_cast<tc::TensorState *>(c->tensor_state);
+    c->tensor_state = nullptr;
+}
+
+template <int KMAX>
+static siso_status_t run_tensor(Cache *c, tc::TensorState *ts, int slot, const CUtensorMap &map_q, int64_t B,
+                                int tiles_per_split, int n_tiles, int splits, int m_tiles, unsigned long long *partial,
+                                cudaStream_t s) {
+    auto kern = tc::lookup_tensor_kernel<KMAX>;
+    if (!ts->attr_set[slot]) {
+        SISO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES));
+        ts->attr_set[slot] = true;
+    }
+    dim3 grid(splits, m_tiles);
+    kern<<<grid, tc::THREADS, tc::SMEM_BYTES, s>>>(map_q, ts->map_c, c->valid, B, c->dim, tiles_per_split, n_tiles,
+                                                   partial, splits, c->status);
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
+
 siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const float *theta, float theta_s, int k,
                                    int32_t *idx, float *sim, uint8_t *hit, cudaStream_t s) {
-    return launch_lookup_simt(c, q, B, theta, theta_s, k, idx, sim, hit, s);
+    if (c->dtype != SISO_BF16) return SISO_ERR_UNSUPPORTED;
+    auto *ts = static_cast<tc::TensorState *>(c->tensor_state);
+    if (!ts) {
+        ts = new tc::TensorState();
+        memset(ts, 0, sizeof(*ts));
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        SISO_CUDA(cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres));
+        if (!fn || qres != cudaDriverEntryPointSuccess) { delete ts; return check_cuda(cudaErrorNotSupported, "cuTensorMapEncodeTiled lookup"); }
+        ts->encode = reinterpret_cast<tc::EncodeTiledFn>(fn);
+        siso_status_t st = tc::encode_map(ts->encode, &ts->map_c, c->vecs, static_cast<uint64_t>(c->rows_alloc),
+                                          static_cast<uint64_t>(c->dim), tc::TN);
+        if (st != SISO_OK) { delete ts; return st; }
+        c->tensor_state = ts;
+    }
+    CUtensorMap map_q;
+    SISO_TRY(tc::encode_map(ts->encode, &map_q, q, static_cast<uint64_t>(B), static_cast<uint64_t>(c->dim), tc::TM));
+
+    const int kmax = k == 1 ? 1 : (k <= 4 ? 4 : 8);
+    const int n_tiles = static_cast<int>((c->capacity + tc::TN - 1) / tc::TN);
+    const int64_t m_tiles64 = (B + tc::TM - 1) / tc::TM;
+    if (m_tiles64 > 65535) return SISO_ERR_UNSUPPORTED;
+    const int m_tiles = static_cast<int>(m_tiles64);
+    // one CTA per SM at a time: aim at a whole number of waves with at least ~8 tiles per CTA
+    const int64_t units = static_cast<int64_t>(m_tiles) * n_tiles;
+    const int waves = static_cast<int>(std::min<int64_t>(16, std::max<int64_t>(1, units / (8ll * c->sm_count))));
+    int splits = std::max(1, std::min(n_tiles, (c->sm_count * waves) / m_tiles));
+    const int tiles_per_split = (n_tiles + splits - 1) / splits;
+    splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
+
+    Scratch scr;
+    SISO_TRY(scratch_reserve(c, pad256(sizeof(unsigned long long) * B * splits * kmax), s, &scr));
+    unsigned long long *partial = scr.take<unsigned long long>(static_cast<size_t>(B) * splits * kmax);
+    siso_status_t st = kmax == 1 ? run_tensor<1>(c, ts, 0, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s)
+                     : kmax == 4 ? run_tensor<4>(c, ts, 1, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s)
+                                 : run_tensor<8>(c, ts, 2, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s);
+    SISO_TRY(st);
+    return launch_topk_finalize(c, partial, B, splits, kmax, k, theta, theta_s, idx, sim, hit, s);
 }
+
 }  // namespace siso
