@@ -130,8 +130,10 @@ lookup_tensor_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
     volatile int *abort_flag = &bars->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int split = blockIdx.x;
-    const int q0 = blockIdx.y * TM;
+    // blockIdx.x walks the query tiles, so CTAs that run at the same time sweep the SAME centroid range
+    // and every centroid tile leaves HBM once and is then served from L2
+    const int split = blockIdx.y;
+    const int q0 = blockIdx.x * TM;
     const int t_begin = split * tiles_per_split;
     const int t_end = min(n_tiles, t_begin + tiles_per_split);
     const int k_slabs = (D + TK - 1) / TK;
@@ -302,7 +304,7 @@ static siso_status_t run_tensor(Cache *c, tc::TensorState *ts, int slot, const C
         SISO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc::SMEM_BYTES));
         ts->attr_set[slot] = true;
     }
-    dim3 grid(splits, m_tiles);
+    dim3 grid(m_tiles, splits);
     kern<<<grid, tc::THREADS, tc::SMEM_BYTES, s>>>(map_q, ts->map_c, c->valid, B, c->dim, tiles_per_split, n_tiles,
                                                    partial, splits, c->status);
     SISO_LAUNCHED(c);
@@ -332,12 +334,12 @@ siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const flo
     const int kmax = k == 1 ? 1 : (k <= 4 ? 4 : 8);
     const int n_tiles = static_cast<int>((c->capacity + tc::TN - 1) / tc::TN);
     const int64_t m_tiles64 = (B + tc::TM - 1) / tc::TM;
-    if (m_tiles64 > 65535) return SISO_ERR_UNSUPPORTED;
+    if (m_tiles64 > 0x7FFFFFFF) return SISO_ERR_UNSUPPORTED;
     const int m_tiles = static_cast<int>(m_tiles64);
     // one CTA per SM at a time: aim at a whole number of waves with at least ~8 tiles per CTA
     const int64_t units = static_cast<int64_t>(m_tiles) * n_tiles;
     const int waves = static_cast<int>(std::min<int64_t>(16, std::max<int64_t>(1, units / (8ll * c->sm_count))));
-    int splits = std::max(1, std::min(n_tiles, (c->sm_count * waves) / m_tiles));
+    int splits = std::max(1, std::min(std::min(n_tiles, 65535), (c->sm_count * waves) / m_tiles));
     const int tiles_per_split = (n_tiles + splits - 1) / splits;
     splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
 
