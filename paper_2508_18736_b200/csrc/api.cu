@@ -207,9 +207,10 @@ siso_status_t siso_lookup(siso_cache_t *c, const void *d_queries, int64_t n_quer
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     int path = c->lookup_path;
     if (path == SISO_PATH_AUTO) {
-        if (n_queries <= 4) path = SISO_PATH_STREAM;
-        else if (c->dtype == SISO_BF16 && n_queries >= 16) path = SISO_PATH_TENSOR;
-        else path = SISO_PATH_SIMT;
+        // measured on B200: the streaming kernel holds 92 % of HBM peak for 1-2 queries and falls off beyond;
+        // the tensor-core kernel is HBM-bound (76-95 % of peak) from 3 queries up to one 128-query tile
+        if (c->dtype == SISO_BF16) path = n_queries <= 2 ? SISO_PATH_STREAM : SISO_PATH_TENSOR;
+        else path = n_queries <= 4 ? SISO_PATH_STREAM : SISO_PATH_SIMT;
     }
     switch (path) {
         case SISO_PATH_STREAM: return launch_lookup_stream(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);

@@ -1,40 +1,46 @@
 // Eviction (FilteringCentroids of Algorithm 1) and insertion of new entries.
 //
 // Eviction removes the m entries that come first in ascending (cluster_size, access_count,
-// last_access, slot) order.  Sorting the whole cache for a few victims would cost far more
-// than the metadata scan, so the kernels select instead:
-//   plan    one CTA ranks a strided sample of live entries and picks a pivot key that, with
-//           overwhelming probability, has at least m entries at or below it but not many more;
-//   filter  every live entry with key <= pivot is appended to a candidate list;
-//   rank    each candidate counts the candidates below it; rank < m means victim number `rank`.
-// If the pivot turned out too low (fewer than m candidates), a second filter/rank pair with an
-// infinite pivot redoes the selection exactly; both pairs are always launched and the second is a
-// no-op when the first succeeded.  The result never depends on the sample: it is the exact order.
+// last_access, slot) order.  Sorting the whole cache for a few victims would cost far more than the
+// metadata scan, so the kernels select, exactly, in the manner of a sample sort:
+//   sample   one CTA gathers a strided sample of 1024 live entries and sorts it (bitonic, in
+//            shared memory): the sorted sample keys are splitters
+//   bucket   every live entry finds its bucket (number of splitters below its key, binary search)
+//            and the buckets are counted
+//   collect  the smallest bucket index p whose cumulative count reaches m is found from the counts;
+//            entries in buckets <= p (at least m of them, about m + capacity/1024) become candidates
+//   rank     one warp per candidate counts the candidates below it; rank < m means victim number rank
+// Keys are compared as three 64-bit integers (order-preserving image of the fp64 cluster_size, then
+// access_count | last_access | slot), so the order is the exact lexicographic order and total.
 #include "common.cuh"
 
 namespace siso {
 
-struct EvictKey {
-    double size;
-    unsigned long long last;
-    uint32_t access;
-    int32_t slot;
+struct Key3 {
+    unsigned long long w0, w1, w2;
 };
-__device__ __forceinline__ bool key_less(const EvictKey &a, const EvictKey &b) {
-    if (a.size != b.size) return a.size < b.size;
-    if (a.access != b.access) return a.access < b.access;
-    if (a.last != b.last) return a.last < b.last;
-    return a.slot < b.slot;
+__device__ __forceinline__ bool key_less(const Key3 &a, const Key3 &b) {
+    if (a.w0 != b.w0) return a.w0 < b.w0;
+    if (a.w1 != b.w1) return a.w1 < b.w1;
+    return a.w2 < b.w2;
+}
+__device__ __forceinline__ Key3 make_key(double size, uint32_t access, unsigned long long last, uint32_t slot) {
+    const unsigned long long u = static_cast<unsigned long long>(__double_as_longlong(size));
+    Key3 k;
+    k.w0 = (u >> 63) ? ~u : (u | 0x8000000000000000ull);          // order-preserving for every finite double
+    k.w1 = (static_cast<unsigned long long>(access) << 32) | (last >> 32);
+    k.w2 = (last << 32) | slot;
+    return k;
 }
 
-struct EvictPlan {
-    EvictKey pivot;
-    long long m;            // victims to produce (clamped to the occupancy)
-    int pivot_all;          // 1: pivot is +infinity
-    unsigned int ncand[2];  // candidates found by attempt 0 / 1
-};
-
 constexpr int EV_SAMPLE = 1024;
+
+struct EvictPlan {
+    long long m;             // victims to produce (clamped to the occupancy)
+    int n_sample;            // live splitters
+    unsigned int n_cand;
+    unsigned int hist[EV_SAMPLE + 1];
+};
 
 __device__ __forceinline__ int block_exclusive_scan_1024(int v, int *total, int *warp_sum) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -62,11 +68,12 @@ __device__ __forceinline__ int block_exclusive_scan_1024(int v, int *total, int 
 }
 
 __global__ void __launch_bounds__(1024)
-evict_plan_kernel(long long m_req, const uint8_t *__restrict__ hit, long long n_hit, long long capacity,
-                  const double *__restrict__ size, const uint32_t *__restrict__ access,
-                  const unsigned long long *__restrict__ last, const uint8_t *__restrict__ valid,
-                  const long long *__restrict__ counters, EvictPlan *plan, int32_t *victims, long long n_victims_out) {
-    __shared__ EvictKey sample[EV_SAMPLE];
+evict_sample_kernel(long long m_req, const uint8_t *__restrict__ hit, long long n_hit, long long capacity,
+                    const double *__restrict__ size, const uint32_t *__restrict__ access,
+                    const unsigned long long *__restrict__ last, const uint8_t *__restrict__ valid,
+                    const long long *__restrict__ counters, EvictPlan *plan, Key3 *__restrict__ splitters,
+                    int32_t *victims, long long n_victims_out) {
+    __shared__ unsigned long long k0[EV_SAMPLE], k1[EV_SAMPLE], k2[EV_SAMPLE];
     __shared__ int warp_sum[32];
     __shared__ long long m_s;
     const int tid = threadIdx.x;
@@ -87,102 +94,151 @@ evict_plan_kernel(long long m_req, const uint8_t *__restrict__ hit, long long n_
     __syncthreads();
     const long long m = m_s < occupancy ? m_s : occupancy;
     for (long long r = m + tid; r < n_victims_out; r += 1024) victims[r] = -1;
-    if (tid == 0) { plan->m = m; plan->ncand[0] = 0; plan->ncand[1] = 0; plan->pivot_all = 0; }
+    if (tid == 0) { plan->m = m; plan->n_cand = 0; }
+    plan->hist[tid] = 0;
+    if (tid == 0) plan->hist[EV_SAMPLE] = 0;
     if (m == 0) return;
-    // strided sample: thread t looks at slots [t*stride, (t+1)*stride) and takes the first live one
+    // strided sample: thread t takes the first live slot of window [t*stride, (t+1)*stride), starting at an
+    // offset that changes from call to call (at most 64 probes)
     const long long stride = (capacity + EV_SAMPLE - 1) / EV_SAMPLE;
-    int have = 0;
-    EvictKey mine;
-    mine.size = 0.0; mine.last = 0; mine.access = 0; mine.slot = -1;
     const long long lo = tid * stride, hi = min(capacity, lo + stride);
-    for (long long sl = lo; sl < hi && sl < lo + 64; ++sl) {
-        if (valid[sl]) {
-            mine.size = size[sl]; mine.access = access[sl]; mine.last = last[sl]; mine.slot = static_cast<int32_t>(sl);
-            have = 1;
-            break;
+    const long long span = hi - lo;
+    int have = 0;
+    Key3 mine;
+    mine.w0 = mine.w1 = mine.w2 = ~0ull;                 // sentinel: sorts after every real key
+    if (span > 0) {
+        const long long start = static_cast<long long>((static_cast<unsigned long long>(counters[CNT_CLOCK]) * 2654435761ull) % static_cast<unsigned long long>(span));
+        const long long probes = span < 64 ? span : 64;
+        for (long long i = 0; i < probes; ++i) {
+            long long sl = lo + start + i;
+            if (sl >= hi) sl -= span;
+            if (valid[sl]) { mine = make_key(size[sl], access[sl], last[sl], static_cast<uint32_t>(sl)); have = 1; break; }
         }
     }
-    sample[tid] = mine;
+    k0[tid] = mine.w0; k1[tid] = mine.w1; k2[tid] = mine.w2;
     int n_sample;
     block_exclusive_scan_1024(have, &n_sample, warp_sum);
     __syncthreads();
-    // which rank of the sample becomes the pivot
-    long long r;
-    if (stride == 1) {
-        r = m;                                     // the sample is the whole cache: exact
-    } else {
-        const double mu = static_cast<double>(m) * n_sample / static_cast<double>(occupancy);
-        r = static_cast<long long>(ceil(mu + 12.0 + 8.0 * sqrt(mu)));
-    }
-    if (r > n_sample || n_sample == 0) {
-        if (tid == 0) plan->pivot_all = 1;
-        return;
-    }
-    if (have) {
-        int rank = 0;
-        for (int j = 0; j < EV_SAMPLE; ++j) {
-            const EvictKey o = sample[j];
-            rank += (o.slot >= 0 && key_less(o, mine)) ? 1 : 0;
+    // bitonic sort, ascending
+    for (int k = 2; k <= EV_SAMPLE; k <<= 1) {
+        for (int j = k >> 1; j > 0; j >>= 1) {
+            const int partner = tid ^ j;
+            if (partner > tid) {
+                Key3 a, b;
+                a.w0 = k0[tid]; a.w1 = k1[tid]; a.w2 = k2[tid];
+                b.w0 = k0[partner]; b.w1 = k1[partner]; b.w2 = k2[partner];
+                const bool up = (tid & k) == 0;
+                if (key_less(b, a) == up) {
+                    k0[tid] = b.w0; k1[tid] = b.w1; k2[tid] = b.w2;
+                    k0[partner] = a.w0; k1[partner] = a.w1; k2[partner] = a.w2;
+                }
+            }
+            __syncthreads();
         }
-        if (rank == r - 1) plan->pivot = mine;
     }
+    Key3 out;
+    out.w0 = k0[tid]; out.w1 = k1[tid]; out.w2 = k2[tid];
+    splitters[tid] = out;
+    if (tid == 0) plan->n_sample = n_sample;
+}
+
+// bucket(key) = number of live splitters strictly below the key, in [0, n_sample]
+__global__ void __launch_bounds__(256)
+evict_bucket_kernel(long long capacity, const double *__restrict__ size, const uint32_t *__restrict__ access,
+                    const unsigned long long *__restrict__ last, const uint8_t *__restrict__ valid, EvictPlan *plan,
+                    const Key3 *__restrict__ splitters, uint16_t *__restrict__ bucket) {
+    if (plan->m == 0) return;
+    __shared__ unsigned long long s0[EV_SAMPLE], s1[EV_SAMPLE], s2[EV_SAMPLE];
+    __shared__ unsigned int hist[EV_SAMPLE + 1];
+    const int n_sample = plan->n_sample;
+    for (int i = threadIdx.x; i < EV_SAMPLE; i += 256) {
+        const Key3 k = splitters[i];
+        s0[i] = k.w0; s1[i] = k.w1; s2[i] = k.w2;
+        hist[i] = 0;
+    }
+    if (threadIdx.x == 0) hist[EV_SAMPLE] = 0;
+    __syncthreads();
+    for (long long sl = static_cast<long long>(blockIdx.x) * 256 + threadIdx.x; sl < capacity;
+         sl += static_cast<long long>(gridDim.x) * 256) {
+        if (!valid[sl]) continue;
+        const Key3 k = make_key(size[sl], access[sl], last[sl], static_cast<uint32_t>(sl));
+        int lo = 0, hi = n_sample;                       // first index whose splitter is >= k
+        while (lo < hi) {
+            const int mid = (lo + hi) >> 1;
+            Key3 sp;
+            sp.w0 = s0[mid]; sp.w1 = s1[mid]; sp.w2 = s2[mid];
+            if (key_less(sp, k)) lo = mid + 1; else hi = mid;
+        }
+        bucket[sl] = static_cast<uint16_t>(lo);
+        atomicAdd(&hist[lo], 1u);
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i <= EV_SAMPLE; i += 256)
+        if (hist[i]) atomicAdd(&plan->hist[i], hist[i]);
 }
 
 __global__ void __launch_bounds__(256)
-evict_filter_kernel(int attempt, long long capacity, const double *__restrict__ size,
-                    const uint32_t *__restrict__ access, const unsigned long long *__restrict__ last,
-                    const uint8_t *__restrict__ valid, EvictPlan *plan, EvictKey *__restrict__ cand) {
+evict_collect_kernel(long long capacity, const double *__restrict__ size, const uint32_t *__restrict__ access,
+                     const unsigned long long *__restrict__ last, const uint8_t *__restrict__ valid, EvictPlan *plan,
+                     const uint16_t *__restrict__ bucket, Key3 *__restrict__ cand) {
     const long long m = plan->m;
     if (m == 0) return;
-    if (attempt == 1 && plan->ncand[0] >= m) return;
-    const bool all = attempt == 1 || plan->pivot_all;
-    const EvictKey pivot = plan->pivot;
-    const int lane = threadIdx.x & 31;
-    for (long long base = static_cast<long long>(blockIdx.x) * blockDim.x; base < capacity;
-         base += static_cast<long long>(gridDim.x) * blockDim.x) {
-        const long long sl = base + threadIdx.x;
-        bool take = false;
-        EvictKey k;
-        if (sl < capacity && valid[sl]) {
-            k.size = size[sl]; k.access = access[sl]; k.last = last[sl]; k.slot = static_cast<int32_t>(sl);
-            take = all || !key_less(pivot, k);
+    __shared__ int p_s;
+    if (threadIdx.x < 32) {
+        // smallest p with hist[0] + ... + hist[p] >= m (exists: the live entries number at least m)
+        long long run = 0;
+        int found = EV_SAMPLE;
+        for (int base = 0; base <= EV_SAMPLE && found == EV_SAMPLE; base += 32) {
+            const int i = base + threadIdx.x;
+            long long x = i <= EV_SAMPLE ? plan->hist[i] : 0;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const long long y = __shfl_up_sync(0xFFFFFFFFu, x, o);
+                if (static_cast<int>(threadIdx.x) >= o) x += y;
+            }
+            const unsigned reach = __ballot_sync(0xFFFFFFFFu, run + x >= m);
+            if (reach) found = base + __ffs(reach) - 1;
+            run += __shfl_sync(0xFFFFFFFFu, x, 31);
         }
+        if (threadIdx.x == 0) p_s = found;
+    }
+    __syncthreads();
+    const int p = p_s;
+    const int lane = threadIdx.x & 31;
+    for (long long base = static_cast<long long>(blockIdx.x) * 256; base < capacity;
+         base += static_cast<long long>(gridDim.x) * 256) {
+        const long long sl = base + threadIdx.x;
+        const bool take = sl < capacity && valid[sl] && bucket[sl] <= p;
         const unsigned ballot = __ballot_sync(0xFFFFFFFFu, take);
         if (ballot) {
             unsigned int warp_base = 0;
-            if (lane == 0) warp_base = atomicAdd(&plan->ncand[attempt], static_cast<unsigned int>(__popc(ballot)));
+            if (lane == 0) warp_base = atomicAdd(&plan->n_cand, static_cast<unsigned int>(__popc(ballot)));
             warp_base = __shfl_sync(0xFFFFFFFFu, warp_base, 0);
-            if (take) cand[warp_base + __popc(ballot & ((1u << lane) - 1u))] = k;
+            if (take) cand[warp_base + __popc(ballot & ((1u << lane) - 1u))] =
+                          make_key(size[sl], access[sl], last[sl], static_cast<uint32_t>(sl));
         }
     }
 }
 
+// one warp per candidate
 __global__ void __launch_bounds__(256)
-evict_rank_kernel(int attempt, EvictPlan *plan, const EvictKey *__restrict__ cand, uint8_t *__restrict__ valid,
+evict_rank_kernel(EvictPlan *plan, const Key3 *__restrict__ cand, uint8_t *__restrict__ valid,
                   int32_t *__restrict__ victims, long long *counters) {
     const long long m = plan->m;
     if (m == 0) return;
-    if (attempt == 1 && plan->ncand[0] >= m) return;
-    const unsigned int n = plan->ncand[attempt];
-    if (n < m) return;                 // attempt 0 fell short: attempt 1 redoes it; attempt 1 never falls short
-    __shared__ EvictKey tile[256];
-    const unsigned int rounds = (n + gridDim.x * blockDim.x - 1) / (gridDim.x * blockDim.x);
-    for (unsigned int rd = 0; rd < rounds; ++rd) {
-        const unsigned int i = (rd * gridDim.x + blockIdx.x) * blockDim.x + threadIdx.x;
-        EvictKey mine;
-        if (i < n) mine = cand[i];
+    const unsigned int n = plan->n_cand;
+    const int lane = threadIdx.x & 31;
+    const unsigned int warps = gridDim.x * (blockDim.x >> 5);
+    for (unsigned int i = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5); i < n; i += warps) {
+        const Key3 mine = cand[i];
         unsigned int rank = 0;
-        for (unsigned int t0 = 0; t0 < n; t0 += 256) {
-            __syncthreads();
-            if (t0 + threadIdx.x < n) tile[threadIdx.x] = cand[t0 + threadIdx.x];
-            __syncthreads();
-            const unsigned int lim = min(256u, n - t0);
-            if (i < n)
-                for (unsigned int j = 0; j < lim; ++j) rank += key_less(tile[j], mine) ? 1u : 0u;
-        }
-        if (i < n && rank < m) {
-            if (victims) victims[rank] = mine.slot;
-            valid[mine.slot] = 0;
+        for (unsigned int j = lane; j < n; j += 32) rank += key_less(cand[j], mine) ? 1u : 0u;
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
+        if (lane == 0 && rank < m) {
+            const int32_t slot = static_cast<int32_t>(mine.w2 & 0xFFFFFFFFull);
+            if (victims) victims[rank] = slot;
+            valid[slot] = 0;
         }
     }
     if (blockIdx.x == 0 && threadIdx.x == 0) {
@@ -204,19 +260,22 @@ __global__ void decay_kernel(long long capacity, double decay, double *__restric
 siso_status_t launch_evict(Cache *c, int64_t n_evict, const uint8_t *hit, int64_t n_hit, uint32_t flags,
                            int32_t *victims, int64_t n_victims_out, cudaStream_t s) {
     Scratch scr;
-    SISO_TRY(scratch_reserve(c, pad256(sizeof(EvictPlan)) + pad256(sizeof(EvictKey) * c->capacity), s, &scr));
+    SISO_TRY(scratch_reserve(c, pad256(sizeof(EvictPlan)) + pad256(sizeof(Key3) * EV_SAMPLE) +
+                                    pad256(sizeof(uint16_t) * c->capacity) + pad256(sizeof(Key3) * c->capacity), s, &scr));
     EvictPlan *plan = scr.take<EvictPlan>(1);
-    EvictKey *cand = scr.take<EvictKey>(c->capacity);
-    evict_plan_kernel<<<1, 1024, 0, s>>>(n_evict, hit, n_hit, c->capacity, c->size, c->access, c->last, c->valid,
-                                         c->counters, plan, victims, victims ? n_victims_out : 0);
+    Key3 *splitters = scr.take<Key3>(EV_SAMPLE);
+    uint16_t *bucket = scr.take<uint16_t>(c->capacity);
+    Key3 *cand = scr.take<Key3>(c->capacity);
+    evict_sample_kernel<<<1, 1024, 0, s>>>(n_evict, hit, n_hit, c->capacity, c->size, c->access, c->last, c->valid,
+                                           c->counters, plan, splitters, victims, victims ? n_victims_out : 0);
     SISO_LAUNCHED(c);
     const int grid = static_cast<int>(std::min<int64_t>((c->capacity + 255) / 256, 4ll * c->sm_count));
-    for (int attempt = 0; attempt < 2; ++attempt) {
-        evict_filter_kernel<<<grid, 256, 0, s>>>(attempt, c->capacity, c->size, c->access, c->last, c->valid, plan, cand);
-        SISO_LAUNCHED(c);
-        evict_rank_kernel<<<grid, 256, 0, s>>>(attempt, plan, cand, c->valid, victims, c->counters);
-        SISO_LAUNCHED(c);
-    }
+    evict_bucket_kernel<<<grid, 256, 0, s>>>(c->capacity, c->size, c->access, c->last, c->valid, plan, splitters, bucket);
+    SISO_LAUNCHED(c);
+    evict_collect_kernel<<<grid, 256, 0, s>>>(c->capacity, c->size, c->access, c->last, c->valid, plan, bucket, cand);
+    SISO_LAUNCHED(c);
+    evict_rank_kernel<<<grid, 256, 0, s>>>(plan, cand, c->valid, victims, c->counters);
+    SISO_LAUNCHED(c);
     if (flags & SISO_EVICT_DECAY) {
         decay_kernel<<<static_cast<unsigned>((c->capacity + 255) / 256), 256, 0, s>>>(c->capacity, c->decay, c->size,
                                                                                       c->access, c->valid);

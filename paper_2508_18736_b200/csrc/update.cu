@@ -27,10 +27,13 @@ __global__ void update_keys_kernel(const int32_t *__restrict__ idx, int idx_stri
     vals[b] = static_cast<uint32_t>(b);
 }
 
-template <typename T> __device__ __forceinline__ double elem_f64(const T *p);
-template <> __device__ __forceinline__ double elem_f64<float>(const float *p) { return static_cast<double>(*p); }
-template <> __device__ __forceinline__ double elem_f64<__nv_bfloat16>(const __nv_bfloat16 *p) {
-    return static_cast<double>(__bfloat162float(*p));
+// four consecutive elements of a row as fp32 (one 8- or 16-byte load)
+template <typename T> __device__ __forceinline__ float4 load4(const T *p);
+template <> __device__ __forceinline__ float4 load4<float>(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
+template <> __device__ __forceinline__ float4 load4<__nv_bfloat16>(const __nv_bfloat16 *p) {
+    const uint2 u = __ldg(reinterpret_cast<const uint2 *>(p));
+    return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xFFFF0000u), __uint_as_float(u.y << 16),
+                       __uint_as_float(u.y & 0xFFFF0000u));
 }
 
 __device__ __forceinline__ double block_sum_f64(double v, double *red) {
@@ -62,11 +65,30 @@ update_apply_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restric
     const double n_old = size[slot];
     float *m = master + static_cast<int64_t>(slot) * D;
     for (int d = threadIdx.x; d < D; d += UP_THREADS) acc[d] = n_old * static_cast<double>(m[d]);
+    __syncthreads();      // the accumulation below uses a different thread-to-element mapping
+    // group extent, then the rows four at a time: the loads of a quartet are in flight together, the
+    // additions stay in ascending query order
     int64_t e = p;
-    for (; e < B && keys[e] == slot; ++e) {
-        const T *q = Q + static_cast<int64_t>(rows[e]) * D;
-        for (int d = threadIdx.x; d < D; d += UP_THREADS) acc[d] += elem_f64<T>(q + d);   // each thread owns its d
+    while (e < B && keys[e] == slot) ++e;
+    const int quads = D / 4;
+    for (int64_t t = p; t < e; t += 4) {
+        const int nrow = static_cast<int>(e - t < 4 ? e - t : 4);
+        const T *q[4];
+#pragma unroll
+        for (int r = 0; r < 4; ++r) q[r] = Q + static_cast<int64_t>(rows[t + (r < nrow ? r : 0)]) * D;
+        for (int g = threadIdx.x; g < quads; g += UP_THREADS) {
+            float4 v[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) v[r] = load4<T>(q[r] + 4 * g);
+            double a0 = acc[4 * g], a1 = acc[4 * g + 1], a2 = acc[4 * g + 2], a3 = acc[4 * g + 3];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) {
+                if (r < nrow) { a0 += v[r].x; a1 += v[r].y; a2 += v[r].z; a3 += v[r].w; }
+            }
+            acc[4 * g] = a0; acc[4 * g + 1] = a1; acc[4 * g + 2] = a2; acc[4 * g + 3] = a3;   // each thread owns its g
+        }
     }
+    __syncthreads();
     const long long count = e - p;
     double ss = 0.0;
     for (int d = threadIdx.x; d < D; d += UP_THREADS) ss += acc[d] * acc[d];
