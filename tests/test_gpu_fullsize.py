@@ -1,0 +1,168 @@
+"""Parity at the stated full sizes of configurations 2-5, in the launch configuration the benchmark times:
+oracle comparison on sampled outputs plus properties that hold for every output."""
+import os
+
+import numpy as np
+import pytest
+import torch
+
+import oracle
+from gen import workloads as W
+from util import TOL, check_lookup, to_dev, widen64
+
+pytestmark = pytest.mark.gpu
+
+siso = pytest.importorskip("paper_2508_18736_b200")
+THREADS = os.cpu_count() or 1
+
+
+def fill(cache, centroids, dtype, step=1 << 16):
+    for lo in range(0, centroids.shape[0], step):
+        cache.insert(to_dev(centroids[lo:lo + step], dtype))
+    cache.check_status()
+
+
+def check_all_rows(idx, sim, hit, w, tol, rng):
+    """Properties of every output row, checked without the oracle's full sweep."""
+    B, k = idx.shape
+    assert (idx >= 0).all() and (idx < w.centroids.shape[0]).all()
+    assert (np.diff(sim, axis=1) <= 0).all(), "similarities not descending"
+    srt = np.sort(idx, axis=1)
+    assert (np.diff(srt, axis=1) > 0).all(), "duplicate slot in a row"
+    # every reported similarity is the true similarity of the reported slot
+    Q = widen64(w.queries)
+    for j in range(k):
+        true = np.einsum("ij,ij->i", Q, widen64(w.centroids[idx[:, j]]))
+        assert np.abs(true - sim[:, j]).max() <= tol
+    assert (hit == (sim[:, 0] > w.theta)).all()
+    # no sampled centroid beats the reported ones by more than the tolerance
+    sub = rng.choice(w.centroids.shape[0], min(4096, (1 << 26) // B), replace=False)     # bounded host memory
+    S = w.queries_f32() @ w.centroids_f32()[sub].T
+    part = -np.partition(-S, k - 1, axis=1)[:, :k]
+    part.sort(axis=1)
+    assert (sim[:, ::-1] >= part - tol).all() if k > 1 else (sim[:, 0] >= S.max(1) - tol).all()
+
+
+def test_config4_full_size_lookup():
+    w = W.config(4, threads=THREADS)
+    cache = siso.SisoCache(w.centroids.shape[0], w.dim, "bf16")
+    fill(cache, w.centroids, "bf16")
+    idx, sim, hit = cache.lookup(to_dev(w.queries, "bf16"), torch.from_numpy(w.theta).cuda(), 4)
+    cache.check_status()
+    idx, sim, hit = idx.cpu().numpy(), sim.cpu().numpy(), hit.cpu().numpy()
+    cache.close()
+    rng = np.random.default_rng(0)
+    check_all_rows(idx, sim, hit, w, TOL["bf16"], rng)
+    rows = np.concatenate([rng.choice(8192, 20, replace=False), np.flatnonzero(w.query_labels < 0)[:4]])
+    ora = oracle.lookup(w.centroids, w.queries[rows], w.theta[rows], 4)
+    check_lookup((idx[rows], sim[rows], hit[rows]), ora, w.centroids, w.queries[rows], w.theta[rows], TOL["bf16"])
+    ind = w.query_labels >= 0
+    same_cluster = w.centroid_labels[idx[ind, 0]] == w.query_labels[ind]
+    assert same_cluster.mean() > 0.999            # in-distribution queries find their own cluster
+    assert hit[ind].mean() > 0.99 and hit[~ind].mean() < 0.01
+
+
+def test_config2_full_size_lookup_and_update():
+    w = W.config(2, threads=THREADS)
+    cache = siso.SisoCache(65536, 768, "bf16")
+    fill(cache, w.centroids, "bf16")
+    q = to_dev(w.queries, "bf16")
+    idx_t, sim_t, hit_t = cache.lookup(q, torch.from_numpy(w.theta).cuda(), 1)
+    idx, sim, hit = idx_t.cpu().numpy(), sim_t.cpu().numpy(), hit_t.cpu().numpy()
+    rng = np.random.default_rng(1)
+    check_all_rows(idx, sim, hit, w, TOL["bf16"], rng)
+    rows = rng.choice(65536, 48, replace=False)
+    ora = oracle.lookup(w.centroids, w.queries[rows], w.theta[rows], 1)
+    check_lookup((idx[rows], sim[rows], hit[rows]), ora, w.centroids, w.queries[rows], w.theta[rows], TOL["bf16"])
+    cache.update(q, idx_t, hit_t)
+    cache.check_status()
+    st = cache.export()
+    master, size = st["master"].cpu().numpy(), st["size"].cpu().numpy()
+    access = st["access"].cpu().numpy().view(np.uint32)
+    vecs = st["vecs"].view(torch.int16).cpu().numpy().view(np.uint16)
+    cache.close()
+    # closed form of the running mean on sampled centroids: the hottest ones and random ones
+    counts = np.bincount(idx[hit == 1, 0], minlength=65536)
+    assert (size == 1 + counts).all() and (access == siso.ACCESS_INF).all()
+    C64, Q64 = widen64(w.centroids), widen64(w.queries)
+    sample = np.concatenate([np.argsort(-counts)[:8], rng.choice(np.flatnonzero(counts > 0), 24),
+                             rng.choice(np.flatnonzero(counts == 0), 8)])
+    assert counts.max() > 200                    # Zipf: some centroids take hundreds of hits in one batch
+    for j in sample:
+        H = np.flatnonzero((hit == 1) & (idx[:, 0] == j))
+        if len(H) == 0:
+            assert (vecs[j] == w.centroids[j]).all()
+            continue
+        v = 1.0 * C64[j] + Q64[H].sum(0)
+        want = v / np.linalg.norm(v)
+        assert np.abs(master[j] - want).max() <= 1e-6
+        assert (vecs[j] == torch.from_numpy(master[j]).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)).all()
+
+
+def test_config3_full_size_self_merge():
+    w = W.config(3, threads=THREADS)
+    cache = siso.SisoCache(32768, 768, "f32")
+    fill(cache, w.centroids, "f32")
+    mm, n = cache.merge(W.MERGE_THRESHOLD_CONFIG3, siso.MERGE_WEIGHTED_MEAN)
+    cache.check_status()
+    mm = mm.cpu().numpy()
+    st = cache.export()
+    ora = oracle.OracleCache(32768, 768, "f32")
+    ora.insert(w.centroids)
+    entry = ora.master.copy()
+    o_mm, o_n = ora.merge(W.MERGE_THRESHOLD_CONFIG3, True)
+    assert n == o_n and (mm == o_mm).all()
+    live = ora.valid == 1
+    assert (st["valid"].cpu().numpy() == ora.valid).all()
+    assert (st["size"].cpu().numpy()[live] == ora.size[live]).all()
+    assert np.abs(st["master"].cpu().numpy()[live] - ora.master[live]).max() <= 1e-6
+    assert 1500 < live.sum() < 2100               # about one survivor per generating cluster
+    assert (w.centroid_labels[mm] == w.centroid_labels).all()      # merged only within a cluster
+    cache.close()
+
+
+def test_config5_full_scale_sampled_batches():
+    sp = W.StreamSpec()                          # 262,144 x 768, batches of 256, P-mode, theta 0.86
+    stream = W.QueryStream(sp, threads=THREADS)
+    n_batches = 1400
+    q_all = to_dev(stream.block(0, n_batches, threads=THREADS), "bf16")
+    cache = siso.SisoCache(sp.capacity, sp.dim, "bf16")
+    # start from a nearly full cache so that the sampled batches evict: fill with the stream's own later queries
+    filler = stream.block(20000, 20000 + (sp.capacity - 3000) // 256, threads=THREADS)
+    fill(cache, filler, "bf16")
+    sampled = {700, 1399}
+    out = None
+    for t in range(n_batches):
+        q = q_all[t * 256:(t + 1) * 256]
+        if t in sampled:
+            st = cache.export()
+            torch.cuda.synchronize()
+            ora = oracle.OracleCache(sp.capacity, sp.dim, "bf16")
+            ora.load_state(st["master"].cpu().numpy(), st["size"].cpu().numpy(),
+                           st["access"].cpu().numpy().view(np.uint32), st["last"].cpu().numpy().view(np.uint64),
+                           st["valid"].cpu().numpy(), cache.stats()["clock"])
+            pre_copy, pre_valid = ora.lookup_copy(), ora.valid.copy()
+        out = cache.stream_step(q, float(sp.theta), out=out)
+        if t in sampled:
+            idx, sim, hit, victims, slots = [x.cpu().numpy() for x in out]
+            qn = q.view(torch.int16).cpu().numpy().view(np.uint16)
+            theta = np.full(256, sp.theta, np.float32)
+            o_idx, o_sim, o_hit, o_victims, o_slots = ora.stream_step(qn, theta, forced=(idx, hit))
+            check_lookup((idx, sim, hit), (o_idx, o_sim, o_hit), pre_copy, qn, theta, TOL["bf16"], valid=pre_valid)
+            nv = len(o_victims)
+            assert nv > 0, "the sampled batch did not evict"
+            assert (victims[:nv] == o_victims).all() and (victims[nv:] == -1).all()
+            assert (slots == o_slots).all()
+            post = cache.export()
+            live = ora.valid == 1
+            assert (post["valid"].cpu().numpy() == ora.valid).all()
+            assert (post["size"].cpu().numpy()[live] == ora.size[live]).all()
+            assert (post["access"].cpu().numpy().view(np.uint32)[live] == ora.access[live]).all()
+            assert (post["last"].cpu().numpy().view(np.uint64)[live] == ora.last[live]).all()
+            touched = np.unique(np.concatenate([idx[hit == 1, 0], slots[slots >= 0]]))
+            assert np.abs(post["master"].cpu().numpy()[touched] - ora.master[touched]).max() <= 1e-6
+    s = cache.stats()
+    assert s["occupancy"] == sp.capacity and s["evictions"] > 0
+    assert s["inserts"] - s["evictions"] == s["occupancy"]
+    cache.check_status()
+    cache.close()
