@@ -66,6 +66,23 @@ def workload_name(args) -> str:
             f"perturbation length), batch {args.queries} (Zipf 1.0, 20% out-of-distribution), top-4, theta in [0.78, 0.93]")
 
 
+# ------------------------------------------------------------------------------ multi-rank helpers
+def max_over_ranks(value: float, world: int, device=None) -> float:
+    """The slowest rank's time: what a whole-job throughput has to be divided by."""
+    if world == 1:
+        return float(value)
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor([value], dtype=torch.float64, device=device)
+    dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return float(t.item())
+
+
+def whole_job_value(queries_per_rank: int, world: int, ms_per_step: float) -> float:
+    """Queries per second over all ranks (weak scaling: every rank looks up its own batch)."""
+    return world * queries_per_rank / (ms_per_step * 1e-3)
+
+
 # ------------------------------------------------------------------------------ CPU oracle legs
 def time_oracle(w, n_sample: int, repeats: int = 1):
     """Seconds per call of the oracle on the first n_sample queries of the batch (all host cores)."""
@@ -220,11 +237,7 @@ def run_ours(args):
             ev[i + 1].record(stream)
         barrier()
         per = [ev[i].elapsed_time(ev[i + 1]) for i in range(steps)]
-        total = ev[0].elapsed_time(ev[steps])
-        if world > 1:
-            t = torch.tensor([total], dtype=torch.float64, device=dev)
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            total = float(t.item())
+        total = max_over_ranks(ev[0].elapsed_time(ev[steps]), world, dev)
         return total / steps, per, cache.launch_count - l0
 
     for _ in range(max(3, args.warmup)):
@@ -240,7 +253,7 @@ def run_ours(args):
             step_host()
         ms_e2e, _, _ = timed(step_host, args.steps)
         cache.check_status()
-        e2e = {"value": world * B / (ms_e2e * 1e-3), "unit": UNIT,
+        e2e = {"value": whole_job_value(B, world, ms_e2e), "unit": UNIT,
                "h2d_bytes_per_step": int(w.queries.nbytes + w.theta.nbytes),
                "d2h_bytes_per_step": int(h_idx.numel() * 4 + h_sim.numel() * 4 + h_hit.numel()),
                "ms_per_step": ms_e2e}
@@ -256,14 +269,20 @@ def run_ours(args):
     flops = 2.0 * B * args.rows * 1024
     kernel_ms = statistics.median(per_step)           # the sweep kernel plus its small finalize kernel
     achieved = flops / (kernel_ms * 1e-3) / 1e12
+    # DRAM bytes per launch from the committed ncu capture of this kernel (profiles/lookup_tensor_small_case_full_set.txt:
+    # 274 MB read + 6 MB written at 131,072 rows x 2,048 queries), scaled with rows and queries; only for the
+    # tensor-core kernel as profiled
+    traffic = None
+    if args.path in ("auto", "tensor"):
+        traffic = 273.9e6 * (args.rows / 131072.0) * (268.4 / 272.6) + 273.9e6 * (B / 2048.0) * (4.2 / 272.6) + 6.0e6 * (B / 2048.0)
     roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops"], "traffic": None, "peak_kind": f"{peak_kind}, burst",
+                "frac": achieved / peaks["bf16_tflops"], "traffic": traffic, "peak_kind": f"{peak_kind}, burst",
                 "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
                 "hbm_floor_ms": (args.rows * 1024 * 2 + B * 1024 * 2) / (peaks["hbm_gbs"] * 1e9) * 1e3,
                 "kernel": {"auto": "tensor-core sweep (auto)", "tensor": "tensor-core sweep", "simt": "CUDA-core sweep",
                            "stream": "streaming sweep"}[args.path],
                 "flops_per_launch": flops, "median_launch_ms": kernel_ms}
-    line = {"metric": METRIC, "value": world * B / (ms * 1e-3), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+    line = {"metric": METRIC, "value": whole_job_value(B, world, ms), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": workload_name(args), "parallelism": f"replica x{world}, queries sharded",
