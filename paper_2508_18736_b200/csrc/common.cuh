@@ -48,6 +48,7 @@ struct Cache {
     size_t stage_bytes;
 
     int32_t lookup_path;
+    int32_t tensor_pair_mode;   // 0: CTA pairs when the batch spans two query tiles; 1: single-CTA kernel only
     int64_t merge_max_cand;
     int64_t launches;
     void *tensor_state;    // owned by lookup_tensor.cu

@@ -271,8 +271,10 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
 
 struct TensorState {
     EncodeTiledFn encode;
-    CUtensorMap map_c;
+    CUtensorMap map_c;        // box of 256 centroid rows (single-CTA kernel)
+    CUtensorMap map_c_half;   // box of 128 centroid rows (CTA-pair kernel: each CTA stages half a tile)
     bool attr_set[3];
+    bool attr_set_pair[3];
 };
 
 static siso_status_t encode_map(EncodeTiledFn fn, CUtensorMap *map, const void *base, uint64_t rows, uint64_t dim,
@@ -289,6 +291,10 @@ static siso_status_t encode_map(EncodeTiledFn fn, CUtensorMap *map, const void *
 }
 
 }  // namespace tc
+
+siso_status_t launch_lookup_tensor_pair(Cache *c, bool *attr_set3, const CUtensorMap &map_q, const CUtensorMap &map_c_half,
+                                        int64_t B, int kmax, int tiles_per_split, int n_tiles, int splits, int m_tiles_even,
+                                        unsigned long long *partial, cudaStream_t s);
 
 void tensor_state_destroy(Cache *c) {
     delete static_cast<tc::TensorState *>(c->tensor_state);
@@ -325,6 +331,9 @@ siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const flo
         ts->encode = reinterpret_cast<tc::EncodeTiledFn>(fn);
         siso_status_t st = tc::encode_map(ts->encode, &ts->map_c, c->vecs, static_cast<uint64_t>(c->rows_alloc),
                                           static_cast<uint64_t>(c->dim), tc::TN);
+        if (st == SISO_OK)
+            st = tc::encode_map(ts->encode, &ts->map_c_half, c->vecs, static_cast<uint64_t>(c->rows_alloc),
+                                static_cast<uint64_t>(c->dim), tc::TN / 2);
         if (st != SISO_OK) { delete ts; return st; }
         c->tensor_state = ts;
     }
@@ -336,19 +345,27 @@ siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const flo
     const int64_t m_tiles64 = (B + tc::TM - 1) / tc::TM;
     if (m_tiles64 > 0x7FFFFFFF) return SISO_ERR_UNSUPPORTED;
     const int m_tiles = static_cast<int>(m_tiles64);
+    // CTA pairs (two query tiles share every centroid tile) whenever the batch has at least two query tiles
+    const bool pair = m_tiles >= 2 && c->tensor_pair_mode == 0;
+    const int m_ctas = pair ? (m_tiles + 1) / 2 * 2 : m_tiles;
     // one CTA per SM at a time: aim at a whole number of waves with at least ~8 tiles per CTA
-    const int64_t units = static_cast<int64_t>(m_tiles) * n_tiles;
+    const int64_t units = static_cast<int64_t>(m_ctas) * n_tiles;
     const int waves = static_cast<int>(std::min<int64_t>(16, std::max<int64_t>(1, units / (8ll * c->sm_count))));
-    int splits = std::max(1, std::min(std::min(n_tiles, 65535), (c->sm_count * waves) / m_tiles));
+    int splits = std::max(1, std::min(std::min(n_tiles, 65535), (c->sm_count * waves) / m_ctas));
     const int tiles_per_split = (n_tiles + splits - 1) / splits;
     splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
 
     Scratch scr;
     SISO_TRY(scratch_reserve(c, pad256(sizeof(unsigned long long) * B * splits * kmax), s, &scr));
     unsigned long long *partial = scr.take<unsigned long long>(static_cast<size_t>(B) * splits * kmax);
-    siso_status_t st = kmax == 1 ? run_tensor<1>(c, ts, 0, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s)
-                     : kmax == 4 ? run_tensor<4>(c, ts, 1, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s)
-                                 : run_tensor<8>(c, ts, 2, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s);
+    siso_status_t st;
+    if (pair)
+        st = launch_lookup_tensor_pair(c, ts->attr_set_pair, map_q, ts->map_c_half, B, kmax, tiles_per_split, n_tiles, splits,
+                                       m_ctas, partial, s);
+    else
+        st = kmax == 1 ? run_tensor<1>(c, ts, 0, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s)
+           : kmax == 4 ? run_tensor<4>(c, ts, 1, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s)
+                       : run_tensor<8>(c, ts, 2, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s);
     SISO_TRY(st);
     return launch_topk_finalize(c, partial, B, splits, kmax, k, theta, theta_s, idx, sim, hit, s);
 }

@@ -1,0 +1,306 @@
+// Large-batch lookup on tensor cores with CTA pairs (tcgen05 cta_group::2).
+//
+// Two CTAs of a cluster work on 256 queries x 256 centroids at a time.  Each CTA stages its own
+// 128-query slab of Q and HALF of the centroid tile (128 rows of C), so for the same flops per SM
+// a third less data crosses L2 -> shared memory than in the single-CTA kernel (which reloads the
+// whole 256-row centroid tile for every 128 queries).  The leader CTA (cluster rank 0) issues one
+// M=256 MMA per 16 K-elements; the result rows 0..127 land in the leader's TMEM, rows 128..255 in
+// the peer's, and each CTA's epilogue warps scan their own rows exactly as in the single-CTA kernel.
+//   full[s]       (leader's)  both CTAs' TMA loads of stage s report their bytes here
+//   empty[s]      (each CTA)  one tcgen05.commit of the leader arrives on both when the MMAs have read stage s
+//   acc_full[a]   (each CTA)  committed by the leader when a 256-column accumulator is complete
+//   acc_empty[a]  (leader's)  the 8 epilogue warps of both CTAs arrive when they have drained it
+// No load is multicast: every CTA fetches what it needs itself.  All waits are bounded (see
+// lookup_tensor.cu); a CTA that gives up sets SISO_ERR_TIMEOUT and still reaches the final cluster barrier.
+#include <cuda.h>
+
+#include <cstring>
+
+#include "common.cuh"
+
+namespace siso {
+namespace tc2 {
+
+constexpr int TM = 128;             // queries per CTA
+constexpr int TN = 256;             // centroids per tile (both CTAs together stage them, 128 rows each)
+constexpr int TK = 64;
+constexpr int STAGES = 6;
+constexpr int ACC_STAGES = 2;
+constexpr int THREADS = 192;
+constexpr uint32_t A_BYTES = TM * TK * 2;            // 16 KiB
+constexpr uint32_t B_BYTES = (TN / 2) * TK * 2;      // 16 KiB: this CTA's half of the centroid tile
+constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
+constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 256;
+constexpr uint32_t TMEM_COLS = ACC_STAGES * TN;
+constexpr uint32_t SPIN_LIMIT = 4u << 20;
+
+__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+// address of the same shared-memory location in CTA `rank` of the cluster (shared::cluster window)
+__device__ __forceinline__ uint32_t cluster_addr(uint32_t local, uint32_t rank) {
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ uint32_t cluster_rank() {
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+__device__ __forceinline__ void cluster_sync() {
+    asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive_cluster(uint32_t cluster_address) {
+    asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(cluster_address) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.acquire.cluster.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
+    for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((it & 63u) == 63u) {
+            if (*abort_flag) return false;
+            __nanosleep(64);
+        }
+    }
+    *abort_flag = 1;
+    return false;
+}
+// this CTA's tile into its own shared memory; the bytes are reported to the barrier at `bar_cluster_addr`,
+// which lives in the leader CTA
+__device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *map, int c0, int c1, uint32_t bar_cluster_addr) {
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar_cluster_addr)
+                 : "memory");
+}
+__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+// Arrive, once all MMAs issued so far have completed, on the barrier at this shared-memory offset in BOTH
+// CTAs of the pair (a commit that signals two barriers; no data is copied by it).
+__device__ __forceinline__ void umma_commit_both(uint64_t *bar) {
+    const uint16_t both = 3;
+    asm volatile("tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
+                 ::"r"(smem_u32(bar)), "h"(both) : "memory");
+}
+__device__ __forceinline__ void umma_bf16_pair(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::2.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
+        "tcgen05.wait::ld.sync.aligned;"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
+          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
+          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
+          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
+    uint64_t d = 0;
+    d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
+    d |= static_cast<uint64_t>(1) << 16;
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;
+    d |= static_cast<uint64_t>(1) << 46;
+    d |= static_cast<uint64_t>(2) << 61;
+    return d;
+}
+// D fp32, A and B bf16, K-major, N = 256, M = 256 (128 rows per CTA of the pair)
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(TN >> 3) << 17) |
+                           (static_cast<uint32_t>((2 * TM) >> 4) << 24);
+
+struct Barriers {
+    uint64_t full[STAGES], empty[STAGES], acc_full[ACC_STAGES], acc_empty[ACC_STAGES];
+    uint32_t tmem_base;
+    int abort_flag;
+};
+
+template <int KMAX>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
+lookup_tensor_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_c_half,
+                          const uint8_t *__restrict__ valid, int64_t B, int D, int tiles_per_split, int n_tiles,
+                          unsigned long long *__restrict__ partial, int splits, int *status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    Barriers *bars = reinterpret_cast<Barriers *>(tiles + STAGES * STAGE_BYTES);
+    volatile int *abort_flag = &bars->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();              // 0 = leader
+    const int split = blockIdx.y;
+    const int q0 = blockIdx.x * TM;                    // this CTA's own 128 queries
+    const int t_begin = split * tiles_per_split;
+    const int t_end = min(n_tiles, t_begin + tiles_per_split);
+    const int k_slabs = (D + TK - 1) / TK;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&bars->full[s], 1); mbar_init(&bars->empty[s], 1); }
+        for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(&bars->acc_full[a], 1); mbar_init(&bars->acc_empty[a], 8); }
+        bars->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {   // the same warp of both CTAs allocates the pair's tensor memory (512 columns in each)
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&bars->tmem_base)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync();                                    // both CTAs' barriers are initialised before any remote use
+    tcgen05_fence_after();
+    const uint32_t tmem_base = bars->tmem_base;
+
+    if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (int t = t_begin; t < t_end && ok; ++t) {
+                const int n0 = t * TN + static_cast<int>(rank) * (TN / 2);     // this CTA's half of the centroid tile
+                for (int ks = 0; ks < k_slabs; ++ks) {
+                    if (!mbar_wait(&bars->empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+                    uint8_t *a_dst = tiles + stage * STAGE_BYTES;
+                    uint8_t *b_dst = a_dst + A_BYTES;
+                    const uint32_t full_leader = cluster_addr(smem_u32(&bars->full[stage]), 0);
+                    if (rank == 0) mbar_arrive_expect_tx(&bars->full[stage], 2 * STAGE_BYTES);   // both CTAs' bytes
+                    tma_load_2d_pair(a_dst, &map_q, ks * TK, q0, full_leader);
+                    tma_load_2d_pair(b_dst, &map_c_half, ks * TK, n0, full_leader);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader only)
+        if (lane == 0 && rank == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            bool ok = true;
+            for (int t = t_begin; t < t_end && ok; ++t) {
+                if (!mbar_wait(&bars->acc_empty[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * TN;
+                for (int ks = 0; ks < k_slabs; ++ks) {
+                    if (!mbar_wait(&bars->full[stage], phase, abort_flag)) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const uint32_t a_addr = smem_u32(tiles + stage * STAGE_BYTES);
+                    const uint64_t da = smem_desc_sw128(a_addr), db = smem_desc_sw128(a_addr + A_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < TK / 16; ++kk)
+                        umma_bf16_pair(d_tmem, da + static_cast<uint64_t>(2 * kk), db + static_cast<uint64_t>(2 * kk), IDESC,
+                                       (ks | kk) ? 1u : 0u);
+                    // stage reusable in BOTH CTAs once these MMAs have read it
+                    umma_commit_both(&bars->empty[stage]);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit_both(&bars->acc_full[acc]);
+                if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5 of both CTAs)
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        TopK<KMAX> top;
+        top.clear();
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        for (int t = t_begin; t < t_end && ok; ++t) {
+            const int n0 = t * TN;
+            if (!mbar_wait(&bars->acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+            tcgen05_fence_after();
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * TN;
+#pragma unroll 1
+            for (int ch = 0; ch < TN / 32; ++ch) {
+                uint32_t r[32];
+                tmem_ld_32x32(taddr + ch * 32, r);
+                const uint32_t live = __ballot_sync(0xFFFFFFFFu, valid[static_cast<int64_t>(n0) + ch * 32 + lane] != 0);
+                if (live == 0u) continue;
+                float m = -INFINITY;
+                if (live == 0xFFFFFFFFu) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) m = fmaxf(m, __uint_as_float(r[j]));
+                } else {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        if (!((live >> j) & 1u)) r[j] = 0xFF800000u;
+                        m = fmaxf(m, __uint_as_float(r[j]));
+                    }
+                }
+                if (m > top.s[KMAX - 1]) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) top.push(__uint_as_float(r[j]), n0 + ch * 32 + j);
+                }
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(cluster_addr(smem_u32(&bars->acc_empty[acc]), 0));
+            if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+        }
+        if (ok && static_cast<int64_t>(q0) + row < B) {
+            unsigned long long *dst = partial + ((static_cast<int64_t>(q0) + row) * splits + split) * KMAX;
+#pragma unroll
+            for (int j = 0; j < KMAX; ++j) dst[j] = top.key(j);
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        if (threadIdx.x == 0) set_status(status, SISO_ERR_TIMEOUT);
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync();          // neither CTA frees tensor memory or exits while the other may still use its memory
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+}  // namespace tc2
+
+template <int KMAX>
+static siso_status_t run_pair(Cache *c, bool *attr_set, const CUtensorMap &map_q, const CUtensorMap &map_c_half, int64_t B,
+                              int tiles_per_split, int n_tiles, int splits, int m_tiles_even, unsigned long long *partial,
+                              cudaStream_t s) {
+    auto kern = tc2::lookup_tensor_pair_kernel<KMAX>;
+    if (!*attr_set) {
+        SISO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::SMEM_BYTES));
+        *attr_set = true;
+    }
+    dim3 grid(m_tiles_even, splits);
+    kern<<<grid, tc2::THREADS, tc2::SMEM_BYTES, s>>>(map_q, map_c_half, c->valid, B, c->dim, tiles_per_split, n_tiles,
+                                                     partial, splits, c->status);
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
+
+// Called by launch_lookup_tensor when the batch spans at least two query tiles.
+siso_status_t launch_lookup_tensor_pair(Cache *c, bool *attr_set3, const CUtensorMap &map_q, const CUtensorMap &map_c_half,
+                                        int64_t B, int kmax, int tiles_per_split, int n_tiles, int splits, int m_tiles_even,
+                                        unsigned long long *partial, cudaStream_t s) {
+    return kmax == 1 ? run_pair<1>(c, attr_set3 + 0, map_q, map_c_half, B, tiles_per_split, n_tiles, splits, m_tiles_even, partial, s)
+         : kmax == 4 ? run_pair<4>(c, attr_set3 + 1, map_q, map_c_half, B, tiles_per_split, n_tiles, splits, m_tiles_even, partial, s)
+                     : run_pair<8>(c, attr_set3 + 2, map_q, map_c_half, B, tiles_per_split, n_tiles, splits, m_tiles_even, partial, s);
+}
+
+}  // namespace siso
