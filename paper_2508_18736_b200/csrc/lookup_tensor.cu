@@ -84,18 +84,28 @@ __device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint
         "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
         ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
 }
-// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp receives row (lane base + i)
+// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp receives row (lane base + i).  The load is
+// asynchronous: the registers hold the data only after tmem_ld_fence() on the same array.
 __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
     asm volatile(
         "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
         "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];\n\t"
-        "tcgen05.wait::ld.sync.aligned;"     // same statement: no use of the registers can be scheduled before the wait
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
         : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
           "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
           "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
           "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
         : "r"(taddr) : "memory");
+}
+// Wait for all tensor-memory loads issued so far.  The registers pass through the statement as in/out operands,
+// so the compiler cannot schedule any use of them before the wait.
+__device__ __forceinline__ void tmem_ld_fence(uint32_t (&r)[32]) {
+    asm volatile("tcgen05.wait::ld.sync.aligned;"
+        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
+          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
+          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
+          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
+        :: "memory");
 }
 
 // Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes and 128-byte swizzled
@@ -211,16 +221,21 @@ lookup_tensor_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         bool ok = true;
         for (int t = t_begin; t < t_end && ok; ++t) {
             const int n0 = t * TN;
+            // live flags of the tile's 256 slots (lane l holds slots l, l+32, ...): fetched before the wait
+            unsigned long long vflags = 0ull;       // bit ch: slot n0 + 32*ch + lane is live
+#pragma unroll
+            for (int ch = 0; ch < TN / 32; ++ch)
+                vflags |= static_cast<unsigned long long>(valid[static_cast<int64_t>(n0) + ch * 32 + lane] != 0) << ch;
             if (!mbar_wait(&bars->acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
             tcgen05_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * TN;
-#pragma unroll 1
-            for (int ch = 0; ch < TN / 32; ++ch) {
-                uint32_t r[32];
-                tmem_ld_32x32(taddr + ch * 32, r);
-                // live mask of these 32 slots: lane l reads the flag of slot l, the ballot shares them
-                const uint32_t live = __ballot_sync(0xFFFFFFFFu, valid[static_cast<int64_t>(n0) + ch * 32 + lane] != 0);
-                if (live == 0u) continue;
+            // two register buffers: while one chunk of 32 columns is scanned the next is in flight from tensor
+            // memory.  The loop stays rolled (two chunks per trip): unrolled eight times the scan code no longer
+            // fits the instruction cache.
+            uint32_t ra[32], rb[32];
+            auto scan = [&](uint32_t (&r)[32], int ch) {
+                const uint32_t live = __ballot_sync(0xFFFFFFFFu, ((vflags >> ch) & 1ull) != 0ull);
+                if (live == 0u) return;
                 float m = -INFINITY;
                 if (live == 0xFFFFFFFFu) {
 #pragma unroll
@@ -236,6 +251,16 @@ lookup_tensor_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
 #pragma unroll
                     for (int j = 0; j < 32; ++j) top.push(__uint_as_float(r[j]), n0 + ch * 32 + j);
                 }
+            };
+            tmem_ld_32x32(taddr, ra);
+#pragma unroll 1
+            for (int ch = 0; ch < TN / 32; ch += 2) {
+                tmem_ld_fence(ra);
+                tmem_ld_32x32(taddr + (ch + 1) * 32, rb);
+                scan(ra, ch);
+                tmem_ld_fence(rb);
+                if (ch + 2 < TN / 32) tmem_ld_32x32(taddr + (ch + 2) * 32, ra);
+                scan(rb, ch + 1);
             }
             tcgen05_fence_before();
             __syncwarp();
