@@ -18,7 +18,7 @@ constexpr int kMaxK = 8;
 constexpr uint32_t kNoSlot = 0xFFFFFFFFu;
 
 // device counters, int64 each
-enum Counter { CNT_OCCUPANCY = 0, CNT_LOOKUPS, CNT_HITS, CNT_INSERTS, CNT_EVICTIONS, CNT_MERGES, CNT_CLOCK, CNT_SPARE, CNT_N };
+enum Counter { CNT_OCCUPANCY = 0, CNT_LOOKUPS, CNT_HITS, CNT_INSERTS, CNT_EVICTIONS, CNT_MERGES, CNT_CLOCK, CNT_SPARE, CNT_SYNC, CNT_N };
 
 struct Cache {
     int64_t capacity;

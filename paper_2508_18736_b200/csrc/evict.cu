@@ -3,12 +3,12 @@
 // Eviction removes the m entries that come first in ascending (cluster_size, access_count,
 // last_access, slot) order.  Sorting the whole cache for a few victims would cost far more than the
 // metadata scan, so the kernels select, exactly, in the manner of a sample sort:
-//   sample   one CTA gathers a strided sample of 1024 live entries and sorts it (bitonic, in
+//   sample   one CTA gathers a strided sample of 256 live entries and sorts it (bitonic, in
 //            shared memory): the sorted sample keys are splitters
 //   bucket   every live entry finds its bucket (number of splitters below its key, binary search)
 //            and the buckets are counted
 //   collect  the smallest bucket index p whose cumulative count reaches m is found from the counts;
-//            entries in buckets <= p (at least m of them, about m + capacity/1024) become candidates
+//            entries in buckets <= p (at least m of them, about m + capacity/256) become candidates
 //   rank     one warp per candidate counts the candidates below it; rank < m means victim number rank
 // Keys are compared as three 64-bit integers (order-preserving image of the fp64 cluster_size, then
 // access_count | last_access | slot), so the order is the exact lexicographic order and total.
@@ -33,7 +33,7 @@ __device__ __forceinline__ Key3 make_key(double size, uint32_t access, unsigned 
     return k;
 }
 
-constexpr int EV_SAMPLE = 1024;
+constexpr int EV_SAMPLE = 256;
 
 struct EvictPlan {
     long long m;             // victims to produce (clamped to the occupancy)
@@ -95,13 +95,12 @@ evict_sample_kernel(long long m_req, const uint8_t *__restrict__ hit, long long 
     const long long m = m_s < occupancy ? m_s : occupancy;
     for (long long r = m + tid; r < n_victims_out; r += 1024) victims[r] = -1;
     if (tid == 0) { plan->m = m; plan->n_cand = 0; }
-    plan->hist[tid] = 0;
-    if (tid == 0) plan->hist[EV_SAMPLE] = 0;
+    if (tid <= EV_SAMPLE) plan->hist[tid] = 0;
     if (m == 0) return;
-    // strided sample: thread t takes the first live slot of window [t*stride, (t+1)*stride), starting at an
-    // offset that changes from call to call (at most 64 probes)
+    // strided sample: thread t < EV_SAMPLE takes the first live slot of window [t*stride, (t+1)*stride), starting
+    // at an offset that changes from call to call (at most 64 probes)
     const long long stride = (capacity + EV_SAMPLE - 1) / EV_SAMPLE;
-    const long long lo = tid * stride, hi = min(capacity, lo + stride);
+    const long long lo = tid * stride, hi = tid < EV_SAMPLE ? min(capacity, lo + stride) : lo;
     const long long span = hi - lo;
     int have = 0;
     Key3 mine;
@@ -115,7 +114,7 @@ evict_sample_kernel(long long m_req, const uint8_t *__restrict__ hit, long long 
             if (valid[sl]) { mine = make_key(size[sl], access[sl], last[sl], static_cast<uint32_t>(sl)); have = 1; break; }
         }
     }
-    k0[tid] = mine.w0; k1[tid] = mine.w1; k2[tid] = mine.w2;
+    if (tid < EV_SAMPLE) { k0[tid] = mine.w0; k1[tid] = mine.w1; k2[tid] = mine.w2; }
     int n_sample;
     block_exclusive_scan_1024(have, &n_sample, warp_sum);
     __syncthreads();
@@ -123,7 +122,7 @@ evict_sample_kernel(long long m_req, const uint8_t *__restrict__ hit, long long 
     for (int k = 2; k <= EV_SAMPLE; k <<= 1) {
         for (int j = k >> 1; j > 0; j >>= 1) {
             const int partner = tid ^ j;
-            if (partner > tid) {
+            if (tid < EV_SAMPLE && partner > tid) {
                 Key3 a, b;
                 a.w0 = k0[tid]; a.w1 = k1[tid]; a.w2 = k2[tid];
                 b.w0 = k0[partner]; b.w1 = k1[partner]; b.w2 = k2[partner];
@@ -136,9 +135,11 @@ evict_sample_kernel(long long m_req, const uint8_t *__restrict__ hit, long long 
             __syncthreads();
         }
     }
-    Key3 out;
-    out.w0 = k0[tid]; out.w1 = k1[tid]; out.w2 = k2[tid];
-    splitters[tid] = out;
+    if (tid < EV_SAMPLE) {
+        Key3 out;
+        out.w0 = k0[tid]; out.w1 = k1[tid]; out.w2 = k2[tid];
+        splitters[tid] = out;
+    }
     if (tid == 0) plan->n_sample = n_sample;
 }
 
@@ -270,7 +271,8 @@ siso_status_t launch_evict(Cache *c, int64_t n_evict, const uint8_t *hit, int64_
                                            c->counters, plan, splitters, victims, victims ? n_victims_out : 0);
     SISO_LAUNCHED(c);
     const int grid = static_cast<int>(std::min<int64_t>((c->capacity + 255) / 256, 4ll * c->sm_count));
-    evict_bucket_kernel<<<grid, 256, 0, s>>>(c->capacity, c->size, c->access, c->last, c->valid, plan, splitters, bucket);
+    const int grid_bucket = static_cast<int>(std::min<int64_t>((c->capacity + 2047) / 2048, 2ll * c->sm_count));
+    evict_bucket_kernel<<<grid_bucket, 256, 0, s>>>(c->capacity, c->size, c->access, c->last, c->valid, plan, splitters, bucket);
     SISO_LAUNCHED(c);
     evict_collect_kernel<<<grid, 256, 0, s>>>(c->capacity, c->size, c->access, c->last, c->valid, plan, bucket, cand);
     SISO_LAUNCHED(c);

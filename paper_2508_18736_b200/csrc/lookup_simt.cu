@@ -59,41 +59,59 @@ lookup_simt_kernel(const T *__restrict__ Q, int64_t B, const T *__restrict__ C, 
     }
 }
 
-// One thread per query: k best of splits*kmax packed keys, then the strict threshold test.
+// One warp per query: the lanes split the splits*kmax packed keys, merge their lists with shuffles, and lane 0
+// writes the k best and applies the strict threshold test.
 template <int KMAX>
-__global__ void topk_finalize_kernel(const unsigned long long *__restrict__ partial, int64_t B, int splits, int k,
-                                     const float *__restrict__ theta, float theta_s, int32_t *__restrict__ idx,
-                                     float *__restrict__ sim, uint8_t *__restrict__ hit, long long *counters) {
-    const int64_t b = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
-    int is_hit = 0;
+__global__ void __launch_bounds__(1024)
+topk_finalize_kernel(const unsigned long long *__restrict__ partial, int64_t B, int splits, int k,
+                     const float *__restrict__ theta, float theta_s, int32_t *__restrict__ idx,
+                     float *__restrict__ sim, uint8_t *__restrict__ hit, long long *counters) {
+    __shared__ int hits_s;
+    if (threadIdx.x == 0) hits_s = 0;
+    __syncthreads();
+    const int lane = threadIdx.x & 31;
+    const int64_t b = static_cast<int64_t>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
     if (b < B) {
         KeyList<KMAX> out;
         out.clear();
         const unsigned long long *src = partial + b * splits * KMAX;
-        for (int s = 0; s < splits * KMAX; ++s) out.insert(src[s]);
+        for (int s = lane; s < splits * KMAX; s += 32) out.insert(src[s]);
 #pragma unroll
-        for (int j = 0; j < KMAX; ++j) {
-            if (j < k) {
-                const unsigned long long key = out.k[j];
-                idx[b * k + j] = key ? key_slot(key) : -1;
-                sim[b * k + j] = key ? key_sim(key) : -INFINITY;
-            }
+        for (int o = 16; o >= 1; o >>= 1) {
+            unsigned long long other[KMAX];
+#pragma unroll
+            for (int j = 0; j < KMAX; ++j) other[j] = __shfl_xor_sync(0xFFFFFFFFu, out.k[j], o);
+#pragma unroll
+            for (int j = 0; j < KMAX; ++j) out.insert(other[j]);
         }
-        const float th = theta ? theta[b] : theta_s;
-        is_hit = (out.k[0] != 0ull && key_sim(out.k[0]) > th) ? 1 : 0;
-        hit[b] = static_cast<uint8_t>(is_hit);
+        if (lane == 0) {
+#pragma unroll
+            for (int j = 0; j < KMAX; ++j) {
+                if (j < k) {
+                    const unsigned long long key = out.k[j];
+                    idx[b * k + j] = key ? key_slot(key) : -1;
+                    sim[b * k + j] = key ? key_sim(key) : -INFINITY;
+                }
+            }
+            const float th = theta ? theta[b] : theta_s;
+            const int is_hit = (out.k[0] != 0ull && key_sim(out.k[0]) > th) ? 1 : 0;
+            hit[b] = static_cast<uint8_t>(is_hit);
+            if (is_hit) atomicAdd(&hits_s, 1);
+        }
     }
-    const unsigned ballot = __ballot_sync(0xFFFFFFFFu, is_hit);
-    if ((threadIdx.x & 31) == 0 && ballot) atomicAdd(reinterpret_cast<unsigned long long *>(counters + CNT_HITS),
-                                                      static_cast<unsigned long long>(__popc(ballot)));
-    if (b == 0) atomicAdd(reinterpret_cast<unsigned long long *>(counters + CNT_LOOKUPS), static_cast<unsigned long long>(B));
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        if (hits_s) atomicAdd(reinterpret_cast<unsigned long long *>(counters + CNT_HITS), static_cast<unsigned long long>(hits_s));
+        if (blockIdx.x == 0) atomicAdd(reinterpret_cast<unsigned long long *>(counters + CNT_LOOKUPS), static_cast<unsigned long long>(B));
+    }
 }
 
 siso_status_t launch_topk_finalize(Cache *c, const unsigned long long *partial, int64_t B, int splits, int kmax, int k,
                                    const float *theta, float theta_s, int32_t *idx, float *sim, uint8_t *hit,
                                    cudaStream_t s) {
-    const int threads = 128;
-    const unsigned blocks = static_cast<unsigned>((B + threads - 1) / threads);
+    const int threads = B >= 4096 ? 1024 : 256;              // one warp per query
+    const int per_block = threads / 32;
+    const unsigned blocks = static_cast<unsigned>((B + per_block - 1) / per_block);
     if (kmax == 1) topk_finalize_kernel<1><<<blocks, threads, 0, s>>>(partial, B, splits, k, theta, theta_s, idx, sim, hit, c->counters);
     else if (kmax == 4) topk_finalize_kernel<4><<<blocks, threads, 0, s>>>(partial, B, splits, k, theta, theta_s, idx, sim, hit, c->counters);
     else topk_finalize_kernel<8><<<blocks, threads, 0, s>>>(partial, B, splits, k, theta, theta_s, idx, sim, hit, c->counters);

@@ -107,9 +107,125 @@ update_apply_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restric
     }
 }
 
+// Small batches (at most UPS_MAX_B rows): one launch.  CTA b looks at row b; it works only if row b is the first
+// hit of its slot in the batch, then collects the later hits of that slot in ascending order (an ordered
+// compaction in shared memory) and applies them exactly like update_apply_kernel.  Every CTA reads the clock
+// before it signs off on a completion counter; the last CTA to sign off advances the clock, so no CTA can
+// see the new value.
+constexpr int UPS_MAX_B = 1024;
+
+template <typename T>
+__global__ void __launch_bounds__(UP_THREADS)
+update_small_kernel(const int32_t *__restrict__ idx, int idx_stride, const uint8_t *__restrict__ hit, int B,
+                    int64_t capacity, int D, const T *__restrict__ Q, float *__restrict__ master, T *__restrict__ vecs,
+                    double *__restrict__ size, uint32_t *__restrict__ access, unsigned long long *__restrict__ last,
+                    const uint8_t *__restrict__ valid, long long *counters, int *status) {
+    extern __shared__ double acc[];          // [D]
+    __shared__ double red[UP_THREADS / 32];
+    __shared__ uint16_t members[UPS_MAX_B];
+    __shared__ int warp_cnt[UP_THREADS / 32];
+    __shared__ long long clock_s;
+    __shared__ int n_members_s;
+    const int b = blockIdx.x, tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (tid == 0) clock_s = counters[CNT_CLOCK];
+    bool work = false;
+    int64_t slot = -1;
+    if (hit[b]) {
+        slot = idx[static_cast<int64_t>(b) * idx_stride];
+        if (slot >= 0 && slot < capacity && valid[slot]) work = true;
+        else if (tid == 0) set_status(status, SISO_ERR_INVALID_ARG);     // a hit must name a live slot; the row is skipped
+    }
+    if (work) {
+        // is an earlier row a hit on the same slot?  then that row's CTA owns the group
+        int earlier = 0;
+        for (int r = tid; r < b; r += UP_THREADS) earlier |= (hit[r] && idx[static_cast<int64_t>(r) * idx_stride] == slot) ? 1 : 0;
+        work = __syncthreads_or(earlier) == 0;
+    }
+    if (work) {
+        // members of the group in ascending row order: rows b.. in chunks of 256, ballot-ordered
+        int base_count = 0;
+        for (int r0 = b; r0 < B; r0 += UP_THREADS) {
+            const int r = r0 + tid;
+            const bool mine = r < B && hit[r] && idx[static_cast<int64_t>(r) * idx_stride] == slot;
+            const unsigned ballot = __ballot_sync(0xFFFFFFFFu, mine);
+            if (lane == 0) warp_cnt[warp] = __popc(ballot);
+            __syncthreads();
+            int before = base_count, total = 0;
+            for (int w = 0; w < UP_THREADS / 32; ++w) { if (w < warp) before += warp_cnt[w]; total += warp_cnt[w]; }
+            if (mine) members[before + __popc(ballot & ((1u << lane) - 1u))] = static_cast<uint16_t>(r);
+            base_count += total;
+            __syncthreads();
+        }
+        if (tid == 0) n_members_s = base_count;
+        const double n_old = size[slot];
+        float *m = master + slot * D;
+        for (int d = tid; d < D; d += UP_THREADS) acc[d] = n_old * static_cast<double>(m[d]);
+        __syncthreads();
+        const int count = n_members_s;
+        const int quads = D / 4;
+        for (int t = 0; t < count; t += 4) {
+            const int nrow = count - t < 4 ? count - t : 4;
+            const T *q[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) q[r] = Q + static_cast<int64_t>(members[t + (r < nrow ? r : 0)]) * D;
+            for (int g = tid; g < quads; g += UP_THREADS) {
+                float4 v[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) v[r] = load4<T>(q[r] + 4 * g);
+                double a0 = acc[4 * g], a1 = acc[4 * g + 1], a2 = acc[4 * g + 2], a3 = acc[4 * g + 3];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    if (r < nrow) { a0 += v[r].x; a1 += v[r].y; a2 += v[r].z; a3 += v[r].w; }
+                }
+                acc[4 * g] = a0; acc[4 * g + 1] = a1; acc[4 * g + 2] = a2; acc[4 * g + 3] = a3;
+            }
+        }
+        __syncthreads();
+        double ss = 0.0;
+        for (int d = tid; d < D; d += UP_THREADS) ss += acc[d] * acc[d];
+        const double norm = sqrt(block_sum_f64(ss, red));
+        T *v = vecs + slot * D;
+        for (int d = tid; d < D; d += UP_THREADS) {
+            const float f = static_cast<float>(acc[d] / norm);
+            m[d] = f;
+            if constexpr (sizeof(T) == 2) v[d] = __float2bfloat16_rn(f);
+        }
+        if (tid == 0) {
+            size[slot] = n_old + static_cast<double>(count);
+            const unsigned long long a = static_cast<unsigned long long>(access[slot]) + static_cast<unsigned long long>(count);
+            access[slot] = (access[slot] == SISO_ACCESS_INF || a >= SISO_ACCESS_INF) ? SISO_ACCESS_INF : static_cast<uint32_t>(a);
+            last[slot] = static_cast<unsigned long long>(clock_s + 1);
+        }
+    }
+    // sign off; the last CTA advances the clock (every CTA has read it by then) and re-arms the counter
+    __syncthreads();
+    if (tid == 0) {
+        __threadfence();
+        const unsigned long long done = atomicAdd(reinterpret_cast<unsigned long long *>(counters + CNT_SYNC), 1ull);
+        if (done == gridDim.x - 1) {
+            counters[CNT_CLOCK] = clock_s + 1;
+            counters[CNT_SYNC] = 0;
+        }
+    }
+}
+
 siso_status_t launch_update(Cache *c, const void *q, int64_t B, const int32_t *idx, int idx_stride, const uint8_t *hit,
                             cudaStream_t s) {
     if (B >= (1ll << 31)) return SISO_ERR_UNSUPPORTED;
+    if (B >= 1 && B <= UPS_MAX_B) {
+        const size_t smem_small = sizeof(double) * c->dim;
+        if (c->dtype == SISO_F32)
+            update_small_kernel<float><<<static_cast<unsigned>(B), UP_THREADS, smem_small, s>>>(
+                idx, idx_stride, hit, static_cast<int>(B), c->capacity, c->dim, static_cast<const float *>(q), c->master,
+                static_cast<float *>(c->vecs), c->size, c->access, c->last, c->valid, c->counters, c->status);
+        else
+            update_small_kernel<__nv_bfloat16><<<static_cast<unsigned>(B), UP_THREADS, smem_small, s>>>(
+                idx, idx_stride, hit, static_cast<int>(B), c->capacity, c->dim, static_cast<const __nv_bfloat16 *>(q),
+                c->master, static_cast<__nv_bfloat16 *>(c->vecs), c->size, c->access, c->last, c->valid, c->counters,
+                c->status);
+        SISO_LAUNCHED(c);
+        return SISO_OK;
+    }
     Scratch scr;
     const size_t need = 4 * pad256(sizeof(uint32_t) * B) + sort_pairs_scratch_bytes(B);
     SISO_TRY(scratch_reserve(c, need, s, &scr));
