@@ -40,6 +40,10 @@ def parse_args():
     ap.add_argument("--rows", type=int, default=1 << 20, help="cached centroids (default: the full 1,048,576)")
     ap.add_argument("--queries", type=int, default=8192, help="query batch per step")
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor", "stream"])
+    ap.add_argument("--workload", default="config4",
+                    choices=["config4", "config1", "config2", "config3", "config5", "stream_probe"],
+                    help="config4 (default) is the benchmark contract; the others print one line each for the other "
+                         "configurations (single GPU only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -312,10 +316,147 @@ def run_ours(args):
     return 0
 
 
+# ------------------------------------------------------------------------------ the other configurations
+def run_other(args):
+    """One JSON line for configuration 1, 2, 3, 5 or the small-batch streaming probe (single GPU, device-resident)."""
+    import torch
+    from paper_2508_18736_b200 import build as _b
+    _b.build()
+    import paper_2508_18736_b200 as siso
+    from gen import workloads as W
+    peaks, peak_kind = load_peaks()
+    cores = os.cpu_count() or 1
+    dev = torch.device("cuda", 0)
+    torch.cuda.set_device(0)
+
+    def to_dev(a, dtype):
+        if dtype == "bf16":
+            return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+        return torch.from_numpy(a).to(dev)
+
+    def fill(cache, cent, dtype):
+        for lo in range(0, cent.shape[0], 1 << 16):
+            cache.insert(to_dev(cent[lo:lo + (1 << 16)], dtype))
+        cache.check_status()
+
+    def time_ms(fn, steps, warm):
+        for _ in range(warm):
+            fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(steps):
+            fn()
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / steps
+
+    steps, warm = args.steps, max(3, args.warmup)
+    line = {"workload": args.workload, "n_gpus": 1, "steps": steps, "warmup": warm, "data": "synthetic",
+            "peaks": peak_kind}
+    fp32_peak = 148 * 128 * 2 * 1.965e9 / 1e12            # FFMA lanes x 2 flop x max SM clock
+    if args.workload == "config1":
+        w = W.config(1)
+        cache = siso.SisoCache(1024, 384, "f32")
+        fill(cache, w.centroids, "f32")
+        q = to_dev(w.queries, "f32")
+        ms = time_ms(lambda: cache.lookup(q, 0.85, 1), steps, warm)
+        fl = 2.0 * 4096 * 1024 * 384
+        line.update(metric="lookup queries/s, 1,024 x 384 fp32, batch 4,096", value=4096 / ms * 1e3, unit=UNIT,
+                    ms_per_step=ms, dtype="f32",
+                    roofline={"bound": "alu", "achieved": fl / ms / 1e9, "peak": fp32_peak, "unit": "TFLOP/s",
+                              "frac": fl / ms / 1e9 / fp32_peak, "peak_kind": "derived: 148 SMs x 128 FFMA lanes x 2 x 1.965 GHz"})
+    elif args.workload == "config2":
+        w = W.config(2, threads=cores)
+        cache = siso.SisoCache(65536, 768, "bf16")
+        fill(cache, w.centroids, "bf16")
+        q, th = to_dev(w.queries, "bf16"), torch.from_numpy(w.theta).to(dev)
+        ms_l = time_ms(lambda: cache.lookup(q, th, 1), steps, warm)
+        idx, sim, hit = cache.lookup(q, th, 1)
+        ms_u = time_ms(lambda: cache.update(q, idx, hit), max(3, steps // 4), 1)
+        fl = 2.0 * 65536 * 65536 * 768
+        line.update(metric="lookup + update queries/s, 65,536 x 768 bf16, batch 65,536", value=65536 / (ms_l + ms_u) * 1e3,
+                    unit=UNIT, ms_per_step=ms_l + ms_u, lookup_ms=ms_l, update_ms=ms_u, dtype="bf16",
+                    hit_ratio=float(hit.float().mean().item()),
+                    roofline={"bound": "tensor", "achieved": fl / ms_l / 1e9, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                              "frac": fl / ms_l / 1e9 / peaks["bf16_tflops"], "kernel": "lookup only"})
+    elif args.workload == "config3":
+        w = W.config(3, threads=cores)
+        cache = siso.SisoCache(32768, 768, "f32")
+        fill(cache, w.centroids, "f32")
+        st = cache.export()
+        times, merged = [], None
+        for _ in range(max(3, steps // 4)):
+            cache.import_(st["master"], st["size"], st["access"], st["last"], st["valid"], 0)
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            _, merged = cache.merge(W.MERGE_THRESHOLD_CONFIG3, siso.MERGE_WEIGHTED_MEAN)
+            e1.record()
+            torch.cuda.synchronize()
+            times.append(e0.elapsed_time(e1))
+        ms = statistics.median(times)
+        fl = 32768.0 * 32767 / 2 * 768 * 2
+        line.update(metric="self-merge pass, 32,768 x 768 fp32, theta_C 0.90, weighted mean", value=32768 / ms * 1e3,
+                    unit="centroids/s", ms_per_step=ms, merged=merged, survivors=cache.stats()["occupancy"], dtype="f32",
+                    roofline={"bound": "alu", "achieved": fl / ms / 1e9, "peak": fp32_peak, "unit": "TFLOP/s",
+                              "frac": fl / ms / 1e9 / fp32_peak, "peak_kind": "derived: 148 SMs x 128 FFMA lanes x 2 x 1.965 GHz"})
+    elif args.workload == "config5":
+        sp = W.StreamSpec()
+        stream = W.QueryStream(sp, threads=cores)
+        n_warm, n_timed = 600, min(4000, max(500, steps * 100))
+        q_all = to_dev(stream.block(0, n_warm + n_timed, threads=cores), "bf16")
+        cache = siso.SisoCache(sp.capacity, sp.dim, "bf16")
+        # the stream starts on an empty cache; to time the steady state (full cache, evicting every batch) the cache
+        # is first filled with later queries of the same stream
+        fill(cache, stream.block(20000, 20000 + (sp.capacity - 2048) // sp.batch, threads=cores), "bf16")
+        out = None
+        for t in range(n_warm):
+            out = cache.stream_step(q_all[t * 256:(t + 1) * 256], float(sp.theta), out=out)
+        torch.cuda.synchronize()
+        s0, l0 = cache.stats(), cache.launch_count
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for t in range(n_warm, n_warm + n_timed):
+            out = cache.stream_step(q_all[t * 256:(t + 1) * 256], float(sp.theta), out=out)
+        e1.record()
+        torch.cuda.synchronize()
+        cache.check_status()
+        s1 = cache.stats()
+        us = e0.elapsed_time(e1) / n_timed * 1e3
+        gbs = sp.capacity * sp.dim * 2 / (us * 1e-6) / 1e9
+        line.update(metric="streaming cache queries/s, 262,144 x 768 bf16, micro-batches of 256 (lookup, update, evict, insert)",
+                    value=256 / us * 1e6, unit=UNIT, us_per_batch=us, batches_timed=n_timed, dtype="bf16",
+                    hit_ratio=(s1["hits"] - s0["hits"]) / (256.0 * n_timed), evictions=s1["evictions"] - s0["evictions"],
+                    inserts=s1["inserts"] - s0["inserts"], gpu_launches=cache.launch_count - l0,
+                    roofline={"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                              "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                              "note": "384 MiB of centroids per batch over the whole step time"})
+    else:   # stream_probe
+        rows = []
+        for (N, D) in ((1 << 20, 1024), (262144, 768)):
+            cache = siso.SisoCache(N, D, "bf16")
+            w = W.config(4, threads=cores, n_centroids=N, dim=D, n_queries=256, n_clusters=max(64, N // 16))
+            fill(cache, w.centroids, "bf16")
+            for B in (1, 2, 4, 8, 16, 32, 64, 128, 256):
+                q = to_dev(w.queries[:B], "bf16")
+                ms = time_ms(lambda: cache.lookup(q, 0.86, 1), steps, warm)
+                gbs = N * D * 2 / ms / 1e6
+                rows.append({"rows": N, "dim": D, "batch": B, "us": ms * 1e3, "GB/s": gbs, "frac": gbs / peaks["hbm_gbs"]})
+            cache.close()
+        line.update(metric="small-batch lookup: centroid bytes per second", unit="GB/s", rows=rows, dtype="bf16",
+                    value=max(r["GB/s"] for r in rows),
+                    roofline={"bound": "hbm", "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                              "achieved": max(r["GB/s"] for r in rows), "frac": max(r["frac"] for r in rows)})
+    print(json.dumps(line), flush=True)
+    return 0
+
+
 def main():
     args = parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.workload != "config4":
+        return run_other(args)
     return run_ours(args)
 
 
