@@ -273,12 +273,12 @@ def run_ours(args):
     flops = 2.0 * B * args.rows * 1024
     kernel_ms = statistics.median(per_step)           # the sweep kernel plus its small finalize kernel
     achieved = flops / (kernel_ms * 1e-3) / 1e12
-    # DRAM bytes per launch from the committed ncu capture of this kernel (profiles/lookup_tensor_small_case_full_set.txt:
-    # 274 MB read + 6 MB written at 131,072 rows x 2,048 queries), scaled with rows and queries; only for the
-    # tensor-core kernel as profiled
+    # DRAM bytes per launch of the dominant kernel, from the committed one-pass ncu capture of this very command
+    # (profiles/lookup_tensor_config4_launches.txt: 5.74e9 / 6.51e9 read, 1.3e7 / 1.0e7 written in two launches);
+    # only known for the full-size workload on the tensor-core kernel as profiled
     traffic = None
-    if args.path in ("auto", "tensor"):
-        traffic = 273.9e6 * (args.rows / 131072.0) * (268.4 / 272.6) + 273.9e6 * (B / 2048.0) * (4.2 / 272.6) + 6.0e6 * (B / 2048.0)
+    if args.path in ("auto", "tensor") and args.rows == (1 << 20) and B == 8192:
+        traffic = 0.5 * (5738814976 + 6508273664) + 0.5 * (12964608 + 10215168)
     roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": achieved / peaks["bf16_tflops"], "traffic": traffic, "peak_kind": f"{peak_kind}, burst",
                 "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
