@@ -433,7 +433,8 @@ def run_other(args):
                               "note": "384 MiB of centroids per batch over the whole step time"})
     else:   # stream_probe
         rows = []
-        for (N, D) in ((1 << 20, 1024), (262144, 768)):
+        # the two stated matrices; an explicit --rows probes that many rows x 1024 only (small profiler captures)
+        for (N, D) in (((1 << 20, 1024), (262144, 768)) if args.rows == (1 << 20) else ((args.rows, 1024),)):
             cache = siso.SisoCache(N, D, "bf16")
             w = W.config(4, threads=cores, n_centroids=N, dim=D, n_queries=256, n_clusters=max(64, N // 16))
             fill(cache, w.centroids, "bf16")
