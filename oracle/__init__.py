@@ -52,6 +52,12 @@ def lib():
         L.siso_oracle_evict.restype = i64
         L.siso_oracle_insert.argtypes = [vp, vp, vp, vp, vp, i64, i32, vp, i32, i64, vp, vp, ctypes.c_uint64, vp]
         L.siso_oracle_insert.restype = i64
+        L.siso_oracle_t2h.argtypes = [vp, i64, vp, i32, vp, vp]
+        L.siso_oracle_t2h.restype = None
+        L.siso_oracle_md1_wait.argtypes = [f64, f64, f64]
+        L.siso_oracle_md1_wait.restype = f64
+        L.siso_oracle_choose_theta.argtypes = [vp, vp, i32, f64, f64, f64, ctypes.POINTER(f64)]
+        L.siso_oracle_choose_theta.restype = i32
         _lib = L
     return _lib
 
@@ -106,6 +112,30 @@ def lookup(centroids: np.ndarray, queries: np.ndarray, theta, k: int = 1, valid:
     if rc:
         raise RuntimeError(f"oracle lookup failed ({rc})")
     return idx, sim, hit
+
+
+def t2h_table(best_sims: np.ndarray, thetas: np.ndarray):
+    """Threshold-to-hit-ratio table of Sec. 4.3: (hits int64 [T], ratio fp64 [T]) for a grid of thresholds."""
+    b = _c(np.asarray(best_sims, dtype=np.float64))
+    th = _c(np.asarray(thetas, dtype=np.float32))
+    hits = np.empty(th.shape[0], dtype=np.int64)
+    ratio = np.empty(th.shape[0], dtype=np.float64)
+    lib().siso_oracle_t2h(_p(b), b.shape[0], _p(th), th.shape[0], _p(hits), _p(ratio))
+    return hits, ratio
+
+
+def md1_wait(L: float, lam: float, h: float) -> float:
+    """Eq. 2: W = L(1-h) + lam L^2 (1-h)^2 / (2 (1 - lam L (1-h))); inf when lam L (1-h) >= 1."""
+    return float(lib().siso_oracle_md1_wait(float(L), float(lam), float(h)))
+
+
+def choose_theta(thetas: np.ndarray, ratio: np.ndarray, L: float, lam: float, slo: float):
+    """Index of the highest threshold with W < slo (or -1), and that W."""
+    th = _c(np.asarray(thetas, dtype=np.float32))
+    r = _c(np.asarray(ratio, dtype=np.float64))
+    w = ctypes.c_double(0.0)
+    i = lib().siso_oracle_choose_theta(_p(th), _p(r), th.shape[0], float(L), float(lam), float(slo), ctypes.byref(w))
+    return int(i), float(w.value)
 
 
 class OracleCache:

@@ -316,3 +316,43 @@ int64_t siso_oracle_insert(double *master, double *size, uint32_t *access, uint6
     }
     return n_ins;
 }
+
+/* ---------------------------------------------------------------------------
+ * Threshold control (Sec. 4.3, "Adjusting theta_R to meet SLO").
+ *
+ * T2H table: for each threshold of a grid, the hit ratio of a sample of queries,
+ * h(theta) = #{queries whose best similarity > theta} / n  (the same strict test
+ * as lookup).  best[] holds the best similarity of each sampled query.
+ * ------------------------------------------------------------------------- */
+void siso_oracle_t2h(const double *best, int64_t n, const float *thetas, int n_thetas, int64_t *hits, double *ratio) {
+    for (int t = 0; t < n_thetas; ++t) {
+        int64_t c = 0;
+        for (int64_t i = 0; i < n; ++i) c += (best[i] > (double)thetas[t]) ? 1 : 0;
+        hits[t] = c;
+        ratio[t] = n > 0 ? (double)c / (double)n : 0.0;
+    }
+}
+
+/* Eq. 1 with E = L (1 - h) (Eq. 2): mean waiting time of the M/D/1 queue,
+ *     W = E + lambda E^2 / (2 (1 - lambda E)),
+ * +infinity when the queue is not stable (lambda E >= 1). */
+double siso_oracle_md1_wait(double L, double lambda, double h) {
+    double E = L * (1.0 - h);
+    double rho = lambda * E;
+    if (rho >= 1.0) return INFINITY;
+    return E + lambda * E * E / (2.0 * (1.0 - rho));
+}
+
+/* The highest threshold of the table whose estimated W is below the SLO S
+ * ("find the highest theta_R ... that satisfies S > W").  Returns its index,
+ * or -1 if no entry qualifies.  W of the chosen entry goes to *w_out. */
+int siso_oracle_choose_theta(const float *thetas, const double *ratio, int n_thetas, double L, double lambda,
+                             double slo, double *w_out) {
+    int best = -1;
+    for (int t = 0; t < n_thetas; ++t) {
+        double W = siso_oracle_md1_wait(L, lambda, ratio[t]);
+        if (W < slo && (best < 0 || thetas[t] > thetas[best])) best = t;
+    }
+    if (w_out) *w_out = best >= 0 ? siso_oracle_md1_wait(L, lambda, ratio[best]) : INFINITY;
+    return best;
+}
