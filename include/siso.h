@@ -192,6 +192,27 @@ siso_status_t siso_lookup_small_noalloc(const void *d_centroids, const uint8_t *
                                         const float *d_theta, float theta_scalar, int32_t k, int32_t *d_idx,
                                         float *d_sim, uint8_t *d_hit, void *stream);
 
+/* Threshold control (Sec. 4.3, the part on adjusting theta_R to meet the SLO).
+ * siso_t2h builds the threshold-to-hit-ratio table: it looks up a sample of queries (k = 1, exact, no hit is
+ * recorded in the statistics) and counts, for every threshold of the grid, the queries whose best similarity
+ * is strictly above it.  d_queries [n_queries, dim] in the cache dtype; d_thetas [n_thetas] fp32 (the paper
+ * sweeps 0.98 down to 0.6; at most 1024 values); d_hits [n_thetas] int64 receives the counts (hit ratio =
+ * count / n_queries).  Asynchronous on `stream`. */
+siso_status_t siso_t2h(siso_cache_t *c, const void *d_queries, int64_t n_queries, const float *d_thetas,
+                       int32_t n_thetas, int64_t *d_hits, void *stream);
+/* Eq. 1 with E = L (1 - h) (Eq. 2): mean waiting time of the M/D/1 queue in front of the LLM,
+ * W = E + lambda E^2 / (2 (1 - lambda E)); +infinity if lambda E >= 1.  Host arithmetic only. */
+double siso_md1_wait(double llm_latency, double arrival_rate, double hit_ratio);
+/* Index of the highest threshold of the table whose W is below the SLO (strictly), or -1; *h_wait_out (may be
+ * NULL) receives that W.  Host arrays. */
+int32_t siso_choose_theta(const float *h_thetas, const double *h_hit_ratio, int32_t n_thetas, double llm_latency,
+                          double arrival_rate, double slo, double *h_wait_out);
+/* Correction step of Sec. 4.3: if the measured waiting time differs from the estimate by more than 10 % (relative to
+ * the measured one), move to the next lower threshold of the table when the measured time is the longer one,
+ * to the next higher when it is the shorter; otherwise, or if there is no such entry, keep `chosen`. */
+int32_t siso_correct_theta(const float *h_thetas, int32_t n_thetas, int32_t chosen, double wait_estimated,
+                           double wait_measured);
+
 /* Copy the state out (checkpoint, parity checks).  Any pointer may be NULL.
  *   d_vecs   [capacity, dim] lookup copy in the cache dtype     d_master [capacity, dim] fp32 master
  *   d_sizes  [capacity] fp64   d_access [capacity] u32   d_last [capacity] u64   d_valid [capacity] u8 */

@@ -58,6 +58,8 @@ def lib():
         L.siso_oracle_md1_wait.restype = f64
         L.siso_oracle_choose_theta.argtypes = [vp, vp, i32, f64, f64, f64, ctypes.POINTER(f64)]
         L.siso_oracle_choose_theta.restype = i32
+        L.siso_oracle_correct_theta.argtypes = [vp, i32, i32, f64, f64]
+        L.siso_oracle_correct_theta.restype = i32
         _lib = L
     return _lib
 
@@ -136,6 +138,12 @@ def choose_theta(thetas: np.ndarray, ratio: np.ndarray, L: float, lam: float, sl
     w = ctypes.c_double(0.0)
     i = lib().siso_oracle_choose_theta(_p(th), _p(r), th.shape[0], float(L), float(lam), float(slo), ctypes.byref(w))
     return int(i), float(w.value)
+
+
+def correct_theta(thetas: np.ndarray, chosen: int, w_est: float, w_meas: float) -> int:
+    """Sec. 4.3 correction: one table entry down (measured wait longer) or up (shorter) if they differ by > 10 %."""
+    th = _c(np.asarray(thetas, dtype=np.float32))
+    return int(lib().siso_oracle_correct_theta(_p(th), th.shape[0], int(chosen), float(w_est), float(w_meas)))
 
 
 class OracleCache:

@@ -356,3 +356,19 @@ int siso_oracle_choose_theta(const float *thetas, const double *ratio, int n_the
     if (w_out) *w_out = best >= 0 ? siso_oracle_md1_wait(L, lambda, ratio[best]) : INFINITY;
     return best;
 }
+
+/* Correction step of Sec. 4.3: when the estimate W and the measured W' differ by more than 10 % (of W'), theta_R
+ * moves one table entry further: down if W' is the longer (less traffic to the LLM), up if it is the shorter. */
+int siso_oracle_correct_theta(const float *thetas, int n_thetas, int chosen, double w_est, double w_meas) {
+    if (chosen < 0 || chosen >= n_thetas || !(w_meas > 0.0)) return chosen;
+    if (fabs(w_est - w_meas) / w_meas <= 0.10) return chosen;
+    int next = -1;
+    for (int t = 0; t < n_thetas; ++t) {
+        if (w_meas > w_est) {            /* next lower threshold */
+            if (thetas[t] < thetas[chosen] && (next < 0 || thetas[t] > thetas[next])) next = t;
+        } else {                          /* next higher threshold */
+            if (thetas[t] > thetas[chosen] && (next < 0 || thetas[t] < thetas[next])) next = t;
+        }
+    }
+    return next < 0 ? chosen : next;
+}

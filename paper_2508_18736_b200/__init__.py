@@ -4,7 +4,7 @@ MergeCentroids / FilteringCentroids and spare-space insertion, behind the C ABI 
 ``include/siso.h``.  This package is the thin Python binding: it marshals torch tensors to
 pointers and calls ``libsiso.so``; every step runs in the library's own CUDA kernels."""
 from .binding import (ACCESS_INF, EVICT_DECAY, MERGE_SIZES_ONLY, MERGE_WEIGHTED_MEAN, PATH_AUTO, PATH_SIMT,
-                      PATH_STREAM, PATH_TENSOR, SisoCache, SisoError, load_library, lookup_small_noalloc)
+                      PATH_STREAM, PATH_TENSOR, SisoCache, SisoError, load_library, lookup_small_noalloc, md1_wait, choose_theta, correct_theta)
 
-__all__ = ["SisoCache", "SisoError", "load_library", "lookup_small_noalloc", "ACCESS_INF", "EVICT_DECAY", "MERGE_SIZES_ONLY",
+__all__ = ["SisoCache", "SisoError", "load_library", "lookup_small_noalloc", "md1_wait", "choose_theta", "correct_theta", "ACCESS_INF", "EVICT_DECAY", "MERGE_SIZES_ONLY",
            "MERGE_WEIGHTED_MEAN", "PATH_AUTO", "PATH_SIMT", "PATH_STREAM", "PATH_TENSOR"]

@@ -21,7 +21,8 @@ _STATUS_NAMES = {0: "SISO_OK", 1: "SISO_ERR_INVALID_ARG", 2: "SISO_ERR_UNSUPPORT
 EXPORTS = ["siso_cache_create", "siso_cache_destroy", "siso_set_option", "siso_insert", "siso_lookup",
            "siso_lookup_host", "siso_update", "siso_merge", "siso_evict", "siso_make_room", "siso_insert_misses",
            "siso_stream_step", "siso_export", "siso_import", "siso_get_stats", "siso_sync_status",
-           "siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_lookup_small_noalloc"]
+           "siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_lookup_small_noalloc", "siso_t2h", "siso_md1_wait",
+           "siso_choose_theta", "siso_correct_theta"]
 
 
 class SisoError(RuntimeError):
@@ -72,6 +73,12 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_insert_misses.argtypes = [vp, vp, i64, vp, vp, vp]
     L.siso_stream_step.argtypes = [vp, vp, i64, vp, f32, vp, vp, vp, vp, vp, vp]
     L.siso_lookup_small_noalloc.argtypes = [vp, vp, i64, i32, i32, vp, i64, vp, f32, i32, vp, vp, vp, vp]
+    L.siso_t2h.argtypes = [vp, vp, i64, vp, i32, vp, vp]
+    L.siso_md1_wait.argtypes = [ctypes.c_double] * 3
+    L.siso_md1_wait.restype = ctypes.c_double
+    L.siso_choose_theta.argtypes = [vp, vp, i32, ctypes.c_double, ctypes.c_double, ctypes.c_double,
+                                    ctypes.POINTER(ctypes.c_double)]
+    L.siso_correct_theta.argtypes = [vp, i32, i32, ctypes.c_double, ctypes.c_double]
     L.siso_export.argtypes = [vp, vp, vp, vp, vp, vp, vp, vp]
     L.siso_import.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_uint64, vp]
     L.siso_get_stats.argtypes = [vp, ctypes.POINTER(i64), vp]
@@ -83,7 +90,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_last_cuda_error.argtypes = []
     L.siso_last_cuda_error.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name not in ("siso_launch_count", "siso_status_string", "siso_last_cuda_error"):
+        if name not in ("siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_md1_wait"):
             getattr(L, name).restype = i32
     if path is None:
         _lib = L
@@ -250,6 +257,15 @@ class SisoCache:
                                                _ptr(victims), _ptr(slots), _stream(stream)), "siso_stream_step")
         return out
 
+    def t2h(self, queries: torch.Tensor, thetas: torch.Tensor, stream=None) -> torch.Tensor:
+        """Threshold-to-hit-ratio counts: int64 [len(thetas)] = sampled queries whose best similarity > theta."""
+        q = self._vec(queries, "queries")
+        th = thetas.to(device=self._dev, dtype=torch.float32).contiguous()
+        hits = self._new((th.numel(),), torch.int64)
+        self._check(self._lib.siso_t2h(self._h, _ptr(q), q.shape[0], _ptr(th), th.numel(), _ptr(hits), _stream(stream)),
+                    "siso_t2h")
+        return hits
+
     def export(self, stream=None) -> dict:
         out = dict(vecs=self._new((self.capacity, self.dim), self.torch_dtype),
                    master=self._new((self.capacity, self.dim), torch.float32),
@@ -307,3 +323,24 @@ def lookup_small_noalloc(centroids: torch.Tensor, queries: torch.Tensor, theta, 
                                          _ptr(hit), _stream(stream))
     if st != 0:
         raise SisoError(st, "siso_lookup_small_noalloc", L.siso_last_cuda_error().decode() if st == 7 else "")
+
+
+def md1_wait(llm_latency: float, arrival_rate: float, hit_ratio: float) -> float:
+    """Eq. 2 of the paper (M/D/1 mean waiting time with E = L(1 - h)); host arithmetic in the library."""
+    return float(load_library().siso_md1_wait(float(llm_latency), float(arrival_rate), float(hit_ratio)))
+
+
+def choose_theta(thetas, hit_ratio, llm_latency: float, arrival_rate: float, slo: float):
+    """(index of the highest threshold whose estimated wait is below the SLO or -1, that wait)."""
+    th = (ctypes.c_float * len(thetas))(*[float(x) for x in thetas])
+    hr = (ctypes.c_double * len(hit_ratio))(*[float(x) for x in hit_ratio])
+    w = ctypes.c_double(0.0)
+    i = load_library().siso_choose_theta(th, hr, len(thetas), float(llm_latency), float(arrival_rate), float(slo),
+                                         ctypes.byref(w))
+    return int(i), float(w.value)
+
+
+def correct_theta(thetas, chosen: int, wait_estimated: float, wait_measured: float) -> int:
+    """One table entry down/up when estimate and measurement differ by more than 10 % (Sec. 4.3)."""
+    th = (ctypes.c_float * len(thetas))(*[float(x) for x in thetas])
+    return int(load_library().siso_correct_theta(th, len(thetas), int(chosen), float(wait_estimated), float(wait_measured)))

@@ -56,3 +56,33 @@ def test_choose_theta_takes_the_highest_threshold_that_meets_the_slo():
     p = np.array([3, 0, 4, 2, 1])
     i, _ = oracle.choose_theta(thetas[p], ratio[p], L, lam, 11.0)
     assert thetas[p][i] == np.float32(0.8)
+
+
+def test_correction_step_moves_one_entry_when_estimate_is_off_by_more_than_ten_percent():
+    thetas = np.array([0.9, 0.98, 0.8, 0.7], dtype=np.float32)          # unordered on purpose
+    assert oracle.correct_theta(thetas, 0, 10.0, 10.9) == 0             # |10 - 10.9| / 10.9 = 8 %: keep
+    assert oracle.correct_theta(thetas, 0, 10.0, 12.0) == 2             # measured longer: next lower threshold (0.8)
+    assert oracle.correct_theta(thetas, 0, 10.0, 8.0) == 1              # measured shorter: next higher (0.98)
+    assert oracle.correct_theta(thetas, 3, 10.0, 20.0) == 3             # already the lowest entry
+    assert oracle.correct_theta(thetas, 1, 10.0, 5.0) == 1              # already the highest entry
+
+
+def test_library_host_functions_equal_the_oracle():
+    """The library's scalar threshold-control functions need no GPU: compare them with the oracle here."""
+    import paper_2508_18736_b200 as siso
+    from paper_2508_18736_b200 import build
+    build.build()
+    rng = np.random.default_rng(3)
+    thetas = np.round(np.arange(0.98, 0.59, -0.02), 2).astype(np.float32)
+    for _ in range(200):
+        ratio = np.sort(rng.random(20))
+        L, lam, slo = rng.uniform(0.5, 15), rng.uniform(0.0, 0.5), rng.uniform(0.5, 30)
+        for h in ratio[::5]:
+            a, b = siso.md1_wait(L, lam, h), oracle.md1_wait(L, lam, h)
+            assert a == b or abs(a - b) <= 1e-12 * abs(b)
+        gi, gw = siso.choose_theta(thetas, ratio, L, lam, slo)
+        oi, ow = oracle.choose_theta(thetas, ratio, L, lam, slo)
+        assert gi == oi and (gw == ow or abs(gw - ow) <= 1e-12 * abs(ow))
+        c = int(rng.integers(0, 20))
+        w_est, w_meas = rng.uniform(1, 20), rng.uniform(1, 20)
+        assert siso.correct_theta(thetas, c, w_est, w_meas) == oracle.correct_theta(thetas, c, w_est, w_meas)
