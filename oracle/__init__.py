@@ -46,7 +46,7 @@ def lib():
         L.siso_oracle_lookup.restype = i32
         L.siso_oracle_update.argtypes = [vp, vp, vp, vp, vp, i64, i32, vp, i32, i64, vp, i64, vp, ctypes.c_uint64]
         L.siso_oracle_update.restype = i32
-        L.siso_oracle_merge.argtypes = [vp, vp, vp, vp, i64, i32, i64, f64, i32, i32, vp]
+        L.siso_oracle_merge.argtypes = [vp, vp, vp, vp, i64, i32, vp, f64, i32, i32, vp]
         L.siso_oracle_merge.restype = i64
         L.siso_oracle_evict.argtypes = [vp, vp, vp, vp, i64, i64, i32, f64, vp]
         L.siso_oracle_evict.restype = i64
@@ -194,11 +194,16 @@ class OracleCache:
         if rc:
             raise RuntimeError(f"oracle update failed ({rc})")
 
-    def merge(self, theta_c: float, weighted_mean: bool, n_seed: int = 0, new_access_inf: bool = False):
-        """MergeCentroids over the slot array (n_seed = 0: self-merge).  Returns (merge_map, n_merged)."""
+    def merge(self, theta_c: float, weighted_mean: bool, n_seed: int = 0, new_access_inf: bool = False,
+              seed_mask=None):
+        """MergeCentroids over the slot array.  Seeds (C_cur) are the slots below n_seed, or those set in
+        seed_mask; none = self-merge.  Returns (merge_map, n_merged)."""
         mm = np.empty(self.capacity, dtype=np.int32)
+        if seed_mask is None and n_seed > 0:
+            seed_mask = (np.arange(self.capacity) < n_seed)
+        sm = None if seed_mask is None else _c(np.asarray(seed_mask).astype(np.uint8))
         n = lib().siso_oracle_merge(_p(self.master), _p(self.size), _p(self.access), _p(self.valid), self.capacity,
-                                    self.dim, int(n_seed), float(theta_c), int(weighted_mean), int(new_access_inf),
+                                    self.dim, _p(sm), float(theta_c), int(weighted_mean), int(new_access_inf),
                                     _p(mm))
         if n < 0:
             raise MemoryError

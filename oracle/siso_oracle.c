@@ -174,23 +174,24 @@ int siso_oracle_update(double *master, double *size, uint32_t *access, uint64_t 
 }
 
 /* ---------------------------------------------------------------------------
- * O3  MergeCentroids over one slot array.  Slots [0, n_seed) that are valid form
- * C_cur: they are survivors unconditionally and are never compared with each
- * other.  Valid slots i >= n_seed are the repository entries, taken in ascending
+ * O3  MergeCentroids over one slot array.  Valid slots whose seed_mask is set form
+ * C_cur: they are survivors unconditionally, are never compared with each other and
+ * head the survivor list in ascending slot order.  The other valid slots are the
+ * repository entries, taken in ascending slot
  * i: find the closest current survivor (largest dot product with the survivor's
  * vector AS IT WAS AT ENTRY; ties to the earliest survivor); if that similarity
  * is > theta_c the entry joins it (merge_map[i] = survivor, survivor's size grows
  * by the entry's size at entry, the entry's slot becomes invalid), otherwise the
- * entry becomes a survivor itself.  n_seed = 0 is the self-merge of one set.
+ * entry becomes a survivor itself.  seed_mask = NULL is the self-merge of one set.
  * After the pass, with weighted_mean != 0, each survivor's vector becomes
- * normalise(sum over its members m in ascending slot of size_m(entry)*c_m(entry)),
- * the survivor itself being its first member; otherwise vectors are untouched.
- * new_access_inf != 0 sets access = infinity for survivors with i >= n_seed
+ * normalise(size_s(entry)*c_s(entry) + sum over its other members m in ascending slot of
+ * size_m(entry)*c_m(entry)); otherwise vectors are untouched.
+ * new_access_inf != 0 sets access = infinity for surviving repository entries
  * (the else-branch of the algorithm); 0 leaves their counters as they are.
  * merge_map: -1 for invalid slots, own slot for survivors.  Returns #merged.
  * ------------------------------------------------------------------------- */
 int64_t siso_oracle_merge(double *vec, double *size, uint32_t *access, uint8_t *valid, int64_t N, int D,
-                          int64_t n_seed, double theta_c, int weighted_mean, int new_access_inf,
+                          const uint8_t *seed_mask, double theta_c, int weighted_mean, int new_access_inf,
                           int32_t *merge_map) {
     int64_t *surv = (int64_t *)malloc(sizeof(int64_t) * (size_t)(N > 0 ? N : 1));
     double *s = (double *)malloc(sizeof(double) * (size_t)(N > 0 ? N : 1));
@@ -198,9 +199,11 @@ int64_t siso_oracle_merge(double *vec, double *size, uint32_t *access, uint8_t *
     if (!surv || !s || !size0) { free(surv); free(s); free(size0); return -1; }
     memcpy(size0, size, sizeof(double) * (size_t)N);
     int64_t n_surv = 0, n_merged = 0;
+    for (int64_t i = 0; i < N; ++i)              /* C_new <- C_cur */
+        if (valid[i] && seed_mask && seed_mask[i]) { merge_map[i] = (int32_t)i; surv[n_surv++] = i; }
     for (int64_t i = 0; i < N; ++i) {
         if (!valid[i]) { merge_map[i] = -1; continue; }
-        if (i < n_seed) { merge_map[i] = (int32_t)i; surv[n_surv++] = i; continue; }
+        if (seed_mask && seed_mask[i]) continue;
         /* FindClosestCentroid over the survivors so far; vec[] is not modified until the pass ends */
 #pragma omp parallel for schedule(static)
         for (int64_t t = 0; t < n_surv; ++t) s[t] = dot_rows(vec, ORACLE_F64, (size_t)i, vec, ORACLE_F64, (size_t)surv[t], D);
@@ -223,9 +226,10 @@ int64_t siso_oracle_merge(double *vec, double *size, uint32_t *access, uint8_t *
         for (int64_t t = 0; t < n_surv; ++t) {
             int64_t sv = surv[t];
             int members = 0;
-            for (int d = 0; d < D; ++d) acc[d] = 0.0;
-            for (int64_t m = sv; m < N; ++m) {          /* members have slots >= the survivor's */
-                if (merge_map[m] != (int32_t)sv) continue;
+            for (int d = 0; d < D; ++d) acc[d] = size0[sv] * vec[(size_t)sv * D + d];
+            members = 1;
+            for (int64_t m = 0; m < N; ++m) {
+                if (m == sv || !valid[m] || merge_map[m] != (int32_t)sv) continue;
                 for (int d = 0; d < D; ++d) acc[d] += size0[m] * vec[(size_t)m * D + d];
                 members += 1;
             }

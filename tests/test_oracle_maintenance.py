@@ -307,3 +307,43 @@ def test_stream_conservation_and_recovery_after_reshuffle():
     assert hits[50:60].mean() > hits[:5].mean()                     # the cache warms up
     assert hits[60:63].mean() < hits[50:60].mean()                  # popularity reshuffle hurts ...
     assert hits[110:].mean() > hits[60:63].mean()                   # ... and the cache recovers
+
+
+def test_two_set_merge_with_interleaved_slots_equals_transcription():
+    """C_cur and the repository entries may sit in any slots: seeds are given by a mask."""
+    w = W.config(3, n_centroids=180, dim=20, n_clusters=14, mode="P")
+    rng = np.random.default_rng(8)
+    sizes = rng.integers(1, 6, 180).astype(np.float64)
+    seed = rng.random(180) < 0.4
+    c = make_cache(w.centroids, sizes=sizes)
+    c.valid[rng.random(180) < 0.1] = 0
+    c.access[:] = 5
+    entry, valid0 = c.master.copy(), c.valid.copy()
+    mm, n = c.merge(0.9, weighted_mean=True, seed_mask=seed, new_access_inf=True)
+    # Algorithm 1 by hand: C_new starts as C_cur (slot order); repository entries in slot order
+    c_new = [i for i in range(180) if valid0[i] and seed[i]]
+    size, mp = list(sizes), [i if valid0[i] else -1 for i in range(180)]
+    for i in range(180):
+        if not valid0[i] or seed[i]:
+            continue
+        sims = [float(entry[i] @ entry[j]) for j in c_new]
+        b = int(np.argmax(sims)) if sims else -1          # argmax returns the first maximum: earliest in C_new
+        if b >= 0 and sims[b] > 0.9:
+            size[c_new[b]] += sizes[i]
+            mp[i] = c_new[b]
+        else:
+            c_new.append(i)
+    assert mm.tolist() == mp and n == sum(1 for i, t in enumerate(mp) if t >= 0 and t != i) and n > 5
+    assert sorted(np.flatnonzero(c.valid)) == sorted(c_new)
+    np.testing.assert_array_equal(c.size[c_new], np.array(size)[c_new])
+    new = [i for i in c_new if not seed[i]]
+    assert (c.access[new] == INF).all() and (c.access[[i for i in c_new if seed[i]]] == 5).all()
+    for s in c_new:                                        # weighted mean: survivor first, then members by slot
+        members = [m for m in range(180) if mp[m] == s and m != s]
+        if members:
+            v = sizes[s] * entry[s] + sum(sizes[m] * entry[m] for m in members)
+            np.testing.assert_allclose(c.master[s], v / np.linalg.norm(v), atol=1e-13)
+    # a tie between a seed in a high slot and an earlier repository survivor goes to the seed (earlier in C_new)
+    c = make_cache(np.array([[1.0, 0], [0, 1.0], [1.0, 0], [1.0, 0]]))
+    mm, n = c.merge(0.5, weighted_mean=False, seed_mask=np.array([0, 0, 0, 1]))
+    assert mm.tolist() == [3, 1, 3, 3] and n == 2
