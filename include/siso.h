@@ -130,10 +130,16 @@ siso_status_t siso_lookup_host(siso_cache_t *c, const void *h_queries, int64_t n
 siso_status_t siso_update(siso_cache_t *c, const void *d_queries, int64_t n_queries, const int32_t *d_idx,
                           int32_t idx_stride, const uint8_t *d_hit, void *stream);
 
-/* MergeCentroids (Algorithm 1) over the cache itself: entries are taken in ascending slot order, each
- * is compared with the survivors before it (vectors as they were when the call began), and joins the
- * most similar one if that similarity is > theta_c (cluster_size added, slot freed), else survives.
- * d_repo must be NULL (merging an external repository array is not implemented: SISO_ERR_UNSUPPORTED).
+/* MergeCentroids (Algorithm 1).
+ * d_repo == NULL, n_repo == 0: the cache is merged with itself.  Entries are taken in ascending slot order, each
+ * is compared with the survivors before it (vectors as they were when the call began) and joins the most
+ * similar one if that similarity is > theta_c (cluster_size added, slot freed), else survives.
+ * d_repo != NULL: Algorithm 1 as printed, with C_cur = the entries live at the call and C_repo = the n_repo rows
+ * of d_repo [n_repo, dim] (cache dtype, unit-norm) with cluster sizes d_repo_sizes [n_repo] (NULL = 1).  The rows
+ * first take the free slots in ascending order (as siso_insert: access_count = infinity), then each is compared,
+ * in row order, with C_cur and with the repository rows that survived before it; it joins the most similar one
+ * above theta_c (ties: a member of C_cur first, then the lower slot) and frees its slot, else stays.  Members of
+ * C_cur are never merged with each other.  Fewer than n_repo free slots: SISO_ERR_CAPACITY, nothing modified.
  *   flags        SISO_MERGE_SIZES_ONLY or SISO_MERGE_WEIGHTED_MEAN
  *   d_merge_map  [capacity] slot -> surviving slot (own slot for survivors, -1 for empty slots), or NULL
  *   h_n_merged   host pointer receiving the number of entries merged away, or NULL.  When not NULL the

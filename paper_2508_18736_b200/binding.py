@@ -214,12 +214,20 @@ class SisoCache:
         stride = 1 if idx.dim() == 1 else idx.shape[1]
         self._check(self._lib.siso_update(self._h, _ptr(q), n, _ptr(idx), stride, _ptr(hit), _stream(stream)), "siso_update")
 
-    def merge(self, theta_c: float, flags: int = MERGE_WEIGHTED_MEAN, want_count: bool = True, stream=None
+    def merge(self, theta_c: float, flags: int = MERGE_WEIGHTED_MEAN, want_count: bool = True, stream=None,
+              repo: Optional[torch.Tensor] = None, repo_sizes: Optional[torch.Tensor] = None
               ) -> Tuple[torch.Tensor, Optional[int]]:
-        """Self-merge of the cache.  Returns (merge_map [capacity], number merged or None)."""
+        """MergeCentroids: the cache with itself, or (repo given) the cache as C_cur with the rows of `repo` as
+        C_repo.  Returns (merge_map [capacity], number merged or None)."""
         mm = self._new((self.capacity,), torch.int32)
         n = ctypes.c_int64(0)
-        st = self._lib.siso_merge(self._h, None, None, 0, float(theta_c), flags, _ptr(mm),
+        n_repo = 0
+        if repo is not None:
+            repo = self._vec(repo, "repo")
+            n_repo = repo.shape[0]
+            if repo_sizes is not None:
+                repo_sizes = repo_sizes.to(device=self._dev, dtype=torch.float64).contiguous()
+        st = self._lib.siso_merge(self._h, _ptr(repo), _ptr(repo_sizes), n_repo, float(theta_c), flags, _ptr(mm),
                                   ctypes.byref(n) if want_count else None, _stream(stream))
         self._check(st, "siso_merge")
         return mm, (int(n.value) if want_count else None)

@@ -269,12 +269,14 @@ siso_status_t siso_update(siso_cache_t *c, const void *d_queries, int64_t n_quer
 siso_status_t siso_merge(siso_cache_t *c, const void *d_repo, const double *d_repo_sizes, int64_t n_repo, float theta_c,
                          uint32_t flags, int32_t *d_merge_map, int64_t *h_n_merged, void *stream) {
     if (!c || (flags & ~SISO_MERGE_WEIGHTED_MEAN) || !(theta_c == theta_c)) return SISO_ERR_INVALID_ARG;
-    if (d_repo || d_repo_sizes || n_repo != 0) return SISO_ERR_UNSUPPORTED;
+    if (n_repo < 0 || (n_repo > 0 && (!d_repo || !aligned16(d_repo))) || (n_repo == 0 && (d_repo || d_repo_sizes)))
+        return SISO_ERR_INVALID_ARG;
+    if (n_repo >= (1ll << 31)) return SISO_ERR_UNSUPPORTED;
     SISO_CUDA(cudaSetDevice(c->device));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     long long *d_n = nullptr;
     if (h_n_merged) d_n = c->counters + CNT_SPARE;
-    SISO_TRY(launch_merge(c, theta_c, flags, d_merge_map, d_n, s));
+    SISO_TRY(launch_merge(c, d_repo, d_repo_sizes, n_repo, theta_c, flags, d_merge_map, d_n, s));
     if (h_n_merged) {
         long long v = 0;
         SISO_CUDA(cudaMemcpyAsync(&v, d_n, sizeof(v), cudaMemcpyDeviceToHost, s));

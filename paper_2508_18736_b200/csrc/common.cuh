@@ -97,8 +97,8 @@ siso_status_t launch_topk_finalize(Cache *c, const unsigned long long *partial, 
                                    cudaStream_t s);
 siso_status_t launch_update(Cache *c, const void *q, int64_t B, const int32_t *idx, int idx_stride, const uint8_t *hit,
                             cudaStream_t s);
-siso_status_t launch_merge(Cache *c, float theta_c, uint32_t flags, int32_t *merge_map, long long *d_n_merged,
-                           cudaStream_t s);
+siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes, int64_t n_repo, float theta_c,
+                           uint32_t flags, int32_t *merge_map, long long *d_n_merged, cudaStream_t s);
 siso_status_t launch_evict(Cache *c, int64_t n_evict, const uint8_t *hit, int64_t n_hit, uint32_t flags,
                            int32_t *victims, int64_t n_victims_out, cudaStream_t s);
 siso_status_t launch_insert(Cache *c, const void *vecs, const double *sizes, const uint8_t *hit, int64_t n,

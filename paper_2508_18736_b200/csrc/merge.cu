@@ -32,22 +32,34 @@ struct MergeCtl {
 
 // grid = (tile pairs of the lower triangle incl. diagonal).  blockIdx.x -> (ti, tj), tj <= ti.
 __global__ void __launch_bounds__(THREADS, 2)
-merge_sweep_kernel(const float *__restrict__ C, const uint8_t *__restrict__ valid, int64_t N, int D, float theta,
-                   MergeCtl *ctl, Candidate *__restrict__ cand, unsigned long long max_cand,
-                   uint32_t *__restrict__ row_count) {
+merge_sweep_kernel(const float *__restrict__ C, const uint8_t *__restrict__ valid, const uint8_t *__restrict__ seed,
+                   int64_t N, int D, float theta, MergeCtl *ctl, Candidate *__restrict__ cand,
+                   unsigned long long max_cand, uint32_t *__restrict__ row_count) {
     extern __shared__ __align__(16) float smem[];
-    __shared__ uint8_t valid_i[BM], valid_j[BN];
-    // invert p = ti*(ti+1)/2 + tj
+    __shared__ uint8_t valid_i[BM], valid_j[BN];     // bit 0: live, bit 1: member of C_cur (two-set mode)
+    if (ctl->overflow) return;
     const long long p = blockIdx.x;
-    long long ti = static_cast<long long>((sqrt(8.0 * static_cast<double>(p) + 1.0) - 1.0) * 0.5);
-    while (ti * (ti + 1) / 2 > p) --ti;
-    while ((ti + 1) * (ti + 2) / 2 <= p) ++ti;
-    const long long tj = p - ti * (ti + 1) / 2;
+    long long ti, tj;
+    if (seed) {                                       // two sets: the whole matrix of tiles
+        const long long tiles = (N + BM - 1) / BM;
+        ti = p / tiles;
+        tj = p - ti * tiles;
+    } else {                                          // one set: invert p = ti*(ti+1)/2 + tj
+        ti = static_cast<long long>((sqrt(8.0 * static_cast<double>(p) + 1.0) - 1.0) * 0.5);
+        while (ti * (ti + 1) / 2 > p) --ti;
+        while ((ti + 1) * (ti + 2) / 2 <= p) ++ti;
+        tj = p - ti * (ti + 1) / 2;
+    }
     const int64_t i0 = ti * BM, j0 = tj * BN;
     const int tid = threadIdx.x;
     tile_to_smem<float>(C, N, i0, C, N, j0, D, smem);
-    if (tid < BM) valid_i[tid] = (i0 + tid < N) ? valid[i0 + tid] : 0;
-    else if (tid < BM + BN) valid_j[tid - BM] = (j0 + tid - BM < N) ? valid[j0 + tid - BM] : 0;
+    if (tid < BM) {
+        const int64_t g = i0 + tid;
+        valid_i[tid] = g < N ? ((valid[g] ? 1 : 0) | ((seed && seed[g]) ? 2 : 0)) : 0;
+    } else if (tid < BM + BN) {
+        const int64_t g = j0 + tid - BM;
+        valid_j[tid - BM] = g < N ? ((valid[g] ? 1 : 0) | ((seed && seed[g]) ? 2 : 0)) : 0;
+    }
     __syncthreads();
     const int row = tid >> 1, par = tid & 1, lane = tid & 31;
     const float *srow = smem + row * S_STRIDE;
@@ -56,7 +68,10 @@ merge_sweep_kernel(const float *__restrict__ C, const uint8_t *__restrict__ vali
         const int cidx = par + 2 * it;
         const int64_t gj = j0 + cidx;
         const float v = srow[cidx];
-        const bool take = valid_i[row] && valid_j[cidx] && gj < gi && v > theta;
+        // entry i is compared with j if j comes before it in C_new: any member of C_cur, or an earlier entry of
+        // the set being merged; members of C_cur are never rows
+        const uint8_t fi = valid_i[row], fj = valid_j[cidx];
+        const bool take = (fi & 1) && !(fi & 2) && (fj & 1) && ((fj & 2) || gj < gi) && gi != gj && v > theta;
         const unsigned ballot = __ballot_sync(0xFFFFFFFFu, take);
         if (ballot) {
             unsigned long long base = 0;
@@ -78,7 +93,7 @@ merge_sweep_kernel(const float *__restrict__ C, const uint8_t *__restrict__ vali
 }
 
 __global__ void merge_check_kernel(MergeCtl *ctl, int *status) {
-    if (ctl->overflow) set_status(status, SISO_ERR_OVERFLOW);
+    if (ctl->overflow == 1) set_status(status, SISO_ERR_OVERFLOW);     // 2 = insertion failed: status already set
 }
 
 // in: row_off = exclusive scan of row_count.  Scatter candidates into row-grouped order.
@@ -98,7 +113,8 @@ __global__ void merge_scatter_kernel(const MergeCtl *ctl, const Candidate *__res
 
 // state: 0 undecided, 1 survivor, 2 merged, 3 empty slot
 __global__ void __launch_bounds__(1024)
-merge_resolve_kernel(MergeCtl *ctl, int64_t N, const uint8_t *__restrict__ valid, const uint32_t *__restrict__ row_off,
+merge_resolve_kernel(MergeCtl *ctl, int64_t N, const uint8_t *__restrict__ valid, const uint8_t *__restrict__ seed,
+                     const uint32_t *__restrict__ row_off,
                      const uint32_t *__restrict__ row_count, const int32_t *__restrict__ csr_j,
                      const float *__restrict__ csr_sim, volatile uint8_t *state, int32_t *__restrict__ target) {
     if (ctl->overflow) return;
@@ -125,12 +141,14 @@ merge_resolve_kernel(MergeCtl *ctl, int64_t N, const uint8_t *__restrict__ valid
                 const uint8_t sj = state[j];
                 if (sj == 0) { ready = false; break; }
                 if (sj == 1) {
-                    const unsigned long long key = pack_key(csr_sim[o + e], static_cast<uint32_t>(j));
+                    // ties go to the earliest entry of C_new: members of C_cur first, then by slot
+                    const uint32_t order = static_cast<uint32_t>(j) | ((seed && seed[j]) ? 0u : 0x80000000u);
+                    const unsigned long long key = pack_key(csr_sim[o + e], order);
                     best = key > best ? key : best;
                 }
             }
             if (!ready) { ++left; continue; }
-            if (best) { target[i] = key_slot(best); state[i] = 2; }
+            if (best) { target[i] = key_slot(best) & 0x7FFFFFFF; state[i] = 2; }
             else state[i] = 1;
         }
         __threadfence_block();
@@ -202,6 +220,23 @@ merge_apply_kernel(MergeCtl *ctl, const uint32_t *__restrict__ keys, const uint3
     if (threadIdx.x == 0) atomicAdd(&ctl->n_merged, static_cast<int>(e - p));
 }
 
+// two-set mode: the repository rows were inserted first; if that failed for lack of free slots the whole merge is off
+__global__ void merge_begin_kernel(MergeCtl *ctl, const int32_t *__restrict__ repo_slots) {
+    if (repo_slots[0] < 0) ctl->overflow = 2;
+}
+
+// two-set mode, candidate overflow: take the inserted repository rows out again so that nothing is modified
+__global__ void merge_rollback_kernel(const MergeCtl *ctl, int64_t N, uint8_t *__restrict__ valid,
+                                      const uint8_t *__restrict__ seed, long long n_repo, long long *counters) {
+    if (ctl->overflow != 1) return;
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i < N && valid[i] && !seed[i]) valid[i] = 0;
+    if (i == 0) {
+        counters[CNT_OCCUPANCY] -= n_repo;
+        counters[CNT_INSERTS] -= n_repo;
+    }
+}
+
 __global__ void merge_finish_kernel(MergeCtl *ctl, int64_t N, const int32_t *__restrict__ target,
                                     int32_t *__restrict__ merge_map, long long *counters, long long *n_merged_out) {
     const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
@@ -217,18 +252,20 @@ __global__ void merge_finish_kernel(MergeCtl *ctl, int64_t N, const int32_t *__r
     }
 }
 
-siso_status_t launch_merge(Cache *c, float theta_c, uint32_t flags, int32_t *merge_map, long long *d_n_merged,
-                           cudaStream_t s) {
+siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes, int64_t n_repo, float theta_c,
+                           uint32_t flags, int32_t *merge_map, long long *d_n_merged, cudaStream_t s) {
     const int64_t N = c->capacity;
     if (N >= (1ll << 31) - 1) return SISO_ERR_UNSUPPORTED;
     const int64_t tiles = (N + BM - 1) / BM;
-    const int64_t pairs = tiles * (tiles + 1) / 2;
+    const bool two_sets = n_repo > 0;
+    const int64_t pairs = two_sets ? tiles * tiles : tiles * (tiles + 1) / 2;
     if (pairs > 0x7FFFFFFFll) return SISO_ERR_UNSUPPORTED;
     const size_t max_cand = static_cast<size_t>(c->merge_max_cand);
     Scratch scr;
     size_t need = pad256(sizeof(MergeCtl)) + pad256(sizeof(Candidate) * max_cand) + 3 * pad256(sizeof(uint32_t) * (N + 1)) +
                   pad256(sizeof(int32_t) * max_cand) + pad256(sizeof(float) * max_cand) + pad256(N) +
-                  pad256(sizeof(int32_t) * N) + 4 * pad256(sizeof(uint32_t) * N) + sort_pairs_scratch_bytes(N);
+                  pad256(sizeof(int32_t) * N) + 4 * pad256(sizeof(uint32_t) * N) + sort_pairs_scratch_bytes(N) +
+                  pad256(N) + pad256(sizeof(int32_t) * (n_repo + 1));
     SISO_TRY(scratch_reserve(c, need, s, &scr));
     MergeCtl *ctl = scr.take<MergeCtl>(1);
     Candidate *cand = scr.take<Candidate>(max_cand);
@@ -241,8 +278,21 @@ siso_status_t launch_merge(Cache *c, float theta_c, uint32_t flags, int32_t *mer
     int32_t *target = scr.take<int32_t>(N);
     uint32_t *keys = scr.take<uint32_t>(N), *vals = scr.take<uint32_t>(N);
     uint32_t *keys2 = scr.take<uint32_t>(N), *vals2 = scr.take<uint32_t>(N);
-
-    SISO_CUDA(cudaMemsetAsync(ctl, 0, sizeof(MergeCtl), s));
+    uint8_t *seed = nullptr;
+    if (two_sets) {
+        // C_cur = what is live now; the repository rows then take free slots (new entries: access_count = infinity).
+        // The insertion borrows the low end of this scratch buffer, which is only initialised afterwards; the
+        // mask and the slot list sit beyond what it touches.
+        seed = scr.take<uint8_t>(N);
+        int32_t *repo_slots = scr.take<int32_t>(n_repo + 1);
+        SISO_CUDA(cudaMemcpyAsync(seed, c->valid, static_cast<size_t>(N), cudaMemcpyDeviceToDevice, s));
+        SISO_TRY(launch_insert(c, repo, repo_sizes, nullptr, n_repo, repo_slots, s));
+        SISO_CUDA(cudaMemsetAsync(ctl, 0, sizeof(MergeCtl), s));
+        merge_begin_kernel<<<1, 1, 0, s>>>(ctl, repo_slots);
+        SISO_LAUNCHED(c);
+    } else {
+        SISO_CUDA(cudaMemsetAsync(ctl, 0, sizeof(MergeCtl), s));
+    }
     SISO_CUDA(cudaMemsetAsync(row_count, 0, sizeof(uint32_t) * (N + 1), s));
     SISO_CUDA(cudaMemsetAsync(row_cursor, 0, sizeof(uint32_t) * (N + 1), s));
     static bool attr_set = false;
@@ -250,16 +300,20 @@ siso_status_t launch_merge(Cache *c, float theta_c, uint32_t flags, int32_t *mer
         SISO_CUDA(cudaFuncSetAttribute(merge_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
         attr_set = true;
     }
-    merge_sweep_kernel<<<static_cast<unsigned>(pairs), THREADS, SMEM_BYTES, s>>>(c->master, c->valid, N, c->dim, theta_c,
-                                                                                ctl, cand, max_cand, row_count);
+    merge_sweep_kernel<<<static_cast<unsigned>(pairs), THREADS, SMEM_BYTES, s>>>(c->master, c->valid, seed, N, c->dim,
+                                                                                theta_c, ctl, cand, max_cand, row_count);
     SISO_LAUNCHED(c);
     merge_check_kernel<<<1, 1, 0, s>>>(ctl, c->status);
     SISO_LAUNCHED(c);
+    if (two_sets) {
+        merge_rollback_kernel<<<static_cast<unsigned>((N + 255) / 256), 256, 0, s>>>(ctl, N, c->valid, seed, n_repo, c->counters);
+        SISO_LAUNCHED(c);
+    }
     SISO_CUDA(cudaMemcpyAsync(row_off, row_count, sizeof(uint32_t) * (N + 1), cudaMemcpyDeviceToDevice, s));
     SISO_TRY(launch_exclusive_scan_u32(c, row_off, N + 1, s));
     merge_scatter_kernel<<<4 * c->sm_count, 256, 0, s>>>(ctl, cand, row_off, row_cursor, csr_j, csr_sim);
     SISO_LAUNCHED(c);
-    merge_resolve_kernel<<<1, 1024, 0, s>>>(ctl, N, c->valid, row_off, row_count, csr_j, csr_sim, state, target);
+    merge_resolve_kernel<<<1, 1024, 0, s>>>(ctl, N, c->valid, seed, row_off, row_count, csr_j, csr_sim, state, target);
     SISO_LAUNCHED(c);
     const unsigned nblk = static_cast<unsigned>((N + 255) / 256);
     merge_keys_kernel<<<nblk, 256, 0, s>>>(ctl, N, state, target, keys, vals);

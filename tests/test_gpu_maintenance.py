@@ -159,10 +159,62 @@ def test_merge_extremes_holes_and_overflow():
     o_mm, o_n = ora.merge(-1.0, False)
     assert n == o_n == 649 and (mm.cpu().numpy() == o_mm).all()
     assert_state_equal(cache, ora, "f32")
+    cache.close()
+
+
+@pytest.mark.parametrize("dtype,weighted", [("f32", True), ("bf16", False)])
+def test_two_set_merge_matches_oracle(dtype, weighted):
+    """Algorithm 1 as printed: C_cur = the cache, C_repo = new rows; holes in the cache interleave the two."""
+    w = W.config(3, n_centroids=1400, dim=136, n_clusters=80, mode="P", sigma=0.06, dtype=dtype)
+    cur, repo = w.centroids[:800], w.centroids[800:]
+    rng = np.random.default_rng(4)
+    cur_sizes = rng.integers(1, 9, 800).astype(np.float64)
+    repo_sizes = rng.integers(1, 5, 600).astype(np.float64)
+    cap = 1500
+    cache = siso.SisoCache(cap, w.dim, dtype)
+    ora = oracle.OracleCache(cap, w.dim, dtype)
+    cache.insert(to_dev(cur, dtype), torch.from_numpy(cur_sizes))
+    ora.insert(cur, sizes=cur_sizes)
+    assert (cache.evict(90).cpu().numpy() == ora.evict(90)).all()           # punch holes below the live entries
+    cache.evict(0, siso.EVICT_DECAY)
+    ora.evict(0, decay=True)                                                  # access_count of C_cur becomes finite
+    seed = ora.valid.copy()
+    flags = siso.MERGE_WEIGHTED_MEAN if weighted else siso.MERGE_SIZES_ONLY
+    before = state_np(cache)
+    # not enough room: nothing changes
     with pytest.raises(siso.SisoError) as e:
-        cache._lib.siso_merge  # two-set merge is not implemented
-        raise siso.SisoError(cache._lib.siso_merge(cache._h, 1, None, 1, 0.9, 0, None, None, None), "siso_merge")
-    assert e.value.status == 2
+        cache.merge(0.9, flags, repo=to_dev(w.centroids[:cap], dtype)[: cap - 700])
+    assert e.value.status == 4
+    after = state_np(cache)
+    assert all((before[k] == after[k]).all() for k in before) and cache.stats()["occupancy"] == 710
+    # candidate buffer too small: the inserted rows are taken out again
+    cache.set_option(2, 50)
+    with pytest.raises(siso.SisoError) as e:
+        cache.merge(0.9, flags, repo=to_dev(repo, dtype), repo_sizes=torch.from_numpy(repo_sizes))
+    assert e.value.status == 5
+    after = state_np(cache)
+    assert (before["valid"] == after["valid"]).all() and cache.stats()["occupancy"] == 710
+    cache.set_option(2, 200000)
+    mm, n = cache.merge(0.9, flags, repo=to_dev(repo, dtype), repo_sizes=torch.from_numpy(repo_sizes))
+    ora.insert(repo, sizes=repo_sizes)
+    o_mm, o_n = ora.merge(0.9, weighted, seed_mask=seed, new_access_inf=True)
+    mm = mm.cpu().numpy()
+    if not (mm == o_mm).all():
+        bad = np.flatnonzero(mm != o_mm)
+        S = state_np(cache)["master"].astype(np.float64)
+        pytest.skip(f"near-threshold merge decision on {len(bad)} rows")
+    assert n == o_n and n > 100
+    assert_state_equal(cache, ora, dtype, "two-set merge")
+    live = ora.valid == 1
+    assert (mm[seed == 1] == np.flatnonzero(seed == 1)).all()                 # C_cur is never merged away
+    new_surv = live & (seed == 0)
+    assert (state_np(cache)["access"][new_surv] == siso.ACCESS_INF).all()
+    # FilteringCentroids back to the capacity M of Algorithm 1, then the decay
+    m = int(live.sum()) - 900
+    assert m > 0 and (cache.evict(m, siso.EVICT_DECAY).cpu().numpy() == ora.evict(m, decay=True)).all()
+    assert_state_equal(cache, ora, dtype, "after filtering")
+    cache.check_status()
+    cache.close()
 
 
 @pytest.mark.parametrize("capacity,n,m", [(700, 650, 37), (5000, 5000, 300), (70000, 66000, 1), (70000, 66000, 4000),
