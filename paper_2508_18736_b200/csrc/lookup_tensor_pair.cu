@@ -250,20 +250,23 @@ lookup_tensor_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
             auto scan = [&](uint32_t (&r)[32], int ch) {
                 const uint32_t live = __ballot_sync(0xFFFFFFFFu, ((vflags >> ch) & 1ull) != 0ull);
                 if (live == 0u) return;
-                float m = -INFINITY;
-                if (live == 0xFFFFFFFFu) {
+                if (live != 0xFFFFFFFFu) {
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) m = fmaxf(m, __uint_as_float(r[j]));
-                } else {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
+                    for (int j = 0; j < 32; ++j)
                         if (!((live >> j) & 1u)) r[j] = 0xFF800000u;      // -inf: never enters a list
-                        m = fmaxf(m, __uint_as_float(r[j]));
-                    }
                 }
-                if (m > top.s[KMAX - 1]) {
+                // Groups of 8 columns: a group is looked at value by value only if its maximum beats the row's
+                // k-th best.  A warp pays for that path when ANY of its 32 rows takes it, so small groups keep
+                // the common case (nothing to insert) down to 7 max operations and one comparison per group.
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) top.push(__uint_as_float(r[j]), n0 + ch * 32 + j);
+                for (int g8 = 0; g8 < 4; ++g8) {
+                    float m = __uint_as_float(r[g8 * 8]);
+#pragma unroll
+                    for (int j = 1; j < 8; ++j) m = fmaxf(m, __uint_as_float(r[g8 * 8 + j]));
+                    if (m > top.s[KMAX - 1]) {
+#pragma unroll
+                        for (int j = 0; j < 8; ++j) top.push(__uint_as_float(r[g8 * 8 + j]), n0 + ch * 32 + g8 * 8 + j);
+                    }
                 }
             };
             tmem_ld_32x32(taddr, ra);
