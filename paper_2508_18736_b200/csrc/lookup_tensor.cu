@@ -245,13 +245,13 @@ lookup_tensor_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                 // k-th best.  A warp pays for that path when ANY of its 32 rows takes it, so small groups keep
                 // the common case (nothing to insert) down to 7 max operations and one comparison per group.
 #pragma unroll
-                for (int g8 = 0; g8 < 4; ++g8) {
-                    float m = __uint_as_float(r[g8 * 8]);
+                for (int g8 = 0; g8 < 8; ++g8) {
+                    float m = __uint_as_float(r[g8 * 4]);
 #pragma unroll
-                    for (int j = 1; j < 8; ++j) m = fmaxf(m, __uint_as_float(r[g8 * 8 + j]));
+                    for (int j = 1; j < 4; ++j) m = fmaxf(m, __uint_as_float(r[g8 * 4 + j]));
                     if (m > top.s[KMAX - 1]) {
 #pragma unroll
-                        for (int j = 0; j < 8; ++j) top.push(__uint_as_float(r[g8 * 8 + j]), n0 + ch * 32 + g8 * 8 + j);
+                        for (int j = 0; j < 4; ++j) top.push(__uint_as_float(r[g8 * 4 + j]), n0 + ch * 32 + g8 * 4 + j);
                     }
                 }
             };
