@@ -376,12 +376,23 @@ siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const flo
     // CTA pairs (two query tiles share every centroid tile) whenever the batch has at least two query tiles
     const bool pair = m_tiles >= 2 && c->tensor_pair_mode == 0;
     const int m_ctas = pair ? (m_tiles + 1) / 2 * 2 : m_tiles;
-    // one CTA per SM at a time: aim at a whole number of waves with at least ~8 tiles per CTA
+    // One CTA per SM at a time.  Few, long splits keep each row's running top-k warm (a fresh CTA inserts often
+    // until its k-th best has risen) but quantise badly into waves of sm_count CTAs; try a few wave counts and
+    // take the cheapest by a simple model: rounds x (tiles per CTA + a fixed start-up/drain cost in tiles).
     const int64_t units = static_cast<int64_t>(m_ctas) * n_tiles;
-    const int waves = static_cast<int>(std::min<int64_t>(16, std::max<int64_t>(1, units / (8ll * c->sm_count))));
-    int splits = std::max(1, std::min(std::min(n_tiles, 65535), (c->sm_count * waves) / m_ctas));
-    const int tiles_per_split = (n_tiles + splits - 1) / splits;
-    splits = (n_tiles + tiles_per_split - 1) / tiles_per_split;
+    const int wave_cap = static_cast<int>(std::min<int64_t>(16, std::max<int64_t>(1, units / (8ll * c->sm_count))));
+    int splits = 1, tiles_per_split = n_tiles;
+    int64_t best_cost = -1;
+    const int candidates[] = {4, 6, 8, 12, 16};
+    for (int ci = 0; ci < 5; ++ci) {
+        const int w = std::min(candidates[ci], wave_cap);
+        int sp = std::max(1, std::min(std::min(n_tiles, 65535), (c->sm_count * w) / m_ctas));
+        const int tps = (n_tiles + sp - 1) / sp;
+        sp = (n_tiles + tps - 1) / tps;
+        const int64_t rounds = (static_cast<int64_t>(m_ctas) * sp + c->sm_count - 1) / c->sm_count;
+        const int64_t cost = rounds * (tps + 6);
+        if (best_cost < 0 || cost < best_cost) { best_cost = cost; splits = sp; tiles_per_split = tps; }
+    }
 
     Scratch scr;
     SISO_TRY(scratch_reserve(c, pad256(sizeof(unsigned long long) * B * splits * kmax), s, &scr));
