@@ -49,27 +49,40 @@ __device__ __forceinline__ double block_sum_f64(double v, double *red) {
     return t;
 }
 
-// One CTA per position of the sorted hit list; the CTA at the head of a group does the group.
+// One CTA per position of the sorted hit list.  A group (the hits of one slot, ascending query order) is cut into
+// chunks of `chunk` rows; the CTA at the first row of a chunk sums that chunk in fp64.  A group of one chunk is
+// finished on the spot.  Otherwise the chunk sums go to scratch and the CTA that arrives last (a counter per
+// group) adds them up in chunk order and finishes, so a centroid that takes hundreds of hits is not one CTA's
+// serial work and the result is still the same on every run.
 template <typename T>
 __global__ void __launch_bounds__(UP_THREADS)
 update_apply_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restrict__ rows, int64_t B, int64_t capacity,
-                    int D, const T *__restrict__ Q, float *__restrict__ master, T *__restrict__ vecs,
+                    int D, int chunk, const T *__restrict__ Q, float *__restrict__ master, T *__restrict__ vecs,
                     double *__restrict__ size, uint32_t *__restrict__ access, unsigned long long *__restrict__ last,
-                    const long long *__restrict__ counters) {
+                    const long long *__restrict__ counters, double *__restrict__ partial,
+                    unsigned int *__restrict__ arrived) {
     extern __shared__ double acc[];          // [D]
     __shared__ double red[UP_THREADS / 32];
+    __shared__ int last_s;
     const int64_t p = blockIdx.x;
     const uint32_t slot = keys[p];
     if (slot >= capacity) return;
-    if (p > 0 && keys[p - 1] == slot) return;
+    int64_t lo = 0, hi = p;                  // first position of this slot in the sorted list
+    while (lo < hi) {
+        const int64_t mid = (lo + hi) >> 1;
+        if (keys[mid] < slot) lo = mid + 1; else hi = mid;
+    }
+    const int64_t head = lo;
+    if ((p - head) % chunk != 0) return;
+    const bool is_head = p == head;
+    int64_t e = p;
+    while (e < B && e < p + chunk && keys[e] == slot) ++e;
+    const bool more = e < B && keys[e] == slot;
     const double n_old = size[slot];
     float *m = master + static_cast<int64_t>(slot) * D;
-    for (int d = threadIdx.x; d < D; d += UP_THREADS) acc[d] = n_old * static_cast<double>(m[d]);
+    for (int d = threadIdx.x; d < D; d += UP_THREADS) acc[d] = is_head ? n_old * static_cast<double>(m[d]) : 0.0;
     __syncthreads();      // the accumulation below uses a different thread-to-element mapping
-    // group extent, then the rows four at a time: the loads of a quartet are in flight together, the
-    // additions stay in ascending query order
-    int64_t e = p;
-    while (e < B && keys[e] == slot) ++e;
+    // the rows four at a time: the loads of a quartet are in flight together, additions stay in ascending order
     const int quads = D / 4;
     for (int64_t t = p; t < e; t += 4) {
         const int nrow = static_cast<int>(e - t < 4 ? e - t : 4);
@@ -89,7 +102,36 @@ update_apply_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restric
         }
     }
     __syncthreads();
-    const long long count = e - p;
+    long long count = e - p;
+    if (!(is_head && !more)) {
+        // several chunks: publish this chunk's sum, the last arriver combines.  A chunk's scratch row is
+        // 2 * (start / chunk) + (1 if it is the group's first chunk): unique, because chunks of one group start
+        // `chunk` rows apart and a first chunk of a several-chunk group is at least `chunk` rows from the next group.
+        const int64_t my_id = 2 * (p / chunk) + (is_head ? 1 : 0);
+        for (int d = threadIdx.x; d < D; d += UP_THREADS) partial[my_id * D + d] = acc[d];
+        int64_t glo = e, ghi = B;            // first position past the group
+        while (glo < ghi) {
+            const int64_t mid = (glo + ghi) >> 1;
+            if (keys[mid] <= slot) glo = mid + 1; else ghi = mid;
+        }
+        const int64_t gend = glo;
+        const int64_t n_chunks = (gend - head + chunk - 1) / chunk;
+        const int64_t head_id = 2 * (head / chunk) + 1;
+        __threadfence();
+        __syncthreads();
+        if (threadIdx.x == 0) last_s = (atomicAdd(&arrived[head_id], 1u) == static_cast<unsigned int>(n_chunks - 1)) ? 1 : 0;
+        __syncthreads();
+        if (!last_s) return;
+        __threadfence();
+        for (int d = threadIdx.x; d < D; d += UP_THREADS) {
+            double v = __ldcg(&partial[head_id * D + d]);
+            for (int64_t cidx = 1; cidx < n_chunks; ++cidx)
+                v += __ldcg(&partial[(2 * ((head + cidx * chunk) / chunk)) * D + d]);
+            acc[d] = v;
+        }
+        __syncthreads();
+        count = gend - head;
+    }
     double ss = 0.0;
     for (int d = threadIdx.x; d < D; d += UP_THREADS) ss += acc[d] * acc[d];
     const double norm = sqrt(block_sum_f64(ss, red));
@@ -227,7 +269,10 @@ siso_status_t launch_update(Cache *c, const void *q, int64_t B, const int32_t *i
         return SISO_OK;
     }
     Scratch scr;
-    const size_t need = 4 * pad256(sizeof(uint32_t) * B) + sort_pairs_scratch_bytes(B);
+    const int chunk = static_cast<int>(std::max<int64_t>(32, (B + 4095) / 4096));
+    const size_t n_ids = 2 * static_cast<size_t>(B / chunk + 1);
+    const size_t need = 4 * pad256(sizeof(uint32_t) * B) + sort_pairs_scratch_bytes(B) +
+                        pad256(sizeof(double) * n_ids * c->dim) + pad256(sizeof(unsigned int) * n_ids);
     SISO_TRY(scratch_reserve(c, need, s, &scr));
     uint32_t *keys = scr.take<uint32_t>(B), *vals = scr.take<uint32_t>(B);
     uint32_t *keys2 = scr.take<uint32_t>(B), *vals2 = scr.take<uint32_t>(B);
@@ -243,14 +288,17 @@ siso_status_t launch_update(Cache *c, const void *q, int64_t B, const int32_t *i
     uint32_t *ks, *vs;
     SISO_TRY(launch_sort_pairs(c, &scr, keys, vals, keys2, vals2, B, key_bits, &ks, &vs, s));
     const size_t smem = sizeof(double) * c->dim;
+    double *partial = scr.take<double>(n_ids * c->dim);
+    unsigned int *arrived = scr.take<unsigned int>(n_ids);
+    SISO_CUDA(cudaMemsetAsync(arrived, 0, sizeof(unsigned int) * n_ids, s));
     if (c->dtype == SISO_F32) {
         update_apply_kernel<float><<<static_cast<unsigned>(B), UP_THREADS, smem, s>>>(
-            ks, vs, B, c->capacity, c->dim, static_cast<const float *>(q), c->master, static_cast<float *>(c->vecs),
-            c->size, c->access, c->last, c->counters);
+            ks, vs, B, c->capacity, c->dim, chunk, static_cast<const float *>(q), c->master, static_cast<float *>(c->vecs),
+            c->size, c->access, c->last, c->counters, partial, arrived);
     } else {
         update_apply_kernel<__nv_bfloat16><<<static_cast<unsigned>(B), UP_THREADS, smem, s>>>(
-            ks, vs, B, c->capacity, c->dim, static_cast<const __nv_bfloat16 *>(q), c->master,
-            static_cast<__nv_bfloat16 *>(c->vecs), c->size, c->access, c->last, c->counters);
+            ks, vs, B, c->capacity, c->dim, chunk, static_cast<const __nv_bfloat16 *>(q), c->master,
+            static_cast<__nv_bfloat16 *>(c->vecs), c->size, c->access, c->last, c->counters, partial, arrived);
     }
     SISO_LAUNCHED(c);
     return SISO_OK;
