@@ -274,11 +274,11 @@ def run_ours(args):
     kernel_ms = statistics.median(per_step)           # the sweep kernel plus its small finalize kernel
     achieved = flops / (kernel_ms * 1e-3) / 1e12
     # DRAM bytes per launch of the dominant kernel, from the committed one-pass ncu capture of this very command
-    # (profiles/lookup_tensor_config4_launches.txt: 5.74e9 / 6.51e9 read, 1.3e7 / 1.0e7 written in two launches);
+    # (profiles/lookup_tensor_config4_launches.txt: 2.888e9 read, 5.5e6 / 2.4e6 written in two launches);
     # only known for the full-size workload on the tensor-core kernel as profiled
     traffic = None
     if args.path in ("auto", "tensor") and args.rows == (1 << 20) and B == 8192:
-        traffic = 0.5 * (5738814976 + 6508273664) + 0.5 * (12964608 + 10215168)
+        traffic = 0.5 * (2888013568 + 2888555520) + 0.5 * (5518080 + 2418432)
     roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": achieved / peaks["bf16_tflops"], "traffic": traffic, "peak_kind": f"{peak_kind}, burst",
                 "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
