@@ -52,6 +52,9 @@ struct Cache {
     int64_t merge_max_cand;
     int64_t launches;
     void *tensor_state;    // owned by lookup_tensor.cu
+    // large-shared-memory opt-in is a per-device function attribute: remembered per cache, not per process
+    bool simt_attr_set[2][3];   // [dtype][k class] of lookup_simt_kernel
+    bool merge_attr_set;
 };
 
 // ---- scratch bump allocator -------------------------------------------------

@@ -271,7 +271,7 @@ siso_status_t launch_evict(Cache *c, int64_t n_evict, const uint8_t *hit, int64_
                                            c->counters, plan, splitters, victims, victims ? n_victims_out : 0);
     SISO_LAUNCHED(c);
     const int grid = static_cast<int>(std::min<int64_t>((c->capacity + 255) / 256, 4ll * c->sm_count));
-    const int grid_bucket = static_cast<int>(std::min<int64_t>((c->capacity + 2047) / 2048, 2ll * c->sm_count));
+    const int grid_bucket = static_cast<int>(std::min<int64_t>((c->capacity + 255) / 256, 8ll * c->sm_count));
     evict_bucket_kernel<<<grid_bucket, 256, 0, s>>>(c->capacity, c->size, c->access, c->last, c->valid, plan, splitters, bucket);
     SISO_LAUNCHED(c);
     evict_collect_kernel<<<grid, 256, 0, s>>>(c->capacity, c->size, c->access, c->last, c->valid, plan, bucket, cand);

@@ -123,7 +123,7 @@ template <typename T, int KMAX>
 static siso_status_t run_simt(Cache *c, const void *q, int64_t B, int tiles_per_split, int n_tiles, int splits,
                               int m_tiles, unsigned long long *partial, cudaStream_t s) {
     auto kern = lookup_simt_kernel<T, KMAX>;
-    static bool attr_set = false;   // per instantiation
+    bool &attr_set = c->simt_attr_set[sizeof(T) == 2 ? 1 : 0][KMAX == 1 ? 0 : (KMAX == 4 ? 1 : 2)];
     if (!attr_set) {
         SISO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
         attr_set = true;

@@ -295,10 +295,9 @@ siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes,
     }
     SISO_CUDA(cudaMemsetAsync(row_count, 0, sizeof(uint32_t) * (N + 1), s));
     SISO_CUDA(cudaMemsetAsync(row_cursor, 0, sizeof(uint32_t) * (N + 1), s));
-    static bool attr_set = false;
-    if (!attr_set) {
+    if (!c->merge_attr_set) {
         SISO_CUDA(cudaFuncSetAttribute(merge_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-        attr_set = true;
+        c->merge_attr_set = true;
     }
     merge_sweep_kernel<<<static_cast<unsigned>(pairs), THREADS, SMEM_BYTES, s>>>(c->master, c->valid, seed, N, c->dim,
                                                                                 theta_c, ctl, cand, max_cand, row_count);

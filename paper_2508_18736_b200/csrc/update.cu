@@ -205,18 +205,19 @@ update_small_kernel(const int32_t *__restrict__ idx, int idx_stride, const uint8
         __syncthreads();
         const int count = n_members_s;
         const int quads = D / 4;
-        for (int t = 0; t < count; t += 4) {
-            const int nrow = count - t < 4 ? count - t : 4;
-            const T *q[4];
+        constexpr int R = 8;                 // rows in flight per trip; additions stay in ascending row order
+        for (int t = 0; t < count; t += R) {
+            const int nrow = count - t < R ? count - t : R;
+            const T *q[R];
 #pragma unroll
-            for (int r = 0; r < 4; ++r) q[r] = Q + static_cast<int64_t>(members[t + (r < nrow ? r : 0)]) * D;
+            for (int r = 0; r < R; ++r) q[r] = Q + static_cast<int64_t>(members[t + (r < nrow ? r : 0)]) * D;
             for (int g = tid; g < quads; g += UP_THREADS) {
-                float4 v[4];
+                float4 v[R];
 #pragma unroll
-                for (int r = 0; r < 4; ++r) v[r] = load4<T>(q[r] + 4 * g);
+                for (int r = 0; r < R; ++r) v[r] = load4<T>(q[r] + 4 * g);
                 double a0 = acc[4 * g], a1 = acc[4 * g + 1], a2 = acc[4 * g + 2], a3 = acc[4 * g + 3];
 #pragma unroll
-                for (int r = 0; r < 4; ++r) {
+                for (int r = 0; r < R; ++r) {
                     if (r < nrow) { a0 += v[r].x; a1 += v[r].y; a2 += v[r].z; a3 += v[r].w; }
                 }
                 acc[4 * g] = a0; acc[4 * g + 1] = a1; acc[4 * g + 2] = a2; acc[4 * g + 3] = a3;
