@@ -374,7 +374,8 @@ siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const flo
     if (m_tiles64 > 0x7FFFFFFF) return SISO_ERR_UNSUPPORTED;
     const int m_tiles = static_cast<int>(m_tiles64);
     // CTA pairs (two query tiles share every centroid tile) whenever the batch has at least two query tiles
-    const bool pair = m_tiles >= 2 && c->tensor_pair_mode == 0;
+    // (an odd tile count is padded with an idle CTA: not worth it for 3, 5 or 7 query tiles)
+    const bool pair = m_tiles >= 2 && (m_tiles % 2 == 0 || m_tiles >= 9) && c->tensor_pair_mode == 0;
     const int m_ctas = pair ? (m_tiles + 1) / 2 * 2 : m_tiles;
     // One CTA per SM at a time.  Few, long splits keep each row's running top-k warm (a fresh CTA inserts often
     // until its k-th best has risen) but quantise badly into waves of sm_count CTAs; try a few wave counts and
