@@ -41,6 +41,12 @@ CASES = [
     (4, dict(n_centroids=2049, n_queries=129, dim=1024, n_clusters=64), "L", 4, ["simt", "tensor", "stream"]),
     (4, dict(n_centroids=999, n_queries=7, dim=1024, n_clusters=64), "P", 8, ["stream", "auto"]),
     (2, dict(n_centroids=640, n_queries=64, dim=72, n_clusters=32), "P", 2, ["simt", "tensor", "stream"]),
+    # largest supported dimension, a single query, three query tiles (single-CTA tensor kernel), nine (CTA pairs + padding)
+    (2, dict(n_centroids=300, n_queries=33, dim=4096, n_clusters=16), "L", 8, ["simt", "tensor", "stream"]),
+    (1, dict(n_centroids=300, n_queries=9, dim=4096, n_clusters=16), "L", 4, ["simt", "stream"]),
+    (4, dict(n_centroids=1500, n_queries=1, dim=1024, n_clusters=64), "P", 4, ["simt", "tensor", "stream", "auto"]),
+    (2, dict(n_centroids=1111, n_queries=300, dim=768, n_clusters=64), "L", 1, ["tensor"]),
+    (2, dict(n_centroids=700, n_queries=1100, dim=264, n_clusters=64), "L", 4, ["tensor", "auto"]),
 ]
 
 
