@@ -130,6 +130,7 @@ siso_status_t siso_cache_create(siso_cache_t **out, const siso_config_t *cfg) {
     if (cfg->allocator.alloc) { c->alloc = cfg->allocator; c->own_alloc = false; }
     else { c->alloc.alloc = default_alloc; c->alloc.free = default_free; c->alloc.ctx = nullptr; c->own_alloc = true; }
     c->lookup_path = SISO_PATH_AUTO;
+    c->stream_fused = 1;
     c->merge_max_cand = 16 * c->capacity + (1ll << 20);
 
     const size_t rows = static_cast<size_t>(c->rows_alloc), D = static_cast<size_t>(c->dim);
@@ -185,6 +186,10 @@ siso_status_t siso_set_option(siso_cache_t *c, int32_t key, int64_t value) {
         case SISO_OPT_TENSOR_CTA_PAIR:
             if (value != 0 && value != 1) return SISO_ERR_INVALID_ARG;
             c->tensor_pair_mode = static_cast<int32_t>(value);
+            return SISO_OK;
+        case SISO_OPT_STREAM_FUSED:
+            if (value != 0 && value != 1) return SISO_ERR_INVALID_ARG;
+            c->stream_fused = static_cast<int32_t>(value);
             return SISO_OK;
         case SISO_OPT_MERGE_MAX_CANDIDATES:
             if (value < 1 || value > (1ll << 31)) return SISO_ERR_INVALID_ARG;
@@ -313,6 +318,12 @@ siso_status_t siso_stream_step(siso_cache_t *c, const void *d_queries, int64_t n
     if (!c || n < 0) return SISO_ERR_INVALID_ARG;
     if (n == 0) return SISO_OK;
     SISO_TRY(siso_lookup(c, d_queries, n, d_theta, theta_scalar, 1, d_idx, d_sim, d_hit, stream));
+    // small batches: update, make-room and insertion in one cooperative launch
+    if (c->stream_fused) {
+        const siso_status_t st = launch_stream_maint(c, d_queries, n, d_idx, d_hit, d_victims, d_slots_out,
+                                                     static_cast<cudaStream_t>(stream));
+        if (st != SISO_ERR_UNSUPPORTED) return st;
+    }
     SISO_TRY(siso_update(c, d_queries, n, d_idx, 1, d_hit, stream));
     SISO_TRY(siso_make_room(c, d_hit, n, 0, d_victims, stream));
     return siso_insert_misses(c, d_queries, n, d_hit, d_slots_out, stream);

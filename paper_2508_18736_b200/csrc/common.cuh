@@ -48,6 +48,7 @@ struct Cache {
     size_t stage_bytes;
 
     int32_t lookup_path;
+    int32_t stream_fused;       // 1: siso_stream_step uses the fused maintenance kernel for small batches
     int32_t tensor_pair_mode;   // 0: CTA pairs when the batch spans two query tiles; 1: single-CTA kernel only
     int64_t merge_max_cand;
     int64_t launches;
@@ -55,6 +56,7 @@ struct Cache {
     // large-shared-memory opt-in is a per-device function attribute: remembered per cache, not per process
     bool simt_attr_set[2][3];   // [dtype][k class] of lookup_simt_kernel
     bool merge_attr_set;
+    int maint_grid;             // CTAs of the fused streaming maintenance kernel (0: not yet asked, -1: unavailable)
 };
 
 // ---- scratch bump allocator -------------------------------------------------
@@ -110,6 +112,8 @@ siso_status_t launch_sort_pairs(Cache *c, Scratch *scr, uint32_t *keys, uint32_t
                                 uint32_t *vals_tmp, int64_t n, int key_bits, uint32_t **keys_out, uint32_t **vals_out,
                                 cudaStream_t s);
 size_t sort_pairs_scratch_bytes(int64_t n);
+siso_status_t launch_stream_maint(Cache *c, const void *q, int64_t B, const int32_t *idx, const uint8_t *hit,
+                                  int32_t *victims, int32_t *slots_out, cudaStream_t s);
 siso_status_t launch_exclusive_scan_u32(Cache *c, uint32_t *a, int64_t n, cudaStream_t s);
 
 #ifdef __CUDACC__

@@ -12,26 +12,9 @@
 //   rank     one warp per candidate counts the candidates below it; rank < m means victim number rank
 // Keys are compared as three 64-bit integers (order-preserving image of the fp64 cluster_size, then
 // access_count | last_access | slot), so the order is the exact lexicographic order and total.
-#include "common.cuh"
+#include "evict_keys.cuh"
 
 namespace siso {
-
-struct Key3 {
-    unsigned long long w0, w1, w2;
-};
-__device__ __forceinline__ bool key_less(const Key3 &a, const Key3 &b) {
-    if (a.w0 != b.w0) return a.w0 < b.w0;
-    if (a.w1 != b.w1) return a.w1 < b.w1;
-    return a.w2 < b.w2;
-}
-__device__ __forceinline__ Key3 make_key(double size, uint32_t access, unsigned long long last, uint32_t slot) {
-    const unsigned long long u = static_cast<unsigned long long>(__double_as_longlong(size));
-    Key3 k;
-    k.w0 = (u >> 63) ? ~u : (u | 0x8000000000000000ull);          // order-preserving for every finite double
-    k.w1 = (static_cast<unsigned long long>(access) << 32) | (last >> 32);
-    k.w2 = (last << 32) | slot;
-    return k;
-}
 
 constexpr int EV_SAMPLE = 256;
 

@@ -300,3 +300,28 @@ def test_streaming_step_lockstep_on_a_scaled_twin(theta_mode):
     s = cache.stats()
     assert s["inserts"] - s["evictions"] == s["occupancy"] and s["lookups"] == sp.n_queries
     cache.check_status()
+
+
+def test_fused_streaming_maintenance_equals_separate_kernels_bit_for_bit():
+    sp = W.StreamSpec(capacity=1000, dim=72, n_queries=256 * 40, batch=256, n_clusters=700, zipf_s=1.2,
+                      reshuffle_every=256 * 20, theta=0.86, mode="P", dtype="bf16")
+    st = W.QueryStream(sp)
+    caches = []
+    for fused in (1, 0):
+        c = siso.SisoCache(sp.capacity, sp.dim, "bf16")
+        c.set_option(4, fused)
+        caches.append(c)
+    for t, q, _ in st.batches():
+        outs = [[x.cpu().numpy() for x in c.stream_step(to_dev(q, "bf16"), float(sp.theta))] for c in caches]
+        for x, y in zip(*outs):
+            assert (x == y).all(), f"batch {t}"
+    a, b = state_np(caches[0]), state_np(caches[1])
+    live = a["valid"] == 1
+    assert (a["valid"] == b["valid"]).all() and caches[0].stats() == caches[1].stats()
+    for k in ("master", "vecs", "size", "access", "last"):
+        assert (a[k][live] == b[k][live]).all(), k
+    assert caches[0].stats()["evictions"] > 0
+    assert caches[0].launch_count < caches[1].launch_count
+    for c in caches:
+        c.check_status()
+        c.close()
