@@ -207,13 +207,8 @@ siso_status_t siso_insert(siso_cache_t *c, const void *d_vecs, const double *d_s
     return launch_insert(c, d_vecs, d_sizes, nullptr, n, d_slots_out, static_cast<cudaStream_t>(stream));
 }
 
-siso_status_t siso_lookup(siso_cache_t *c, const void *d_queries, int64_t n_queries, const float *d_theta,
-                          float theta_scalar, int32_t k, int32_t *d_idx, float *d_sim, uint8_t *d_hit, void *stream) {
-    if (!c || n_queries < 0 || k < 1 || k > kMaxK) return SISO_ERR_INVALID_ARG;
-    if (n_queries == 0) return SISO_OK;
-    if (!d_queries || !d_idx || !d_sim || !d_hit || !aligned16(d_queries)) return SISO_ERR_INVALID_ARG;
-    SISO_CUDA(cudaSetDevice(c->device));
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
+// which kernel family serves a lookup of n_queries rows
+static int resolve_lookup_path(const siso_cache_t *c, int64_t n_queries) {
     int path = c->lookup_path;
     if (path == SISO_PATH_AUTO) {
         // measured on B200: the streaming kernel holds 92 % of HBM peak for 1-2 queries and falls off beyond;
@@ -221,7 +216,17 @@ siso_status_t siso_lookup(siso_cache_t *c, const void *d_queries, int64_t n_quer
         if (c->dtype == SISO_BF16) path = n_queries <= 2 ? SISO_PATH_STREAM : SISO_PATH_TENSOR;
         else path = n_queries <= 4 ? SISO_PATH_STREAM : SISO_PATH_SIMT;
     }
-    switch (path) {
+    return path;
+}
+
+siso_status_t siso_lookup(siso_cache_t *c, const void *d_queries, int64_t n_queries, const float *d_theta,
+                          float theta_scalar, int32_t k, int32_t *d_idx, float *d_sim, uint8_t *d_hit, void *stream) {
+    if (!c || n_queries < 0 || k < 1 || k > kMaxK) return SISO_ERR_INVALID_ARG;
+    if (n_queries == 0) return SISO_OK;
+    if (!d_queries || !d_idx || !d_sim || !d_hit || !aligned16(d_queries)) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    switch (resolve_lookup_path(c, n_queries)) {
         case SISO_PATH_STREAM: return launch_lookup_stream(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);
         case SISO_PATH_TENSOR: return launch_lookup_tensor(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);
         default: return launch_lookup_simt(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);
@@ -317,13 +322,23 @@ siso_status_t siso_stream_step(siso_cache_t *c, const void *d_queries, int64_t n
                                int32_t *d_slots_out, void *stream) {
     if (!c || n < 0) return SISO_ERR_INVALID_ARG;
     if (n == 0) return SISO_OK;
-    SISO_TRY(siso_lookup(c, d_queries, n, d_theta, theta_scalar, 1, d_idx, d_sim, d_hit, stream));
-    // small batches: update, make-room and insertion in one cooperative launch
-    if (c->stream_fused) {
-        const siso_status_t st = launch_stream_maint(c, d_queries, n, d_idx, d_hit, d_victims, d_slots_out,
-                                                     static_cast<cudaStream_t>(stream));
-        if (st != SISO_ERR_UNSUPPORTED) return st;
+    if (!d_queries || !d_idx || !d_sim || !d_hit || !aligned16(d_queries)) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // small batches: update, make-room and insertion in one cooperative launch, which also finishes the lookup
+    // (best key over the splits, threshold test) when the tensor-core kernel produced it
+    if (c->stream_fused && stream_maint_supported(c, n)) {
+        if (resolve_lookup_path(c, n) == SISO_PATH_TENSOR) {
+            DeferredTop1 top1;
+            void *tail = nullptr;
+            SISO_TRY(launch_lookup_tensor(c, d_queries, n, d_theta, theta_scalar, 1, d_idx, d_sim, d_hit, s, &top1,
+                                          stream_maint_scratch_bytes(c, n), &tail));
+            return launch_stream_maint(c, d_queries, n, d_idx, d_hit, d_victims, d_slots_out, &top1, tail, s);
+        }
+        SISO_TRY(siso_lookup(c, d_queries, n, d_theta, theta_scalar, 1, d_idx, d_sim, d_hit, stream));
+        return launch_stream_maint(c, d_queries, n, d_idx, d_hit, d_victims, d_slots_out, nullptr, nullptr, s);
     }
+    SISO_TRY(siso_lookup(c, d_queries, n, d_theta, theta_scalar, 1, d_idx, d_sim, d_hit, stream));
     SISO_TRY(siso_update(c, d_queries, n, d_idx, 1, d_hit, stream));
     SISO_TRY(siso_make_room(c, d_hit, n, 0, d_victims, stream));
     return siso_insert_misses(c, d_queries, n, d_hit, d_slots_out, stream);

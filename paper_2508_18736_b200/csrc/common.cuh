@@ -94,8 +94,19 @@ siso_status_t launch_lookup_simt(Cache *c, const void *q, int64_t B, const float
                                  int32_t *idx, float *sim, uint8_t *hit, cudaStream_t s);
 siso_status_t launch_lookup_stream(Cache *c, const void *q, int64_t B, const float *theta, float theta_s, int k,
                                    int32_t *idx, float *sim, uint8_t *hit, cudaStream_t s);
+// A top-1 lookup whose last step (best key over the splits, threshold test) is left to a later kernel.
+struct DeferredTop1 {
+    const unsigned long long *partial;     // [B, splits] packed (similarity, slot) keys, 0 = no entry
+    int splits;
+    const float *theta;
+    float theta_s;
+    float *sim;                            // [B] out
+};
+// With `defer` (k must be 1) the finalisation kernel is not launched; *defer receives the partial results and
+// *tail points to `tail_bytes` of the cache's scratch that stay untouched by the lookup.
 siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const float *theta, float theta_s, int k,
-                                   int32_t *idx, float *sim, uint8_t *hit, cudaStream_t s);
+                                   int32_t *idx, float *sim, uint8_t *hit, cudaStream_t s,
+                                   DeferredTop1 *defer = nullptr, size_t tail_bytes = 0, void **tail = nullptr);
 void tensor_state_destroy(Cache *c);
 siso_status_t launch_topk_finalize(Cache *c, const unsigned long long *partial, int64_t B, int splits, int kmax, int k,
                                    const float *theta, float theta_s, int32_t *idx, float *sim, uint8_t *hit,
@@ -112,8 +123,10 @@ siso_status_t launch_sort_pairs(Cache *c, Scratch *scr, uint32_t *keys, uint32_t
                                 uint32_t *vals_tmp, int64_t n, int key_bits, uint32_t **keys_out, uint32_t **vals_out,
                                 cudaStream_t s);
 size_t sort_pairs_scratch_bytes(int64_t n);
-siso_status_t launch_stream_maint(Cache *c, const void *q, int64_t B, const int32_t *idx, const uint8_t *hit,
-                                  int32_t *victims, int32_t *slots_out, cudaStream_t s);
+bool stream_maint_supported(Cache *c, int64_t B);
+size_t stream_maint_scratch_bytes(const Cache *c, int64_t B);
+siso_status_t launch_stream_maint(Cache *c, const void *q, int64_t B, int32_t *idx, uint8_t *hit, int32_t *victims,
+                                  int32_t *slots_out, const DeferredTop1 *deferred, void *scratch_tail, cudaStream_t s);
 siso_status_t launch_exclusive_scan_u32(Cache *c, uint32_t *a, int64_t n, cudaStream_t s);
 
 #ifdef __CUDACC__

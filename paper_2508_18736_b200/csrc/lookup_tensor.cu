@@ -72,6 +72,18 @@ __device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, i
                  ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar))
                  : "memory");
 }
+// the same load with an L2 eviction policy: used for centroid tiles that no other CTA will read again, so that the
+// one-pass stream does not push the queries, the cache's metadata and the kernels' code out of L2
+__device__ __forceinline__ void tma_load_2d_hint(void *dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar, uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar)), "l"(policy)
+                 : "memory");
+}
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void umma_commit(uint64_t *bar) {
@@ -133,7 +145,7 @@ template <int KMAX>
 __global__ void __launch_bounds__(THREADS, 1)
 lookup_tensor_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_c,
                      const uint8_t *__restrict__ valid, int64_t B, int D, int tiles_per_split, int n_tiles,
-                     unsigned long long *__restrict__ partial, int splits, int *status) {
+                     unsigned long long *__restrict__ partial, int splits, int stream_c, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     Barriers *bars = reinterpret_cast<Barriers *>(tiles + STAGES * STAGE_BYTES);
@@ -170,6 +182,7 @@ lookup_tensor_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
+            const uint64_t policy = stream_c ? l2_evict_first_policy() : 0ull;
             for (int t = t_begin; t < t_end && ok; ++t) {
                 const int n0 = t * TN;
                 for (int ks = 0; ks < k_slabs; ++ks) {
@@ -178,7 +191,8 @@ lookup_tensor_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
                     uint8_t *b_dst = a_dst + A_BYTES;
                     mbar_arrive_expect_tx(&bars->full[stage], STAGE_BYTES);
                     tma_load_2d(a_dst, &map_q, ks * TK, q0, &bars->full[stage]);
-                    tma_load_2d(b_dst, &map_c, ks * TK, n0, &bars->full[stage]);
+                    if (stream_c) tma_load_2d_hint(b_dst, &map_c, ks * TK, n0, &bars->full[stage], policy);
+                    else tma_load_2d(b_dst, &map_c, ks * TK, n0, &bars->full[stage]);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -339,15 +353,18 @@ static siso_status_t run_tensor(Cache *c, tc::TensorState *ts, int slot, const C
         ts->attr_set[slot] = true;
     }
     dim3 grid(m_tiles, splits);
+    // one query tile: every centroid tile is read by exactly one CTA, so it need not stay in L2
     kern<<<grid, tc::THREADS, tc::SMEM_BYTES, s>>>(map_q, ts->map_c, c->valid, B, c->dim, tiles_per_split, n_tiles,
-                                                   partial, splits, c->status);
+                                                   partial, splits, m_tiles == 1 ? 1 : 0, c->status);
     SISO_LAUNCHED(c);
     return SISO_OK;
 }
 
 siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const float *theta, float theta_s, int k,
-                                   int32_t *idx, float *sim, uint8_t *hit, cudaStream_t s) {
+                                   int32_t *idx, float *sim, uint8_t *hit, cudaStream_t s, DeferredTop1 *defer,
+                                   size_t tail_bytes, void **tail) {
     if (c->dtype != SISO_BF16) return SISO_ERR_UNSUPPORTED;
+    if (defer && (k != 1 || !tail)) return SISO_ERR_INVALID_ARG;
     auto *ts = static_cast<tc::TensorState *>(c->tensor_state);
     if (!ts) {
         ts = new tc::TensorState();
@@ -396,7 +413,7 @@ siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const flo
     }
 
     Scratch scr;
-    SISO_TRY(scratch_reserve(c, pad256(sizeof(unsigned long long) * B * splits * kmax), s, &scr));
+    SISO_TRY(scratch_reserve(c, pad256(sizeof(unsigned long long) * B * splits * kmax) + (defer ? tail_bytes : 0), s, &scr));
     unsigned long long *partial = scr.take<unsigned long long>(static_cast<size_t>(B) * splits * kmax);
     siso_status_t st;
     if (pair)
@@ -407,6 +424,15 @@ siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const flo
            : kmax == 4 ? run_tensor<4>(c, ts, 1, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s)
                        : run_tensor<8>(c, ts, 2, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s);
     SISO_TRY(st);
+    if (defer) {
+        defer->partial = partial;
+        defer->splits = splits;
+        defer->theta = theta;
+        defer->theta_s = theta_s;
+        defer->sim = sim;
+        *tail = scr.base + scr.off;
+        return SISO_OK;
+    }
     return launch_topk_finalize(c, partial, B, splits, kmax, k, theta, theta_s, idx, sim, hit, s);
 }
 

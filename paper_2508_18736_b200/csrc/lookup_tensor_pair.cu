@@ -85,6 +85,18 @@ __device__ __forceinline__ void tma_load_2d_pair(void *dst, const CUtensorMap *m
                  ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar_cluster_addr)
                  : "memory");
 }
+// the same load with an L2 eviction policy (centroid tiles that no other cluster will read again)
+__device__ __forceinline__ void tma_load_2d_pair_hint(void *dst, const CUtensorMap *map, int c0, int c1, uint32_t bar_cluster_addr,
+                                                      uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.2d.cta_group::2.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar_cluster_addr), "l"(policy)
+                 : "memory");
+}
+__device__ __forceinline__ uint64_t l2_evict_first_policy() {
+    uint64_t p;
+    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
+    return p;
+}
 __device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
 __device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
 // Arrive, once all MMAs issued so far have completed, on the barrier at this shared-memory offset in BOTH
@@ -147,7 +159,7 @@ template <int KMAX>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 lookup_tensor_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_c_half,
                           const uint8_t *__restrict__ valid, int64_t B, int D, int tiles_per_split, int n_tiles,
-                          unsigned long long *__restrict__ partial, int splits, int *status) {
+                          unsigned long long *__restrict__ partial, int splits, int stream_c, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     Barriers *bars = reinterpret_cast<Barriers *>(tiles + STAGES * STAGE_BYTES);
@@ -184,6 +196,7 @@ lookup_tensor_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
+            const uint64_t policy = stream_c ? l2_evict_first_policy() : 0ull;
             for (int t = t_begin; t < t_end && ok; ++t) {
                 const int n0 = t * TN + static_cast<int>(rank) * (TN / 2);     // this CTA's half of the centroid tile
                 for (int ks = 0; ks < k_slabs; ++ks) {
@@ -193,7 +206,8 @@ lookup_tensor_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
                     const uint32_t full_leader = cluster_addr(smem_u32(&bars->full[stage]), 0);
                     if (rank == 0) mbar_arrive_expect_tx(&bars->full[stage], 2 * STAGE_BYTES);   // both CTAs' bytes
                     tma_load_2d_pair(a_dst, &map_q, ks * TK, q0, full_leader);
-                    tma_load_2d_pair(b_dst, &map_c_half, ks * TK, n0, full_leader);
+                    if (stream_c) tma_load_2d_pair_hint(b_dst, &map_c_half, ks * TK, n0, full_leader, policy);
+                    else tma_load_2d_pair(b_dst, &map_c_half, ks * TK, n0, full_leader);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -318,8 +332,9 @@ static siso_status_t run_pair(Cache *c, bool *attr_set, const CUtensorMap &map_q
         *attr_set = true;
     }
     dim3 grid(m_tiles_even, splits);
+    // one pair covers the whole batch: every centroid tile is read by exactly one cluster, so it need not stay in L2
     kern<<<grid, tc2::THREADS, tc2::SMEM_BYTES, s>>>(map_q, map_c_half, c->valid, B, c->dim, tiles_per_split, n_tiles,
-                                                     partial, splits, c->status);
+                                                     partial, splits, m_tiles_even == 2 ? 1 : 0, c->status);
     SISO_LAUNCHED(c);
     return SISO_OK;
 }

@@ -1,14 +1,23 @@
-// Maintenance of one streaming micro-batch in ONE cooperative launch: hit update, eviction of what the misses
-// lack in free slots, insertion of the misses.  As separate launches these are eight small kernels whose
-// launch and drain latencies add up to about as much as the lookup itself; here the phases are separated by
-// grid-wide barriers instead.  The arithmetic and every ordering rule are those of update.cu and evict.cu:
-//   U   CTA per row: the first hit of a slot owns the slot's group (ascending query order, fp64 sums)
-//   E1  CTA 0: m = max(0, misses - free slots); strided sample of 256 live entries, sorted -> splitters
-//   E2  all: bucket of every live entry (binary search among the splitters), bucket counts
-//   E3  all: entries in the buckets up to the one where the cumulative count reaches m -> candidates
-//   E4  all: one warp per candidate counts the candidates below it; rank < m = victim number rank
-//   I1  all: free slots per CTA slice;  I2 all: first #miss free slots in ascending order
-//   I3  CTA per row: miss number r takes free slot number r
+// Maintenance of one streaming micro-batch in ONE cooperative launch: (top-1 finalisation of the lookup,) hit
+// update, eviction of what the misses lack in free slots, insertion of the misses.  As separate launches these
+// are ten small kernels whose launch and drain latencies add up to about as much as the lookup itself; here the
+// phases are separated by grid-wide barriers, four of them in the steady state.  The arithmetic and every
+// ordering rule are those of update.cu and evict.cu (Alg. 1 FilteringCentroids order; running-mean update):
+//   F   (only when the lookup left its per-split partial results) one warp per row: best key, threshold test
+//   U   CTA per row: the first hit of a slot owns the slot's group (ascending query order, fp64 sums);
+//       meanwhile the last CTA draws a strided sample of 256 live entries and puts its P+1 smallest keys in
+//       order -> splitters 0..P (P chosen so that about 3 m entries lie below splitter P)
+//   S   CTA g owns the contiguous slice g of the slots: free slots of the slice; entries whose key is at most
+//       splitter P become candidates, counted per bucket
+//   R   p = first bucket where the cumulative count reaches m; every fourth CTA copies the candidates up to
+//       splitter p to shared memory and ranks its share of them (one warp per candidate); rank < m = victim
+//       number rank
+//   I   the first #miss free slots in ascending order take the misses in ascending row order.  A full cache has
+//       no free slots but the victims, so every CTA sorts the victims by slot and copies its share of the rows;
+//       otherwise each CTA lists the free slots of its slice, and after one more barrier all CTAs copy
+// If the sample misleads (fewer than m candidates) the selection falls back to a full sort of the sample, a full
+// histogram pass and a collection pass, as evict.cu does.  Whatever the splitters are, the victims are the m
+// smallest keys exactly.
 // Used by siso_stream_step for batches of at most 1024 rows; larger batches take the separate kernels.
 #include <cooperative_groups.h>
 
@@ -22,20 +31,22 @@ constexpr int SM_THREADS = 256;
 constexpr int SM_WARPS = SM_THREADS / 32;
 constexpr int SM_MAX_B = 1024;
 constexpr int SM_SAMPLE = 256;
+constexpr int SM_STAGE = 2048;      // candidates a CTA can hold in shared memory while ranking
+constexpr int SM_SELECT = 16;       // up to this many splitters are extracted one by one instead of sorting the sample
+constexpr int SM_RANK_STRIDE = 4;   // every fourth CTA ranks candidates
 
 struct MaintCtl {
-    long long m;                       // victims of this batch
+    unsigned int n_cand;                 // candidates appended in phase S
+    unsigned int n_cand_full;            // candidates of the fall-back collection
     int n_sample;
-    unsigned int n_cand;
-    int n_miss;
-    int insert_ok;
-    unsigned int hist[SM_SAMPLE + 1];
+    unsigned int hist[SM_SAMPLE + 1];    // phase S: buckets 0..P
+    unsigned int hist_full[SM_SAMPLE + 1];
 };
 
 struct MaintArgs {
     const void *Q;
-    const int32_t *idx;                // [B] best slot per row (stride 1)
-    const uint8_t *hit;                // [B]
+    int32_t *idx;                      // [B] best slot per row (stride 1); written by phase F
+    uint8_t *hit;                      // [B]
     int B, D;
     long long capacity;
     void *vecs;
@@ -48,14 +59,39 @@ struct MaintArgs {
     int *status;
     int32_t *victims;                  // [B] or NULL
     int32_t *slots_out;                // [B] or NULL
+    // phase F (partial == NULL: idx and hit are inputs)
+    const unsigned long long *partial; // [B, splits] packed (similarity, slot) keys
+    int splits;
+    const float *theta;
+    float theta_s;
+    float *sim;                        // [B]
     // scratch
     MaintCtl *ctl;
     Key3 *splitters;                   // [SM_SAMPLE]
-    uint16_t *bucket;                  // [capacity]
-    Key3 *cand;                        // [capacity]
+    uint16_t *bucket;                  // [capacity] (fall-back only)
+    unsigned long long *cand0, *cand1, *cand2;   // [capacity] each: the candidates' key words
+    int32_t *victim_buf;               // [B] victims in key order (always present, unlike `victims`)
     int *cta_free;                     // [grid]
     int32_t *free_list;                // [B]
 };
+
+// fixed part of the shared memory; it follows the 48 KiB that hold the fp64 row accumulator during the update and
+// the candidates during ranking
+struct MaintSmem {
+    unsigned long long k0[SM_SAMPLE], k1[SM_SAMPLE], k2[SM_SAMPLE];    // splitters (sorting area of the sampler)
+    double red[SM_WARPS];
+    unsigned int hist[SM_SAMPLE + 1];
+    int warp_sum[SM_WARPS];
+    int32_t idx[SM_MAX_B];
+    uint16_t miss_list[SM_MAX_B];
+    uint16_t members[SM_MAX_B];
+    uint8_t hit[SM_MAX_B];
+    int n_stage;
+    int p;
+};
+constexpr size_t SM_UNION_BYTES = 3 * sizeof(unsigned long long) * SM_STAGE;      // 48 KiB >= 8 * kMaxDim
+constexpr size_t SM_SMEM_BYTES = SM_UNION_BYTES + sizeof(MaintSmem);
+static_assert(SM_UNION_BYTES >= sizeof(double) * kMaxDim, "row accumulator must fit");
 
 __device__ __forceinline__ int block_exclusive_scan_256(int v, int *total, int *warp_sum) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
@@ -78,6 +114,18 @@ __device__ __forceinline__ int block_exclusive_scan_256(int v, int *total, int *
     return before + x - v;
 }
 
+__device__ __forceinline__ int block_max_256(int v, int *warp_sum) {
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) v = max(v, __shfl_xor_sync(0xFFFFFFFFu, v, o));
+    __syncthreads();
+    if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = v;
+    __syncthreads();
+    int r = warp_sum[0];
+#pragma unroll
+    for (int w = 1; w < SM_WARPS; ++w) r = max(r, warp_sum[w]);
+    return r;
+}
+
 template <typename T> __device__ __forceinline__ float4 maint_load4(const T *p);
 template <> __device__ __forceinline__ float4 maint_load4<float>(const float *p) { return __ldg(reinterpret_cast<const float4 *>(p)); }
 template <> __device__ __forceinline__ float4 maint_load4<__nv_bfloat16>(const __nv_bfloat16 *p) {
@@ -86,15 +134,43 @@ template <> __device__ __forceinline__ float4 maint_load4<__nv_bfloat16>(const _
                        __uint_as_float(u.y & 0xFFFF0000u));
 }
 
-struct MaintSmem {
-    double red[SM_WARPS];
-    int warp_sum[SM_WARPS];
-    int n_members;
-    int p;
-    uint16_t members[SM_MAX_B];
-    unsigned long long k0[SM_SAMPLE], k1[SM_SAMPLE], k2[SM_SAMPLE];
-    unsigned int hist[SM_SAMPLE + 1];
-};
+__device__ __forceinline__ Key3 smem_key(const MaintSmem &sm, int i) {
+    Key3 k;
+    k.w0 = sm.k0[i]; k.w1 = sm.k1[i]; k.w2 = sm.k2[i];
+    return k;
+}
+
+// number of splitters among the first n that are smaller than k
+__device__ __forceinline__ int splitter_lower_bound(const MaintSmem &sm, int n, const Key3 &k) {
+    int lo = 0, hi = n;
+    while (lo < hi) {
+        const int mid = (lo + hi) >> 1;
+        if (key_less(smem_key(sm, mid), k)) lo = mid + 1; else hi = mid;
+    }
+    return lo;
+}
+
+// ---- phase F: best key of every row over the lookup's splits, strict threshold test --------------------------
+__device__ void maint_finalize(const MaintArgs &a) {
+    const int lane = threadIdx.x & 31;
+    const int warps = gridDim.x * SM_WARPS;
+    for (int b = blockIdx.x * SM_WARPS + (threadIdx.x >> 5); b < a.B; b += warps) {
+        const unsigned long long *src = a.partial + static_cast<long long>(b) * a.splits;
+        unsigned long long best = 0ull;
+        for (int s = lane; s < a.splits; s += 32) { const unsigned long long v = src[s]; best = v > best ? v : best; }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) {
+            const unsigned long long v = __shfl_xor_sync(0xFFFFFFFFu, best, o);
+            best = v > best ? v : best;
+        }
+        if (lane == 0) {
+            a.idx[b] = best ? key_slot(best) : -1;
+            a.sim[b] = best ? key_sim(best) : -INFINITY;
+            const float th = a.theta ? a.theta[b] : a.theta_s;
+            a.hit[b] = (best != 0ull && key_sim(best) > th) ? 1 : 0;
+        }
+    }
+}
 
 // ---- phase U: hit update of the group that row b heads (see update_small_kernel in update.cu) ----------------
 template <typename T>
@@ -102,22 +178,35 @@ __device__ void maint_update_row(const MaintArgs &a, int b, long long clock_new,
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const T *Q = static_cast<const T *>(a.Q);
     T *vecs = static_cast<T *>(a.vecs);
-    bool work = false;
+    constexpr int MR = 4;                       // master elements per thread fetched ahead (covers D <= 1024)
     long long slot = -1;
-    if (a.hit[b]) {
-        slot = a.idx[b];
-        if (slot >= 0 && slot < a.capacity && a.valid[slot]) work = true;
-        else if (tid == 0) set_status(a.status, SISO_ERR_INVALID_ARG);
+    bool work = false;
+    double n_old = 0.0;
+    uint32_t ac_old = 0;
+    float mreg[MR];
+    if (sm.hit[b]) {
+        slot = sm.idx[b];
+        if (slot >= 0 && slot < a.capacity) {
+            // everything the update reads of the slot is requested at once, before the ownership test below
+            const uint8_t live = a.valid[slot];
+            n_old = a.size[slot];
+            ac_old = a.access[slot];
+            const float *m = a.master + slot * a.D;
+#pragma unroll
+            for (int j = 0; j < MR; ++j) { const int d = tid + j * SM_THREADS; mreg[j] = d < a.D ? m[d] : 0.0f; }
+            work = live != 0;
+        }
+        if (!work && tid == 0) set_status(a.status, SISO_ERR_INVALID_ARG);
     }
     int earlier = 0;
     if (work)
-        for (int r = tid; r < b; r += SM_THREADS) earlier |= (a.hit[r] && a.idx[r] == slot) ? 1 : 0;
+        for (int r = tid; r < b; r += SM_THREADS) earlier |= (sm.hit[r] && sm.idx[r] == slot) ? 1 : 0;
     if (__syncthreads_or(earlier) != 0) work = false;      // an earlier row owns this slot's group
     if (!work) return;                                      // uniform for the CTA
     int base_count = 0;
     for (int r0 = b; r0 < a.B; r0 += SM_THREADS) {
         const int r = r0 + tid;
-        const bool mine = r < a.B && a.hit[r] && a.idx[r] == slot;
+        const bool mine = r < a.B && sm.hit[r] && sm.idx[r] == slot;
         const unsigned ballot = __ballot_sync(0xFFFFFFFFu, mine);
         if (lane == 0) sm.warp_sum[warp] = __popc(ballot);
         __syncthreads();
@@ -128,12 +217,13 @@ __device__ void maint_update_row(const MaintArgs &a, int b, long long clock_new,
         __syncthreads();
     }
     const int count = base_count;
-    const double n_old = a.size[slot];
     float *m = a.master + slot * a.D;
-    for (int d = tid; d < a.D; d += SM_THREADS) acc[d] = n_old * static_cast<double>(m[d]);
+#pragma unroll
+    for (int j = 0; j < MR; ++j) { const int d = tid + j * SM_THREADS; if (d < a.D) acc[d] = n_old * static_cast<double>(mreg[j]); }
+    for (int d = tid + MR * SM_THREADS; d < a.D; d += SM_THREADS) acc[d] = n_old * static_cast<double>(m[d]);
     __syncthreads();
     const int quads = a.D / 4;
-    constexpr int R = 8;
+    constexpr int R = 16;                       // rows in flight per thread
     for (int t = 0; t < count; t += R) {
         const int nrow = count - t < R ? count - t : R;
         const T *q[R];
@@ -169,29 +259,50 @@ __device__ void maint_update_row(const MaintArgs &a, int b, long long clock_new,
     }
     if (tid == 0) {
         a.size[slot] = n_old + static_cast<double>(count);
-        const unsigned long long ac = static_cast<unsigned long long>(a.access[slot]) + static_cast<unsigned long long>(count);
-        a.access[slot] = (a.access[slot] == SISO_ACCESS_INF || ac >= SISO_ACCESS_INF) ? SISO_ACCESS_INF : static_cast<uint32_t>(ac);
+        const unsigned long long ac = static_cast<unsigned long long>(ac_old) + static_cast<unsigned long long>(count);
+        a.access[slot] = (ac_old == SISO_ACCESS_INF || ac >= SISO_ACCESS_INF) ? SISO_ACCESS_INF : static_cast<uint32_t>(ac);
         a.last[slot] = static_cast<unsigned long long>(clock_new);
     }
     __syncthreads();      // acc and members are reused by the CTA's next row
 }
 
-// ---- phase E1 (CTA 0): how many victims; sample and sort the splitters ------------------------------------------
-__device__ void maint_evict_sample(const MaintArgs &a, long long clock_new, MaintSmem &sm) {
+// splitter index P: entries with a key up to splitter P are looked at (about 3 m of them are expected)
+__device__ __forceinline__ int maint_spec_buckets(long long m, int n_sample, long long occupancy) {
+    if (n_sample == 0) return 0;
+    const long long want = (3 * m * (n_sample + 1) + occupancy - 1) / occupancy + 1;
+    return static_cast<int>(want < n_sample ? want : n_sample);
+}
+
+// smallest key of the CTA's 256 (each thread passes its own); all threads get it
+__device__ __forceinline__ Key3 block_min_key(Key3 k, MaintSmem &sm) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        Key3 y;
+        y.w0 = __shfl_xor_sync(0xFFFFFFFFu, k.w0, o);
+        y.w1 = __shfl_xor_sync(0xFFFFFFFFu, k.w1, o);
+        y.w2 = __shfl_xor_sync(0xFFFFFFFFu, k.w2, o);
+        if (key_less(y, k)) k = y;
+    }
+    __syncthreads();
+    if (lane == 0) { sm.k0[warp] = k.w0; sm.k1[warp] = k.w1; sm.k2[warp] = k.w2; }
+    __syncthreads();
+    Key3 best = smem_key(sm, 0);
+#pragma unroll
+    for (int w = 1; w < SM_WARPS; ++w) {
+        const Key3 y = smem_key(sm, w);
+        if (key_less(y, best)) best = y;
+    }
+    return best;
+}
+
+// ---- sampler (one CTA): strided sample of live entries -> splitters ------------------------------------------
+// The sample only steers the selection (which entries are looked at closely), so it may see an entry before or
+// after this batch's update of it.  With `all` the whole sample is sorted; otherwise only its P+1 smallest keys
+// are put in order (P as maint_spec_buckets gives it), which is all that phases S and R read.
+__device__ void maint_evict_sample(const MaintArgs &a, long long clock_new, long long m, long long occupancy, bool all,
+                                   MaintSmem &sm) {
     const int tid = threadIdx.x;
-    const long long occupancy = a.counters[CNT_OCCUPANCY];
-    int miss = 0;
-    for (int b = tid; b < a.B; b += SM_THREADS) miss += a.hit[b] ? 0 : 1;
-    int n_miss;
-    block_exclusive_scan_256(miss, &n_miss, sm.warp_sum);
-    long long m = static_cast<long long>(n_miss) - (a.capacity - occupancy);
-    m = m > 0 ? m : 0;
-    m = m < occupancy ? m : occupancy;
-    if (a.victims)
-        for (long long r = m + tid; r < a.B; r += SM_THREADS) a.victims[r] = -1;
-    if (tid == 0) { a.ctl->m = m; a.ctl->n_cand = 0; a.ctl->n_miss = n_miss; }
-    for (int i = tid; i <= SM_SAMPLE; i += SM_THREADS) a.ctl->hist[i] = 0;
-    if (m == 0) return;
     const long long stride = (a.capacity + SM_SAMPLE - 1) / SM_SAMPLE;
     const long long lo = tid * stride, hi = min(a.capacity, lo + stride);
     const long long span = hi - lo;
@@ -199,82 +310,150 @@ __device__ void maint_evict_sample(const MaintArgs &a, long long clock_new, Main
     Key3 mine;
     mine.w0 = mine.w1 = mine.w2 = ~0ull;
     if (span > 0) {
-        // the same window offset as evict_sample_kernel uses, which reads the clock after the update advanced it
         const long long start = static_cast<long long>((static_cast<unsigned long long>(clock_new) * 2654435761ull) % static_cast<unsigned long long>(span));
         const long long probes = span < 64 ? span : 64;
         for (long long i = 0; i < probes; ++i) {
             long long sl = lo + start + i;
             if (sl >= hi) sl -= span;
-            if (a.valid[sl]) { mine = make_key(a.size[sl], a.access[sl], a.last[sl], static_cast<uint32_t>(sl)); have = 1; break; }
+            // the four loads do not wait for one another: a full cache answers at the first probe
+            const uint8_t live = a.valid[sl];
+            const double sz = a.size[sl];
+            const uint32_t ac = a.access[sl];
+            const unsigned long long la = a.last[sl];
+            if (live) { mine = make_key(sz, ac, la, static_cast<uint32_t>(sl)); have = 1; break; }
         }
     }
-    sm.k0[tid] = mine.w0; sm.k1[tid] = mine.w1; sm.k2[tid] = mine.w2;
     int n_sample;
     block_exclusive_scan_256(have, &n_sample, sm.warp_sum);
-    __syncthreads();
-    for (int k = 2; k <= SM_SAMPLE; k <<= 1) {
-        for (int j = k >> 1; j > 0; j >>= 1) {
-            const int partner = tid ^ j;
-            if (partner > tid) {
-                Key3 x, y;
-                x.w0 = sm.k0[tid]; x.w1 = sm.k1[tid]; x.w2 = sm.k2[tid];
-                y.w0 = sm.k0[partner]; y.w1 = sm.k1[partner]; y.w2 = sm.k2[partner];
-                const bool up = (tid & k) == 0;
-                if (key_less(y, x) == up) {
-                    sm.k0[tid] = y.w0; sm.k1[tid] = y.w1; sm.k2[tid] = y.w2;
-                    sm.k0[partner] = x.w0; sm.k1[partner] = x.w1; sm.k2[partner] = x.w2;
-                }
-            }
-            __syncthreads();
+    const int P = maint_spec_buckets(m, n_sample, occupancy);
+    if (!all && P < SM_SELECT && P < n_sample) {
+        // the P+1 smallest, one block-wide minimum at a time (keys differ in their slot word)
+        for (int r = 0; r <= P; ++r) {
+            const Key3 best = block_min_key(mine, sm);
+            if (tid == 0) a.splitters[r] = best;
+            if (mine.w0 == best.w0 && mine.w1 == best.w1 && mine.w2 == best.w2) mine.w0 = mine.w1 = mine.w2 = ~0ull;
         }
+    } else {
+        __syncthreads();
+        sm.k0[tid] = mine.w0; sm.k1[tid] = mine.w1; sm.k2[tid] = mine.w2;
+        __syncthreads();
+        for (int k = 2; k <= SM_SAMPLE; k <<= 1) {
+            for (int j = k >> 1; j > 0; j >>= 1) {
+                const int partner = tid ^ j;
+                if (partner > tid) {
+                    const Key3 x = smem_key(sm, tid), y = smem_key(sm, partner);
+                    const bool up = (tid & k) == 0;
+                    if (key_less(y, x) == up) {
+                        sm.k0[tid] = y.w0; sm.k1[tid] = y.w1; sm.k2[tid] = y.w2;
+                        sm.k0[partner] = x.w0; sm.k1[partner] = x.w1; sm.k2[partner] = x.w2;
+                    }
+                }
+                __syncthreads();
+            }
+        }
+        a.splitters[tid] = smem_key(sm, tid);
     }
-    Key3 out;
-    out.w0 = sm.k0[tid]; out.w1 = sm.k1[tid]; out.w2 = sm.k2[tid];
-    a.splitters[tid] = out;
     if (tid == 0) a.ctl->n_sample = n_sample;
 }
 
-// ---- phase E2 (all CTAs): bucket of every live entry ------------------------------------------------------------
-__device__ void maint_evict_bucket(const MaintArgs &a, MaintSmem &sm) {
-    if (a.ctl->m == 0) return;
-    const int tid = threadIdx.x;
-    const int n_sample = a.ctl->n_sample;
-    {
-        const Key3 k = a.splitters[tid];
-        sm.k0[tid] = k.w0; sm.k1[tid] = k.w1; sm.k2[tid] = k.w2;
+// ---- phase S (all CTAs): free slots of the slice; candidates up to splitter P ----------------------------------
+struct MetaChunk {
+    static constexpr int U = 4;
+    uint8_t v[U];
+    double sz[U];
+    uint32_t ac[U];
+    unsigned long long la[U];
+};
+__device__ __forceinline__ void maint_load_chunk(const MaintArgs &a, long long base, long long hi, MetaChunk &c) {
+#pragma unroll
+    for (int j = 0; j < MetaChunk::U; ++j) {
+        const long long sl = base + j * SM_THREADS + threadIdx.x;
+        const bool in = sl < hi;
+        c.v[j] = in ? a.valid[sl] : 1;
+        c.sz[j] = in ? a.size[sl] : 0.0;
+        c.ac[j] = in ? a.access[sl] : 0u;
+        c.la[j] = in ? a.last[sl] : 0ull;
     }
-    for (int i = tid; i <= SM_SAMPLE; i += SM_THREADS) sm.hist[i] = 0;
-    __syncthreads();
-    for (long long sl = static_cast<long long>(blockIdx.x) * SM_THREADS + tid; sl < a.capacity;
-         sl += static_cast<long long>(gridDim.x) * SM_THREADS) {
-        if (!a.valid[sl]) continue;
-        const Key3 k = make_key(a.size[sl], a.access[sl], a.last[sl], static_cast<uint32_t>(sl));
-        int lo = 0, hi = n_sample;
-        while (lo < hi) {
-            const int mid = (lo + hi) >> 1;
-            Key3 sp;
-            sp.w0 = sm.k0[mid]; sp.w1 = sm.k1[mid]; sp.w2 = sm.k2[mid];
-            if (key_less(sp, k)) lo = mid + 1; else hi = mid;
-        }
-        a.bucket[sl] = static_cast<uint16_t>(lo);
-        atomicAdd(&sm.hist[lo], 1u);
-    }
-    __syncthreads();
-    for (int i = tid; i <= SM_SAMPLE; i += SM_THREADS)
-        if (sm.hist[i]) atomicAdd(&a.ctl->hist[i], sm.hist[i]);
 }
 
-// ---- phase E3 (all CTAs): candidates = entries in buckets 0..p, p the first bucket where the count reaches m ----
-__device__ void maint_evict_collect(const MaintArgs &a, MaintSmem &sm) {
-    const long long m = a.ctl->m;
-    if (m == 0) return;
-    const int tid = threadIdx.x, lane = tid & 31;
+__device__ void maint_slice_pass(const MaintArgs &a, long long m, long long occupancy, long long per, MaintSmem &sm) {
+    const int tid = threadIdx.x;
+    const long long lo = min(a.capacity, static_cast<long long>(blockIdx.x) * per), hi = min(a.capacity, lo + per);
+    int nfree = 0;
+    if (m == 0) {
+        for (long long sl = lo + tid; sl < hi; sl += SM_THREADS) nfree += a.valid[sl] ? 0 : 1;
+    } else {
+        MetaChunk cur;
+        maint_load_chunk(a, lo, hi, cur);              // in flight while the splitters are fetched
+        const int n_sample = a.ctl->n_sample;
+        const int P = maint_spec_buckets(m, n_sample, occupancy);
+        if (tid <= P && tid < SM_SAMPLE) {
+            const Key3 k = a.splitters[tid];
+            sm.k0[tid] = k.w0; sm.k1[tid] = k.w1; sm.k2[tid] = k.w2;
+        }
+        for (int i = tid; i <= SM_SAMPLE; i += SM_THREADS) sm.hist[i] = 0;
+        __syncthreads();
+        const bool has_bound = P < n_sample;
+        Key3 bound;
+        bound.w0 = bound.w1 = bound.w2 = ~0ull;
+        if (has_bound) bound = smem_key(sm, P);
+        for (long long base = lo; base < hi; base += MetaChunk::U * SM_THREADS) {
+            MetaChunk nxt;
+            const long long nb = base + MetaChunk::U * SM_THREADS;
+            if (nb < hi) maint_load_chunk(a, nb, hi, nxt);
+            // the CTA's candidates of this chunk get consecutive places: one global atomic per CTA and chunk
+            if (tid == 0) sm.n_stage = 0;
+            __syncthreads();
+            Key3 k[MetaChunk::U];
+            int place[MetaChunk::U];
+#pragma unroll
+            for (int j = 0; j < MetaChunk::U; ++j) {
+                const long long sl = base + j * SM_THREADS + tid;
+                const bool in = sl < hi;
+                nfree += (in && !cur.v[j]) ? 1 : 0;
+                place[j] = -1;
+                if (in && cur.v[j]) {
+                    k[j] = make_key(cur.sz[j], cur.ac[j], cur.la[j], static_cast<uint32_t>(sl));
+                    if (!has_bound || !key_less(bound, k[j])) {
+                        atomicAdd(&sm.hist[splitter_lower_bound(sm, P, k[j])], 1u);
+                        place[j] = atomicAdd(&sm.n_stage, 1);
+                    }
+                }
+            }
+            __syncthreads();
+            if (tid == 0 && sm.n_stage > 0) sm.p = static_cast<int>(atomicAdd(&a.ctl->n_cand, static_cast<unsigned int>(sm.n_stage)));
+            __syncthreads();
+            if (sm.n_stage > 0) {
+                const unsigned int cta_base = static_cast<unsigned int>(sm.p);
+#pragma unroll
+                for (int j = 0; j < MetaChunk::U; ++j) {
+                    if (place[j] >= 0) {
+                        const unsigned int at = cta_base + place[j];
+                        a.cand0[at] = k[j].w0; a.cand1[at] = k[j].w1; a.cand2[at] = k[j].w2;
+                    }
+                }
+            }
+            if (nb < hi) cur = nxt;
+        }
+        __syncthreads();
+        for (int i = tid; i <= P; i += SM_THREADS)
+            if (sm.hist[i]) atomicAdd(&a.ctl->hist[i], sm.hist[i]);
+    }
+    int total;
+    block_exclusive_scan_256(nfree, &total, sm.warp_sum);
+    if (tid == 0) a.cta_free[blockIdx.x] = total;
+}
+
+// first bucket in hist[0..last] where the cumulative count reaches m, or -1 (the same value in all threads)
+__device__ int maint_find_bucket(const unsigned int *hist, int last, long long m, MaintSmem &sm) {
+    const int tid = threadIdx.x;
+    __syncthreads();
     if (tid < 32) {
         long long run = 0;
-        int found = SM_SAMPLE;
-        for (int base = 0; base <= SM_SAMPLE && found == SM_SAMPLE; base += 32) {
+        int found = -1;
+        for (int base = 0; base <= last && found < 0; base += 32) {
             const int i = base + tid;
-            long long x = i <= SM_SAMPLE ? a.ctl->hist[i] : 0;
+            long long x = i <= last ? hist[i] : 0;
 #pragma unroll
             for (int o = 1; o < 32; o <<= 1) {
                 const long long y = __shfl_up_sync(0xFFFFFFFFu, x, o);
@@ -287,7 +466,34 @@ __device__ void maint_evict_collect(const MaintArgs &a, MaintSmem &sm) {
         if (tid == 0) sm.p = found;
     }
     __syncthreads();
-    const int p = sm.p;
+    return sm.p;
+}
+
+// ---- fall-back (all CTAs): bucket of every live entry over all splitters, then the candidates -------------------
+__device__ __noinline__ void maint_full_bucket(const MaintArgs &a, MaintSmem &sm) {
+    const int tid = threadIdx.x;
+    const int n_sample = a.ctl->n_sample;
+    {
+        const Key3 k = a.splitters[tid];
+        sm.k0[tid] = k.w0; sm.k1[tid] = k.w1; sm.k2[tid] = k.w2;
+    }
+    for (int i = tid; i <= SM_SAMPLE; i += SM_THREADS) sm.hist[i] = 0;
+    __syncthreads();
+    for (long long sl = static_cast<long long>(blockIdx.x) * SM_THREADS + tid; sl < a.capacity;
+         sl += static_cast<long long>(gridDim.x) * SM_THREADS) {
+        if (!a.valid[sl]) continue;
+        const Key3 k = make_key(a.size[sl], a.access[sl], a.last[sl], static_cast<uint32_t>(sl));
+        const int b = splitter_lower_bound(sm, n_sample, k);
+        a.bucket[sl] = static_cast<uint16_t>(b);
+        atomicAdd(&sm.hist[b], 1u);
+    }
+    __syncthreads();
+    for (int i = tid; i <= SM_SAMPLE; i += SM_THREADS)
+        if (sm.hist[i]) atomicAdd(&a.ctl->hist_full[i], sm.hist[i]);
+}
+
+__device__ __noinline__ void maint_full_collect(const MaintArgs &a, int p) {
+    const int tid = threadIdx.x, lane = tid & 31;
     for (long long base = static_cast<long long>(blockIdx.x) * SM_THREADS; base < a.capacity;
          base += static_cast<long long>(gridDim.x) * SM_THREADS) {
         const long long sl = base + tid;
@@ -295,189 +501,363 @@ __device__ void maint_evict_collect(const MaintArgs &a, MaintSmem &sm) {
         const unsigned ballot = __ballot_sync(0xFFFFFFFFu, take);
         if (ballot) {
             unsigned int warp_base = 0;
-            if (lane == 0) warp_base = atomicAdd(&a.ctl->n_cand, static_cast<unsigned int>(__popc(ballot)));
+            if (lane == 0) warp_base = atomicAdd(&a.ctl->n_cand_full, static_cast<unsigned int>(__popc(ballot)));
             warp_base = __shfl_sync(0xFFFFFFFFu, warp_base, 0);
-            if (take) a.cand[warp_base + __popc(ballot & ((1u << lane) - 1u))] =
-                          make_key(a.size[sl], a.access[sl], a.last[sl], static_cast<uint32_t>(sl));
+            if (take) {
+                const Key3 k = make_key(a.size[sl], a.access[sl], a.last[sl], static_cast<uint32_t>(sl));
+                const unsigned int at = warp_base + __popc(ballot & ((1u << lane) - 1u));
+                a.cand0[at] = k.w0; a.cand1[at] = k.w1; a.cand2[at] = k.w2;
+            }
         }
     }
 }
 
-// ---- phase E4 (all CTAs): rank the candidates, the m lowest are the victims -------------------------------------
-__device__ void maint_evict_rank(const MaintArgs &a) {
-    const long long m = a.ctl->m;
-    if (m == 0) return;
-    const unsigned int n = a.ctl->n_cand;
-    const int lane = threadIdx.x & 31;
-    const unsigned int warps = gridDim.x * SM_WARPS;
-    for (unsigned int i = blockIdx.x * SM_WARPS + (threadIdx.x >> 5); i < n; i += warps) {
-        const Key3 mine = a.cand[i];
-        unsigned int rank = 0;
-        for (unsigned int j = lane; j < n; j += 32) rank += key_less(a.cand[j], mine) ? 1u : 0u;
+__device__ __forceinline__ Key3 cand_key(const MaintArgs &a, unsigned int i) {
+    Key3 k;
+    k.w0 = a.cand0[i]; k.w1 = a.cand1[i]; k.w2 = a.cand2[i];
+    return k;
+}
+
+__device__ __forceinline__ void maint_take_victim(const MaintArgs &a, int32_t slot, unsigned int rank, long long per) {
+    a.victim_buf[rank] = slot;
+    if (a.victims) a.victims[rank] = slot;
+    a.valid[slot] = 0;
+    atomicAdd(&a.cta_free[slot / per], 1);
+}
+
+// ---- phase R (every SM_RANK_STRIDE-th CTA): rank the candidates whose key is at most `limit`; the m lowest are
+// the victims.  A candidate above the limit is larger than every candidate below it, so it never counts toward
+// a rank.
+__device__ void maint_rank(const MaintArgs &a, long long m, unsigned int n, bool has_limit, const Key3 &limit, long long per,
+                           unsigned long long *stage, MaintSmem &sm) {
+    const int tid = threadIdx.x, lane = tid & 31;
+    unsigned long long *s0 = stage, *s1 = stage + SM_STAGE, *s2 = stage + 2 * SM_STAGE;
+    if (tid == 0) sm.n_stage = 0;
+    __syncthreads();
+    constexpr int SU = 6;
+    for (unsigned int i0 = 0; i0 < n; i0 += SU * SM_THREADS) {
+        Key3 k[SU];
 #pragma unroll
-        for (int o = 16; o >= 1; o >>= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
-        if (lane == 0 && rank < m) {
-            const int32_t slot = static_cast<int32_t>(mine.w2 & 0xFFFFFFFFull);
-            if (a.victims) a.victims[rank] = slot;
-            a.valid[slot] = 0;
+        for (int u = 0; u < SU; ++u) {
+            const unsigned int i = i0 + u * SM_THREADS + tid;
+            if (i < n) k[u] = cand_key(a, i);
+        }
+#pragma unroll
+        for (int u = 0; u < SU; ++u) {
+            const unsigned int i = i0 + u * SM_THREADS + tid;
+            if (i < n && (!has_limit || !key_less(limit, k[u]))) {
+                const int j = atomicAdd(&sm.n_stage, 1);
+                if (j < SM_STAGE) { s0[j] = k[u].w0; s1[j] = k[u].w1; s2[j] = k[u].w2; }
+            }
+        }
+    }
+    __syncthreads();
+    const int n_stage = sm.n_stage;
+    const unsigned int rankers = (gridDim.x + SM_RANK_STRIDE - 1) / SM_RANK_STRIDE;
+    const unsigned int warps = rankers * SM_WARPS;
+    const unsigned int me = (blockIdx.x / SM_RANK_STRIDE) * SM_WARPS + (tid >> 5);
+    if (n_stage <= SM_STAGE) {
+        // the copy's order differs from CTA to CTA, so the work is dealt out by slot: this warp ranks the
+        // candidates whose slot is congruent to its number
+        for (int j0 = 0; j0 < n_stage; j0 += 32) {
+            const int j = j0 + lane;
+            const bool own = j < n_stage && static_cast<uint32_t>(s2[j] & 0xFFFFFFFFull) % warps == me;
+            unsigned todo = __ballot_sync(0xFFFFFFFFu, own);
+            while (todo) {
+                const int jj = j0 + __ffs(todo) - 1;
+                todo &= todo - 1;
+                Key3 mine;
+                mine.w0 = s0[jj]; mine.w1 = s1[jj]; mine.w2 = s2[jj];
+                unsigned int rank = 0;
+                for (int t = lane; t < n_stage; t += 32) {
+                    Key3 o;
+                    o.w0 = s0[t]; o.w1 = s1[t]; o.w2 = s2[t];
+                    rank += key_less(o, mine) ? 1u : 0u;
+                }
+#pragma unroll
+                for (int o = 16; o >= 1; o >>= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
+                if (lane == 0 && rank < m) maint_take_victim(a, static_cast<int32_t>(mine.w2 & 0xFFFFFFFFull), rank, per);
+            }
+        }
+    } else {
+        // too many for shared memory: by position in the list, against the list in global memory
+#pragma unroll 1
+        for (unsigned int i = me; i < n; i += warps) {
+            const Key3 mine = cand_key(a, i);
+            if (has_limit && key_less(limit, mine)) continue;          // the same for all lanes
+            unsigned int rank = 0;
+            for (unsigned int j = lane; j < n; j += 32) rank += key_less(cand_key(a, j), mine) ? 1u : 0u;
+#pragma unroll
+            for (int o = 16; o >= 1; o >>= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
+            if (lane == 0 && rank < m) maint_take_victim(a, static_cast<int32_t>(mine.w2 & 0xFFFFFFFFull), rank, per);
         }
     }
 }
 
-// ---- phases I1/I2 (all CTAs): the first n_miss free slots in ascending order ------------------------------------
-// CTA g owns the contiguous slice [g * per, (g + 1) * per) of the slots; thread t owns `chunk` consecutive slots of it.
-__device__ void maint_free_count(const MaintArgs &a, long long per, MaintSmem &sm) {
-    const long long lo = static_cast<long long>(blockIdx.x) * per, hi = min(a.capacity, lo + per);
-    int c = 0;
-    for (long long sl = lo + threadIdx.x; sl < hi; sl += SM_THREADS) c += a.valid[sl] ? 0 : 1;
-    int total;
-    block_exclusive_scan_256(c, &total, sm.warp_sum);
-    if (threadIdx.x == 0) a.cta_free[blockIdx.x] = total;
-}
-
-__device__ void maint_free_list(const MaintArgs &a, long long per, MaintSmem &sm) {
-    const int tid = threadIdx.x;
-    const int n_miss = a.ctl->n_miss;
-    // free slots in the slices before this one, and in all slices
-    int mine = 0, all = 0;
-    for (int g = tid; g < static_cast<int>(gridDim.x); g += SM_THREADS) {
-        const int f = a.cta_free[g];
-        all += f;
-        if (g < static_cast<int>(blockIdx.x)) mine += f;
-    }
-    int dummy;
-    // two block-wide sums through the scan helper (the total is what is wanted)
-    block_exclusive_scan_256(mine, &dummy, sm.warp_sum);
-    const int base = dummy;
-    __syncthreads();
-    block_exclusive_scan_256(all, &dummy, sm.warp_sum);
-    const int n_free = dummy;
-    __syncthreads();
-    if (blockIdx.x == 0 && tid == 0) {
-        const int ok = n_miss <= n_free ? 1 : 0;
-        a.ctl->insert_ok = ok;
-        if (!ok) set_status(a.status, SISO_ERR_CAPACITY);
-    }
-    if (n_miss > n_free || base >= n_miss) return;       // nothing of this slice is needed
-    const long long lo = static_cast<long long>(blockIdx.x) * per, hi = min(a.capacity, lo + per);
-    const long long chunk = (per + SM_THREADS - 1) / SM_THREADS;
-    const long long t_lo = lo + tid * chunk, t_hi = min(hi, t_lo + chunk);
-    int c = 0;
-    for (long long sl = t_lo; sl < t_hi; ++sl) c += a.valid[sl] ? 0 : 1;
-    int total;
-    int rank = base + block_exclusive_scan_256(c, &total, sm.warp_sum);
-    for (long long sl = t_lo; sl < t_hi; ++sl) {
-        if (!a.valid[sl]) {
-            if (rank < n_miss) a.free_list[rank] = static_cast<int32_t>(sl);
-            ++rank;
-        }
-    }
-}
-
-// ---- phase I3: row b, if it is a miss, takes free slot number (misses before b) ---------------------------------
+// ---- phase I: row `b` (a miss) into `slot` by one warp --------------------------------------------------------
 template <typename T>
-__device__ void maint_insert_row(const MaintArgs &a, int b, long long clock_new, MaintSmem &sm) {
-    const int tid = threadIdx.x;
-    const bool ok = a.ctl->insert_ok != 0;
-    if (a.hit[b] || !ok) {
-        if (tid == 0 && a.slots_out) a.slots_out[b] = -1;
-        return;
-    }
-    int before = 0;
-    for (int r = tid; r < b; r += SM_THREADS) before += a.hit[r] ? 0 : 1;
-    int rank;
-    block_exclusive_scan_256(before, &rank, sm.warp_sum);
-    const int32_t slot = a.free_list[rank];
+__device__ __forceinline__ void maint_insert_row(const MaintArgs &a, int b, int32_t slot, long long clock_new) {
+    const int lane = threadIdx.x & 31;
     const T *src = static_cast<const T *>(a.Q) + static_cast<long long>(b) * a.D;
     T *dv = static_cast<T *>(a.vecs) + static_cast<long long>(slot) * a.D;
     float *dm = a.master + static_cast<long long>(slot) * a.D;
-    for (int d = tid; d < a.D; d += SM_THREADS) {
-        const T x = src[d];
-        dv[d] = x;
-        if constexpr (sizeof(T) == 2) dm[d] = __bfloat162float(x);
+    if constexpr (sizeof(T) == 2) {
+        for (int d = lane * 8; d < a.D; d += 256) {
+            const uint4 u = __ldg(reinterpret_cast<const uint4 *>(src + d));
+            *reinterpret_cast<uint4 *>(dv + d) = u;
+            const float4 f0 = make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xFFFF0000u),
+                                          __uint_as_float(u.y << 16), __uint_as_float(u.y & 0xFFFF0000u));
+            const float4 f1 = make_float4(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xFFFF0000u),
+                                          __uint_as_float(u.w << 16), __uint_as_float(u.w & 0xFFFF0000u));
+            *reinterpret_cast<float4 *>(dm + d) = f0;
+            *reinterpret_cast<float4 *>(dm + d + 4) = f1;
+        }
+    } else {
+        for (int d = lane * 4; d < a.D; d += 128)
+            *reinterpret_cast<float4 *>(dv + d) = __ldg(reinterpret_cast<const float4 *>(src + d));
     }
-    if (tid == 0) {
+    if (lane == 0) {
         a.size[slot] = 1.0;
         a.access[slot] = SISO_ACCESS_INF;
         a.last[slot] = static_cast<unsigned long long>(clock_new);
         a.valid[slot] = 1;
         if (a.slots_out) a.slots_out[b] = slot;
     }
-    __syncthreads();
 }
 
 template <typename T>
-__global__ void __launch_bounds__(SM_THREADS)
+__global__ void __launch_bounds__(SM_THREADS, 2)
 stream_maint_kernel(const MaintArgs a) {
-    extern __shared__ double acc[];          // [D]
-    __shared__ MaintSmem sm;
+    extern __shared__ __align__(16) unsigned char smem_raw[];
+    double *acc = reinterpret_cast<double *>(smem_raw);                              // [D] during the update
+    unsigned long long *stage = reinterpret_cast<unsigned long long *>(smem_raw);    // [3][SM_STAGE] while ranking
+    int32_t *sorted = reinterpret_cast<int32_t *>(smem_raw);                         // [2][SM_MAX_B] while inserting
+    MaintSmem &sm = *reinterpret_cast<MaintSmem *>(smem_raw + SM_UNION_BYTES);
     cg::grid_group grid = cg::this_grid();
-    const long long clock_new = a.counters[CNT_CLOCK] + 1;      // nobody writes the clock before the first barrier
+    const int tid = threadIdx.x, warp = tid >> 5;
+    // nobody writes the counters before the last barrier
+    const long long clock_new = a.counters[CNT_CLOCK] + 1;
+    const long long occupancy = a.counters[CNT_OCCUPANCY];
+
+    if (a.partial) {
+        maint_finalize(a);
+        grid.sync();
+    }
+
+    // ---- every CTA: the batch's hit flags and slots, the misses in row order, the number of victims
+    for (int b = tid; b < a.B; b += SM_THREADS) { sm.hit[b] = a.hit[b]; sm.idx[b] = a.idx[b]; }
+    __syncthreads();
+    int n_miss;
+    {
+        constexpr int PER = SM_MAX_B / SM_THREADS;
+        int c = 0;
+#pragma unroll
+        for (int j = 0; j < PER; ++j) { const int b = tid * PER + j; c += (b < a.B && !sm.hit[b]) ? 1 : 0; }
+        int r = block_exclusive_scan_256(c, &n_miss, sm.warp_sum);
+#pragma unroll
+        for (int j = 0; j < PER; ++j) {
+            const int b = tid * PER + j;
+            if (b < a.B && !sm.hit[b]) sm.miss_list[r++] = static_cast<uint16_t>(b);
+        }
+    }
+    const long long free0 = a.capacity - occupancy;         // free slots before this batch
+    long long m = static_cast<long long>(n_miss) - free0;
+    m = m > 0 ? m : 0;
+    m = m < occupancy ? m : occupancy;
+    __syncthreads();
+
+    // ---- U (+ sampler)
+    if (blockIdx.x == 0) {
+        if (tid == 0) { a.ctl->n_cand = 0; a.ctl->n_cand_full = 0; }
+        for (int i = tid; i <= SM_SAMPLE; i += SM_THREADS) { a.ctl->hist[i] = 0; a.ctl->hist_full[i] = 0; }
+        if (a.victims)
+            for (long long r = m + tid; r < a.B; r += SM_THREADS) a.victims[r] = -1;
+        if (a.slots_out)
+            for (int b = tid; b < a.B; b += SM_THREADS)
+                if (sm.hit[b]) a.slots_out[b] = -1;
+    }
+    if (m > 0 && blockIdx.x == gridDim.x - 1) maint_evict_sample(a, clock_new, m, occupancy, false, sm);
     for (int b = blockIdx.x; b < a.B; b += gridDim.x) maint_update_row<T>(a, b, clock_new, acc, sm);
     grid.sync();
-    if (blockIdx.x == 0) {
-        if (threadIdx.x == 0) a.counters[CNT_CLOCK] = clock_new;
-        maint_evict_sample(a, clock_new, sm);
-    }
-    grid.sync();
-    maint_evict_bucket(a, sm);
-    grid.sync();
-    maint_evict_collect(a, sm);
-    grid.sync();
-    maint_evict_rank(a);
+
+    // ---- S
     const long long per = (a.capacity + gridDim.x - 1) / gridDim.x;
+    maint_slice_pass(a, m, occupancy, per, sm);
     grid.sync();
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
-        a.counters[CNT_OCCUPANCY] -= a.ctl->m;
-        a.counters[CNT_EVICTIONS] += a.ctl->m;
+
+    // ---- R
+    if (m > 0) {
+        int n_sample = a.ctl->n_sample;
+        const int P = maint_spec_buckets(m, n_sample, occupancy);
+        unsigned int n = a.ctl->n_cand;
+        int p = maint_find_bucket(a.ctl->hist, P, m, sm);
+        if (p < 0) {
+            // the whole sample in order (the entries are final by now), every entry's bucket, the candidates
+            if (blockIdx.x == 0) maint_evict_sample(a, clock_new, m, occupancy, true, sm);
+            grid.sync();
+            n_sample = a.ctl->n_sample;
+            maint_full_bucket(a, sm);
+            grid.sync();
+            p = maint_find_bucket(a.ctl->hist_full, SM_SAMPLE, m, sm);      // m <= occupancy, so it exists
+            maint_full_collect(a, p);
+            grid.sync();
+            n = a.ctl->n_cand_full;
+            p = n_sample;                                                   // every collected entry is ranked
+        }
+        if (blockIdx.x % SM_RANK_STRIDE == 0) {
+            const bool has_limit = p < n_sample;
+            Key3 limit;
+            limit.w0 = limit.w1 = limit.w2 = ~0ull;
+            if (has_limit) limit = smem_key(sm, p);
+            maint_rank(a, m, n, has_limit, limit, per, stage, sm);
+        }
+        grid.sync();
     }
-    maint_free_count(a, per, sm);
-    grid.sync();
-    maint_free_list(a, per, sm);
-    grid.sync();
-    for (int b = blockIdx.x; b < a.B; b += gridDim.x) maint_insert_row<T>(a, b, clock_new, sm);
-    if (blockIdx.x == 0 && threadIdx.x == 0 && a.ctl->insert_ok) {
-        a.counters[CNT_OCCUPANCY] += a.ctl->n_miss;
-        a.counters[CNT_INSERTS] += a.ctl->n_miss;
+
+    // ---- I
+    bool insert_ok;
+    if (free0 == 0) {
+        // a full cache: the free slots are the victims; every CTA puts them in slot order
+        insert_ok = n_miss <= m;
+        if (insert_ok) {
+            int32_t *vict = sorted, *by_slot = sorted + SM_MAX_B;
+            for (int r = tid; r < n_miss; r += SM_THREADS) vict[r] = a.victim_buf[r];
+            __syncthreads();
+            for (int r = tid; r < n_miss; r += SM_THREADS) {
+                const int32_t mine = vict[r];
+                int rank = 0;
+                for (int j = 0; j < n_miss; ++j) rank += vict[j] < mine ? 1 : 0;
+                by_slot[rank] = mine;
+            }
+            __syncthreads();
+            const int warps = gridDim.x * SM_WARPS;
+            for (int r = blockIdx.x * SM_WARPS + warp; r < n_miss; r += warps)
+                maint_insert_row<T>(a, sm.miss_list[r], by_slot[r], clock_new);
+        }
+    } else {
+        // free slots before this CTA's slice and in all slices
+        int base = 0, n_free = 0;
+        {
+            const int G = static_cast<int>(gridDim.x);
+            const int cs = (G + SM_THREADS - 1) / SM_THREADS;
+            int c = 0;
+            for (int j = 0; j < cs; ++j) { const int g = tid * cs + j; c += g < G ? a.cta_free[g] : 0; }
+            int run = block_exclusive_scan_256(c, &n_free, sm.warp_sum);
+            __syncthreads();
+            for (int j = 0; j < cs; ++j) {
+                const int g = tid * cs + j;
+                if (g >= G) break;
+                if (g == static_cast<int>(blockIdx.x)) sm.p = run;
+                run += a.cta_free[g];
+            }
+            __syncthreads();
+            base = sm.p;
+        }
+        insert_ok = n_miss <= n_free;
+        if (insert_ok) {          // the same in every CTA
+            // the free slots of this slice that are taken, in ascending order
+            const long long lo = min(a.capacity, static_cast<long long>(blockIdx.x) * per), hi = min(a.capacity, lo + per);
+            const int my_need = max(0, min(a.cta_free[blockIdx.x], n_miss - base));
+            if (my_need > 0) {        // uniform for the CTA
+                const long long chunk = (per + SM_THREADS - 1) / SM_THREADS;
+                const long long t_lo = min(hi, lo + tid * chunk), t_hi = min(hi, t_lo + chunk);
+                int c = 0;
+                for (long long sl = t_lo; sl < t_hi; ++sl) c += a.valid[sl] ? 0 : 1;
+                int total;
+                int r = block_exclusive_scan_256(c, &total, sm.warp_sum);
+                for (long long sl = t_lo; sl < t_hi; ++sl) {
+                    if (!a.valid[sl]) {
+                        if (r < my_need) a.free_list[base + r] = static_cast<int32_t>(sl);
+                        ++r;
+                    }
+                }
+            }
+            grid.sync();
+            const int warps = gridDim.x * SM_WARPS;
+            for (int r = blockIdx.x * SM_WARPS + warp; r < n_miss; r += warps)
+                maint_insert_row<T>(a, sm.miss_list[r], a.free_list[r], clock_new);
+        }
+    }
+    if (!insert_ok && blockIdx.x == 0) {
+        if (tid == 0) set_status(a.status, SISO_ERR_CAPACITY);
+        if (a.slots_out)
+            for (int r = tid; r < n_miss; r += SM_THREADS) a.slots_out[sm.miss_list[r]] = -1;
+    }
+    if (blockIdx.x == 0 && tid == 0) {
+        a.counters[CNT_CLOCK] = clock_new;
+        a.counters[CNT_OCCUPANCY] = occupancy - m + (insert_ok ? n_miss : 0);
+        a.counters[CNT_EVICTIONS] += m;
+        if (insert_ok) a.counters[CNT_INSERTS] += n_miss;
+        if (a.partial) {
+            a.counters[CNT_LOOKUPS] += a.B;
+            a.counters[CNT_HITS] += a.B - n_miss;
+        }
     }
 }
 
-// Returns SISO_ERR_UNSUPPORTED if this batch cannot take the fused path (the caller then uses the separate kernels).
-siso_status_t launch_stream_maint(Cache *c, const void *q, int64_t B, const int32_t *idx, const uint8_t *hit,
-                                  int32_t *victims, int32_t *slots_out, cudaStream_t s) {
-    if (B < 1 || B > SM_MAX_B) return SISO_ERR_UNSUPPORTED;
+// With `deferred` the lookup's top-1 finalisation (best key over the splits, threshold test, idx/sim/hit) runs as the
+// kernel's first phase; `scratch_tail` is then the part of the cache's scratch that the lookup set aside for this call.
+size_t stream_maint_scratch_bytes(const Cache *c, int64_t B) {
+    const int grid_cap = c->sm_count * 2;
+    return pad256(sizeof(MaintCtl)) + pad256(sizeof(Key3) * SM_SAMPLE) + pad256(sizeof(uint16_t) * c->capacity) +
+           3 * pad256(sizeof(unsigned long long) * c->capacity) + pad256(sizeof(int) * grid_cap) +
+           2 * pad256(sizeof(int32_t) * B) + 256;
+}
+
+bool stream_maint_supported(Cache *c, int64_t B) {
+    if (B < 1 || B > SM_MAX_B) return false;
     if (c->maint_grid == 0) {
         int coop = 0;
-        SISO_CUDA(cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device));
+        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device) != cudaSuccess) coop = 0;
         int per_sm = 0;
-        const size_t smem = sizeof(double) * c->dim;
-        cudaError_t e = c->dtype == SISO_F32
-            ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, stream_maint_kernel<float>, SM_THREADS, smem)
-            : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, stream_maint_kernel<__nv_bfloat16>, SM_THREADS, smem);
-        SISO_CUDA(e);
+        const void *fn = c->dtype == SISO_F32 ? reinterpret_cast<const void *>(stream_maint_kernel<float>)
+                                              : reinterpret_cast<const void *>(stream_maint_kernel<__nv_bfloat16>);
+        cudaError_t e = cudaFuncSetAttribute(fn, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(SM_SMEM_BYTES));
+        if (e == cudaSuccess)
+            e = c->dtype == SISO_F32
+                ? cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, stream_maint_kernel<float>, SM_THREADS, SM_SMEM_BYTES)
+                : cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, stream_maint_kernel<__nv_bfloat16>, SM_THREADS, SM_SMEM_BYTES);
+        if (e != cudaSuccess) { cudaGetLastError(); per_sm = 0; }
         c->maint_grid = (coop && per_sm >= 1) ? c->sm_count * std::min(per_sm, 2) : -1;
     }
-    if (c->maint_grid < 0) return SISO_ERR_UNSUPPORTED;
+    return c->maint_grid > 0;
+}
+
+// Returns SISO_ERR_UNSUPPORTED if this batch cannot take the fused path (the caller then uses the separate kernels).
+siso_status_t launch_stream_maint(Cache *c, const void *q, int64_t B, int32_t *idx, uint8_t *hit, int32_t *victims,
+                                  int32_t *slots_out, const DeferredTop1 *deferred, void *scratch_tail, cudaStream_t s) {
+    if (!stream_maint_supported(c, B)) return SISO_ERR_UNSUPPORTED;
     const int grid = c->maint_grid;
     Scratch scr;
-    const size_t need = pad256(sizeof(MaintCtl)) + pad256(sizeof(Key3) * SM_SAMPLE) + pad256(sizeof(uint16_t) * c->capacity) +
-                        pad256(sizeof(Key3) * c->capacity) + pad256(sizeof(int) * grid) + pad256(sizeof(int32_t) * B);
-    SISO_TRY(scratch_reserve(c, need, s, &scr));
+    if (scratch_tail) {
+        scr.base = static_cast<char *>(scratch_tail);
+        scr.off = 0;
+        scr.cap = stream_maint_scratch_bytes(c, B);
+    } else {
+        SISO_TRY(scratch_reserve(c, stream_maint_scratch_bytes(c, B), s, &scr));
+    }
     MaintArgs a;
     a.Q = q; a.idx = idx; a.hit = hit; a.B = static_cast<int>(B); a.D = c->dim; a.capacity = c->capacity;
     a.vecs = c->vecs; a.master = c->master; a.size = c->size; a.access = c->access; a.last = c->last; a.valid = c->valid;
     a.counters = c->counters; a.status = c->status; a.victims = victims; a.slots_out = slots_out;
+    a.partial = deferred ? deferred->partial : nullptr;
+    a.splits = deferred ? deferred->splits : 0;
+    a.theta = deferred ? deferred->theta : nullptr;
+    a.theta_s = deferred ? deferred->theta_s : 0.0f;
+    a.sim = deferred ? deferred->sim : nullptr;
     a.ctl = scr.take<MaintCtl>(1);
     a.splitters = scr.take<Key3>(SM_SAMPLE);
     a.bucket = scr.take<uint16_t>(c->capacity);
-    a.cand = scr.take<Key3>(c->capacity);
+    a.cand0 = scr.take<unsigned long long>(c->capacity);
+    a.cand1 = scr.take<unsigned long long>(c->capacity);
+    a.cand2 = scr.take<unsigned long long>(c->capacity);
+    a.victim_buf = scr.take<int32_t>(B);
     a.cta_free = scr.take<int>(grid);
     a.free_list = scr.take<int32_t>(B);
     void *args[] = {&a};
-    const size_t smem = sizeof(double) * c->dim;
     const void *fn = c->dtype == SISO_F32 ? reinterpret_cast<const void *>(stream_maint_kernel<float>)
                                           : reinterpret_cast<const void *>(stream_maint_kernel<__nv_bfloat16>);
-    SISO_CUDA(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(SM_THREADS), args, smem, s));
+    SISO_CUDA(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(SM_THREADS), args, SM_SMEM_BYTES, s));
     c->launches += 1;
     return SISO_OK;
 }

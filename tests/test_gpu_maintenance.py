@@ -325,3 +325,32 @@ def test_fused_streaming_maintenance_equals_separate_kernels_bit_for_bit():
     for c in caches:
         c.check_status()
         c.close()
+
+
+def test_streaming_eviction_is_exact_when_the_sample_misleads():
+    """The fused step chooses its victims with the help of a strided sample of 256 entries.  Here exactly the
+    sampled entries hold the smallest keys, so the sample says that hardly any entry is small; the selection
+    must notice (fewer candidates than victims) and still return the m smallest keys in key order."""
+    cap, D, B = 4096, 64, 256
+    cent = W.f32_to_bf16_bits(W.unit_gaussian_rows(cap, D, 5, 901))
+    cache = siso.SisoCache(cap, D, "bf16")
+    cache.insert(to_dev(cent, "bf16"))
+    g = state_np(cache)
+    clock = cache.stats()["clock"]
+    # the step's sampler looks at slot 16 w + ((clock + 1) * 2654435761 mod 16) of every 16-slot window w
+    off = ((clock + 1) * 2654435761) % (cap // 256)
+    size = np.ones(cap)
+    size[np.arange(256) * (cap // 256) + off] = 0.5
+    cache.import_(torch.from_numpy(g["master"]), torch.from_numpy(size), torch.from_numpy(g["access"].view(np.int32)),
+                  torch.from_numpy(g["last"].view(np.int64)), torch.from_numpy(g["valid"]), clock)
+    ora = oracle.OracleCache(cap, D, "bf16")
+    ora.load_state(g["master"], size, g["access"], g["last"], g["valid"], clock)
+    q = W.f32_to_bf16_bits(W.unit_gaussian_rows(B, D, 6, 902))          # unrelated directions: every row misses
+    idx, sim, hit, victims, slots = [x.cpu().numpy() for x in cache.stream_step(to_dev(q, "bf16"), 0.86)]
+    assert hit.sum() == 0
+    o_idx, o_sim, o_hit, o_victims, o_slots = ora.stream_step(q, np.full(B, 0.86, np.float32), forced=(idx, hit))
+    assert len(o_victims) == B and (np.sort(o_victims) == np.arange(256) * (cap // 256) + off).all()
+    assert (victims == o_victims).all() and (slots == o_slots).all()
+    assert_state_equal(cache, ora, "bf16")
+    cache.check_status()
+    cache.close()
