@@ -62,6 +62,8 @@ typedef enum { SISO_F32 = 0, SISO_BF16 = 1 } siso_dtype_t;
 #define SISO_OPT_MERGE_MAX_CANDIDATES 2 /* capacity of the merge candidate buffer, in pairs */
 #define SISO_OPT_STREAM_FUSED 4         /* 1 (default): siso_stream_step fuses update, make-room and insertion of batches
                                            of at most 1024 rows into one cooperative launch; 0: separate kernels */
+#define SISO_OPT_MERGE_PATH 5           /* pairwise sweep of siso_merge: SISO_PATH_AUTO (default: tensor cores from 4096
+                                           entries), SISO_PATH_SIMT or SISO_PATH_TENSOR; the results are the same */
 #define SISO_OPT_TENSOR_CTA_PAIR 3      /* 0 (default): tensor-core lookup runs CTA pairs for >= 2 query tiles; 1: never */
 #define SISO_PATH_AUTO 0
 #define SISO_PATH_SIMT 1   /* CUDA-core tiled sweep (fp32 accumulate of exact products)        */

@@ -3,8 +3,10 @@ cosine lookup with top-k and a per-query hit threshold, running-mean hit updates
 MergeCentroids / FilteringCentroids and spare-space insertion, behind the C ABI of
 ``include/siso.h``.  This package is the thin Python binding: it marshals torch tensors to
 pointers and calls ``libsiso.so``; every step runs in the library's own CUDA kernels."""
-from .binding import (ACCESS_INF, EVICT_DECAY, MERGE_SIZES_ONLY, MERGE_WEIGHTED_MEAN, PATH_AUTO, PATH_SIMT,
+from .binding import (ACCESS_INF, EVICT_DECAY, MERGE_SIZES_ONLY, MERGE_WEIGHTED_MEAN, OPT_LOOKUP_PATH,
+                      OPT_MERGE_MAX_CANDIDATES, OPT_MERGE_PATH, OPT_STREAM_FUSED, OPT_TENSOR_CTA_PAIR, PATH_AUTO, PATH_SIMT,
                       PATH_STREAM, PATH_TENSOR, SisoCache, SisoError, load_library, lookup_small_noalloc, md1_wait, choose_theta, correct_theta)
 
 __all__ = ["SisoCache", "SisoError", "load_library", "lookup_small_noalloc", "md1_wait", "choose_theta", "correct_theta", "ACCESS_INF", "EVICT_DECAY", "MERGE_SIZES_ONLY",
-           "MERGE_WEIGHTED_MEAN", "PATH_AUTO", "PATH_SIMT", "PATH_STREAM", "PATH_TENSOR"]
+           "MERGE_WEIGHTED_MEAN", "OPT_LOOKUP_PATH", "OPT_MERGE_MAX_CANDIDATES", "OPT_MERGE_PATH", "OPT_STREAM_FUSED",
+           "OPT_TENSOR_CTA_PAIR", "PATH_AUTO", "PATH_SIMT", "PATH_STREAM", "PATH_TENSOR"]

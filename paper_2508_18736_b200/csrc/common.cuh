@@ -56,6 +56,9 @@ struct Cache {
     // large-shared-memory opt-in is a per-device function attribute: remembered per cache, not per process
     bool simt_attr_set[2][3];   // [dtype][k class] of lookup_simt_kernel
     bool merge_attr_set;
+    bool merge_tensor_attr_set;
+    int merge_resolve_grid;     // CTAs of the grid-wide merge resolution (0: not yet asked, -1: unavailable)
+    int32_t merge_path;         // SISO_PATH_AUTO, SISO_PATH_SIMT or SISO_PATH_TENSOR for the pairwise sweep of siso_merge
     int maint_grid;             // CTAs of the fused streaming maintenance kernel (0: not yet asked, -1: unavailable)
 };
 
@@ -115,6 +118,9 @@ siso_status_t launch_update(Cache *c, const void *q, int64_t B, const int32_t *i
                             cudaStream_t s);
 siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes, int64_t n_repo, float theta_c,
                            uint32_t flags, int32_t *merge_map, long long *d_n_merged, cudaStream_t s);
+size_t merge_tensor_scratch_bytes(const Cache *c);
+siso_status_t launch_merge_sweep_tensor(Cache *c, Scratch *scr, const uint8_t *seed, float theta_c, void *ctl, void *cand,
+                                        size_t max_cand, uint32_t *row_count, cudaStream_t s);
 siso_status_t launch_evict(Cache *c, int64_t n_evict, const uint8_t *hit, int64_t n_hit, uint32_t flags,
                            int32_t *victims, int64_t n_victims_out, cudaStream_t s);
 siso_status_t launch_insert(Cache *c, const void *vecs, const double *sizes, const uint8_t *hit, int64_t n,

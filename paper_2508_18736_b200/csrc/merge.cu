@@ -13,6 +13,8 @@
 // The similarity used is that of the vectors as they were when the call began: nothing is written
 // before the sweep has finished.  If the candidates do not fit their buffer the status word gets
 // SISO_ERR_OVERFLOW and every later kernel of the call returns without writing.
+#include <cooperative_groups.h>
+
 #include "sweep_simt.cuh"
 
 namespace siso {
@@ -101,10 +103,11 @@ __global__ void merge_scatter_kernel(const MergeCtl *ctl, const Candidate *__res
                                      const uint32_t *__restrict__ row_off, uint32_t *__restrict__ row_cursor,
                                      int32_t *__restrict__ csr_j, float *__restrict__ csr_sim) {
     if (ctl->overflow) return;
-    const unsigned long long n = ctl->n_cand;
+    const unsigned long long n = ctl->n_cand;        // no overflow here, so every one of them is in the buffer
     for (unsigned long long e = static_cast<unsigned long long>(blockIdx.x) * blockDim.x + threadIdx.x; e < n;
          e += static_cast<unsigned long long>(gridDim.x) * blockDim.x) {
         const Candidate cd = cand[e];
+        if (cd.i < 0) continue;          // a pair the tensor-core filter proposed and the exact check rejected
         const uint32_t pos = row_off[cd.i] + atomicAdd(&row_cursor[cd.i], 1u);
         csr_j[pos] = cd.j;
         csr_sim[pos] = cd.sim;
@@ -156,6 +159,63 @@ merge_resolve_kernel(MergeCtl *ctl, int64_t N, const uint8_t *__restrict__ valid
         __syncthreads();
         const int any = undecided_s;
         __syncthreads();
+        if (!any) break;
+    }
+}
+
+// The same resolution spread over the whole GPU: a cooperative launch, one thread per row at a time, a grid-wide
+// barrier per round.  A chain of k entries that each merge into the previous survivor needs k rounds; a round costs
+// a barrier plus a few memory round trips instead of one CTA's walk over all rows.
+namespace cgm = cooperative_groups;
+__global__ void __launch_bounds__(256)
+merge_resolve_grid_kernel(MergeCtl *ctl, int64_t N, const uint8_t *__restrict__ valid, const uint8_t *__restrict__ seed,
+                          const uint32_t *__restrict__ row_off, const uint32_t *__restrict__ row_count,
+                          const int32_t *__restrict__ csr_j, const float *__restrict__ csr_sim, volatile uint8_t *state,
+                          int32_t *__restrict__ target, unsigned int *undecided /* [3], zeroed */) {
+    cgm::grid_group grid = cgm::this_grid();
+    if (ctl->overflow) return;                      // the same in every CTA
+    __shared__ int warp_left[8];
+    const int64_t first = static_cast<int64_t>(blockIdx.x) * 256 + threadIdx.x;
+    const int64_t stride = static_cast<int64_t>(gridDim.x) * 256;
+    for (int64_t i = first; i < N; i += stride) {
+        state[i] = valid[i] ? (row_count[i] == 0 ? 1 : 0) : 3;
+        target[i] = valid[i] ? static_cast<int32_t>(i) : -1;
+    }
+    grid.sync();
+    for (int64_t round = 0; round <= N; ++round) {
+        int left = 0;
+        for (int64_t i = first; i < N; i += stride) {
+            if (state[i] != 0) continue;
+            const uint32_t o = row_off[i], cnt = row_count[i];
+            bool ready = true;
+            unsigned long long best = 0ull;
+            for (uint32_t e = 0; e < cnt; ++e) {
+                const int32_t j = csr_j[o + e];
+                const uint8_t sj = state[j];
+                if (sj == 0) { ready = false; break; }
+                if (sj == 1) {
+                    const uint32_t order = static_cast<uint32_t>(j) | ((seed && seed[j]) ? 0u : 0x80000000u);
+                    const unsigned long long key = pack_key(csr_sim[o + e], order);
+                    best = key > best ? key : best;
+                }
+            }
+            if (!ready) { ++left; continue; }
+            if (best) { target[i] = key_slot(best) & 0x7FFFFFFF; state[i] = 2; }
+            else state[i] = 1;
+        }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) left += __shfl_xor_sync(0xFFFFFFFFu, left, o);
+        if ((threadIdx.x & 31) == 0) warp_left[threadIdx.x >> 5] = left;
+        __syncthreads();
+        if (threadIdx.x == 0) {
+            int t = 0;
+            for (int w = 0; w < 8; ++w) t += warp_left[w];
+            if (t) atomicAdd(&undecided[round % 3], static_cast<unsigned int>(t));
+            // the counter of the round after this one was last read two barriers ago
+            if (blockIdx.x == 0) undecided[(round + 1) % 3] = 0;
+        }
+        grid.sync();
+        const unsigned int any = *reinterpret_cast<volatile unsigned int *>(&undecided[round % 3]);
         if (!any) break;
     }
 }
@@ -262,10 +322,12 @@ siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes,
     if (pairs > 0x7FFFFFFFll) return SISO_ERR_UNSUPPORTED;
     const size_t max_cand = static_cast<size_t>(c->merge_max_cand);
     Scratch scr;
-    size_t need = pad256(sizeof(MergeCtl)) + pad256(sizeof(Candidate) * max_cand) + 3 * pad256(sizeof(uint32_t) * (N + 1)) +
+    // the tensor-core sweep pays off once the matrix of pairs is large; small caches take the CUDA-core sweep
+    const bool tensor = c->merge_path == SISO_PATH_TENSOR || (c->merge_path == SISO_PATH_AUTO && N >= 4096);
+    size_t need = (tensor ? merge_tensor_scratch_bytes(c) : 0) + pad256(sizeof(MergeCtl)) + pad256(sizeof(Candidate) * max_cand) + 3 * pad256(sizeof(uint32_t) * (N + 1)) +
                   pad256(sizeof(int32_t) * max_cand) + pad256(sizeof(float) * max_cand) + pad256(N) +
                   pad256(sizeof(int32_t) * N) + 4 * pad256(sizeof(uint32_t) * N) + sort_pairs_scratch_bytes(N) +
-                  pad256(N) + pad256(sizeof(int32_t) * (n_repo + 1));
+                  pad256(N) + pad256(sizeof(int32_t) * (n_repo + 1)) + 256;
     SISO_TRY(scratch_reserve(c, need, s, &scr));
     MergeCtl *ctl = scr.take<MergeCtl>(1);
     Candidate *cand = scr.take<Candidate>(max_cand);
@@ -278,6 +340,7 @@ siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes,
     int32_t *target = scr.take<int32_t>(N);
     uint32_t *keys = scr.take<uint32_t>(N), *vals = scr.take<uint32_t>(N);
     uint32_t *keys2 = scr.take<uint32_t>(N), *vals2 = scr.take<uint32_t>(N);
+    unsigned int *undecided = scr.take<unsigned int>(3);
     uint8_t *seed = nullptr;
     if (two_sets) {
         // C_cur = what is live now; the repository rows then take free slots (new entries: access_count = infinity).
@@ -295,13 +358,17 @@ siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes,
     }
     SISO_CUDA(cudaMemsetAsync(row_count, 0, sizeof(uint32_t) * (N + 1), s));
     SISO_CUDA(cudaMemsetAsync(row_cursor, 0, sizeof(uint32_t) * (N + 1), s));
-    if (!c->merge_attr_set) {
-        SISO_CUDA(cudaFuncSetAttribute(merge_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
-        c->merge_attr_set = true;
+    if (tensor) {
+        SISO_TRY(launch_merge_sweep_tensor(c, &scr, seed, theta_c, ctl, cand, max_cand, row_count, s));
+    } else {
+        if (!c->merge_attr_set) {
+            SISO_CUDA(cudaFuncSetAttribute(merge_sweep_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES));
+            c->merge_attr_set = true;
+        }
+        merge_sweep_kernel<<<static_cast<unsigned>(pairs), THREADS, SMEM_BYTES, s>>>(c->master, c->valid, seed, N, c->dim,
+                                                                                    theta_c, ctl, cand, max_cand, row_count);
+        SISO_LAUNCHED(c);
     }
-    merge_sweep_kernel<<<static_cast<unsigned>(pairs), THREADS, SMEM_BYTES, s>>>(c->master, c->valid, seed, N, c->dim,
-                                                                                theta_c, ctl, cand, max_cand, row_count);
-    SISO_LAUNCHED(c);
     merge_check_kernel<<<1, 1, 0, s>>>(ctl, c->status);
     SISO_LAUNCHED(c);
     if (two_sets) {
@@ -312,8 +379,30 @@ siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes,
     SISO_TRY(launch_exclusive_scan_u32(c, row_off, N + 1, s));
     merge_scatter_kernel<<<4 * c->sm_count, 256, 0, s>>>(ctl, cand, row_off, row_cursor, csr_j, csr_sim);
     SISO_LAUNCHED(c);
-    merge_resolve_kernel<<<1, 1024, 0, s>>>(ctl, N, c->valid, seed, row_off, row_count, csr_j, csr_sim, state, target);
-    SISO_LAUNCHED(c);
+    if (c->merge_resolve_grid == 0) {
+        int coop = 0, per_sm = 0;
+        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device) != cudaSuccess) coop = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, merge_resolve_grid_kernel, 256, 0) != cudaSuccess) {
+            cudaGetLastError();
+            per_sm = 0;
+        }
+        c->merge_resolve_grid = (coop && per_sm >= 1) ? c->sm_count * std::min(per_sm, 4) : -1;
+    }
+    if (c->merge_resolve_grid > 0) {
+        SISO_CUDA(cudaMemsetAsync(undecided, 0, 3 * sizeof(unsigned int), s));
+        const uint8_t *valid_p = c->valid;
+        const uint8_t *seed_p = seed;
+        int64_t n_arg = N;
+        volatile uint8_t *state_p = state;
+        void *args[] = {&ctl, &n_arg, &valid_p, &seed_p, &row_off, &row_count, &csr_j, &csr_sim, &state_p, &target, &undecided};
+        const int grid = static_cast<int>(std::min<int64_t>(c->merge_resolve_grid, (N + 255) / 256));
+        SISO_CUDA(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(merge_resolve_grid_kernel), dim3(grid), dim3(256),
+                                              args, 0, s));
+        c->launches += 1;
+    } else {
+        merge_resolve_kernel<<<1, 1024, 0, s>>>(ctl, N, c->valid, seed, row_off, row_count, csr_j, csr_sim, state, target);
+        SISO_LAUNCHED(c);
+    }
     const unsigned nblk = static_cast<unsigned>((N + 255) / 256);
     merge_keys_kernel<<<nblk, 256, 0, s>>>(ctl, N, state, target, keys, vals);
     SISO_LAUNCHED(c);

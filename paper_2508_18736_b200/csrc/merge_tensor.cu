@@ -1,0 +1,377 @@
+// Pairwise similarity sweep of MergeCentroids (Algorithm 1: every entry against the earlier entries of C_new) as a
+// dense contraction on the tensor cores, for fp32 vectors.
+//
+// An fp32 value x is split as x = hi + lo + r with hi = bf16(x), lo = bf16(x - hi), |r| <= 2^-18 |x|.  The sweep
+// accumulates hi_i.hi_j + hi_i.lo_j + lo_i.hi_j in fp32 on tcgen05 (three MMAs per 16 K-elements, one TMEM
+// accumulator); what it leaves out (lo.lo, the r terms) and the fp32 accumulation stay below 3e-5 for unit
+// vectors.  So the tensor cores only FILTER: every pair whose approximate similarity exceeds theta_C - 1e-4
+// becomes a provisional candidate, and merge_verify_kernel recomputes exactly these pairs from the fp32 vectors
+// in fp64 and keeps those whose exact similarity exceeds theta_C.  The decisions are therefore those of an exact
+// fp64 sweep; the tensor cores do the 2 N^2 D flops, the exact arithmetic touches the few candidates only.
+//
+// Kernel layout (CTA pairs, cta_group::2, as in the large-batch lookup): a cluster works on 256 rows i x 256 rows j
+// at a time; each CTA stages its own 128 rows i (hi and lo) and half of the rows j (hi and lo), 64 KiB per stage,
+// three stages; warp 0 = TMA producer, warp 1 = MMA issuer (leader CTA), warps 2-5 = epilogue (thread = row i)
+// over two TMEM accumulators.  A cluster takes a contiguous run of tile pairs of the lower triangle (one set) or
+// of the whole matrix (two sets).  No load is multicast; every wait is bounded.
+#include <cstring>
+
+#include "umma_pair.cuh"
+
+namespace siso {
+
+struct MergeCandidate {
+    int32_t i, j;
+    float sim;
+};
+struct MergeCtlView {                 // same layout as MergeCtl in merge.cu
+    unsigned long long n_cand;
+    int overflow;
+    int n_merged;
+};
+
+namespace tcm {
+
+using namespace umma2;
+
+constexpr int TM = 128;             // rows i per CTA
+constexpr int TN = 256;             // rows j per tile (128 staged by each CTA)
+constexpr int TK = 64;
+constexpr int STAGES = 3;
+constexpr int ACC_STAGES = 2;
+constexpr int THREADS = 192;
+constexpr uint32_t OPER_BYTES = TM * TK * 2;              // 16 KiB: 128 rows x 64 bf16
+constexpr uint32_t STAGE_BYTES = 4 * OPER_BYTES;          // hi_i, lo_i, hi_j (half), lo_j (half)
+constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 4096;
+constexpr uint32_t TMEM_COLS = ACC_STAGES * TN;
+constexpr float FILTER_MARGIN = 1e-4f;
+
+// D fp32, A and B bf16, K-major, N = 256, M = 256 (128 rows per CTA of the pair)
+constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(TN >> 3) << 17) |
+                           (static_cast<uint32_t>((2 * TM) >> 4) << 24);
+
+struct Shared {
+    uint64_t full[STAGES], empty[STAGES], acc_full[ACC_STAGES], acc_empty[ACC_STAGES];
+    uint32_t tmem_base;
+    int abort_flag;
+    uint8_t jflag[4][TN];                // per epilogue warp; bit 0: live, bit 1: member of C_cur
+};
+
+// tile pair number -> (row tile I, column tile t); one set: lower triangle incl. the diagonal, row by row
+__device__ __forceinline__ void pair_to_tiles(long long p, int tiles, bool two_sets, int *I, int *t) {
+    if (two_sets) {
+        *I = static_cast<int>(p / tiles);
+        *t = static_cast<int>(p - static_cast<long long>(*I) * tiles);
+    } else {
+        long long r = static_cast<long long>((sqrt(8.0 * static_cast<double>(p) + 1.0) - 1.0) * 0.5);
+        while (r * (r + 1) / 2 > p) --r;
+        while ((r + 1) * (r + 2) / 2 <= p) ++r;
+        *I = static_cast<int>(r);
+        *t = static_cast<int>(p - r * (r + 1) / 2);
+    }
+}
+
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
+merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CUtensorMap map_lo,
+                          const uint8_t *__restrict__ valid, const uint8_t *__restrict__ seed, int64_t N, int D, int tiles,
+                          long long n_pairs, long long pairs_per_cluster, float theta_filter, MergeCtlView *ctl,
+                          MergeCandidate *__restrict__ cand, unsigned long long max_cand, int *status) {
+    extern __shared__ uint8_t smem_raw[];
+    uint8_t *stage_mem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
+    Shared *sh = reinterpret_cast<Shared *>(stage_mem + STAGES * STAGE_BYTES);
+    volatile int *abort_flag = &sh->abort_flag;
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const uint32_t rank = cluster_rank();
+    const bool two_sets = seed != nullptr;
+    const long long cluster_id = blockIdx.x >> 1;
+    const long long p_begin = cluster_id * pairs_per_cluster;
+    const long long p_end = min(n_pairs, p_begin + pairs_per_cluster);
+    const int k_slabs = (D + TK - 1) / TK;
+    const bool skip = ctl->overflow != 0;           // set before the launch (two sets: the insertion failed)
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < STAGES; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(&sh->acc_full[a], 1); mbar_init(&sh->acc_empty[a], 8); }
+        sh->abort_flag = 0;
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
+                     ::"r"(smem_u32(&sh->tmem_base)), "r"(TMEM_COLS) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::2.sync.aligned;" ::: "memory");
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync();
+    tcgen05_fence_after();
+    const uint32_t tmem_base = sh->tmem_base;
+
+    if (skip) {
+        // nothing to do; fall through to the common teardown
+    } else if (warp == 0) {
+        // ------------------------------------------------------------------ TMA producer (both CTAs)
+        if (lane == 0) {
+            uint32_t stage = 0, phase = 0;
+            bool ok = true;
+            for (long long p = p_begin; p < p_end && ok; ++p) {
+                int I, t;
+                pair_to_tiles(p, tiles, two_sets, &I, &t);
+                const int i0 = I * (2 * TM) + static_cast<int>(rank) * TM;        // this CTA's own rows i
+                const int n0 = t * TN + static_cast<int>(rank) * (TN / 2);        // its half of the rows j
+                for (int ks = 0; ks < k_slabs; ++ks) {
+                    if (!mbar_wait(&sh->empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
+                    uint8_t *dst = stage_mem + stage * STAGE_BYTES;
+                    const uint32_t full_leader = cluster_addr(smem_u32(&sh->full[stage]), 0);
+                    if (rank == 0) mbar_arrive_expect_tx(&sh->full[stage], 2 * STAGE_BYTES);
+                    tma_load_2d_pair(dst, &map_hi, ks * TK, i0, full_leader);
+                    tma_load_2d_pair(dst + OPER_BYTES, &map_lo, ks * TK, i0, full_leader);
+                    tma_load_2d_pair(dst + 2 * OPER_BYTES, &map_hi, ks * TK, n0, full_leader);
+                    tma_load_2d_pair(dst + 3 * OPER_BYTES, &map_lo, ks * TK, n0, full_leader);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ------------------------------------------------------------------ MMA issuer (leader only)
+        if (lane == 0 && rank == 0) {
+            uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
+            bool ok = true;
+            for (long long p = p_begin; p < p_end && ok; ++p) {
+                if (!mbar_wait(&sh->acc_empty[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
+                tcgen05_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * TN;
+                for (int ks = 0; ks < k_slabs; ++ks) {
+                    if (!mbar_wait(&sh->full[stage], phase, abort_flag)) { ok = false; break; }
+                    tcgen05_fence_after();
+                    const uint32_t base = smem_u32(stage_mem + stage * STAGE_BYTES);
+                    const uint64_t a_hi = smem_desc_sw128(base), a_lo = smem_desc_sw128(base + OPER_BYTES);
+                    const uint64_t b_hi = smem_desc_sw128(base + 2 * OPER_BYTES), b_lo = smem_desc_sw128(base + 3 * OPER_BYTES);
+#pragma unroll
+                    for (int kk = 0; kk < TK / 16; ++kk) {
+                        const uint64_t o = static_cast<uint64_t>(2 * kk);
+                        umma_bf16_pair(d_tmem, a_hi + o, b_hi + o, IDESC, (ks | kk) ? 1u : 0u);
+                        umma_bf16_pair(d_tmem, a_hi + o, b_lo + o, IDESC, 1u);
+                        umma_bf16_pair(d_tmem, a_lo + o, b_hi + o, IDESC, 1u);
+                    }
+                    umma_commit_both(&sh->empty[stage]);
+                    if (++stage == STAGES) { stage = 0; phase ^= 1u; }
+                }
+                if (!ok) break;
+                umma_commit_both(&sh->acc_full[acc]);
+                if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+            }
+        }
+    } else {
+        // ------------------------------------------------------------------ epilogue (warps 2..5 of both CTAs)
+        const int quarter = warp & 3;
+        uint8_t *jflag = sh->jflag[quarter];                 // this warp's own copy: no barrier between the warps
+        uint32_t acc = 0, acc_phase = 0;
+        bool ok = true;
+        int last_I = -1;
+        bool row_ok = false;
+        long long gi = 0;
+        for (long long p = p_begin; p < p_end && ok; ++p) {
+            int I, t;
+            pair_to_tiles(p, tiles, two_sets, &I, &t);
+            const long long n0 = static_cast<long long>(t) * TN;
+            if (I != last_I) {
+                last_I = I;
+                gi = static_cast<long long>(I) * (2 * TM) + static_cast<long long>(rank) * TM + quarter * 32 + lane;
+                // a row takes part if it is live and not a member of C_cur (those are never merged into others)
+                row_ok = gi < N && valid[gi] != 0 && !(two_sets && seed[gi] != 0);
+            }
+            // flags of the tile's 256 rows j
+            __syncwarp();
+#pragma unroll
+            for (int h = 0; h < TN / 32; ++h) {
+                const long long gj = n0 + h * 32 + lane;
+                uint8_t f = 0;
+                if (gj < N) f = (valid[gj] ? 1 : 0) | ((two_sets && seed[gj]) ? 2 : 0);
+                jflag[h * 32 + lane] = f;
+            }
+            __syncwarp();
+            if (!mbar_wait(&sh->acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+            tcgen05_fence_after();
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * TN;
+            uint32_t ra[32], rb[32];
+            auto scan = [&](uint32_t (&r)[32], int ch) {
+                float m = __uint_as_float(r[0]);
+#pragma unroll
+                for (int j = 1; j < 32; ++j) m = fmaxf(m, __uint_as_float(r[j]));
+                if (!(row_ok && m > theta_filter)) return;
+                // this row has values above the filter in this chunk: which of them are pairs of the sweep
+                uint32_t take = 0;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    const long long gj = n0 + ch * 32 + j;
+                    const uint8_t f = jflag[ch * 32 + j];
+                    const bool pair_ok = (f & 1) && ((f & 2) || gj < gi) && gj != gi;
+                    if (pair_ok && __uint_as_float(r[j]) > theta_filter) take |= 1u << j;
+                }
+                if (!take) return;
+                const unsigned long long base = atomicAdd(&ctl->n_cand, static_cast<unsigned long long>(__popc(take)));
+                unsigned long long pos = base;
+#pragma unroll
+                for (int j = 0; j < 32; ++j) {
+                    if ((take >> j) & 1u) {
+                        if (pos < max_cand) {
+                            MergeCandidate cd;
+                            cd.i = static_cast<int32_t>(gi);
+                            cd.j = static_cast<int32_t>(n0 + ch * 32 + j);
+                            cd.sim = __uint_as_float(r[j]);
+                            cand[pos] = cd;
+                        } else {
+                            ctl->overflow = 1;
+                        }
+                        ++pos;
+                    }
+                }
+            };
+            tmem_ld_32x32(taddr, ra);
+#pragma unroll 1
+            for (int ch = 0; ch < TN / 32; ch += 2) {
+                tmem_ld_fence(ra);
+                tmem_ld_32x32(taddr + (ch + 1) * 32, rb);
+                scan(ra, ch);
+                tmem_ld_fence(rb);
+                if (ch + 2 < TN / 32) tmem_ld_32x32(taddr + (ch + 2) * 32, ra);
+                scan(rb, ch + 1);
+            }
+            tcgen05_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive_cluster(cluster_addr(smem_u32(&sh->acc_empty[acc]), 0));
+            if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
+        }
+    }
+
+    // ---------------------------------------------------------------------- teardown
+    __syncwarp();
+    if (*abort_flag) {
+        for (int i = 0; i < 64; ++i) __nanosleep(1000);
+        if (threadIdx.x == 0) set_status(status, SISO_ERR_TIMEOUT);
+    }
+    tcgen05_fence_before();
+    __syncthreads();
+    cluster_sync();
+    if (warp == 1) {
+        tcgen05_fence_after();
+        asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
+    }
+}
+
+// x -> (bf16(x), bf16(x - bf16(x))), four elements per thread
+__global__ void split_bf16_kernel(const float *__restrict__ x, __nv_bfloat16 *__restrict__ hi, __nv_bfloat16 *__restrict__ lo,
+                                  long long n4) {
+    const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n4) return;
+    const float4 v = __ldg(reinterpret_cast<const float4 *>(x) + i);
+    const float f[4] = {v.x, v.y, v.z, v.w};
+    __nv_bfloat16 h[4], l[4];
+#pragma unroll
+    for (int k = 0; k < 4; ++k) {
+        h[k] = __float2bfloat16_rn(f[k]);
+        l[k] = __float2bfloat16_rn(f[k] - __bfloat162float(h[k]));
+    }
+    *reinterpret_cast<uint2 *>(hi + 4 * i) = *reinterpret_cast<const uint2 *>(h);
+    *reinterpret_cast<uint2 *>(lo + 4 * i) = *reinterpret_cast<const uint2 *>(l);
+}
+
+// One warp per provisional candidate: exact similarity of the fp32 vectors (products and sums in fp64).  The pair
+// stays a candidate if it exceeds theta_C (strict, as in Algorithm 1); otherwise its row index becomes -1.
+__global__ void __launch_bounds__(256)
+merge_verify_kernel(const MergeCtlView *ctl, const float *__restrict__ C, int D, float theta, MergeCandidate *__restrict__ cand,
+                    unsigned long long max_cand, uint32_t *__restrict__ row_count) {
+    if (ctl->overflow) return;
+    const unsigned long long n = ctl->n_cand < max_cand ? ctl->n_cand : max_cand;
+    const int lane = threadIdx.x & 31;
+    const unsigned long long warps = static_cast<unsigned long long>(gridDim.x) * (blockDim.x >> 5);
+    for (unsigned long long e = static_cast<unsigned long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); e < n; e += warps) {
+        const MergeCandidate cd = cand[e];
+        const float4 *a = reinterpret_cast<const float4 *>(C + static_cast<long long>(cd.i) * D);
+        const float4 *b = reinterpret_cast<const float4 *>(C + static_cast<long long>(cd.j) * D);
+        double s = 0.0;
+        for (int q = lane; q < D / 4; q += 32) {
+            const float4 x = __ldg(a + q), y = __ldg(b + q);
+            s += static_cast<double>(x.x) * static_cast<double>(y.x) + static_cast<double>(x.y) * static_cast<double>(y.y) +
+                 static_cast<double>(x.z) * static_cast<double>(y.z) + static_cast<double>(x.w) * static_cast<double>(y.w);
+        }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) s += __shfl_xor_sync(0xFFFFFFFFu, s, o);
+        if (lane == 0) {
+            if (s > static_cast<double>(theta)) {
+                cand[e].sim = static_cast<float>(s);
+                atomicAdd(&row_count[cd.i], 1u);
+            } else {
+                cand[e].i = -1;
+            }
+        }
+    }
+}
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static siso_status_t encode_rows_map(EncodeTiledFn fn, CUtensorMap *map, const void *base, uint64_t rows, uint64_t dim) {
+    cuuint64_t gdim[2] = {dim, rows};
+    cuuint64_t gstride[1] = {dim * 2};
+    cuuint32_t box[2] = {static_cast<cuuint32_t>(TK), static_cast<cuuint32_t>(TM)};
+    cuuint32_t estr[2] = {1, 1};
+    CUresult r = fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), gdim, gstride, box, estr,
+                    CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+                    CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) return check_cuda(cudaErrorInvalidValue, "cuTensorMapEncodeTiled");
+    return SISO_OK;
+}
+
+}  // namespace tcm
+
+size_t merge_tensor_scratch_bytes(const Cache *c) {
+    return 2 * pad256(static_cast<size_t>(c->rows_alloc) * c->dim * sizeof(__nv_bfloat16));
+}
+
+// Sweep + exact check.  `ctl` and `row_count` are zeroed (or carry the two-set insertion's failure flag); on return
+// (in stream order) cand[0 .. min(n_cand, max_cand)) holds the provisional pairs, the confirmed ones with their
+// exact similarity and i >= 0, and row_count[i] counts the confirmed pairs of row i.
+siso_status_t launch_merge_sweep_tensor(Cache *c, Scratch *scr, const uint8_t *seed, float theta_c, void *ctl, void *cand,
+                                        size_t max_cand, uint32_t *row_count, cudaStream_t s) {
+    static tcm::EncodeTiledFn encode = nullptr;
+    if (!encode) {
+        void *fn = nullptr;
+        cudaDriverEntryPointQueryResult qres;
+        SISO_CUDA(cudaGetDriverEntryPointByVersion("cuTensorMapEncodeTiled", &fn, 12000, cudaEnableDefault, &qres));
+        if (!fn || qres != cudaDriverEntryPointSuccess) return check_cuda(cudaErrorNotSupported, "cuTensorMapEncodeTiled lookup");
+        encode = reinterpret_cast<tcm::EncodeTiledFn>(fn);
+    }
+    const int64_t N = c->capacity, rows = c->rows_alloc;
+    const size_t elems = static_cast<size_t>(rows) * c->dim;
+    __nv_bfloat16 *hi = scr->take<__nv_bfloat16>(elems);
+    __nv_bfloat16 *lo = scr->take<__nv_bfloat16>(elems);
+    const long long n4 = static_cast<long long>(elems / 4);
+    tcm::split_bf16_kernel<<<static_cast<unsigned>((n4 + 255) / 256), 256, 0, s>>>(c->master, hi, lo, n4);
+    SISO_LAUNCHED(c);
+    CUtensorMap map_hi, map_lo;
+    SISO_TRY(tcm::encode_rows_map(encode, &map_hi, hi, static_cast<uint64_t>(rows), static_cast<uint64_t>(c->dim)));
+    SISO_TRY(tcm::encode_rows_map(encode, &map_lo, lo, static_cast<uint64_t>(rows), static_cast<uint64_t>(c->dim)));
+    const int tiles = static_cast<int>((N + 2 * tcm::TM - 1) / (2 * tcm::TM));       // 256 rows per tile
+    const long long n_pairs = seed ? static_cast<long long>(tiles) * tiles : static_cast<long long>(tiles) * (tiles + 1) / 2;
+    const long long clusters = std::max<long long>(1, std::min<long long>(n_pairs, c->sm_count / 2));
+    const long long per = (n_pairs + clusters - 1) / clusters;
+    const long long used = (n_pairs + per - 1) / per;
+    if (!c->merge_tensor_attr_set) {
+        SISO_CUDA(cudaFuncSetAttribute(tcm::merge_sweep_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tcm::SMEM_BYTES));
+        c->merge_tensor_attr_set = true;
+    }
+    tcm::merge_sweep_tensor_kernel<<<static_cast<unsigned>(2 * used), tcm::THREADS, tcm::SMEM_BYTES, s>>>(
+        map_hi, map_lo, c->valid, seed, N, c->dim, tiles, n_pairs, per, theta_c - tcm::FILTER_MARGIN,
+        static_cast<MergeCtlView *>(ctl), static_cast<MergeCandidate *>(cand), max_cand, c->status);
+    SISO_LAUNCHED(c);
+    tcm::merge_verify_kernel<<<8 * c->sm_count, 256, 0, s>>>(static_cast<const MergeCtlView *>(ctl), c->master, c->dim, theta_c,
+                                                             static_cast<MergeCandidate *>(cand), max_cand, row_count);
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
+
+}  // namespace siso

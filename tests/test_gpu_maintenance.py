@@ -99,10 +99,12 @@ def test_update_counts_accesses_after_decay_reset():
 @pytest.mark.parametrize("dtype,mode,theta_c,weighted", [
     ("f32", "T", 0.90, True), ("f32", "P", 0.90, True), ("f32", "P", 0.86, False), ("bf16", "P", 0.90, True),
 ])
-def test_self_merge_matches_oracle(dtype, mode, theta_c, weighted):
+@pytest.mark.parametrize("sweep", [siso.PATH_SIMT, siso.PATH_TENSOR])
+def test_self_merge_matches_oracle(dtype, mode, theta_c, weighted, sweep):
     w = W.config(3, n_centroids=1500, dim=136, n_clusters=90, mode=mode, sigma=0.06, dtype=dtype)
     sizes = np.random.default_rng(9).integers(1, 9, 1500).astype(np.float64)
     cache, ora = make_pair(w, capacity=1536, sizes=sizes)
+    cache.set_option(siso.OPT_MERGE_PATH, sweep)       # CUDA-core sweep, or tensor-core filter + exact check
     entry = ora.master.copy()
     flags = siso.MERGE_WEIGHTED_MEAN if weighted else siso.MERGE_SIZES_ONLY
     for rounds in range(40):
@@ -140,9 +142,11 @@ def test_self_merge_matches_oracle(dtype, mode, theta_c, weighted):
     cache.check_status()
 
 
-def test_merge_extremes_holes_and_overflow():
+@pytest.mark.parametrize("sweep", [siso.PATH_SIMT, siso.PATH_TENSOR])
+def test_merge_extremes_holes_and_overflow(sweep):
     w = W.config(3, n_centroids=700, dim=64, n_clusters=30, mode="P")
     cache, ora = make_pair(w, capacity=1000)
+    cache.set_option(siso.OPT_MERGE_PATH, sweep)
     victims = cache.evict(50).cpu().numpy()
     assert (victims == ora.evict(50)).all()
     mm, n = cache.merge(1.0, siso.MERGE_WEIGHTED_MEAN)
@@ -163,7 +167,8 @@ def test_merge_extremes_holes_and_overflow():
 
 
 @pytest.mark.parametrize("dtype,weighted", [("f32", True), ("bf16", False)])
-def test_two_set_merge_matches_oracle(dtype, weighted):
+@pytest.mark.parametrize("sweep", [siso.PATH_SIMT, siso.PATH_TENSOR])
+def test_two_set_merge_matches_oracle(dtype, weighted, sweep):
     """Algorithm 1 as printed: C_cur = the cache, C_repo = new rows; holes in the cache interleave the two."""
     w = W.config(3, n_centroids=1400, dim=136, n_clusters=80, mode="P", sigma=0.06, dtype=dtype)
     cur, repo = w.centroids[:800], w.centroids[800:]
@@ -172,6 +177,7 @@ def test_two_set_merge_matches_oracle(dtype, weighted):
     repo_sizes = rng.integers(1, 5, 600).astype(np.float64)
     cap = 1500
     cache = siso.SisoCache(cap, w.dim, dtype)
+    cache.set_option(siso.OPT_MERGE_PATH, sweep)
     ora = oracle.OracleCache(cap, w.dim, dtype)
     cache.insert(to_dev(cur, dtype), torch.from_numpy(cur_sizes))
     ora.insert(cur, sizes=cur_sizes)
