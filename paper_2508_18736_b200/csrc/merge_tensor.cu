@@ -12,9 +12,11 @@
 // Kernel layout (CTA pairs, cta_group::2, as in the large-batch lookup): a cluster works on 256 rows i x 256 rows j
 // at a time; each CTA stages its own 128 rows i (hi and lo) and half of the rows j (hi and lo), 64 KiB per stage,
 // three stages; warp 0 = TMA producer, warp 1 = MMA issuer (leader CTA), warps 2-5 = epilogue (thread = row i)
-// over two TMEM accumulators.  A cluster takes a contiguous run of tile pairs of the lower triangle (one set) or
-// of the whole matrix (two sets).  No load is multicast; every wait is bounded.
+// over two TMEM accumulators.  The tile pairs of the lower triangle (one set) or of the whole matrix (two sets) are
+// listed block by block (9 x 9 tiles) and dealt to the clusters round robin, so the clusters that run at the same
+// time work inside one block and share its rows through L2.  No load is multicast; every wait is bounded.
 #include <cstring>
+#include <vector>
 
 #include "umma_pair.cuh"
 
@@ -57,24 +59,17 @@ struct Shared {
     uint8_t jflag[4][TN];                // per epilogue warp; bit 0: live, bit 1: member of C_cur
 };
 
-// tile pair number -> (row tile I, column tile t); one set: lower triangle incl. the diagonal, row by row
-__device__ __forceinline__ void pair_to_tiles(long long p, int tiles, bool two_sets, int *I, int *t) {
-    if (two_sets) {
-        *I = static_cast<int>(p / tiles);
-        *t = static_cast<int>(p - static_cast<long long>(*I) * tiles);
-    } else {
-        long long r = static_cast<long long>((sqrt(8.0 * static_cast<double>(p) + 1.0) - 1.0) * 0.5);
-        while (r * (r + 1) / 2 > p) --r;
-        while ((r + 1) * (r + 2) / 2 <= p) ++r;
-        *I = static_cast<int>(r);
-        *t = static_cast<int>(p - r * (r + 1) / 2);
-    }
+// tile pair number -> (row tile I, column tile t), from the list the host wrote
+__device__ __forceinline__ void pair_to_tiles(const uint32_t *__restrict__ pair_list, long long p, int *I, int *t) {
+    const uint32_t v = __ldg(pair_list + p);
+    *I = static_cast<int>(v >> 16);
+    *t = static_cast<int>(v & 0xFFFFu);
 }
 
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CUtensorMap map_lo,
-                          const uint8_t *__restrict__ valid, const uint8_t *__restrict__ seed, int64_t N, int D, int tiles,
-                          long long n_pairs, long long pairs_per_cluster, float theta_filter, MergeCtlView *ctl,
+                          const uint8_t *__restrict__ valid, const uint8_t *__restrict__ seed, int64_t N, int D,
+                          const uint32_t *__restrict__ pair_list, long long n_pairs, float theta_filter, MergeCtlView *ctl,
                           MergeCandidate *__restrict__ cand, unsigned long long max_cand, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *stage_mem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -84,9 +79,9 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const uint32_t rank = cluster_rank();
     const bool two_sets = seed != nullptr;
-    const long long cluster_id = blockIdx.x >> 1;
-    const long long p_begin = cluster_id * pairs_per_cluster;
-    const long long p_end = min(n_pairs, p_begin + pairs_per_cluster);
+    const long long p_begin = blockIdx.x >> 1;             // this cluster's tile pairs: p_begin, p_begin + clusters, ...
+    const long long p_step = gridDim.x >> 1;
+    const long long p_end = n_pairs;
     const int k_slabs = (D + TK - 1) / TK;
     const bool skip = ctl->overflow != 0;           // set before the launch (two sets: the insertion failed)
 
@@ -115,9 +110,9 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
         if (lane == 0) {
             uint32_t stage = 0, phase = 0;
             bool ok = true;
-            for (long long p = p_begin; p < p_end && ok; ++p) {
+            for (long long p = p_begin; p < p_end && ok; p += p_step) {
                 int I, t;
-                pair_to_tiles(p, tiles, two_sets, &I, &t);
+                pair_to_tiles(pair_list, p, &I, &t);
                 const int i0 = I * (2 * TM) + static_cast<int>(rank) * TM;        // this CTA's own rows i
                 const int n0 = t * TN + static_cast<int>(rank) * (TN / 2);        // its half of the rows j
                 for (int ks = 0; ks < k_slabs; ++ks) {
@@ -138,7 +133,7 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
         if (lane == 0 && rank == 0) {
             uint32_t stage = 0, phase = 0, acc = 0, acc_phase = 0;
             bool ok = true;
-            for (long long p = p_begin; p < p_end && ok; ++p) {
+            for (long long p = p_begin; p < p_end && ok; p += p_step) {
                 if (!mbar_wait(&sh->acc_empty[acc], acc_phase ^ 1u, abort_flag)) { ok = false; break; }
                 tcgen05_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * TN;
@@ -172,9 +167,9 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
         int last_I = -1;
         bool row_ok = false;
         long long gi = 0;
-        for (long long p = p_begin; p < p_end && ok; ++p) {
+        for (long long p = p_begin; p < p_end && ok; p += p_step) {
             int I, t;
-            pair_to_tiles(p, tiles, two_sets, &I, &t);
+            pair_to_tiles(pair_list, p, &I, &t);
             const long long n0 = static_cast<long long>(t) * TN;
             if (I != last_I) {
                 last_I = I;
@@ -329,7 +324,8 @@ static siso_status_t encode_rows_map(EncodeTiledFn fn, CUtensorMap *map, const v
 }  // namespace tcm
 
 size_t merge_tensor_scratch_bytes(const Cache *c) {
-    return 2 * pad256(static_cast<size_t>(c->rows_alloc) * c->dim * sizeof(__nv_bfloat16));
+    const size_t tiles = static_cast<size_t>((c->capacity + 2 * tcm::TM - 1) / (2 * tcm::TM));
+    return 2 * pad256(static_cast<size_t>(c->rows_alloc) * c->dim * sizeof(__nv_bfloat16)) + pad256(sizeof(uint32_t) * tiles * tiles);
 }
 
 // Sweep + exact check.  `ctl` and `row_count` are zeroed (or carry the two-set insertion's failure flag); on return
@@ -356,16 +352,26 @@ siso_status_t launch_merge_sweep_tensor(Cache *c, Scratch *scr, const uint8_t *s
     SISO_TRY(tcm::encode_rows_map(encode, &map_hi, hi, static_cast<uint64_t>(rows), static_cast<uint64_t>(c->dim)));
     SISO_TRY(tcm::encode_rows_map(encode, &map_lo, lo, static_cast<uint64_t>(rows), static_cast<uint64_t>(c->dim)));
     const int tiles = static_cast<int>((N + 2 * tcm::TM - 1) / (2 * tcm::TM));       // 256 rows per tile
-    const long long n_pairs = seed ? static_cast<long long>(tiles) * tiles : static_cast<long long>(tiles) * (tiles + 1) / 2;
-    const long long clusters = std::max<long long>(1, std::min<long long>(n_pairs, c->sm_count / 2));
-    const long long per = (n_pairs + clusters - 1) / clusters;
-    const long long used = (n_pairs + per - 1) / per;
+    if (tiles > 0xFFFF) return SISO_ERR_UNSUPPORTED;
+    // the tile pairs block by block: blocks of SB x SB tiles, row-major inside a block
+    constexpr int SB = 9;
+    std::vector<uint32_t> list;
+    list.reserve(static_cast<size_t>(tiles) * (tiles + 1) / (seed ? 1 : 2));
+    for (int bi = 0; bi < tiles; bi += SB)
+        for (int bt = 0; bt < (seed ? tiles : bi + 1); bt += SB)
+            for (int I = bi; I < std::min(tiles, bi + SB); ++I)
+                for (int t = bt; t < std::min(seed ? tiles : I + 1, bt + SB); ++t)
+                    list.push_back((static_cast<uint32_t>(I) << 16) | static_cast<uint32_t>(t));
+    const long long n_pairs = static_cast<long long>(list.size());
+    uint32_t *pair_list = scr->take<uint32_t>(list.size());
+    SISO_CUDA(cudaMemcpyAsync(pair_list, list.data(), sizeof(uint32_t) * list.size(), cudaMemcpyHostToDevice, s));
+    const long long used = std::max<long long>(1, std::min<long long>(n_pairs, c->sm_count / 2));
     if (!c->merge_tensor_attr_set) {
         SISO_CUDA(cudaFuncSetAttribute(tcm::merge_sweep_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tcm::SMEM_BYTES));
         c->merge_tensor_attr_set = true;
     }
     tcm::merge_sweep_tensor_kernel<<<static_cast<unsigned>(2 * used), tcm::THREADS, tcm::SMEM_BYTES, s>>>(
-        map_hi, map_lo, c->valid, seed, N, c->dim, tiles, n_pairs, per, theta_c - tcm::FILTER_MARGIN,
+        map_hi, map_lo, c->valid, seed, N, c->dim, pair_list, n_pairs, theta_c - tcm::FILTER_MARGIN,
         static_cast<MergeCtlView *>(ctl), static_cast<MergeCandidate *>(cand), max_cand, c->status);
     SISO_LAUNCHED(c);
     tcm::merge_verify_kernel<<<8 * c->sm_count, 256, 0, s>>>(static_cast<const MergeCtlView *>(ctl), c->master, c->dim, theta_c,
