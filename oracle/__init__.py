@@ -60,6 +60,8 @@ def lib():
         L.siso_oracle_choose_theta.restype = i32
         L.siso_oracle_correct_theta.argtypes = [vp, i32, i32, f64, f64]
         L.siso_oracle_correct_theta.restype = i32
+        L.siso_oracle_cluster.argtypes = [vp, i32, i64, i32, f64, vp, vp, vp, vp]
+        L.siso_oracle_cluster.restype = i64
         _lib = L
     return _lib
 
@@ -144,6 +146,21 @@ def correct_theta(thetas: np.ndarray, chosen: int, w_est: float, w_meas: float) 
     """Sec. 4.3 correction: one table entry down (measured wait longer) or up (shorter) if they differ by > 10 %."""
     th = _c(np.asarray(thetas, dtype=np.float32))
     return int(lib().siso_oracle_correct_theta(_p(th), th.shape[0], int(chosen), float(w_est), float(w_meas)))
+
+
+def cluster(vecs: np.ndarray, theta_c: float, want_centroids: bool = True):
+    """Community detection at theta_c (Sec. 4.1; the steps are stated at siso_oracle_cluster).
+    Returns (label [n] int32, centres [k] int32 in founding order, sizes [k] float64, centroids [k, D] float64 or None)."""
+    v = _c(vecs)
+    n, D = v.shape
+    label = np.empty(n, np.int32)
+    centres = np.empty(n, np.int32)
+    sizes = np.empty(n, np.float64)
+    cent = np.empty((n, D), np.float64) if want_centroids else None
+    k = lib().siso_oracle_cluster(_p(v), _dtype_code(v), n, D, float(theta_c), _p(label), _p(centres), _p(sizes), _p(cent))
+    if k < 0:
+        raise MemoryError("oracle clustering: allocation failed")
+    return label, centres[:k].copy(), sizes[:k].copy(), (cent[:k].copy() if want_centroids else None)
 
 
 class OracleCache:

@@ -23,6 +23,9 @@
  *   evict         FilteringCentroids of Algorithm 1: remove the smallest
  *                 (cluster_size, access_count) entry while over capacity, then
  *                 cluster_size /= 1.1 and access_count = 0 for the rest.
+ *   cluster       the clustering step of Sec. 4.1 (community detection at theta_C); the
+ *                 paper names the method without stating it, so the steps are a reading:
+ *                 see siso_oracle_cluster.
  *   insert        the else-branch of MergeCentroids (new entry, access_count =
  *                 infinity) used for spare-space caching of individual vectors
  *                 (Sec. 5.2.5: left-over space holds single vectors under LRU).
@@ -375,4 +378,76 @@ int siso_oracle_correct_theta(const float *thetas, int n_thetas, int chosen, dou
         }
     }
     return next < 0 ? chosen : next;
+}
+
+/* ---------------------------------------------------------------------------
+ * Clustering of Sec. 4.1: community detection at the clustering threshold
+ * theta_C.  The paper only names the method; the reading taken here:
+ *   - u and v are neighbours if their cosine (dot product of unit vectors, summed
+ *     in index order in binary64) is strictly above theta_C; every vector is its
+ *     own neighbour;
+ *   - vectors are visited by neighbourhood size, largest first, ties by index;
+ *   - a visited vector that belongs to no community yet founds one: it is the
+ *     centre, and every neighbour that belongs to no community yet joins it;
+ *     a visited vector that already belongs to a community is passed over.
+ * So every vector ends in exactly one community (possibly alone), communities
+ * are disjoint, and cluster_size is the number of members (Sec. 4.1: "the number
+ * of vectors in the cluster").
+ * Outputs: label[v] = index of the centre of v's community; centres[] in the order
+ * they were founded; sizes[] alongside; if centroids != NULL, row c = the mean of
+ * the members of community c (members added in ascending index) scaled to unit
+ * length (Sec. 3.1: a centroid is the mean point of its group).  Returns the
+ * number of communities.
+ * ------------------------------------------------------------------------- */
+typedef struct { int64_t degree; int64_t index; } visit_t;
+static int visit_cmp(const void *a, const void *b) {
+    const visit_t *x = (const visit_t *)a, *y = (const visit_t *)b;
+    if (x->degree != y->degree) return x->degree > y->degree ? -1 : 1;
+    return x->index < y->index ? -1 : (x->index > y->index ? 1 : 0);
+}
+
+int64_t siso_oracle_cluster(const void *V, int dtype, int64_t n, int D, double theta, int32_t *label,
+                            int32_t *centres, double *sizes, double *centroids) {
+    uint8_t *nb = (uint8_t *)calloc((size_t)n * (size_t)n, 1);   /* neighbour matrix */
+    visit_t *order = (visit_t *)malloc(sizeof(visit_t) * (size_t)n);
+    if (!nb || !order) { free(nb); free(order); return -1; }
+#pragma omp parallel for schedule(dynamic, 16)
+    for (int64_t u = 0; u < n; ++u)
+        for (int64_t v = 0; v < n; ++v)
+            nb[u * n + v] = (u == v) || (dot_rows(V, dtype, (size_t)u, V, dtype, (size_t)v, D) > theta);
+    for (int64_t v = 0; v < n; ++v) {
+        int64_t deg = 0;
+        for (int64_t u = 0; u < n; ++u) deg += nb[v * n + u];    /* symmetric: both directions multiply and add alike */
+        order[v].degree = deg;
+        order[v].index = v;
+        label[v] = -1;
+    }
+    qsort(order, (size_t)n, sizeof(visit_t), visit_cmp);
+    int64_t n_comm = 0;
+    for (int64_t k = 0; k < n; ++k) {
+        const int64_t v = order[k].index;
+        if (label[v] >= 0) continue;
+        int64_t members = 0;
+        for (int64_t u = 0; u < n; ++u)
+            if (nb[v * n + u] && label[u] < 0) { label[u] = (int32_t)v; ++members; }
+        centres[n_comm] = (int32_t)v;
+        sizes[n_comm] = (double)members;
+        ++n_comm;
+    }
+    if (centroids) {
+        for (int64_t c = 0; c < n_comm; ++c) {
+            double *row = centroids + (size_t)c * (size_t)D;
+            for (int d = 0; d < D; ++d) row[d] = 0.0;
+            for (int64_t u = 0; u < n; ++u)
+                if (label[u] == centres[c])
+                    for (int d = 0; d < D; ++d) row[d] += widen(V, dtype, (size_t)u * (size_t)D + (size_t)d);
+            double ss = 0.0;
+            for (int d = 0; d < D; ++d) ss += row[d] * row[d];
+            const double norm = sqrt(ss);
+            for (int d = 0; d < D; ++d) row[d] /= norm;
+        }
+    }
+    free(nb);
+    free(order);
+    return n_comm;
 }
