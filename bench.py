@@ -41,7 +41,7 @@ def parse_args():
     ap.add_argument("--queries", type=int, default=8192, help="query batch per step")
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor", "stream"])
     ap.add_argument("--workload", default="config4",
-                    choices=["config4", "config1", "config2", "config3", "config5", "stream_probe"],
+                    choices=["config4", "config1", "config2", "config3", "config5", "stream_probe", "cluster"],
                     help="config4 (default) is the benchmark contract; the others print one line each for the other "
                          "configurations (single GPU only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -407,6 +407,32 @@ def run_other(args):
                               "note": "whole pass (split, sweep, exact check, grouping, resolution, apply) over the "
                                       "lower-triangle flops N(N-1)/2 x 2D; the sweep kernel is about three quarters of it",
                               "fp32_alu_peak": fp32_peak})
+    elif args.workload == "cluster":
+        # stand-in for the query log that SISO-Cluster turns into centroids (Sec. 4.1): 131,072 unit vectors of dim 768
+        # around 13,107 cluster means (the paper's 10 queries per centroid), clustered at theta_C = 0.86
+        n, dim = (131072 if args.rows == (1 << 20) else args.rows), 768
+        w = W.config(3, threads=cores, n_centroids=n, dim=dim, n_clusters=max(2, n // 10), sigma=0.06)
+        cache = siso.SisoCache(64, dim, "f32")
+        v = to_dev(w.centroids, "f32")
+        times, k = [], 0
+        for it in range(max(3, steps // 4) + 1):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            label, centres, sizes, cent = cache.cluster(v, 0.86)
+            e1.record()
+            torch.cuda.synchronize()
+            if it > 0:
+                times.append(e0.elapsed_time(e1))
+            k = len(centres)
+        ms = statistics.median(times)
+        fl = float(n) * (n - 1) / 2 * dim * 2
+        tc_peak = peaks["bf16_tflops"] / 3.0
+        planted = int(len(np.unique(w.centroid_labels)))
+        line.update(metric=f"community detection, {n:,} x {dim} fp32 vectors, theta_C 0.86 (all pairs, order, founders, mean centroids)",
+                    value=n / ms * 1e3, unit="vectors/s", ms_per_step=ms, communities=k, planted_clusters=planted, dtype="f32",
+                    roofline={"bound": "tensor", "achieved": fl / ms / 1e9, "peak": tc_peak, "unit": "TFLOP/s",
+                              "frac": fl / ms / 1e9 / tc_peak, "traffic": None,
+                              "peak_kind": "measured bf16 burst peak / 3 (split-bf16 emulation of fp32 products)"})
     elif args.workload == "config5":
         sp = W.StreamSpec()
         stream = W.QueryStream(sp, threads=cores)

@@ -202,6 +202,27 @@ siso_status_t siso_lookup_small_noalloc(const void *d_centroids, const uint8_t *
                                         const float *d_theta, float theta_scalar, int32_t k, int32_t *d_idx,
                                         float *d_sim, uint8_t *d_hit, void *stream);
 
+/* Clustering of logged query vectors into centroids (Sec. 4.1, SISO-Cluster: community detection at the clustering
+ * threshold theta_C, which yields for every cluster a centroid and cluster_size, "the number of vectors in the
+ * cluster").  The paper names the method without stating its steps; the reading built here: two vectors are neighbours
+ * if their cosine is strictly above theta_c; vectors are visited by neighbourhood size, largest first, ties by index;
+ * a visited vector that belongs to no community founds one and takes every neighbour that belongs to none.
+ * d_vecs [n, dim] in the cache's dtype, unit norm, 16-byte aligned, n < 2^24; the cache's own contents are neither
+ * read nor written (the handle supplies dim, dtype, device, allocator and scratch memory).
+ * Outputs, each optional (NULL), all caller-owned device memory:
+ *   d_label     [n] int32   index of the centre of the vector's community (a centre labels itself)
+ *   d_centres   [n] int32   the centres in founding order; the first *h_n_clusters entries are written
+ *   d_sizes     [n] fp64    cluster_size of the communities, in the same order
+ *   d_centroids [n, dim]    cache dtype: per community the mean of its members (fp64 sums in ascending index), scaled
+ *                           to unit length (Sec. 3.1: a centroid is the mean point of its group); rows beyond the
+ *                           number of communities are not written.  The rows can be handed to siso_merge as C_repo
+ *                           with d_sizes as their cluster_size.
+ * h_n_clusters (host, optional): number of communities; if given the call synchronises the stream and returns the
+ * device status (SISO_ERR_OVERFLOW if the pairs above the threshold exceed the candidate buffer, whose size is the
+ * larger of SISO_OPT_MERGE_MAX_CANDIDATES and 16 n + 2^20; the outputs are then undefined). */
+siso_status_t siso_cluster(siso_cache_t *c, const void *d_vecs, int64_t n, float theta_c, int32_t *d_label,
+                           int32_t *d_centres, double *d_sizes, void *d_centroids, int64_t *h_n_clusters, void *stream);
+
 /* Threshold control (Sec. 4.3, the part on adjusting theta_R to meet the SLO).
  * siso_t2h builds the threshold-to-hit-ratio table: it looks up a sample of queries (k = 1, exact, no hit is
  * recorded in the statistics) and counts, for every threshold of the grid, the queries whose best similarity

@@ -21,7 +21,7 @@ _STATUS_NAMES = {0: "SISO_OK", 1: "SISO_ERR_INVALID_ARG", 2: "SISO_ERR_UNSUPPORT
 EXPORTS = ["siso_cache_create", "siso_cache_destroy", "siso_set_option", "siso_insert", "siso_lookup",
            "siso_lookup_host", "siso_update", "siso_merge", "siso_evict", "siso_make_room", "siso_insert_misses",
            "siso_stream_step", "siso_export", "siso_import", "siso_get_stats", "siso_sync_status",
-           "siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_lookup_small_noalloc", "siso_t2h", "siso_md1_wait",
+           "siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_lookup_small_noalloc", "siso_cluster", "siso_t2h", "siso_md1_wait",
            "siso_choose_theta", "siso_correct_theta"]
 
 
@@ -74,6 +74,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_stream_step.argtypes = [vp, vp, i64, vp, f32, vp, vp, vp, vp, vp, vp]
     L.siso_lookup_small_noalloc.argtypes = [vp, vp, i64, i32, i32, vp, i64, vp, f32, i32, vp, vp, vp, vp]
     L.siso_t2h.argtypes = [vp, vp, i64, vp, i32, vp, vp]
+    L.siso_cluster.argtypes = [vp, vp, i64, f32, vp, vp, vp, vp, ctypes.POINTER(i64), vp]
     L.siso_md1_wait.argtypes = [ctypes.c_double] * 3
     L.siso_md1_wait.restype = ctypes.c_double
     L.siso_choose_theta.argtypes = [vp, vp, i32, ctypes.c_double, ctypes.c_double, ctypes.c_double,
@@ -264,6 +265,20 @@ class SisoCache:
         self._check(self._lib.siso_stream_step(self._h, _ptr(q), n, _ptr(th_t), th_s, _ptr(idx), _ptr(sim), _ptr(hit),
                                                _ptr(victims), _ptr(slots), _stream(stream)), "siso_stream_step")
         return out
+
+    def cluster(self, vecs: torch.Tensor, theta_c: float, want_centroids: bool = True, stream=None):
+        """Community detection at theta_c over the rows of `vecs` (the cache's contents are not touched).
+        Returns (label [n] int32, centres [k] int32 in founding order, sizes [k] float64, centroids [k, dim] or None)."""
+        v = self._vec(vecs, "vecs")
+        n = v.shape[0]
+        label, centres = self._new((n,), torch.int32), self._new((n,), torch.int32)
+        sizes = self._new((n,), torch.float64)
+        cent = self._new((n, self.dim), self.torch_dtype) if want_centroids else None
+        k = ctypes.c_int64(0)
+        self._check(self._lib.siso_cluster(self._h, _ptr(v), n, float(theta_c), _ptr(label), _ptr(centres), _ptr(sizes),
+                                           _ptr(cent), ctypes.byref(k), _stream(stream)), "siso_cluster")
+        k = int(k.value)
+        return label, centres[:k], sizes[:k], (cent[:k] if want_centroids else None)
 
     def t2h(self, queries: torch.Tensor, thetas: torch.Tensor, stream=None) -> torch.Tensor:
         """Threshold-to-hit-ratio counts: int64 [len(thetas)] = sampled queries whose best similarity > theta."""

@@ -301,6 +301,28 @@ siso_status_t siso_merge(siso_cache_t *c, const void *d_repo, const double *d_re
     return SISO_OK;
 }
 
+siso_status_t siso_cluster(siso_cache_t *c, const void *d_vecs, int64_t n, float theta_c, int32_t *d_label, int32_t *d_centres,
+                           double *d_sizes, void *d_centroids, int64_t *h_n_clusters, void *stream) {
+    if (!c || n < 0 || !(theta_c == theta_c)) return SISO_ERR_INVALID_ARG;
+    if (n == 0) {
+        if (h_n_clusters) *h_n_clusters = 0;
+        return SISO_OK;
+    }
+    if (!d_vecs || !aligned16(d_vecs)) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    long long *d_n = h_n_clusters ? c->counters + CNT_SPARE : nullptr;
+    SISO_TRY(launch_cluster(c, d_vecs, n, theta_c, d_label, d_centres, d_sizes, d_centroids, d_n, s));
+    if (h_n_clusters) {
+        long long v = 0;
+        SISO_CUDA(cudaMemcpyAsync(&v, d_n, sizeof(v), cudaMemcpyDeviceToHost, s));
+        SISO_CUDA(cudaStreamSynchronize(s));
+        *h_n_clusters = v;
+        return siso_sync_status(c, stream);
+    }
+    return SISO_OK;
+}
+
 siso_status_t siso_evict(siso_cache_t *c, int64_t n_evict, uint32_t flags, int32_t *d_victims, void *stream) {
     if (!c || n_evict < 0 || (flags & ~SISO_EVICT_DECAY)) return SISO_ERR_INVALID_ARG;
     SISO_CUDA(cudaSetDevice(c->device));

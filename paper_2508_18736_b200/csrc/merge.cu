@@ -312,6 +312,40 @@ __global__ void merge_finish_kernel(MergeCtl *ctl, int64_t N, const int32_t *__r
     }
 }
 
+// Resolution of the candidate graph: state[i] = 1 survivor / 2 merged / 3 empty, target[i] = the survivor that i joins
+// (itself for survivors, -1 for empty slots).  `ctl` is a MergeCtl (only its overflow flag is read).
+siso_status_t launch_merge_resolve(Cache *c, void *ctl_v, int64_t N, const uint8_t *valid, const uint8_t *seed,
+                                   const uint32_t *row_off, const uint32_t *row_count, const int32_t *csr_j,
+                                   const float *csr_sim, uint8_t *state, int32_t *target, unsigned int *undecided,
+                                   cudaStream_t s) {
+    MergeCtl *ctl = static_cast<MergeCtl *>(ctl_v);
+    if (c->merge_resolve_grid == 0) {
+        int coop = 0, per_sm = 0;
+        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device) != cudaSuccess) coop = 0;
+        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, merge_resolve_grid_kernel, 256, 0) != cudaSuccess) {
+            cudaGetLastError();
+            per_sm = 0;
+        }
+        c->merge_resolve_grid = (coop && per_sm >= 1) ? c->sm_count * std::min(per_sm, 4) : -1;
+    }
+    if (c->merge_resolve_grid > 0) {
+        SISO_CUDA(cudaMemsetAsync(undecided, 0, 3 * sizeof(unsigned int), s));
+        const uint8_t *valid_p = valid;
+        const uint8_t *seed_p = seed;
+        int64_t n_arg = N;
+        volatile uint8_t *state_p = state;
+        void *args[] = {&ctl, &n_arg, &valid_p, &seed_p, &row_off, &row_count, &csr_j, &csr_sim, &state_p, &target, &undecided};
+        const int grid = static_cast<int>(std::min<int64_t>(c->merge_resolve_grid, (N + 255) / 256));
+        SISO_CUDA(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(merge_resolve_grid_kernel), dim3(grid), dim3(256),
+                                              args, 0, s));
+        c->launches += 1;
+    } else {
+        merge_resolve_kernel<<<1, 1024, 0, s>>>(ctl, N, valid, seed, row_off, row_count, csr_j, csr_sim, state, target);
+        SISO_LAUNCHED(c);
+    }
+    return SISO_OK;
+}
+
 siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes, int64_t n_repo, float theta_c,
                            uint32_t flags, int32_t *merge_map, long long *d_n_merged, cudaStream_t s) {
     const int64_t N = c->capacity;
@@ -379,30 +413,7 @@ siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes,
     SISO_TRY(launch_exclusive_scan_u32(c, row_off, N + 1, s));
     merge_scatter_kernel<<<4 * c->sm_count, 256, 0, s>>>(ctl, cand, row_off, row_cursor, csr_j, csr_sim);
     SISO_LAUNCHED(c);
-    if (c->merge_resolve_grid == 0) {
-        int coop = 0, per_sm = 0;
-        if (cudaDeviceGetAttribute(&coop, cudaDevAttrCooperativeLaunch, c->device) != cudaSuccess) coop = 0;
-        if (cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, merge_resolve_grid_kernel, 256, 0) != cudaSuccess) {
-            cudaGetLastError();
-            per_sm = 0;
-        }
-        c->merge_resolve_grid = (coop && per_sm >= 1) ? c->sm_count * std::min(per_sm, 4) : -1;
-    }
-    if (c->merge_resolve_grid > 0) {
-        SISO_CUDA(cudaMemsetAsync(undecided, 0, 3 * sizeof(unsigned int), s));
-        const uint8_t *valid_p = c->valid;
-        const uint8_t *seed_p = seed;
-        int64_t n_arg = N;
-        volatile uint8_t *state_p = state;
-        void *args[] = {&ctl, &n_arg, &valid_p, &seed_p, &row_off, &row_count, &csr_j, &csr_sim, &state_p, &target, &undecided};
-        const int grid = static_cast<int>(std::min<int64_t>(c->merge_resolve_grid, (N + 255) / 256));
-        SISO_CUDA(cudaLaunchCooperativeKernel(reinterpret_cast<const void *>(merge_resolve_grid_kernel), dim3(grid), dim3(256),
-                                              args, 0, s));
-        c->launches += 1;
-    } else {
-        merge_resolve_kernel<<<1, 1024, 0, s>>>(ctl, N, c->valid, seed, row_off, row_count, csr_j, csr_sim, state, target);
-        SISO_LAUNCHED(c);
-    }
+    SISO_TRY(launch_merge_resolve(c, ctl, N, c->valid, seed, row_off, row_count, csr_j, csr_sim, state, target, undecided, s));
     const unsigned nblk = static_cast<unsigned>((N + 255) / 256);
     merge_keys_kernel<<<nblk, 256, 0, s>>>(ctl, N, state, target, keys, vals);
     SISO_LAUNCHED(c);

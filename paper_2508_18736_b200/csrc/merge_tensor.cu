@@ -297,7 +297,7 @@ merge_verify_kernel(const MergeCtlView *ctl, const float *__restrict__ C, int D,
         if (lane == 0) {
             if (s > static_cast<double>(theta)) {
                 cand[e].sim = static_cast<float>(s);
-                atomicAdd(&row_count[cd.i], 1u);
+                if (row_count) atomicAdd(&row_count[cd.i], 1u);
             } else {
                 cand[e].i = -1;
             }
@@ -323,16 +323,20 @@ static siso_status_t encode_rows_map(EncodeTiledFn fn, CUtensorMap *map, const v
 
 }  // namespace tcm
 
-size_t merge_tensor_scratch_bytes(const Cache *c) {
-    const size_t tiles = static_cast<size_t>((c->capacity + 2 * tcm::TM - 1) / (2 * tcm::TM));
-    return 2 * pad256(static_cast<size_t>(c->rows_alloc) * c->dim * sizeof(__nv_bfloat16)) + pad256(sizeof(uint32_t) * tiles * tiles);
+size_t pair_sweep_tensor_scratch_bytes(int64_t n, int64_t rows, int dim) {
+    const size_t tiles = static_cast<size_t>((n + 2 * tcm::TM - 1) / (2 * tcm::TM));
+    return 2 * pad256(static_cast<size_t>(rows) * dim * sizeof(__nv_bfloat16)) + pad256(sizeof(uint32_t) * tiles * tiles);
 }
+size_t merge_tensor_scratch_bytes(const Cache *c) { return pair_sweep_tensor_scratch_bytes(c->capacity, c->rows_alloc, c->dim); }
 
-// Sweep + exact check.  `ctl` and `row_count` are zeroed (or carry the two-set insertion's failure flag); on return
-// (in stream order) cand[0 .. min(n_cand, max_cand)) holds the provisional pairs, the confirmed ones with their
-// exact similarity and i >= 0, and row_count[i] counts the confirmed pairs of row i.
-siso_status_t launch_merge_sweep_tensor(Cache *c, Scratch *scr, const uint8_t *seed, float theta_c, void *ctl, void *cand,
-                                        size_t max_cand, uint32_t *row_count, cudaStream_t s) {
+// Sweep + exact check over the rows of X ([rows, dim] fp32, the first N of them taking part, `valid` [N] saying which
+// are live, `seed` [N] or NULL marking the members of C_cur).  `ctl` and `row_count` are zeroed (or carry the two-set
+// insertion's failure flag); on return (in stream order) cand[0 .. min(n_cand, max_cand)) holds the provisional
+// pairs, the confirmed ones with their exact similarity and i >= 0, and row_count[i] (if not NULL) counts the
+// confirmed pairs of row i.
+siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, int64_t N, int64_t rows, const uint8_t *valid,
+                                       const uint8_t *seed, float theta_c, void *ctl, void *cand, size_t max_cand,
+                                       uint32_t *row_count, cudaStream_t s) {
     static tcm::EncodeTiledFn encode = nullptr;
     if (!encode) {
         void *fn = nullptr;
@@ -341,12 +345,11 @@ siso_status_t launch_merge_sweep_tensor(Cache *c, Scratch *scr, const uint8_t *s
         if (!fn || qres != cudaDriverEntryPointSuccess) return check_cuda(cudaErrorNotSupported, "cuTensorMapEncodeTiled lookup");
         encode = reinterpret_cast<tcm::EncodeTiledFn>(fn);
     }
-    const int64_t N = c->capacity, rows = c->rows_alloc;
     const size_t elems = static_cast<size_t>(rows) * c->dim;
     __nv_bfloat16 *hi = scr->take<__nv_bfloat16>(elems);
     __nv_bfloat16 *lo = scr->take<__nv_bfloat16>(elems);
     const long long n4 = static_cast<long long>(elems / 4);
-    tcm::split_bf16_kernel<<<static_cast<unsigned>((n4 + 255) / 256), 256, 0, s>>>(c->master, hi, lo, n4);
+    tcm::split_bf16_kernel<<<static_cast<unsigned>((n4 + 255) / 256), 256, 0, s>>>(X, hi, lo, n4);
     SISO_LAUNCHED(c);
     CUtensorMap map_hi, map_lo;
     SISO_TRY(tcm::encode_rows_map(encode, &map_hi, hi, static_cast<uint64_t>(rows), static_cast<uint64_t>(c->dim)));
@@ -371,13 +374,19 @@ siso_status_t launch_merge_sweep_tensor(Cache *c, Scratch *scr, const uint8_t *s
         c->merge_tensor_attr_set = true;
     }
     tcm::merge_sweep_tensor_kernel<<<static_cast<unsigned>(2 * used), tcm::THREADS, tcm::SMEM_BYTES, s>>>(
-        map_hi, map_lo, c->valid, seed, N, c->dim, pair_list, n_pairs, theta_c - tcm::FILTER_MARGIN,
+        map_hi, map_lo, valid, seed, N, c->dim, pair_list, n_pairs, theta_c - tcm::FILTER_MARGIN,
         static_cast<MergeCtlView *>(ctl), static_cast<MergeCandidate *>(cand), max_cand, c->status);
     SISO_LAUNCHED(c);
-    tcm::merge_verify_kernel<<<8 * c->sm_count, 256, 0, s>>>(static_cast<const MergeCtlView *>(ctl), c->master, c->dim, theta_c,
+    tcm::merge_verify_kernel<<<8 * c->sm_count, 256, 0, s>>>(static_cast<const MergeCtlView *>(ctl), X, c->dim, theta_c,
                                                              static_cast<MergeCandidate *>(cand), max_cand, row_count);
     SISO_LAUNCHED(c);
     return SISO_OK;
+}
+
+siso_status_t launch_merge_sweep_tensor(Cache *c, Scratch *scr, const uint8_t *seed, float theta_c, void *ctl, void *cand,
+                                        size_t max_cand, uint32_t *row_count, cudaStream_t s) {
+    return launch_pair_sweep_tensor(c, scr, c->master, c->capacity, c->rows_alloc, c->valid, seed, theta_c, ctl, cand, max_cand,
+                                    row_count, s);
 }
 
 }  // namespace siso
