@@ -185,6 +185,32 @@ class OracleCache:
         self.valid[...] = valid
         self.clock = int(clock)
 
+    def copy_from(self, other: "OracleCache") -> None:
+        """C_new <- C_cur, the first line of MergeCentroids (Algorithm 1): every slot of `other` into the same slot
+        here (this cache may be larger; its remaining slots become empty)."""
+        assert self.capacity >= other.capacity and self.dim == other.dim and self.dtype == other.dtype
+        n = other.capacity
+        self.valid[:] = 0
+        self.master[:n], self.size[:n], self.access[:n] = other.master, other.size, other.access
+        self.last[:n], self.valid[:n], self.clock = other.last, other.valid, other.clock
+
+    def update_centroids(self, new: "OracleCache", first_slot: int, n_slots: int) -> None:
+        """UpdateCentroids of Algorithm 1 (Sec. 4.2, update step), one group: the live entries of C_new, taken in
+        ascending slot order, are numbered 0, 1, ...; slot d of this cache (first_slot <= d < first_slot + n_slots)
+        receives entry number d, or becomes empty if C_new has no such entry.  Calling it for consecutive groups
+        until the capacity is covered replaces C_cur by C_new."""
+        assert self.dim == new.dim and self.dtype == new.dtype
+        live = np.flatnonzero(new.valid)
+        if len(live) > self.capacity:
+            raise ValueError("C_new holds more entries than C_cur has slots")
+        for d in range(first_slot, min(first_slot + n_slots, self.capacity)):
+            if d < len(live):
+                src = live[d]
+                self.master[d], self.size[d], self.access[d] = new.master[src], new.size[src], new.access[src]
+                self.last[d], self.valid[d] = new.last[src], 1
+            else:
+                self.valid[d] = 0
+
     def lookup_copy(self) -> np.ndarray:
         """What a lookup reads: the master rounded once to the storage type."""
         if self.dtype == "bf16":

@@ -347,3 +347,44 @@ def test_two_set_merge_with_interleaved_slots_equals_transcription():
     c = make_cache(np.array([[1.0, 0], [0, 1.0], [1.0, 0], [1.0, 0]]))
     mm, n = c.merge(0.5, weighted_mean=False, seed_mask=np.array([0, 0, 0, 1]))
     assert mm.tolist() == [3, 1, 3, 3] and n == 2
+
+
+# ---------------------------------------------------------------------------- Algorithm 1 as a whole
+def test_algorithm1_pipeline_and_progressive_update():
+    """MergeCentroids -> FilteringCentroids -> UpdateCentroids (Algorithm 1), the update taken a group of slots at a
+    time (Sec. 4.2, update step): after the last group C_cur holds exactly the entries of C_new, in C_new's slot order;
+    in between, every slot is wholly old or wholly new."""
+    w = W.config(3, seed=21, mode="P", n_centroids=90, dim=16, n_clusters=12, sigma=0.06)
+    M = 50
+    cur = make_cache(w.centroids[:40].astype(np.float64), sizes=np.arange(1, 41, dtype=np.float64), capacity=M)
+    cur.evict(5)                                    # holes in C_cur
+    old = {k: getattr(cur, k).copy() for k in ("master", "size", "access", "last", "valid")}
+    new = oracle.OracleCache(M + 50, 16, "f32")
+    new.copy_from(cur)
+    assert (new.valid[:M] == cur.valid).all() and (new.valid[M:] == 0).all() and (new.master[:M] == cur.master).all()
+    seed = new.valid.copy()
+    new.insert(w.centroids[40:].astype(np.float64), sizes=np.full(50, 2.0))
+    new.merge(0.9, False, seed_mask=seed, new_access_inf=True)
+    over = new.occupancy - M
+    assert over > 0
+    new.evict(over, decay=True)
+    assert new.occupancy == M
+    live = np.flatnonzero(new.valid)
+    for g in range(0, M, 16):
+        cur.update_centroids(new, g, 16)
+        done = min(M, g + 16)
+        assert (cur.valid[:done] == 1).all()
+        assert (cur.master[:done] == new.master[live[:done]]).all() and (cur.size[:done] == new.size[live[:done]]).all()
+        for k in old:                               # the slots not yet reached are untouched
+            assert (getattr(cur, k)[done:] == old[k][done:]).all()
+    assert (cur.access == 0).all()                  # FilteringCentroids reset them
+    np.testing.assert_allclose(cur.size, new.size[live])
+    # a C_new with fewer entries than slots empties the tail
+    new.evict(10)
+    cur.update_centroids(new, 0, M)
+    assert cur.occupancy == M - 10 and (cur.valid[M - 10:] == 0).all()
+    # more entries than slots is refused
+    big = oracle.OracleCache(M + 50, 16, "f32")
+    big.insert(w.centroids[:60].astype(np.float64))
+    with pytest.raises(ValueError):
+        cur.update_centroids(big, 0, 16)
