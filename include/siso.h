@@ -202,6 +202,28 @@ siso_status_t siso_lookup_small_noalloc(const void *d_centroids, const uint8_t *
                                         const float *d_theta, float theta_scalar, int32_t k, int32_t *d_idx,
                                         float *d_sim, uint8_t *d_hit, void *stream);
 
+/* Algorithm 1 as a whole (Sec. 4.2): C_new <- MergeCentroids(C_cur, C_repo, theta_C); C_new <- FilteringCentroids(C_new, M);
+ * UpdateCentroids(C_cur, C_new).  With a second handle as C_new the steps are
+ *     siso_cache_copy(c_new, cur)                       "C_new <- C_cur", the first line of MergeCentroids
+ *     siso_merge(c_new, d_repo, d_repo_sizes, ...)      the rest of MergeCentroids (c_new needs n_repo free slots)
+ *     siso_evict(c_new, occupancy - M, SISO_EVICT_DECAY)   FilteringCentroids
+ *     siso_update_centroids(cur, c_new, g, group) for g = 0, group, 2 group, ... < capacity of cur
+ * and the cache `cur` serves lookups all the while.
+ *
+ * siso_cache_copy: every slot of src (vector, cluster_size, access_count, last_access, live flag) into the same slot of
+ * dst, the counters and the clock too; dst must have the same dim, dtype and device and at least src's capacity (its
+ * further slots become empty), else SISO_ERR_INVALID_ARG / SISO_ERR_CAPACITY.
+ *
+ * siso_update_centroids is the update step: "progressively replaces small groups of centroids one at a time" so that
+ * the cache stays available (the paper gives no group size; 256 slots is a reasonable one).  The live entries of c_new,
+ * in ascending slot order, are numbered 0, 1, ...; slot d of cur, first_slot <= d < first_slot + n_slots, receives entry
+ * number d, or becomes empty if c_new has no such entry.  The numbering is taken when first_slot == 0 is copied, so
+ * c_new must not change until the last group is done; groups may be issued in any order after that first one.  A lookup
+ * ordered between two groups sees every slot either as it was or as it will be.  If c_new holds more live entries than
+ * cur has slots nothing is copied and the device status becomes SISO_ERR_CAPACITY.  Asynchronous on `stream`. */
+siso_status_t siso_cache_copy(siso_cache_t *dst, siso_cache_t *src, void *stream);
+siso_status_t siso_update_centroids(siso_cache_t *cur, siso_cache_t *c_new, int64_t first_slot, int64_t n_slots, void *stream);
+
 /* Clustering of logged query vectors into centroids (Sec. 4.1, SISO-Cluster: community detection at the clustering
  * threshold theta_C, which yields for every cluster a centroid and cluster_size, "the number of vectors in the
  * cluster").  The paper names the method without stating its steps; the reading built here: two vectors are neighbours

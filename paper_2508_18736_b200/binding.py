@@ -21,7 +21,7 @@ _STATUS_NAMES = {0: "SISO_OK", 1: "SISO_ERR_INVALID_ARG", 2: "SISO_ERR_UNSUPPORT
 EXPORTS = ["siso_cache_create", "siso_cache_destroy", "siso_set_option", "siso_insert", "siso_lookup",
            "siso_lookup_host", "siso_update", "siso_merge", "siso_evict", "siso_make_room", "siso_insert_misses",
            "siso_stream_step", "siso_export", "siso_import", "siso_get_stats", "siso_sync_status",
-           "siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_lookup_small_noalloc", "siso_cluster", "siso_t2h", "siso_md1_wait",
+           "siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_lookup_small_noalloc", "siso_cluster", "siso_cache_copy", "siso_update_centroids", "siso_t2h", "siso_md1_wait",
            "siso_choose_theta", "siso_correct_theta"]
 
 
@@ -74,6 +74,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_stream_step.argtypes = [vp, vp, i64, vp, f32, vp, vp, vp, vp, vp, vp]
     L.siso_lookup_small_noalloc.argtypes = [vp, vp, i64, i32, i32, vp, i64, vp, f32, i32, vp, vp, vp, vp]
     L.siso_t2h.argtypes = [vp, vp, i64, vp, i32, vp, vp]
+    L.siso_cache_copy.argtypes = [vp, vp, vp]
+    L.siso_update_centroids.argtypes = [vp, vp, i64, i64, vp]
     L.siso_cluster.argtypes = [vp, vp, i64, f32, vp, vp, vp, vp, ctypes.POINTER(i64), vp]
     L.siso_md1_wait.argtypes = [ctypes.c_double] * 3
     L.siso_md1_wait.restype = ctypes.c_double
@@ -265,6 +267,15 @@ class SisoCache:
         self._check(self._lib.siso_stream_step(self._h, _ptr(q), n, _ptr(th_t), th_s, _ptr(idx), _ptr(sim), _ptr(hit),
                                                _ptr(victims), _ptr(slots), _stream(stream)), "siso_stream_step")
         return out
+
+    def copy_from(self, src: "SisoCache", stream=None) -> None:
+        """C_new <- C_cur (first line of MergeCentroids, Algorithm 1): every slot of `src` into the same slot here."""
+        self._check(self._lib.siso_cache_copy(self._h, src._h, _stream(stream)), "siso_cache_copy")
+
+    def update_centroids(self, c_new: "SisoCache", first_slot: int, n_slots: int, stream=None) -> None:
+        """UpdateCentroids of Algorithm 1, one group of destination slots (see include/siso.h)."""
+        self._check(self._lib.siso_update_centroids(self._h, c_new._h, int(first_slot), int(n_slots), _stream(stream)),
+                    "siso_update_centroids")
 
     def cluster(self, vecs: torch.Tensor, theta_c: float, want_centroids: bool = True, stream=None):
         """Community detection at theta_c over the rows of `vecs` (the cache's contents are not touched).

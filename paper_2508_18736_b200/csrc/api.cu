@@ -26,6 +26,16 @@ static void *cache_alloc(Cache *c, size_t bytes, cudaStream_t s) {
     return c->alloc.alloc(bytes ? bytes : 256, s, c->alloc.ctx);
 }
 
+void *cache_alloc_zeroed(Cache *c, size_t bytes) {
+    void *p = cache_alloc(c, bytes, nullptr);
+    if (p && cudaMemset(p, 0, bytes) != cudaSuccess) {
+        cudaGetLastError();
+        c->alloc.free(p, c->alloc.ctx);
+        return nullptr;
+    }
+    return p;
+}
+
 siso_status_t scratch_reserve(Cache *c, size_t bytes, cudaStream_t s, Scratch *out) {
     bytes += 4096;
     if (bytes > c->ws_bytes) {
@@ -168,7 +178,7 @@ siso_status_t siso_cache_destroy(siso_cache_t *c) {
     cudaDeviceSynchronize();
     tensor_state_destroy(c);
     void *ptrs[] = {c->dtype == SISO_F32 ? nullptr : c->vecs, c->master, c->size, c->access, c->last, c->valid,
-                    c->counters, c->status, c->ws, c->stage};
+                    c->counters, c->status, c->ws, c->stage, c->swap_plan};
     for (void *p : ptrs)
         if (p) c->alloc.free(p, c->alloc.ctx);
     delete c;
@@ -299,6 +309,22 @@ siso_status_t siso_merge(siso_cache_t *c, const void *d_repo, const double *d_re
         return siso_sync_status(c, stream);
     }
     return SISO_OK;
+}
+
+siso_status_t siso_cache_copy(siso_cache_t *dst, siso_cache_t *src, void *stream) {
+    if (!dst || !src || dst == src) return SISO_ERR_INVALID_ARG;
+    if (dst->dim != src->dim || dst->dtype != src->dtype || dst->device != src->device) return SISO_ERR_INVALID_ARG;
+    if (dst->capacity < src->capacity) return SISO_ERR_CAPACITY;
+    SISO_CUDA(cudaSetDevice(dst->device));
+    return launch_cache_copy(dst, src, static_cast<cudaStream_t>(stream));
+}
+
+siso_status_t siso_update_centroids(siso_cache_t *cur, siso_cache_t *c_new, int64_t first_slot, int64_t n_slots, void *stream) {
+    if (!cur || !c_new || cur == c_new || first_slot < 0 || n_slots < 0) return SISO_ERR_INVALID_ARG;
+    if (cur->dim != c_new->dim || cur->dtype != c_new->dtype || cur->device != c_new->device) return SISO_ERR_INVALID_ARG;
+    if (first_slot > cur->capacity) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(cur->device));
+    return launch_update_centroids(cur, c_new, first_slot, n_slots, static_cast<cudaStream_t>(stream));
 }
 
 siso_status_t siso_cluster(siso_cache_t *c, const void *d_vecs, int64_t n, float theta_c, int32_t *d_label, int32_t *d_centres,

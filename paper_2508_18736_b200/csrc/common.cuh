@@ -59,6 +59,7 @@ struct Cache {
     bool merge_tensor_attr_set;
     int merge_resolve_grid;     // CTAs of the grid-wide merge resolution (0: not yet asked, -1: unavailable)
     int32_t merge_path;         // SISO_PATH_AUTO, SISO_PATH_SIMT or SISO_PATH_TENSOR for the pairwise sweep of siso_merge
+    void *swap_plan;            // UpdateCentroids: slot of the d-th live entry, when this cache serves as C_new
     int maint_grid;             // CTAs of the fused streaming maintenance kernel (0: not yet asked, -1: unavailable)
 };
 
@@ -75,6 +76,8 @@ struct Scratch {
 };
 inline size_t pad256(size_t b) { return (b + 255) & ~size_t(255); }
 siso_status_t scratch_reserve(Cache *c, size_t bytes, cudaStream_t s, Scratch *out);
+// memory that lives as long as the cache, set to zero; NULL if the allocator fails
+void *cache_alloc_zeroed(Cache *c, size_t bytes);
 siso_status_t check_cuda(cudaError_t e, const char *what);
 #define SISO_CUDA(expr)                                                  \
     do {                                                                 \
@@ -127,6 +130,8 @@ siso_status_t launch_merge_resolve(Cache *c, void *ctl, int64_t N, const uint8_t
                                    const uint32_t *row_off, const uint32_t *row_count, const int32_t *csr_j,
                                    const float *csr_sim, uint8_t *state, int32_t *target, unsigned int *undecided,
                                    cudaStream_t s);
+siso_status_t launch_cache_copy(Cache *dst, const Cache *src, cudaStream_t s);
+siso_status_t launch_update_centroids(Cache *cur, Cache *c_new, int64_t first, int64_t n, cudaStream_t s);
 siso_status_t launch_cluster(Cache *c, const void *vecs, int64_t n, float theta_c, int32_t *label, int32_t *centres,
                              double *sizes, void *centroids, long long *d_n_clusters, cudaStream_t s);
 siso_status_t launch_merge_sweep_tensor(Cache *c, Scratch *scr, const uint8_t *seed, float theta_c, void *ctl, void *cand,

@@ -41,6 +41,12 @@ def assert_state_equal(cache, ora, dtype, what=""):
     assert cache.stats()["occupancy"] == int(live.sum()) and cache.stats()["clock"] == ora.clock, what
 
 
+def dataclass_slice(w, lo, hi):
+    """The workload with only rows lo..hi of its centroids."""
+    import dataclasses
+    return dataclasses.replace(w, centroids=w.centroids[lo:hi], centroid_labels=w.centroid_labels[lo:hi])
+
+
 def make_pair(w, capacity=None, sizes=None):
     cap = capacity or w.centroids.shape[0]
     cache = siso.SisoCache(cap, w.dim, w.dtype)
@@ -360,3 +366,54 @@ def test_streaming_eviction_is_exact_when_the_sample_misleads():
     assert_state_equal(cache, ora, "bf16")
     cache.check_status()
     cache.close()
+
+
+@pytest.mark.parametrize("dtype", ["f32", "bf16"])
+def test_algorithm1_with_progressive_update_matches_oracle(dtype):
+    """Algorithm 1 end to end on a second handle as C_new (copy, MergeCentroids with a repository, FilteringCentroids with
+    the decay), then UpdateCentroids a group of slots at a time with lookups in between (Sec. 4.2, update step)."""
+    w = W.config(3, seed=31, mode="P", n_centroids=1600, n_queries=300, dim=72, n_clusters=90, sigma=0.06, dtype=dtype)
+    M, n_repo, group = 1000, 700, 256
+    cur, o_cur = make_pair(dataclass_slice(w, 0, 900), capacity=M,
+                           sizes=np.random.default_rng(3).integers(1, 9, 900).astype(np.float64))
+    assert (cur.evict(60).cpu().numpy() == o_cur.evict(60)).all()                      # holes in C_cur
+    new = siso.SisoCache(M + n_repo, w.dim, dtype)
+    o_new = oracle.OracleCache(M + n_repo, w.dim, dtype)
+    new.copy_from(cur)
+    o_new.copy_from(o_cur)
+    assert_state_equal(new, o_new, dtype, "C_new <- C_cur")
+    repo, repo_sizes = w.centroids[900:], np.random.default_rng(4).integers(1, 5, n_repo).astype(np.float64)
+    seed = o_new.valid.copy()
+    mm, n_merged = new.merge(0.9, siso.MERGE_SIZES_ONLY, repo=to_dev(repo, dtype), repo_sizes=torch.from_numpy(repo_sizes))
+    o_new.insert(repo, sizes=repo_sizes)
+    o_mm, o_n = o_new.merge(0.9, False, seed_mask=seed, new_access_inf=True)
+    if not (mm.cpu().numpy() == o_mm).all():
+        pytest.skip("near-threshold merge decision")
+    over = o_new.occupancy - M
+    assert over > 0 and (new.evict(over, siso.EVICT_DECAY).cpu().numpy() == o_new.evict(over, decay=True)).all()
+    assert_state_equal(new, o_new, dtype, "C_new after filtering")
+    # the live cache keeps serving while it is replaced group by group
+    q, theta = w.queries, np.full(300, 0.86, np.float32)
+    for g in range(0, M, group):
+        cur.update_centroids(new, g, group)
+        o_cur.update_centroids(o_new, g, group)
+        got = [x.cpu().numpy() for x in cur.lookup(to_dev(q, dtype), 0.86, 2)]
+        want = o_cur.lookup(q, theta, 2)
+        check_lookup(got, want, o_cur.lookup_copy(), q, theta, TOL[dtype], valid=o_cur.valid)
+        g_state = state_np(cur)
+        assert (g_state["valid"] == o_cur.valid).all(), f"group at {g}"
+    assert cur.stats()["occupancy"] == M == o_cur.occupancy
+    live = np.flatnonzero(o_new.valid)
+    g_state = state_np(cur)
+    assert (g_state["size"] == o_new.size[live]).all() and (g_state["access"] == 0).all()
+    assert np.abs(g_state["master"].astype(np.float64) - o_new.master[live]).max() <= 1e-6
+    # a C_new with more entries than C_cur has slots is refused and nothing changes
+    before = state_np(cur)
+    big = siso.SisoCache(M + n_repo, w.dim, dtype)
+    big.insert(to_dev(w.centroids[:1200], dtype))
+    cur.update_centroids(big, 0, group)
+    assert cur.sync_status() == 4
+    after = state_np(cur)
+    assert all((before[k] == after[k]).all() for k in before)
+    for c in (cur, new, big):
+        c.close()
