@@ -202,6 +202,23 @@ siso_status_t siso_lookup_small_noalloc(const void *d_centroids, const uint8_t *
                                         const float *d_theta, float theta_scalar, int32_t k, int32_t *d_idx,
                                         float *d_sim, uint8_t *d_hit, void *stream);
 
+/* Lookup over a cache whose rows are partitioned across several GPUs (one handle per GPU, each holding a contiguous
+ * range of the global slots).  FindClosestCentroid over the whole cache = the best of the shards' best, so every GPU
+ * scores the full query batch against its own rows and the shards' top-k lists are combined after one exchange.
+ * siso_lookup_keys is a1-a2 on one shard: d_keys [n_queries, k] receives packed 64-bit keys,
+ * (order-preserving similarity bits << 32) | (2^32 - 1 - (slot + slot_offset)), 0 where the shard has fewer than k
+ * entries; a larger key is a better match, ties go to the lower global slot.  The shard's hit statistics are not
+ * touched.  slot_offset + capacity must stay below 2^32.
+ * siso_combine_keys (needs no handle; runs on the current device): d_keys [n_queries, n_lists, k], e.g. the all-gathered
+ * lists of n_lists shards brought into that layout; per query the k largest keys give d_idx [n_queries, k] (int64 global
+ * slot, -1 where none), d_sim [n_queries, k] and the strict threshold test d_hit [n_queries] on the best one (d_theta
+ * per query, or theta_scalar if NULL).  The result is the same for any number and order of shards.
+ * Both are asynchronous on `stream`. */
+siso_status_t siso_lookup_keys(siso_cache_t *c, const void *d_queries, int64_t n_queries, int32_t k, int64_t slot_offset,
+                               uint64_t *d_keys, void *stream);
+siso_status_t siso_combine_keys(const uint64_t *d_keys, int64_t n_queries, int32_t n_lists, int32_t k, const float *d_theta,
+                                float theta_scalar, int64_t *d_idx, float *d_sim, uint8_t *d_hit, void *stream);
+
 /* Algorithm 1 as a whole (Sec. 4.2): C_new <- MergeCentroids(C_cur, C_repo, theta_C); C_new <- FilteringCentroids(C_new, M);
  * UpdateCentroids(C_cur, C_new).  With a second handle as C_new the steps are
  *     siso_cache_copy(c_new, cur)                       "C_new <- C_cur", the first line of MergeCentroids

@@ -21,7 +21,7 @@ _STATUS_NAMES = {0: "SISO_OK", 1: "SISO_ERR_INVALID_ARG", 2: "SISO_ERR_UNSUPPORT
 EXPORTS = ["siso_cache_create", "siso_cache_destroy", "siso_set_option", "siso_insert", "siso_lookup",
            "siso_lookup_host", "siso_update", "siso_merge", "siso_evict", "siso_make_room", "siso_insert_misses",
            "siso_stream_step", "siso_export", "siso_import", "siso_get_stats", "siso_sync_status",
-           "siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_lookup_small_noalloc", "siso_cluster", "siso_cache_copy", "siso_update_centroids", "siso_t2h", "siso_md1_wait",
+           "siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_lookup_small_noalloc", "siso_cluster", "siso_cache_copy", "siso_update_centroids", "siso_lookup_keys", "siso_combine_keys", "siso_t2h", "siso_md1_wait",
            "siso_choose_theta", "siso_correct_theta"]
 
 
@@ -74,6 +74,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_stream_step.argtypes = [vp, vp, i64, vp, f32, vp, vp, vp, vp, vp, vp]
     L.siso_lookup_small_noalloc.argtypes = [vp, vp, i64, i32, i32, vp, i64, vp, f32, i32, vp, vp, vp, vp]
     L.siso_t2h.argtypes = [vp, vp, i64, vp, i32, vp, vp]
+    L.siso_lookup_keys.argtypes = [vp, vp, i64, i32, i64, vp, vp]
+    L.siso_combine_keys.argtypes = [vp, i64, i32, i32, vp, f32, vp, vp, vp, vp]
     L.siso_cache_copy.argtypes = [vp, vp, vp]
     L.siso_update_centroids.argtypes = [vp, vp, i64, i64, vp]
     L.siso_cluster.argtypes = [vp, vp, i64, f32, vp, vp, vp, vp, ctypes.POINTER(i64), vp]
@@ -268,6 +270,14 @@ class SisoCache:
                                                _ptr(victims), _ptr(slots), _stream(stream)), "siso_stream_step")
         return out
 
+    def lookup_keys(self, queries: torch.Tensor, k: int = 1, slot_offset: int = 0, stream=None) -> torch.Tensor:
+        """This shard's top-k as packed keys [n, k] (int64 tensor holding the 64-bit patterns); see siso_lookup_keys."""
+        q = self._vec(queries, "queries")
+        keys = self._new((q.shape[0], k), torch.int64)
+        self._check(self._lib.siso_lookup_keys(self._h, _ptr(q), q.shape[0], k, int(slot_offset), _ptr(keys), _stream(stream)),
+                    "siso_lookup_keys")
+        return keys
+
     def copy_from(self, src: "SisoCache", stream=None) -> None:
         """C_new <- C_cur (first line of MergeCentroids, Algorithm 1): every slot of `src` into the same slot here."""
         self._check(self._lib.siso_cache_copy(self._h, src._h, _stream(stream)), "siso_cache_copy")
@@ -357,6 +367,24 @@ def lookup_small_noalloc(centroids: torch.Tensor, queries: torch.Tensor, theta, 
                                          _ptr(hit), _stream(stream))
     if st != 0:
         raise SisoError(st, "siso_lookup_small_noalloc", L.siso_last_cuda_error().decode() if st == 7 else "")
+
+
+def combine_keys(keys: torch.Tensor, theta, stream=None) -> Tuple[torch.Tensor, torch.Tensor, torch.Tensor]:
+    """keys [n, n_lists, k] (int64 tensor of packed keys on a GPU) -> (idx [n, k] int64 global slots, sim [n, k], hit [n])."""
+    assert keys.dtype == torch.int64 and keys.dim() == 3 and keys.is_cuda
+    keys = keys.contiguous()
+    n, n_lists, k = keys.shape
+    th_t, th_s = (theta.to(device=keys.device, dtype=torch.float32).contiguous(), 0.0) \
+        if isinstance(theta, torch.Tensor) else (None, float(theta))
+    idx = torch.empty((n, k), dtype=torch.int64, device=keys.device)
+    sim = torch.empty((n, k), dtype=torch.float32, device=keys.device)
+    hit = torch.empty((n,), dtype=torch.uint8, device=keys.device)
+    with torch.cuda.device(keys.device):
+        st = load_library().siso_combine_keys(_ptr(keys), n, n_lists, k, _ptr(th_t), th_s, _ptr(idx), _ptr(sim), _ptr(hit),
+                                              _stream(stream))
+    if st != 0:
+        raise SisoError(st, "siso_combine_keys")
+    return idx, sim, hit
 
 
 def md1_wait(llm_latency: float, arrival_rate: float, hit_ratio: float) -> float:

@@ -1,4 +1,5 @@
 // C ABI of libsiso: argument checking, state, scratch memory and kernel launches.
+#include <cmath>
 #include <cstdio>
 #include <cstring>
 #include <new>
@@ -309,6 +310,44 @@ siso_status_t siso_merge(siso_cache_t *c, const void *d_repo, const double *d_re
         return siso_sync_status(c, stream);
     }
     return SISO_OK;
+}
+
+siso_status_t siso_lookup_keys(siso_cache_t *c, const void *d_queries, int64_t n_queries, int32_t k, int64_t slot_offset,
+                               uint64_t *d_keys, void *stream) {
+    if (!c || n_queries < 0 || k < 1 || k > kMaxK || slot_offset < 0) return SISO_ERR_INVALID_ARG;
+    if (slot_offset + c->capacity > 0xFFFFFFFFll) return SISO_ERR_UNSUPPORTED;        // global slots are 32-bit in a key
+    if (n_queries == 0) return SISO_OK;
+    if (!d_queries || !d_keys) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // idx / sim / hit of the shard go to the cache's staging buffer (the lookup itself uses the scratch buffer)
+    const size_t ib = pad256(sizeof(int32_t) * n_queries * k), sb = pad256(sizeof(float) * n_queries * k);
+    const size_t hb = pad256(static_cast<size_t>(n_queries));
+    const size_t need = ib + sb + hb;
+    if (need > c->stage_bytes) {
+        if (c->stage) c->alloc.free(c->stage, c->alloc.ctx);
+        c->stage = nullptr;
+        c->stage_bytes = 0;
+        c->stage = cache_alloc(c, need, s);
+        if (!c->stage) return SISO_ERR_OOM;
+        c->stage_bytes = need;
+    }
+    char *p = static_cast<char *>(c->stage);
+    int32_t *di = reinterpret_cast<int32_t *>(p);
+    float *ds = reinterpret_cast<float *>(p + ib);
+    uint8_t *dh = reinterpret_cast<uint8_t *>(p + ib + sb);
+    // threshold +inf: the shard records no hit; hit or miss is decided on the combined result
+    SISO_TRY(siso_lookup(c, d_queries, n_queries, nullptr, INFINITY, k, di, ds, dh, stream));
+    return launch_shard_pack(c, di, ds, n_queries * k, slot_offset, reinterpret_cast<unsigned long long *>(d_keys), s);
+}
+
+siso_status_t siso_combine_keys(const uint64_t *d_keys, int64_t n_queries, int32_t n_lists, int32_t k, const float *d_theta,
+                                float theta_scalar, int64_t *d_idx, float *d_sim, uint8_t *d_hit, void *stream) {
+    if (n_queries < 0 || n_lists < 1 || k < 1 || k > kMaxK) return SISO_ERR_INVALID_ARG;
+    if (n_queries == 0) return SISO_OK;
+    if (!d_keys || !d_idx || !d_sim || !d_hit) return SISO_ERR_INVALID_ARG;
+    return launch_shard_combine(reinterpret_cast<const unsigned long long *>(d_keys), n_queries, n_lists, k, d_theta,
+                                theta_scalar, reinterpret_cast<long long *>(d_idx), d_sim, d_hit, static_cast<cudaStream_t>(stream));
 }
 
 siso_status_t siso_cache_copy(siso_cache_t *dst, siso_cache_t *src, void *stream) {

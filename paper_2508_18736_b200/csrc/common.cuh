@@ -130,6 +130,10 @@ siso_status_t launch_merge_resolve(Cache *c, void *ctl, int64_t N, const uint8_t
                                    const uint32_t *row_off, const uint32_t *row_count, const int32_t *csr_j,
                                    const float *csr_sim, uint8_t *state, int32_t *target, unsigned int *undecided,
                                    cudaStream_t s);
+siso_status_t launch_shard_pack(Cache *c, const int32_t *idx, const float *sim, int64_t n, int64_t slot_offset,
+                                unsigned long long *keys, cudaStream_t s);
+siso_status_t launch_shard_combine(const unsigned long long *keys, int64_t n, int n_lists, int k, const float *theta,
+                                   float theta_s, long long *idx, float *sim, uint8_t *hit, cudaStream_t s);
 siso_status_t launch_cache_copy(Cache *dst, const Cache *src, cudaStream_t s);
 siso_status_t launch_update_centroids(Cache *cur, Cache *c_new, int64_t first, int64_t n, cudaStream_t s);
 siso_status_t launch_cluster(Cache *c, const void *vecs, int64_t n, float theta_c, int32_t *label, int32_t *centres,

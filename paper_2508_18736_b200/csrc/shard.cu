@@ -1,0 +1,74 @@
+// Centroid-sharded lookup: the cache's rows are partitioned over several GPUs, every GPU scores the whole query batch
+// against its own rows (FindClosestCentroid of Algorithm 1 restricted to a shard), and the shards' results are
+// combined after ONE exchange of a few bytes per query.  What crosses between GPUs are packed 64-bit keys,
+// (order-preserving similarity bits << 32) | (2^32 - 1 - global slot), whose maximum is the best match with ties to the
+// lower global slot, so that the combined result does not depend on the number of shards or on their order.
+//   pack     a shard's (idx, sim) lists -> keys with the shard's slot offset added
+//   combine  per query the k largest of n_lists * k keys -> global slot (int64), similarity, strict threshold test
+#include "common.cuh"
+
+namespace siso {
+
+namespace {
+
+__global__ void shard_pack_kernel(const int32_t *__restrict__ idx, const float *__restrict__ sim, long long n, long long slot_offset,
+                                  unsigned long long *__restrict__ keys) {
+    const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const int32_t s = idx[i];
+    keys[i] = s < 0 ? 0ull : pack_key(sim[i], static_cast<uint32_t>(static_cast<long long>(s) + slot_offset));
+}
+
+// one warp per query; keys [n, n_lists, k]
+template <int KMAX>
+__global__ void __launch_bounds__(256)
+shard_combine_kernel(const unsigned long long *__restrict__ keys, long long n, int n_lists, int k, const float *__restrict__ theta,
+                     float theta_s, long long *__restrict__ idx, float *__restrict__ sim, uint8_t *__restrict__ hit) {
+    const int lane = threadIdx.x & 31;
+    const long long b = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (b >= n) return;
+    KeyList<KMAX> out;
+    out.clear();
+    const unsigned long long *src = keys + b * n_lists * k;
+    for (int s = lane; s < n_lists * k; s += 32) out.insert(src[s]);
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) {
+        unsigned long long other[KMAX];
+#pragma unroll
+        for (int j = 0; j < KMAX; ++j) other[j] = __shfl_xor_sync(0xFFFFFFFFu, out.k[j], o);
+#pragma unroll
+        for (int j = 0; j < KMAX; ++j) out.insert(other[j]);
+    }
+    if (lane == 0) {
+#pragma unroll
+        for (int j = 0; j < KMAX; ++j) {
+            if (j < k) {
+                const unsigned long long key = out.k[j];
+                idx[b * k + j] = key ? static_cast<long long>(0xFFFFFFFFu - static_cast<uint32_t>(key)) : -1ll;
+                sim[b * k + j] = key ? key_sim(key) : -INFINITY;
+            }
+        }
+        const float th = theta ? theta[b] : theta_s;
+        hit[b] = (out.k[0] != 0ull && key_sim(out.k[0]) > th) ? 1 : 0;
+    }
+}
+
+}  // namespace
+
+siso_status_t launch_shard_pack(Cache *c, const int32_t *idx, const float *sim, int64_t n, int64_t slot_offset,
+                                unsigned long long *keys, cudaStream_t s) {
+    shard_pack_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, s>>>(idx, sim, n, slot_offset, keys);
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
+
+siso_status_t launch_shard_combine(const unsigned long long *keys, int64_t n, int n_lists, int k, const float *theta,
+                                   float theta_s, long long *idx, float *sim, uint8_t *hit, cudaStream_t s) {
+    const unsigned blocks = static_cast<unsigned>((n + 7) / 8);
+    if (k == 1) shard_combine_kernel<1><<<blocks, 256, 0, s>>>(keys, n, n_lists, k, theta, theta_s, idx, sim, hit);
+    else if (k <= 4) shard_combine_kernel<4><<<blocks, 256, 0, s>>>(keys, n, n_lists, k, theta, theta_s, idx, sim, hit);
+    else shard_combine_kernel<8><<<blocks, 256, 0, s>>>(keys, n, n_lists, k, theta, theta_s, idx, sim, hit);
+    return check_cuda(cudaGetLastError(), "shard_combine_kernel");
+}
+
+}  // namespace siso
