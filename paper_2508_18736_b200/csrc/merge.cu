@@ -189,14 +189,26 @@ merge_resolve_grid_kernel(MergeCtl *ctl, int64_t N, const uint8_t *__restrict__ 
             const uint32_t o = row_off[i], cnt = row_count[i];
             bool ready = true;
             unsigned long long best = 0ull;
-            for (uint32_t e = 0; e < cnt; ++e) {
-                const int32_t j = csr_j[o + e];
-                const uint8_t sj = state[j];
-                if (sj == 0) { ready = false; break; }
-                if (sj == 1) {
-                    const uint32_t order = static_cast<uint32_t>(j) | ((seed && seed[j]) ? 0u : 0x80000000u);
-                    const unsigned long long key = pack_key(csr_sim[o + e], order);
-                    best = key > best ? key : best;
+            // eight candidates at a time, so that their loads are in flight together
+            for (uint32_t e0 = 0; e0 < cnt && ready; e0 += 8) {
+                int32_t j[8];
+                uint8_t sj[8];
+                float sv[8];
+#pragma unroll
+                for (int u = 0; u < 8; ++u) j[u] = e0 + u < cnt ? csr_j[o + e0 + u] : -1;
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    sj[u] = j[u] >= 0 ? state[j[u]] : 3;
+                    sv[u] = j[u] >= 0 ? csr_sim[o + e0 + u] : 0.0f;
+                }
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    if (sj[u] == 0) ready = false;
+                    if (sj[u] == 1) {
+                        const uint32_t order = static_cast<uint32_t>(j[u]) | ((seed && seed[j[u]]) ? 0u : 0x80000000u);
+                        const unsigned long long key = pack_key(sv[u], order);
+                        best = key > best ? key : best;
+                    }
                 }
             }
             if (!ready) { ++left; continue; }

@@ -56,7 +56,6 @@ struct Shared {
     uint64_t full[STAGES], empty[STAGES], acc_full[ACC_STAGES], acc_empty[ACC_STAGES];
     uint32_t tmem_base;
     int abort_flag;
-    uint8_t jflag[4][TN];                // per epilogue warp; bit 0: live, bit 1: member of C_cur
 };
 
 // tile pair number -> (row tile I, column tile t), from the list the host wrote
@@ -161,9 +160,11 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
     } else {
         // ------------------------------------------------------------------ epilogue (warps 2..5 of both CTAs)
         const int quarter = warp & 3;
-        uint8_t *jflag = sh->jflag[quarter];                 // this warp's own copy: no barrier between the warps
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
+        constexpr int RUN = 256;                 // places of the candidate list a warp reserves at a time
+        unsigned long long run_base = 0;         // the warp's current run (the same in all lanes)
+        int run_left = 0;
         int last_I = -1;
         bool row_ok = false;
         long long gi = 0;
@@ -177,16 +178,15 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
                 // a row takes part if it is live and not a member of C_cur (those are never merged into others)
                 row_ok = gi < N && valid[gi] != 0 && !(two_sets && seed[gi] != 0);
             }
-            // flags of the tile's 256 rows j
-            __syncwarp();
+            // the tile's 256 rows j as bit masks per chunk of 32 (the same in all lanes): live, member of C_cur
+            uint32_t live_mask[TN / 32], seed_mask[TN / 32];
 #pragma unroll
             for (int h = 0; h < TN / 32; ++h) {
                 const long long gj = n0 + h * 32 + lane;
-                uint8_t f = 0;
-                if (gj < N) f = (valid[gj] ? 1 : 0) | ((two_sets && seed[gj]) ? 2 : 0);
-                jflag[h * 32 + lane] = f;
+                const bool lv = gj < N && valid[gj] != 0;
+                live_mask[h] = __ballot_sync(0xFFFFFFFFu, lv);
+                seed_mask[h] = two_sets ? __ballot_sync(0xFFFFFFFFu, lv && seed[gj] != 0) : 0u;
             }
-            __syncwarp();
             if (!mbar_wait(&sh->acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
             tcgen05_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * TN;
@@ -195,19 +195,44 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
                 float m = __uint_as_float(r[0]);
 #pragma unroll
                 for (int j = 1; j < 32; ++j) m = fmaxf(m, __uint_as_float(r[j]));
-                if (!(row_ok && m > theta_filter)) return;
-                // this row has values above the filter in this chunk: which of them are pairs of the sweep
+                const bool look = row_ok && m > theta_filter;
+                if (!__any_sync(0xFFFFFFFFu, look)) return;            // the common case: nothing above the filter
+                // which values of this row are pairs of the sweep
                 uint32_t take = 0;
+                if (look) {
+                    // columns that come before row gi in C_new: members of C_cur, or a lower slot
+                    const long long below = gi - (n0 + ch * 32);             // columns 0..below-1 of the chunk are lower slots
+                    const uint32_t lower = below <= 0 ? 0u : (below >= 32 ? 0xFFFFFFFFu : ((1u << below) - 1u));
+                    uint32_t ok_mask = live_mask[ch] & (seed_mask[ch] | lower);
+                    if (below >= 0 && below < 32) ok_mask &= ~(1u << below);   // never the row itself
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    const long long gj = n0 + ch * 32 + j;
-                    const uint8_t f = jflag[ch * 32 + j];
-                    const bool pair_ok = (f & 1) && ((f & 2) || gj < gi) && gj != gi;
-                    if (pair_ok && __uint_as_float(r[j]) > theta_filter) take |= 1u << j;
+                    for (int j = 0; j < 32; ++j)
+                        if (__uint_as_float(r[j]) > theta_filter) take |= 1u << j;
+                    take &= ok_mask;
                 }
-                if (!take) return;
-                const unsigned long long base = atomicAdd(&ctl->n_cand, static_cast<unsigned long long>(__popc(take)));
-                unsigned long long pos = base;
+                // places in the warp's reserved run of the candidate list: one global atomic per RUN places
+                // instead of one per row (a single counter that every warp hits would serialise them)
+                const int mine = __popc(take);
+                int incl = mine;
+#pragma unroll
+                for (int o = 1; o < 32; o <<= 1) {
+                    const int y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+                    if (lane >= o) incl += y;
+                }
+                const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
+                if (total == 0) return;
+                if (total > run_left) {
+                    // give the rest of the old run back as empty records and take a new one
+                    for (int t = lane; t < run_left; t += 32)
+                        if (run_base + t < max_cand) cand[run_base + t].i = -1;
+                    const int want = total > RUN ? total : RUN;
+                    unsigned long long nb = 0;
+                    if (lane == 0) nb = atomicAdd(&ctl->n_cand, static_cast<unsigned long long>(want));
+                    run_base = __shfl_sync(0xFFFFFFFFu, nb, 0);
+                    run_left = want;
+                    if (run_base + want > max_cand && lane == 0) ctl->overflow = 1;
+                }
+                unsigned long long pos = run_base + static_cast<unsigned long long>(incl - mine);
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     if ((take >> j) & 1u) {
@@ -217,12 +242,12 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
                             cd.j = static_cast<int32_t>(n0 + ch * 32 + j);
                             cd.sim = __uint_as_float(r[j]);
                             cand[pos] = cd;
-                        } else {
-                            ctl->overflow = 1;
                         }
                         ++pos;
                     }
                 }
+                run_base += static_cast<unsigned long long>(total);
+                run_left -= total;
             };
             tmem_ld_32x32(taddr, ra);
 #pragma unroll 1
@@ -239,6 +264,9 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
             if (lane == 0) mbar_arrive_cluster(cluster_addr(smem_u32(&sh->acc_empty[acc]), 0));
             if (++acc == ACC_STAGES) { acc = 0; acc_phase ^= 1u; }
         }
+        // what is left of the last run holds no pair
+        for (int t = lane; t < run_left; t += 32)
+            if (run_base + t < max_cand) cand[run_base + t].i = -1;
     }
 
     // ---------------------------------------------------------------------- teardown
@@ -284,6 +312,7 @@ merge_verify_kernel(const MergeCtlView *ctl, const float *__restrict__ C, int D,
     const unsigned long long warps = static_cast<unsigned long long>(gridDim.x) * (blockDim.x >> 5);
     for (unsigned long long e = static_cast<unsigned long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); e < n; e += warps) {
         const MergeCandidate cd = cand[e];
+        if (cd.i < 0) continue;                      // an unused place of a warp's reserved run
         const float4 *a = reinterpret_cast<const float4 *>(C + static_cast<long long>(cd.i) * D);
         const float4 *b = reinterpret_cast<const float4 *>(C + static_cast<long long>(cd.j) * D);
         double s = 0.0;
