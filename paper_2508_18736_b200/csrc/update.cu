@@ -65,22 +65,55 @@ update_apply_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restric
     __shared__ double red[UP_THREADS / 32];
     __shared__ int last_s;
     const int64_t p = blockIdx.x;
+    // this position, its left neighbour and the position one chunk to the left, requested together: most CTAs
+    // learn from them alone whether they start a chunk
     const uint32_t slot = keys[p];
+    const uint32_t left = p > 0 ? keys[p - 1] : 0xFFFFFFFFu;
+    const uint32_t far_left = p >= chunk ? keys[p - chunk] : 0xFFFFFFFFu;
     if (slot >= capacity) return;
-    int64_t lo = 0, hi = p;                  // first position of this slot in the sorted list
-    while (lo < hi) {
-        const int64_t mid = (lo + hi) >> 1;
-        if (keys[mid] < slot) lo = mid + 1; else hi = mid;
+    int64_t head = p;                        // first position of this slot in the sorted list
+    if (left == slot) {
+        // not the first row of the group.  If the row one chunk to the left belongs to another slot, the group began
+        // less than a chunk ago and this row starts no chunk; only long groups need their first position
+        if (far_left != slot) return;
+        int64_t lo = 0, hi = p;
+        while (lo < hi) {
+            const int64_t mid = (lo + hi) >> 1;
+            if (keys[mid] < slot) lo = mid + 1; else hi = mid;
+        }
+        head = lo;
+        if ((p - head) % chunk != 0) return;
     }
-    const int64_t head = lo;
-    if ((p - head) % chunk != 0) return;
     const bool is_head = p == head;
-    int64_t e = p;
-    while (e < B && e < p + chunk && keys[e] == slot) ++e;
-    const bool more = e < B && keys[e] == slot;
+    // everything the CTA needs of the slot and the first rows of the chunk, requested before the chunk's end is known
     const double n_old = size[slot];
+    const uint32_t access_old = access[slot];
     float *m = master + static_cast<int64_t>(slot) * D;
-    for (int d = threadIdx.x; d < D; d += UP_THREADS) acc[d] = is_head ? n_old * static_cast<double>(m[d]) : 0.0;
+    constexpr int MR = 4;                    // master elements per thread fetched ahead (covers D <= 1024)
+    float mreg[MR];
+#pragma unroll
+    for (int j = 0; j < MR; ++j) { const int d = threadIdx.x + j * UP_THREADS; mreg[j] = (is_head && d < D) ? m[d] : 0.0f; }
+    uint32_t row4[4];
+#pragma unroll
+    for (int r = 0; r < 4; ++r) row4[r] = p + r < B ? rows[p + r] : 0u;
+    // the end of this chunk, eight positions at a time; one position beyond the chunk tells whether the group goes on
+    int64_t e = p + 1;
+    const int64_t limit = min(B, p + static_cast<int64_t>(chunk) + 1);
+    while (e < limit) {
+        uint32_t k8[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) k8[u] = e + u < limit ? keys[e + u] : 0xFFFFFFFFu;
+        int same = 0;
+#pragma unroll
+        for (int u = 0; u < 8; ++u) same += (same == u && k8[u] == slot) ? 1 : 0;
+        e += same;
+        if (same < 8) break;
+    }
+    const bool more = e > p + chunk;
+    if (more) e = p + chunk;
+#pragma unroll
+    for (int j = 0; j < MR; ++j) { const int d = threadIdx.x + j * UP_THREADS; if (d < D) acc[d] = is_head ? n_old * static_cast<double>(mreg[j]) : 0.0; }
+    for (int d = threadIdx.x + MR * UP_THREADS; d < D; d += UP_THREADS) acc[d] = is_head ? n_old * static_cast<double>(m[d]) : 0.0;
     __syncthreads();      // the accumulation below uses a different thread-to-element mapping
     // the rows four at a time: the loads of a quartet are in flight together, additions stay in ascending order
     const int quads = D / 4;
@@ -88,7 +121,8 @@ update_apply_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restric
         const int nrow = static_cast<int>(e - t < 4 ? e - t : 4);
         const T *q[4];
 #pragma unroll
-        for (int r = 0; r < 4; ++r) q[r] = Q + static_cast<int64_t>(rows[t + (r < nrow ? r : 0)]) * D;
+        for (int r = 0; r < 4; ++r)
+            q[r] = Q + static_cast<int64_t>(t == p ? row4[r < nrow ? r : 0] : rows[t + (r < nrow ? r : 0)]) * D;
         for (int g = threadIdx.x; g < quads; g += UP_THREADS) {
             float4 v[4];
 #pragma unroll
@@ -143,8 +177,8 @@ update_apply_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restric
     }
     if (threadIdx.x == 0) {
         size[slot] = n_old + static_cast<double>(count);
-        const unsigned long long a = static_cast<unsigned long long>(access[slot]) + static_cast<unsigned long long>(count);
-        access[slot] = (access[slot] == SISO_ACCESS_INF || a >= SISO_ACCESS_INF) ? SISO_ACCESS_INF : static_cast<uint32_t>(a);
+        const unsigned long long a = static_cast<unsigned long long>(access_old) + static_cast<unsigned long long>(count);
+        access[slot] = (access_old == SISO_ACCESS_INF || a >= SISO_ACCESS_INF) ? SISO_ACCESS_INF : static_cast<uint32_t>(a);
         last[slot] = static_cast<unsigned long long>(counters[CNT_CLOCK]);
     }
 }
