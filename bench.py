@@ -41,7 +41,7 @@ def parse_args():
     ap.add_argument("--queries", type=int, default=8192, help="query batch per step")
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor", "stream"])
     ap.add_argument("--workload", default="config4",
-                    choices=["config4", "config1", "config2", "config3", "config5", "stream_probe", "cluster"],
+                    choices=["config4", "config1", "config2", "config3", "config5", "stream_probe", "cluster", "evict"],
                     help="config4 (default) is the benchmark contract; the others print one line each for the other "
                          "configurations (single GPU only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -407,6 +407,36 @@ def run_other(args):
                               "note": "whole pass (split, sweep, exact check, grouping, resolution, apply) over the "
                                       "lower-triangle flops N(N-1)/2 x 2D; the sweep kernel is about three quarters of it",
                               "fp32_alu_peak": fp32_peak})
+    elif args.workload == "evict":
+        # FilteringCentroids on the configuration-5 cache: the 256 lowest (cluster_size, access_count, last_access, slot)
+        # keys of 262,144 entries, then the decay pass; entries are put back between calls
+        sp = W.StreamSpec()
+        n, dim, m = sp.capacity, sp.dim, 256
+        cache = siso.SisoCache(n, dim, "bf16")
+        rows = torch.randn(1 << 16, dim, device=dev).to(torch.bfloat16)
+        sizes = torch.from_numpy(np.random.default_rng(0).integers(1, 64, n).astype(np.float64)).to(dev)
+        for lo in range(0, n, 1 << 16):
+            cache.insert(rows, sizes[lo:lo + (1 << 16)])
+        refill = rows[:m].contiguous()
+        times_e, times_d = [], []
+        for it in range(steps + warm):
+            e0, e1, e2 = (torch.cuda.Event(enable_timing=True) for _ in range(3))
+            e0.record()
+            cache.evict(m)
+            e1.record()
+            cache.evict(0, siso.EVICT_DECAY)
+            e2.record()
+            torch.cuda.synchronize()
+            cache.insert(refill)
+            if it >= warm:
+                times_e.append(e0.elapsed_time(e1)); times_d.append(e1.elapsed_time(e2))
+        ms_e, ms_d = statistics.median(times_e), statistics.median(times_d)
+        meta = n * 21.0                                  # cluster_size 8 + access_count 4 + last_access 8 + live flag 1
+        line.update(metric=f"eviction of the {m} lowest keys of {n:,} entries (exact selection); decay pass", value=n / ms_e * 1e3,
+                    unit="entries/s", ms_per_step=ms_e, decay_ms=ms_d, dtype="u64 keys / f64 sizes",
+                    roofline={"bound": "hbm", "achieved": 2 * meta / ms_e / 1e6, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                              "frac": 2 * meta / ms_e / 1e6 / peaks["hbm_gbs"], "traffic": None,
+                              "note": "two scans of 21 bytes of metadata per entry (5.5 MB each): a launch-latency-sized problem"})
     elif args.workload == "cluster":
         # stand-in for the query log that SISO-Cluster turns into centroids (Sec. 4.1): 131,072 unit vectors of dim 768
         # around 13,107 cluster means (the paper's 10 queries per centroid), clustered at theta_C = 0.86
