@@ -67,7 +67,7 @@ typedef enum { SISO_F32 = 0, SISO_BF16 = 1 } siso_dtype_t;
 #define SISO_OPT_TENSOR_CTA_PAIR 3      /* 0 (default): tensor-core lookup runs CTA pairs for >= 2 query tiles; 1: never */
 #define SISO_PATH_AUTO 0
 #define SISO_PATH_SIMT 1   /* CUDA-core tiled sweep (fp32 accumulate of exact products)        */
-#define SISO_PATH_TENSOR 2 /* tcgen05 tensor-core sweep, bf16 caches only                      */
+#define SISO_PATH_TENSOR 2 /* tcgen05 tensor-core sweep (fp32 caches: split-bf16 selection + exact rescoring, k <= 4) */
 #define SISO_PATH_STREAM 3 /* small-batch streaming sweep, one pass over the centroid matrix   */
 
 /* Device memory for the cache's own state and scratch comes from here.  alloc returns a
@@ -293,7 +293,8 @@ siso_status_t siso_export(siso_cache_t *c, void *d_vecs, float *d_master, double
 siso_status_t siso_import(siso_cache_t *c, const float *d_master, const double *d_sizes, const uint32_t *d_access,
                           const uint64_t *d_last, const uint8_t *d_valid, uint64_t clock, void *stream);
 
-/* h_counts[8] = occupancy, lookups, hits, inserts, evictions, merges, clock, 0.  Synchronises `stream`. */
+/* h_counts[8] = occupancy, lookups, hits, inserts, evictions, merges, clock, rescans (queries of fp32 tensor-core
+ * lookups that the exact rescoring could not settle and that were scanned again).  Synchronises `stream`. */
 siso_status_t siso_get_stats(siso_cache_t *c, int64_t *h_counts, void *stream);
 /* Synchronise `stream`, return the device status word (SISO_OK if clear) and clear it. */
 siso_status_t siso_sync_status(siso_cache_t *c, void *stream);

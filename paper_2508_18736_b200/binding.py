@@ -334,7 +334,7 @@ class SisoCache:
     def stats(self, stream=None) -> dict:
         buf = (ctypes.c_int64 * 8)()
         self._check(self._lib.siso_get_stats(self._h, buf, _stream(stream)), "siso_get_stats")
-        names = ["occupancy", "lookups", "hits", "inserts", "evictions", "merges", "clock"]
+        names = ["occupancy", "lookups", "hits", "inserts", "evictions", "merges", "clock", "rescans"]
         return {n: int(buf[i]) for i, n in enumerate(names)}
 
     def sync_status(self, stream=None) -> int:

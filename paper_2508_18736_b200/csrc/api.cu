@@ -191,7 +191,6 @@ siso_status_t siso_set_option(siso_cache_t *c, int32_t key, int64_t value) {
     switch (key) {
         case SISO_OPT_LOOKUP_PATH:
             if (value < SISO_PATH_AUTO || value > SISO_PATH_STREAM) return SISO_ERR_INVALID_ARG;
-            if (value == SISO_PATH_TENSOR && c->dtype != SISO_BF16) return SISO_ERR_UNSUPPORTED;
             c->lookup_path = static_cast<int32_t>(value);
             return SISO_OK;
         case SISO_OPT_TENSOR_CTA_PAIR:
@@ -229,7 +228,8 @@ static int resolve_lookup_path(const siso_cache_t *c, int64_t n_queries) {
         // measured on B200: the streaming kernel holds 92 % of HBM peak for 1-2 queries and falls off beyond;
         // the tensor-core kernel is HBM-bound (76-95 % of peak) from 3 queries up to one 128-query tile
         if (c->dtype == SISO_BF16) path = n_queries <= 2 ? SISO_PATH_STREAM : SISO_PATH_TENSOR;
-        else path = n_queries <= 4 ? SISO_PATH_STREAM : SISO_PATH_SIMT;
+        // fp32: the tensor-core sweep selects, an exact rescoring decides (k <= 4; otherwise the CUDA-core sweep)
+        else path = n_queries <= 4 ? SISO_PATH_STREAM : (n_queries >= 32 ? SISO_PATH_TENSOR : SISO_PATH_SIMT);
     }
     return path;
 }
@@ -243,7 +243,13 @@ siso_status_t siso_lookup(siso_cache_t *c, const void *d_queries, int64_t n_quer
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     switch (resolve_lookup_path(c, n_queries)) {
         case SISO_PATH_STREAM: return launch_lookup_stream(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);
-        case SISO_PATH_TENSOR: return launch_lookup_tensor(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);
+        case SISO_PATH_TENSOR:
+            if (c->dtype == SISO_BF16) return launch_lookup_tensor(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);
+            else {
+                const siso_status_t st = launch_lookup_tensor_f32(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);
+                if (st != SISO_ERR_UNSUPPORTED) return st;
+            }
+            return launch_lookup_simt(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);
         default: return launch_lookup_simt(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);
     }
 }
@@ -419,7 +425,7 @@ siso_status_t siso_stream_step(siso_cache_t *c, const void *d_queries, int64_t n
     // small batches: update, make-room and insertion in one cooperative launch, which also finishes the lookup
     // (best key over the splits, threshold test) when the tensor-core kernel produced it
     if (c->stream_fused && stream_maint_supported(c, n)) {
-        if (resolve_lookup_path(c, n) == SISO_PATH_TENSOR) {
+        if (c->dtype == SISO_BF16 && resolve_lookup_path(c, n) == SISO_PATH_TENSOR) {
             DeferredTop1 top1;
             void *tail = nullptr;
             SISO_TRY(launch_lookup_tensor(c, d_queries, n, d_theta, theta_scalar, 1, d_idx, d_sim, d_hit, s, &top1,
@@ -483,6 +489,7 @@ siso_status_t siso_get_stats(siso_cache_t *c, int64_t *h_counts, void *stream) {
     SISO_CUDA(cudaMemcpyAsync(tmp, c->counters, sizeof(tmp), cudaMemcpyDeviceToHost, s));
     SISO_CUDA(cudaStreamSynchronize(s));
     for (int i = 0; i < 8; ++i) h_counts[i] = i < CNT_SPARE ? tmp[i] : 0;
+    h_counts[7] = tmp[CNT_RESCANS];
     return SISO_OK;
 }
 

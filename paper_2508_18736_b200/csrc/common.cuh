@@ -18,7 +18,7 @@ constexpr int kMaxK = 8;
 constexpr uint32_t kNoSlot = 0xFFFFFFFFu;
 
 // device counters, int64 each
-enum Counter { CNT_OCCUPANCY = 0, CNT_LOOKUPS, CNT_HITS, CNT_INSERTS, CNT_EVICTIONS, CNT_MERGES, CNT_CLOCK, CNT_SPARE, CNT_SYNC, CNT_N };
+enum Counter { CNT_OCCUPANCY = 0, CNT_LOOKUPS, CNT_HITS, CNT_INSERTS, CNT_EVICTIONS, CNT_MERGES, CNT_CLOCK, CNT_SPARE, CNT_SYNC, CNT_RESCANS, CNT_N };
 
 struct Cache {
     int64_t capacity;
@@ -56,6 +56,7 @@ struct Cache {
     // large-shared-memory opt-in is a per-device function attribute: remembered per cache, not per process
     bool simt_attr_set[2][3];   // [dtype][k class] of lookup_simt_kernel
     bool merge_attr_set;
+    bool split_attr_set;
     bool merge_tensor_attr_set;
     int merge_resolve_grid;     // CTAs of the grid-wide merge resolution (0: not yet asked, -1: unavailable)
     int32_t merge_path;         // SISO_PATH_AUTO, SISO_PATH_SIMT or SISO_PATH_TENSOR for the pairwise sweep of siso_merge
@@ -114,6 +115,10 @@ siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const flo
                                    int32_t *idx, float *sim, uint8_t *hit, cudaStream_t s,
                                    DeferredTop1 *defer = nullptr, size_t tail_bytes = 0, void **tail = nullptr);
 void tensor_state_destroy(Cache *c);
+// fp32 caches on the tensor cores (split-bf16 selection, exact rescoring); SISO_ERR_UNSUPPORTED for bf16 caches or k > 4
+siso_status_t launch_lookup_tensor_f32(Cache *c, const void *q, int64_t B, const float *theta, float theta_s, int k,
+                                       int32_t *idx, float *sim, uint8_t *hit, cudaStream_t s);
+siso_status_t launch_split_bf16(Cache *c, const float *x, __nv_bfloat16 *hi, __nv_bfloat16 *lo, long long n4, cudaStream_t s);
 siso_status_t launch_topk_finalize(Cache *c, const unsigned long long *partial, int64_t B, int splits, int kmax, int k,
                                    const float *theta, float theta_s, int32_t *idx, float *sim, uint8_t *hit,
                                    cudaStream_t s);

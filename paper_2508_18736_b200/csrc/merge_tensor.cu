@@ -352,6 +352,13 @@ static siso_status_t encode_rows_map(EncodeTiledFn fn, CUtensorMap *map, const v
 
 }  // namespace tcm
 
+siso_status_t launch_split_bf16(Cache *c, const float *x, __nv_bfloat16 *hi, __nv_bfloat16 *lo, long long n4, cudaStream_t s) {
+    if (n4 <= 0) return SISO_OK;
+    tcm::split_bf16_kernel<<<static_cast<unsigned>((n4 + 255) / 256), 256, 0, s>>>(x, hi, lo, n4);
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
+
 size_t pair_sweep_tensor_scratch_bytes(int64_t n, int64_t rows, int dim) {
     const size_t tiles = static_cast<size_t>((n + 2 * tcm::TM - 1) / (2 * tcm::TM));
     return 2 * pad256(static_cast<size_t>(rows) * dim * sizeof(__nv_bfloat16)) + pad256(sizeof(uint32_t) * tiles * tiles);

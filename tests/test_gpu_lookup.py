@@ -31,10 +31,12 @@ def run_lookup(w, k, path, valid=None, theta=None):
 
 CASES = [
     # (config, overrides, mode, k, paths)
-    (1, dict(), "T", 1, ["simt", "auto"]),
-    (1, dict(n_centroids=1000, n_queries=333, dim=384), "P", 4, ["simt", "stream"]),
-    (1, dict(n_centroids=517, n_queries=130, dim=136, n_clusters=16), "L", 8, ["simt", "stream"]),
-    (1, dict(n_centroids=3, n_queries=5, dim=8, n_clusters=2), "L", 4, ["simt", "stream"]),
+    (1, dict(), "T", 1, ["simt", "tensor", "auto"]),
+    (1, dict(n_centroids=1000, n_queries=333, dim=384), "P", 4, ["simt", "stream", "tensor"]),
+    (1, dict(n_centroids=517, n_queries=130, dim=136, n_clusters=16), "L", 8, ["simt", "stream", "tensor"]),   # k = 8: CUDA cores
+    (1, dict(n_centroids=3, n_queries=5, dim=8, n_clusters=2), "L", 4, ["simt", "stream", "tensor"]),
+    (1, dict(n_centroids=5000, n_queries=700, dim=768, n_clusters=300), "T", 4, ["tensor"]),       # fp32 on tensor cores
+    (1, dict(n_centroids=2300, n_queries=1, dim=1024, n_clusters=100), "P", 2, ["tensor"]),
     (2, dict(n_centroids=4096 + 77, n_queries=700, dim=768, n_clusters=256), "T", 1, ["simt", "tensor", "auto"]),
     (2, dict(n_centroids=3000, n_queries=257, dim=768, n_clusters=128), "P", 1, ["simt", "tensor"]),
     (4, dict(n_centroids=8192 + 5, n_queries=300, dim=1024, n_clusters=512), "T", 4, ["simt", "tensor"]),
@@ -64,7 +66,7 @@ def test_lookup_matches_oracle(cfg, over, mode, k, paths):
         assert (lab[gpu[0][:, 0]] == lab[ora[0][:, 0]]).all() or mode != "T"
 
 
-@pytest.mark.parametrize("dtype,path", [("f32", "simt"), ("f32", "stream"), ("bf16", "simt"), ("bf16", "tensor"),
+@pytest.mark.parametrize("dtype,path", [("f32", "simt"), ("f32", "stream"), ("f32", "tensor"), ("bf16", "simt"), ("bf16", "tensor"),
                                         ("bf16", "stream")])
 def test_lookup_skips_empty_slots_and_pads_short_results(dtype, path):
     w = W.config(1, n_centroids=300, n_queries=40, dim=64, n_clusters=10, mode="P", dtype=dtype)
@@ -80,7 +82,7 @@ def test_lookup_skips_empty_slots_and_pads_short_results(dtype, path):
     assert (gpu[0] == -1).all() and np.isneginf(gpu[1]).all() and (gpu[2] == 0).all()
 
 
-@pytest.mark.parametrize("dtype,path", [("f32", "simt"), ("bf16", "tensor"), ("bf16", "stream")])
+@pytest.mark.parametrize("dtype,path", [("f32", "simt"), ("f32", "tensor"), ("bf16", "tensor"), ("bf16", "stream")])
 def test_exact_ties_go_to_the_lower_slot_and_threshold_is_strict(dtype, path):
     rng = np.random.default_rng(3)
     C = rng.integers(-1, 2, (200, 64)).astype(np.float32) * 0.125          # exact in bf16, exact dot products
@@ -99,6 +101,25 @@ def test_exact_ties_go_to_the_lower_slot_and_threshold_is_strict(dtype, path):
         gpu = run_lookup(w, 4, path)
         assert (gpu[0] == ora[0]).all() and (gpu[1] == ora[1].astype(np.float32)).all() and (gpu[2] == ora[2]).all()
     assert gpu[0][0, :3].tolist() == [7, 90, 150] and gpu[2].tolist() == [1, 1, 1]
+
+
+def test_fp32_tensor_path_rescans_queries_it_cannot_settle():
+    """The fp32 tensor-core path accepts its answer only if the k-th exact similarity clears the 8th approximate one by a
+    margin.  With a dozen identical rows inside one tile that never happens: those queries must come out of the exact scan, ties to the
+    lower slot; the other queries are settled by the rescoring."""
+    w = W.config(1, n_centroids=900, n_queries=200, dim=72, n_clusters=40, mode="P")
+    C = w.centroids.copy()
+    dup = [5, 17, 30, 31, 100, 101, 120, 130, 140, 150, 160, 170]         # all in the first tile of 256 rows
+    C[dup] = C[5]
+    Q = w.queries.copy()
+    Q[:50] = C[5]                                             # 50 queries whose 12 best rows tie exactly
+    w2 = W.Workload("ties", "f32", 72, C, Q, w.theta, 4, w.centroid_labels, None, {})
+    ora = oracle.lookup(C, Q, w.theta, 4)
+    gpu = run_lookup(w2, 4, "tensor")
+    check_lookup(gpu, ora, C, Q, w.theta, TOL["f32"])
+    assert (gpu[0][:50] == np.array(dup[:4])).all()
+    simt = run_lookup(w2, 4, "simt")
+    assert (simt[0] == gpu[0]).all() and (simt[2] == gpu[2]).all()
 
 
 def test_bad_arguments_return_status_and_touch_nothing():
