@@ -41,7 +41,7 @@ def parse_args():
     ap.add_argument("--queries", type=int, default=8192, help="query batch per step")
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor", "stream"])
     ap.add_argument("--workload", default="config4",
-                    choices=["config4", "config1", "config2", "config3", "config5", "stream_probe", "cluster", "evict"],
+                    choices=["config4", "config1", "config2", "config3", "config5", "stream_probe", "cluster", "evict", "f32_lookup"],
                     help="config4 (default) is the benchmark contract; the others print one line each for the other "
                          "configurations (single GPU only)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -410,6 +410,28 @@ def run_other(args):
                               "peak_kind": "measured bf16 burst peak / 3 (split-bf16 emulation of fp32 products)",
                               "note": "whole pass (split, sweep, exact check, grouping, resolution, apply) over the "
                                       "lower-triangle flops N(N-1)/2 x 2D; the sweep kernel is about three quarters of it",
+                              "fp32_alu_peak": fp32_peak})
+    elif args.workload == "f32_lookup":
+        # an fp32 cache at scale: 262,144 x 1024 fp32 centroids (1 GiB), batch 4,096, top-4; clusters as in configuration 4
+        N = 262144 if args.rows == (1 << 20) else args.rows
+        B = 4096 if args.queries == 8192 else args.queries
+        D = 1024
+        w = W.config(1, threads=cores, n_centroids=N, n_queries=B, dim=D, n_clusters=max(2, N // 16), theta=(0.78, 0.93), k=4)
+        cache = siso.SisoCache(N, D, "f32")
+        fill(cache, w.centroids, "f32")
+        q, th = to_dev(w.queries, "f32"), torch.from_numpy(w.theta).to(dev)
+        res = {}
+        for name, path in (("cuda_cores", siso.PATH_SIMT), ("tensor", siso.PATH_TENSOR)):
+            cache.set_lookup_path(path)
+            res[name] = time_ms(lambda: cache.lookup(q, th, 4), steps if name == "tensor" else max(3, steps // 4), warm)
+        ms = res["tensor"]
+        fl = 2.0 * N * B * D
+        tc_peak = peaks["bf16_tflops"] / 3.0
+        line.update(metric=f"lookup queries/s, {N:,} x {D} fp32, batch {B:,}, top-4", value=B / ms * 1e3, unit=UNIT, ms_per_step=ms,
+                    cuda_core_sweep_ms=res["cuda_cores"], rescans=cache.stats()["rescans"], dtype="f32",
+                    roofline={"bound": "tensor", "achieved": fl / ms / 1e9, "peak": tc_peak, "unit": "TFLOP/s",
+                              "frac": fl / ms / 1e9 / tc_peak, "traffic": None,
+                              "peak_kind": "measured bf16 burst peak / 3 (split-bf16 emulation of fp32 products)",
                               "fp32_alu_peak": fp32_peak})
     elif args.workload == "evict":
         # FilteringCentroids on the configuration-5 cache: the 256 lowest (cluster_size, access_count, last_access, slot)
