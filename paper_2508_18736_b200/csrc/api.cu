@@ -225,9 +225,10 @@ siso_status_t siso_insert(siso_cache_t *c, const void *d_vecs, const double *d_s
 static int resolve_lookup_path(const siso_cache_t *c, int64_t n_queries) {
     int path = c->lookup_path;
     if (path == SISO_PATH_AUTO) {
-        // measured on B200: the streaming kernel holds 92 % of HBM peak for 1-2 queries and falls off beyond;
-        // the tensor-core kernel is HBM-bound (76-95 % of peak) from 3 queries up to one 128-query tile
-        if (c->dtype == SISO_BF16) path = n_queries <= 2 ? SISO_PATH_STREAM : SISO_PATH_TENSOR;
+        // measured on B200: with a small batch padded to a whole query tile the tensor-core kernel streams the matrix at
+        // 100-104 % of the measured copy bandwidth from one query up (2 GiB matrix; 86-92 % on 384 MiB); the streaming
+        // kernel holds 96 % for 1-2 queries and falls off beyond, so bf16 caches always take the tensor-core kernel
+        if (c->dtype == SISO_BF16) path = SISO_PATH_TENSOR;
         // fp32: the tensor-core sweep selects, an exact rescoring decides (k <= 4; otherwise the CUDA-core sweep)
         else path = n_queries <= 4 ? SISO_PATH_STREAM : (n_queries >= 32 ? SISO_PATH_TENSOR : SISO_PATH_SIMT);
     }
