@@ -179,7 +179,7 @@ siso_status_t siso_cache_destroy(siso_cache_t *c) {
     cudaDeviceSynchronize();
     tensor_state_destroy(c);
     void *ptrs[] = {c->dtype == SISO_F32 ? nullptr : c->vecs, c->master, c->size, c->access, c->last, c->valid,
-                    c->counters, c->status, c->ws, c->stage, c->swap_plan};
+                    c->counters, c->status, c->ws, c->stage, c->swap_plan, c->split_hi, c->split_lo};
     for (void *p : ptrs)
         if (p) c->alloc.free(p, c->alloc.ctx);
     delete c;
@@ -461,6 +461,7 @@ siso_status_t siso_export(siso_cache_t *c, void *d_vecs, float *d_master, double
 siso_status_t siso_import(siso_cache_t *c, const float *d_master, const double *d_sizes, const uint32_t *d_access,
                           const uint64_t *d_last, const uint8_t *d_valid, uint64_t clock, void *stream) {
     if (!c || !d_master || !d_sizes || !d_access || !d_last || !d_valid) return SISO_ERR_INVALID_ARG;
+    c->vec_epoch += 1;          // the vectors may change: derived copies (the split-bf16 parts) are stale
     SISO_CUDA(cudaSetDevice(c->device));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t n = static_cast<size_t>(c->capacity), D = static_cast<size_t>(c->dim);

@@ -57,6 +57,9 @@ struct Cache {
     bool simt_attr_set[2][3];   // [dtype][k class] of lookup_simt_kernel
     bool merge_attr_set;
     bool split_attr_set;
+    // fp32 caches: the bf16 parts (hi, lo) of the vectors for the tensor-core lookup, valid while split_epoch == vec_epoch
+    void *split_hi, *split_lo;
+    unsigned long long vec_epoch, split_epoch;
     bool merge_tensor_attr_set;
     int merge_resolve_grid;     // CTAs of the grid-wide merge resolution (0: not yet asked, -1: unavailable)
     int32_t merge_path;         // SISO_PATH_AUTO, SISO_PATH_SIMT or SISO_PATH_TENSOR for the pairwise sweep of siso_merge

@@ -366,6 +366,7 @@ insert_copy_kernel(const T *__restrict__ rows, const double *__restrict__ sizes_
 
 siso_status_t launch_insert(Cache *c, const void *vecs, const double *sizes, const uint8_t *hit, int64_t n,
                             int32_t *slots_out, cudaStream_t s) {
+    c->vec_epoch += 1;          // the vectors may change: derived copies (the split-bf16 parts) are stale
     if (n == 0) return SISO_OK;
     if (n >= (1ll << 31)) return SISO_ERR_UNSUPPORTED;
     Scratch scr;

@@ -461,17 +461,27 @@ siso_status_t launch_lookup_tensor_f32(Cache *c, const void *q, int64_t B, const
     }
     const size_t c_elems = static_cast<size_t>(rows) * D, q_elems = static_cast<size_t>(B) * D;
     Scratch scr;
-    const size_t need = 2 * pad256(c_elems * 2) + 2 * pad256(q_elems * 2) + pad256(sizeof(unsigned long long) * B * splits * tc3::CAND) +
+    const size_t need = 2 * pad256(q_elems * 2) + pad256(sizeof(unsigned long long) * B * splits * tc3::CAND) +
                         pad256(4 * B) + pad256(sizeof(unsigned long long) * 4 * B * c->sm_count) + 512;
     SISO_TRY(scratch_reserve(c, need, s, &scr));
-    __nv_bfloat16 *c_hi = scr.take<__nv_bfloat16>(c_elems), *c_lo = scr.take<__nv_bfloat16>(c_elems);
+    // the centroids' parts are kept until the vectors change (every entry point that writes vectors raises vec_epoch)
+    if (!c->split_hi) {
+        c->split_hi = cache_alloc_zeroed(c, c_elems * 2);
+        c->split_lo = cache_alloc_zeroed(c, c_elems * 2);
+        if (!c->split_hi || !c->split_lo) return SISO_ERR_OOM;
+        c->split_epoch = ~0ull;
+    }
+    __nv_bfloat16 *c_hi = static_cast<__nv_bfloat16 *>(c->split_hi), *c_lo = static_cast<__nv_bfloat16 *>(c->split_lo);
     __nv_bfloat16 *q_hi = scr.take<__nv_bfloat16>(q_elems), *q_lo = scr.take<__nv_bfloat16>(q_elems);
     unsigned long long *partial = scr.take<unsigned long long>(static_cast<size_t>(B) * splits * tc3::CAND);
     int32_t *flagged = scr.take<int32_t>(B);
     unsigned int *n_flagged = scr.take<unsigned int>(1);
     unsigned long long *rescan_keys = scr.take<unsigned long long>(static_cast<size_t>(4) * B * c->sm_count);
     SISO_CUDA(cudaMemsetAsync(n_flagged, 0, sizeof(unsigned int), s));
-    SISO_TRY(launch_split_bf16(c, c->master, c_hi, c_lo, static_cast<long long>(c_elems / 4), s));
+    if (c->split_epoch != c->vec_epoch) {
+        SISO_TRY(launch_split_bf16(c, c->master, c_hi, c_lo, static_cast<long long>(c_elems / 4), s));
+        c->split_epoch = c->vec_epoch;
+    }
     SISO_TRY(launch_split_bf16(c, static_cast<const float *>(q), q_hi, q_lo, static_cast<long long>(q_elems / 4), s));
     CUtensorMap map_q_hi, map_q_lo, map_c_hi, map_c_lo;
     SISO_TRY(tc3::encode_rows_map(encode, &map_q_hi, q_hi, static_cast<uint64_t>(B), static_cast<uint64_t>(D)));

@@ -360,6 +360,7 @@ siso_status_t launch_merge_resolve(Cache *c, void *ctl_v, int64_t N, const uint8
 
 siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes, int64_t n_repo, float theta_c,
                            uint32_t flags, int32_t *merge_map, long long *d_n_merged, cudaStream_t s) {
+    c->vec_epoch += 1;          // the vectors may change: derived copies (the split-bf16 parts) are stale
     const int64_t N = c->capacity;
     if (N >= (1ll << 31) - 1) return SISO_ERR_UNSUPPORTED;
     const int64_t tiles = (N + BM - 1) / BM;

@@ -826,6 +826,7 @@ bool stream_maint_supported(Cache *c, int64_t B) {
 // Returns SISO_ERR_UNSUPPORTED if this batch cannot take the fused path (the caller then uses the separate kernels).
 siso_status_t launch_stream_maint(Cache *c, const void *q, int64_t B, int32_t *idx, uint8_t *hit, int32_t *victims,
                                   int32_t *slots_out, const DeferredTop1 *deferred, void *scratch_tail, cudaStream_t s) {
+    c->vec_epoch += 1;          // the vectors may change: derived copies (the split-bf16 parts) are stale
     if (!stream_maint_supported(c, B)) return SISO_ERR_UNSUPPORTED;
     const int grid = c->maint_grid;
     Scratch scr;

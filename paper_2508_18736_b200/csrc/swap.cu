@@ -97,6 +97,7 @@ __global__ void swap_copy_counters_kernel(const long long *__restrict__ src, lon
 }  // namespace
 
 siso_status_t launch_cache_copy(Cache *dst, const Cache *src, cudaStream_t s) {
+    dst->vec_epoch += 1;          // the vectors may change: derived copies (the split-bf16 parts) are stale
     const size_t n = static_cast<size_t>(src->capacity), D = static_cast<size_t>(src->dim);
     const size_t esz = src->dtype == SISO_F32 ? 4 : 2;
     SISO_CUDA(cudaMemcpyAsync(dst->master, src->master, n * D * 4, cudaMemcpyDeviceToDevice, s));
@@ -116,6 +117,7 @@ siso_status_t launch_cache_copy(Cache *dst, const Cache *src, cudaStream_t s) {
 }
 
 siso_status_t launch_update_centroids(Cache *cur, Cache *c_new, int64_t first, int64_t n, cudaStream_t s) {
+    cur->vec_epoch += 1;          // the vectors may change: derived copies (the split-bf16 parts) are stale
     if (!c_new->swap_plan) {
         // source_of[capacity of C_new] and the live count behind it; lives as long as C_new
         c_new->swap_plan = cache_alloc_zeroed(c_new, pad256(sizeof(int32_t) * c_new->capacity) + 256);

@@ -288,6 +288,7 @@ update_small_kernel(const int32_t *__restrict__ idx, int idx_stride, const uint8
 
 siso_status_t launch_update(Cache *c, const void *q, int64_t B, const int32_t *idx, int idx_stride, const uint8_t *hit,
                             cudaStream_t s) {
+    c->vec_epoch += 1;          // the vectors may change: derived copies (the split-bf16 parts) are stale
     if (B >= (1ll << 31)) return SISO_ERR_UNSUPPORTED;
     if (B >= 1 && B <= UPS_MAX_B) {
         const size_t smem_small = sizeof(double) * c->dim;

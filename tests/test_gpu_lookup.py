@@ -122,6 +122,43 @@ def test_fp32_tensor_path_rescans_queries_it_cannot_settle():
     assert (simt[0] == gpu[0]).all() and (simt[2] == gpu[2]).all()
 
 
+def test_fp32_tensor_path_sees_every_change_of_the_vectors():
+    """The fp32 tensor-core path keeps the bf16 parts of the centroids between calls; every entry point that writes
+    vectors must make it split them again."""
+    w = W.config(1, n_centroids=600, n_queries=64, dim=72, n_clusters=30, mode="P")
+    cache = siso.SisoCache(700, 72, "f32")
+    ora = oracle.OracleCache(700, 72, "f32")
+    cache.set_lookup_path(siso.PATH_TENSOR)
+    cache.insert(to_dev(w.centroids[:500], "f32"))
+    ora.insert(w.centroids[:500])
+    q, theta = to_dev(w.queries, "f32"), np.full(64, 0.85, np.float32)
+
+    def same(what):
+        got = [x.cpu().numpy() for x in cache.lookup(q, 0.85, 2)]
+        check_lookup(got, ora.lookup(w.queries, theta, 2), ora.lookup_copy(), w.queries, theta, TOL["f32"], valid=ora.valid)
+        return got
+
+    same("after the first insert")
+    cache.insert(to_dev(w.centroids[500:], "f32"))                       # insert
+    ora.insert(w.centroids[500:])
+    same("after a second insert")
+    idx, sim, hit = cache.lookup(q, 0.85, 1)                              # running-mean update of the hit rows
+    cache.update(q, idx, hit)
+    ora.update(w.queries, idx.cpu().numpy(), hit.cpu().numpy())
+    got = same("after an update")
+    assert hit.cpu().numpy().sum() > 0
+    mm, n = cache.merge(0.9, siso.MERGE_WEIGHTED_MEAN)                     # merge moves vectors and empties slots
+    ora.merge(0.9, True)
+    same("after a merge")
+    st = cache.export()                                                   # import replaces everything
+    rolled = torch.roll(st["master"], 1, dims=0)
+    cache.import_(rolled, st["size"], st["access"], st["last"], st["valid"], 5)
+    ora.load_state(rolled.cpu().numpy(), st["size"].cpu().numpy(), st["access"].cpu().numpy().view(np.uint32),
+                   st["last"].cpu().numpy().view(np.uint64), st["valid"].cpu().numpy(), 5)
+    same("after an import")
+    cache.close()
+
+
 def test_bad_arguments_return_status_and_touch_nothing():
     cache = siso.SisoCache(64, 64, "bf16")
     q = torch.zeros(4, 64, dtype=torch.bfloat16, device="cuda")
