@@ -283,28 +283,28 @@ def test_insert_misses_and_capacity_error():
     assert all((before[k] == after[k]).all() for k in before)
 
 
-@pytest.mark.parametrize("theta_mode", ["fixed", "per_query"])
-def test_streaming_step_lockstep_on_a_scaled_twin(theta_mode):
+@pytest.mark.parametrize("theta_mode,dtype", [("fixed", "bf16"), ("per_query", "bf16"), ("fixed", "f32")])
+def test_streaming_step_lockstep_on_a_scaled_twin(theta_mode, dtype):
     sp = W.StreamSpec(capacity=1024, dim=128, n_queries=256 * 60, batch=256, n_clusters=400, zipf_s=1.2,
-                      reshuffle_every=256 * 30, theta=0.86, mode="P", dtype="bf16")
+                      reshuffle_every=256 * 30, theta=0.86, mode="P", dtype=dtype)
     st = W.QueryStream(sp)
-    cache = siso.SisoCache(sp.capacity, sp.dim, "bf16")
-    ora = oracle.OracleCache(sp.capacity, sp.dim, "bf16")
+    cache = siso.SisoCache(sp.capacity, sp.dim, dtype)
+    ora = oracle.OracleCache(sp.capacity, sp.dim, dtype)
     rng = np.random.default_rng(2)
     evictions = 0
     for t, q, _ in st.batches():
         theta = np.full(len(q), sp.theta, np.float32) if theta_mode == "fixed" else rng.uniform(0.80, 0.92, len(q)).astype(np.float32)
         th = float(sp.theta) if theta_mode == "fixed" else torch.from_numpy(theta).cuda()
-        idx, sim, hit, victims, slots = [x.cpu().numpy() for x in cache.stream_step(to_dev(q, "bf16"), th)]
+        idx, sim, hit, victims, slots = [x.cpu().numpy() for x in cache.stream_step(to_dev(q, dtype), th)]
         pre_copy, pre_valid = ora.lookup_copy(), ora.valid.copy()
         o_idx, o_sim, o_hit, o_victims, o_slots = ora.stream_step(q, theta, forced=(idx, hit))
-        check_lookup((idx, sim, hit), (o_idx, o_sim, o_hit), pre_copy, q, theta, TOL["bf16"], valid=pre_valid)
+        check_lookup((idx, sim, hit), (o_idx, o_sim, o_hit), pre_copy, q, theta, TOL[dtype], valid=pre_valid)
         nv = len(o_victims)
         assert (victims[:nv] == o_victims).all() and (victims[nv:] == -1).all(), f"batch {t}"
         assert (slots == o_slots).all(), f"batch {t}"
         evictions += nv
         if t % 10 == 9 or t < 3:
-            assert_state_equal(cache, ora, "bf16", f"batch {t}")
+            assert_state_equal(cache, ora, dtype, f"batch {t}")
             # resynchronise the oracle's fp64 master with the GPU's fp32 master so rounding does not accumulate
             g = state_np(cache)
             ora.load_state(g["master"], g["size"], g["access"], g["last"], g["valid"], ora.clock)
