@@ -283,10 +283,11 @@ def test_insert_misses_and_capacity_error():
     assert all((before[k] == after[k]).all() for k in before)
 
 
-@pytest.mark.parametrize("theta_mode,dtype", [("fixed", "bf16"), ("per_query", "bf16"), ("fixed", "f32")])
-def test_streaming_step_lockstep_on_a_scaled_twin(theta_mode, dtype):
-    sp = W.StreamSpec(capacity=1024, dim=128, n_queries=256 * 60, batch=256, n_clusters=400, zipf_s=1.2,
-                      reshuffle_every=256 * 30, theta=0.86, mode="P", dtype=dtype)
+@pytest.mark.parametrize("theta_mode,dtype,batch", [("fixed", "bf16", 256), ("per_query", "bf16", 256), ("fixed", "f32", 256),
+                                                    ("fixed", "bf16", 100)])      # 100: a batch that is padded to a query tile
+def test_streaming_step_lockstep_on_a_scaled_twin(theta_mode, dtype, batch):
+    sp = W.StreamSpec(capacity=1024, dim=128, n_queries=batch * 60, batch=batch, n_clusters=400, zipf_s=1.2,
+                      reshuffle_every=batch * 30, theta=0.86, mode="P", dtype=dtype)
     st = W.QueryStream(sp)
     cache = siso.SisoCache(sp.capacity, sp.dim, dtype)
     ora = oracle.OracleCache(sp.capacity, sp.dim, dtype)
