@@ -34,6 +34,7 @@ constexpr int SM_SAMPLE = 256;
 constexpr int SM_STAGE = 2048;      // candidates a CTA can hold in shared memory while ranking
 constexpr int SM_SELECT = 16;       // up to this many splitters are extracted one by one instead of sorting the sample
 constexpr int SM_RANK_STRIDE = 4;   // every fourth CTA ranks candidates
+constexpr int SM_DENSE = 4;         // entries per sampler thread in the fine sample (4 x 256 entries)
 
 struct MaintCtl {
     unsigned int n_cand;                 // candidates appended in phase S
@@ -305,35 +306,60 @@ __device__ void maint_evict_sample(const MaintArgs &a, long long clock_new, long
     const int tid = threadIdx.x;
     const long long stride = (a.capacity + SM_SAMPLE - 1) / SM_SAMPLE;
     const long long lo = tid * stride, hi = min(a.capacity, lo + stride);
-    const long long span = hi - lo;
-    int have = 0;
-    Key3 mine;
-    mine.w0 = mine.w1 = mine.w2 = ~0ull;
-    if (span > 0) {
-        const long long start = static_cast<long long>((static_cast<unsigned long long>(clock_new) * 2654435761ull) % static_cast<unsigned long long>(span));
-        const long long probes = span < 64 ? span : 64;
-        for (long long i = 0; i < probes; ++i) {
-            long long sl = lo + start + i;
-            if (sl >= hi) sl -= span;
-            // the four loads do not wait for one another: a full cache answers at the first probe
-            const uint8_t live = a.valid[sl];
-            const double sz = a.size[sl];
-            const uint32_t ac = a.access[sl];
-            const unsigned long long la = a.last[sl];
-            if (live) { mine = make_key(sz, ac, la, static_cast<uint32_t>(sl)); have = 1; break; }
+    // up to SM_DENSE live entries of this thread's window, one from each quarter of it (the first one serves the
+    // 256-entry sample that is sorted in full; all of them serve the finer sample of which only the few smallest
+    // keys are needed)
+    Key3 k[SM_DENSE];
+    int have[SM_DENSE];
+    const long long sub = (stride + SM_DENSE - 1) / SM_DENSE;
+#pragma unroll
+    for (int d = 0; d < SM_DENSE; ++d) {
+        k[d].w0 = k[d].w1 = k[d].w2 = ~0ull;
+        have[d] = 0;
+        const long long s_lo = min(hi, lo + d * sub), s_hi = min(hi, s_lo + sub);
+        const long long span = s_hi - s_lo;
+        if (span > 0) {
+            const long long start = static_cast<long long>((static_cast<unsigned long long>(clock_new) * 2654435761ull) % static_cast<unsigned long long>(span));
+            const long long probes = span < 16 ? span : 16;
+            for (long long i = 0; i < probes; ++i) {
+                long long sl = s_lo + start + i;
+                if (sl >= s_hi) sl -= span;
+                // the four loads do not wait for one another: a full cache answers at the first probe
+                const uint8_t live = a.valid[sl];
+                const double sz = a.size[sl];
+                const uint32_t ac = a.access[sl];
+                const unsigned long long la = a.last[sl];
+                if (live) { k[d] = make_key(sz, ac, la, static_cast<uint32_t>(sl)); have[d] = 1; break; }
+            }
         }
     }
-    int n_sample;
-    block_exclusive_scan_256(have, &n_sample, sm.warp_sum);
-    const int P = maint_spec_buckets(m, n_sample, occupancy);
-    if (!all && P < SM_SELECT && P < n_sample) {
-        // the P+1 smallest, one block-wide minimum at a time (keys differ in their slot word)
-        for (int r = 0; r <= P; ++r) {
+    int n_dense, n_sample;
+    {
+        int h = 0;
+#pragma unroll
+        for (int d = 0; d < SM_DENSE; ++d) h += have[d];
+        block_exclusive_scan_256(h, &n_dense, sm.warp_sum);
+        __syncthreads();
+    }
+    const int P_dense = maint_spec_buckets(m, n_dense, occupancy);
+    if (!all && P_dense < SM_SELECT && P_dense < n_dense) {
+        // the P+1 smallest of the fine sample, one block-wide minimum at a time (keys differ in their slot word)
+        n_sample = n_dense;
+        for (int r = 0; r <= P_dense; ++r) {
+            Key3 mine = k[0];
+#pragma unroll
+            for (int d = 1; d < SM_DENSE; ++d)
+                if (key_less(k[d], mine)) mine = k[d];
             const Key3 best = block_min_key(mine, sm);
             if (tid == 0) a.splitters[r] = best;
-            if (mine.w0 == best.w0 && mine.w1 == best.w1 && mine.w2 == best.w2) mine.w0 = mine.w1 = mine.w2 = ~0ull;
+#pragma unroll
+            for (int d = 0; d < SM_DENSE; ++d)
+                if (k[d].w0 == best.w0 && k[d].w1 == best.w1 && k[d].w2 == best.w2) k[d].w0 = k[d].w1 = k[d].w2 = ~0ull;
         }
     } else {
+        // the coarse sample (one entry per thread), sorted in full
+        const Key3 mine = k[0];
+        block_exclusive_scan_256(have[0], &n_sample, sm.warp_sum);
         __syncthreads();
         sm.k0[tid] = mine.w0; sm.k1[tid] = mine.w1; sm.k2[tid] = mine.w2;
         __syncthreads();

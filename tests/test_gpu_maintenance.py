@@ -350,8 +350,9 @@ def test_streaming_eviction_is_exact_when_the_sample_misleads():
     cache.insert(to_dev(cent, "bf16"))
     g = state_np(cache)
     clock = cache.stats()["clock"]
-    # the step's sampler looks at slot 16 w + ((clock + 1) * 2654435761 mod 16) of every 16-slot window w
-    off = ((clock + 1) * 2654435761) % (cap // 256)
+    # for this many victims the step's sampler sorts one entry per 16-slot window w: the first live one of the window's
+    # first quarter, slot 16 w + ((clock + 1) * 2654435761 mod 4)
+    off = ((clock + 1) * 2654435761) % (cap // 256 // 4)
     size = np.ones(cap)
     size[np.arange(256) * (cap // 256) + off] = 0.5
     cache.import_(torch.from_numpy(g["master"]), torch.from_numpy(size), torch.from_numpy(g["access"].view(np.int32)),
