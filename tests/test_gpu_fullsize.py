@@ -166,3 +166,36 @@ def test_config5_full_scale_sampled_batches():
     assert s["inserts"] - s["evictions"] == s["occupancy"]
     cache.check_status()
     cache.close()
+
+
+def test_config5_full_scale_is_reproducible_and_equals_the_separate_kernels():
+    """300 micro-batches on the full-size cache, three times: twice through the one-launch maintenance kernel (grid-wide
+    barriers, atomics on candidate lists) and once through the separate kernels.  Every output of every batch and the
+    final state must be the same bits: the step has no run-to-run freedom."""
+    sp = W.StreamSpec()
+    stream = W.QueryStream(sp, threads=THREADS)
+    n_batches = 300
+    q_all = to_dev(stream.block(0, n_batches, threads=THREADS), "bf16")
+    filler = to_dev(stream.block(20000, 20000 + (sp.capacity - 3000) // 256, threads=THREADS), "bf16")
+
+    def run(fused):
+        cache = siso.SisoCache(sp.capacity, sp.dim, "bf16")
+        cache.set_option(siso.OPT_STREAM_FUSED, fused)
+        for lo in range(0, filler.shape[0], 1 << 16):
+            cache.insert(filler[lo:lo + (1 << 16)])
+        outs = [[x.clone() for x in cache.stream_step(q_all[t * 256:(t + 1) * 256], float(sp.theta))] for t in range(n_batches)]
+        cache.check_status()
+        st, stats = cache.export(), cache.stats()
+        cache.close()
+        return outs, st, stats
+
+    a, sa, ta = run(1)
+    for other in (run(1), run(0)):
+        b, sb, tb = other
+        assert ta == tb and ta["evictions"] > 0
+        for t, (oa, ob) in enumerate(zip(a, b)):
+            assert all((x == y).all().item() for x, y in zip(oa, ob)), f"batch {t}"
+        live = sa["valid"] == 1
+        assert (sa["valid"] == sb["valid"]).all().item()
+        for k in ("master", "vecs", "size", "access", "last"):
+            assert (sa[k][live] == sb[k][live]).all().item(), k
