@@ -278,7 +278,7 @@ def run_ours(args):
     # only known for the full-size workload on the tensor-core kernel as profiled
     traffic = None
     if args.path in ("auto", "tensor") and args.rows == (1 << 20) and B == 8192:
-        traffic = 0.5 * (2888013568 + 2888555520) + 0.5 * (5518080 + 2418432)
+        traffic = 0.5 * (2892656384 + 2893686784) + 0.5 * (5250560 + 1996544)
     roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                 "frac": achieved / peaks["bf16_tflops"], "traffic": traffic, "peak_kind": f"{peak_kind}, burst",
                 "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
