@@ -41,9 +41,10 @@ def parse_args():
     ap.add_argument("--queries", type=int, default=8192, help="query batch per step")
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor", "stream"])
     ap.add_argument("--workload", default="config4",
-                    choices=["config4", "config1", "config2", "config3", "config5", "stream_probe", "cluster", "evict", "f32_lookup"],
+                    choices=["config4", "config1", "config2", "config3", "config5", "stream_probe", "cluster", "evict", "f32_lookup", "config5_full"],
                     help="config4 (default) is the benchmark contract; the others print one line each for the other "
                          "configurations (single GPU only)")
+    ap.add_argument("--seed", type=int, default=0, help="seed of the configuration-5 stream (config5_full)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -489,6 +490,50 @@ def run_other(args):
                     roofline={"bound": "tensor", "achieved": fl / ms / 1e9, "peak": tc_peak, "unit": "TFLOP/s",
                               "frac": fl / ms / 1e9 / tc_peak, "traffic": None,
                               "peak_kind": "measured bf16 burst peak / 3 (split-bf16 emulation of fp32 products)"})
+    elif args.workload == "config5_full":
+        # the whole stream of configuration 5 from an empty cache: 10,000,000 queries in micro-batches of 256, popularity
+        # reshuffled every 1,000,000 queries.  Queries are generated a million at a time on the host (not timed), copied
+        # to the device, and the steps of that chunk are timed with CUDA events.
+        sp = W.StreamSpec(seed=args.seed)
+        stream = W.QueryStream(sp, threads=cores)
+        cache = siso.SisoCache(sp.capacity, sp.dim, "bf16")
+        per_chunk = 3906                                      # batches per chunk (about one popularity epoch)
+        total_ms, done, out = 0.0, 0, None
+        epochs, first_full, prev = [], None, cache.stats()
+        while done < sp.n_batches:
+            stop = min(sp.n_batches, done + per_chunk)
+            q = to_dev(stream.block(done, stop, threads=cores), "bf16")
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            for t in range(done, stop):
+                lo = (t - done) * sp.batch
+                qb = q[lo:lo + sp.batch]
+                if qb.shape[0] != sp.batch:
+                    out = None                                 # the last batch is short
+                out = cache.stream_step(qb, float(sp.theta), out=out)
+            e1.record()
+            torch.cuda.synchronize()
+            total_ms += e0.elapsed_time(e1)
+            st = cache.stats()
+            nq = st["lookups"] - prev["lookups"]
+            epochs.append({"queries": nq, "hit_ratio": round((st["hits"] - prev["hits"]) / max(1, nq), 4),
+                           "inserts": st["inserts"] - prev["inserts"], "evictions": st["evictions"] - prev["evictions"],
+                           "us_per_batch": round(e0.elapsed_time(e1) / (stop - done) * 1e3, 1), "occupancy": st["occupancy"]})
+            if first_full is None and st["occupancy"] == sp.capacity:
+                first_full = len(epochs)
+            prev, done = st, stop
+        cache.check_status()
+        st = cache.stats()
+        assert st["lookups"] == sp.n_queries and st["inserts"] - st["evictions"] == st["occupancy"] <= sp.capacity
+        us = total_ms / sp.n_batches * 1e3
+        gbs = sp.capacity * sp.dim * 2 / (us * 1e-6) / 1e9
+        line.update(metric="streaming cache, whole stream: 10,000,000 queries, 262,144 x 768 bf16, micro-batches of 256, from an empty cache",
+                    value=sp.n_queries / total_ms * 1e3, unit=UNIT, us_per_batch=us, batches=sp.n_batches, seed=args.seed, dtype="bf16",
+                    hit_ratio=st["hits"] / sp.n_queries, inserts=st["inserts"], evictions=st["evictions"],
+                    cache_full_after_chunk=first_full, chunks=epochs,
+                    roofline={"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                              "frac": gbs / peaks["hbm_gbs"], "traffic": None,
+                              "note": "384 MiB of centroid slots per batch over the whole step time (the early batches sweep a partly empty cache)"})
     elif args.workload == "config5":
         sp = W.StreamSpec()
         stream = W.QueryStream(sp, threads=cores)
