@@ -32,7 +32,7 @@ def _worker(rank, world, port, out):
 def test_two_ranks_share_centroids_draw_own_queries_and_time_by_the_slowest():
     world = 2
     port = 29500 + os.getpid() % 2000
-    with mp.Manager() as mgr:
+    with mp.get_context("spawn").Manager() as mgr:
         out = mgr.dict()
         mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
         res = dict(out)

@@ -46,7 +46,7 @@ def _worker(rank, world, port, out):
 def test_two_ranks_gather_and_agree_on_the_global_top_k():
     world = 2
     port = 31500 + os.getpid() % 2000
-    with mp.Manager() as mgr:
+    with mp.get_context("spawn").Manager() as mgr:
         out = mgr.dict()
         mp.spawn(_worker, args=(world, port, out), nprocs=world, join=True)
         res = dict(out)
