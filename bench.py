@@ -44,6 +44,7 @@ def parse_args():
                     choices=["config4", "config1", "config2", "config3", "config5", "stream_probe", "cluster", "evict", "f32_lookup", "config5_full"],
                     help="config4 (default) is the benchmark contract; the others print one line each for the other "
                          "configurations (single GPU only)")
+    ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"], help="vector type of the cluster workload")
     ap.add_argument("--seed", type=int, default=0, help="seed of the configuration-5 stream (config5_full)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
@@ -468,9 +469,9 @@ def run_other(args):
         # stand-in for the query log that SISO-Cluster turns into centroids (Sec. 4.1): 131,072 unit vectors of dim 768
         # around 13,107 cluster means (the paper's 10 queries per centroid), clustered at theta_C = 0.86
         n, dim = (131072 if args.rows == (1 << 20) else args.rows), 768
-        w = W.config(3, threads=cores, n_centroids=n, dim=dim, n_clusters=max(2, n // 10), sigma=0.06)
-        cache = siso.SisoCache(64, dim, "f32")
-        v = to_dev(w.centroids, "f32")
+        w = W.config(3, threads=cores, n_centroids=n, dim=dim, n_clusters=max(2, n // 10), sigma=0.06, dtype=args.dtype)
+        cache = siso.SisoCache(64, dim, args.dtype)
+        v = to_dev(w.centroids, args.dtype)
         times, k = [], 0
         for it in range(max(3, steps // 4) + 1):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -483,13 +484,14 @@ def run_other(args):
             k = len(centres)
         ms = statistics.median(times)
         fl = float(n) * (n - 1) / 2 * dim * 2
-        tc_peak = peaks["bf16_tflops"] / 3.0
+        tc_peak = peaks["bf16_tflops"] / (3.0 if args.dtype == "f32" else 1.0)
         planted = int(len(np.unique(w.centroid_labels)))
-        line.update(metric=f"community detection, {n:,} x {dim} fp32 vectors, theta_C 0.86 (all pairs, order, founders, mean centroids)",
-                    value=n / ms * 1e3, unit="vectors/s", ms_per_step=ms, communities=k, planted_clusters=planted, dtype="f32",
+        line.update(metric=f"community detection, {n:,} x {dim} {args.dtype} vectors, theta_C 0.86 (all pairs, order, founders, mean centroids)",
+                    value=n / ms * 1e3, unit="vectors/s", ms_per_step=ms, communities=k, planted_clusters=planted, dtype=args.dtype,
                     roofline={"bound": "tensor", "achieved": fl / ms / 1e9, "peak": tc_peak, "unit": "TFLOP/s",
                               "frac": fl / ms / 1e9 / tc_peak, "traffic": None,
-                              "peak_kind": "measured bf16 burst peak / 3 (split-bf16 emulation of fp32 products)"})
+                              "peak_kind": "measured bf16 burst peak / 3 (split-bf16 emulation of fp32 products)"
+                              if args.dtype == "f32" else "measured bf16 burst peak"})
     elif args.workload == "config5_full":
         # the whole stream of configuration 5 from an empty cache: 10,000,000 queries in micro-batches of 256, popularity
         # reshuffled every 1,000,000 queries.  Queries are generated a million at a time on the host (not timed), copied

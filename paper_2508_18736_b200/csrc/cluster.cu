@@ -227,7 +227,8 @@ siso_status_t launch_cluster(Cache *c, const void *vecs, int64_t n, float theta_
     SISO_CUDA(cudaMemsetAsync(member_count, 0, sizeof(uint32_t) * n1, s));
 
     // all pairs j < i above the threshold
-    SISO_TRY(launch_pair_sweep_tensor(c, &scr, X, n, n, all_live, nullptr, theta_c, ctl, cand, max_cand, nullptr, s));
+    SISO_TRY(launch_pair_sweep_tensor(c, &scr, X, n, n, all_live, nullptr, theta_c, ctl, cand, max_cand, nullptr, s,
+                                      c->dtype == SISO_BF16 ? vecs : nullptr));
     cluster_check_kernel<<<1, 1, 0, s>>>(ctl, c->status);
     SISO_LAUNCHED(c);
     // visiting order

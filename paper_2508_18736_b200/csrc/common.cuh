@@ -133,7 +133,7 @@ size_t merge_tensor_scratch_bytes(const Cache *c);
 size_t pair_sweep_tensor_scratch_bytes(int64_t n, int64_t rows, int dim);
 siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, int64_t N, int64_t rows, const uint8_t *valid,
                                        const uint8_t *seed, float theta_c, void *ctl, void *cand, size_t max_cand,
-                                       uint32_t *row_count, cudaStream_t s);
+                                       uint32_t *row_count, cudaStream_t s, const void *rows_bf16);
 siso_status_t launch_merge_resolve(Cache *c, void *ctl, int64_t N, const uint8_t *valid, const uint8_t *seed,
                                    const uint32_t *row_off, const uint32_t *row_count, const int32_t *csr_j,
                                    const float *csr_sim, uint8_t *state, int32_t *target, unsigned int *undecided,

@@ -68,7 +68,7 @@ __device__ __forceinline__ void pair_to_tiles(const uint32_t *__restrict__ pair_
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CUtensorMap map_lo,
                           const uint8_t *__restrict__ valid, const uint8_t *__restrict__ seed, int64_t N, int D,
-                          const uint32_t *__restrict__ pair_list, long long n_pairs, float theta_filter, MergeCtlView *ctl,
+                          const uint32_t *__restrict__ pair_list, long long n_pairs, float theta_filter, int split, MergeCtlView *ctl,
                           MergeCandidate *__restrict__ cand, unsigned long long max_cand, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *stage_mem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
@@ -118,11 +118,12 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
                     if (!mbar_wait(&sh->empty[stage], phase ^ 1u, abort_flag)) { ok = false; break; }
                     uint8_t *dst = stage_mem + stage * STAGE_BYTES;
                     const uint32_t full_leader = cluster_addr(smem_u32(&sh->full[stage]), 0);
-                    if (rank == 0) mbar_arrive_expect_tx(&sh->full[stage], 2 * STAGE_BYTES);
+                    // bf16 inputs have no second part: only the hi tiles are loaded and one MMA per K step is issued
+                    if (rank == 0) mbar_arrive_expect_tx(&sh->full[stage], split ? 2 * STAGE_BYTES : STAGE_BYTES);
                     tma_load_2d_pair(dst, &map_hi, ks * TK, i0, full_leader);
-                    tma_load_2d_pair(dst + OPER_BYTES, &map_lo, ks * TK, i0, full_leader);
+                    if (split) tma_load_2d_pair(dst + OPER_BYTES, &map_lo, ks * TK, i0, full_leader);
                     tma_load_2d_pair(dst + 2 * OPER_BYTES, &map_hi, ks * TK, n0, full_leader);
-                    tma_load_2d_pair(dst + 3 * OPER_BYTES, &map_lo, ks * TK, n0, full_leader);
+                    if (split) tma_load_2d_pair(dst + 3 * OPER_BYTES, &map_lo, ks * TK, n0, full_leader);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -146,8 +147,10 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
                     for (int kk = 0; kk < TK / 16; ++kk) {
                         const uint64_t o = static_cast<uint64_t>(2 * kk);
                         umma_bf16_pair(d_tmem, a_hi + o, b_hi + o, IDESC, (ks | kk) ? 1u : 0u);
-                        umma_bf16_pair(d_tmem, a_hi + o, b_lo + o, IDESC, 1u);
-                        umma_bf16_pair(d_tmem, a_lo + o, b_hi + o, IDESC, 1u);
+                        if (split) {
+                            umma_bf16_pair(d_tmem, a_hi + o, b_lo + o, IDESC, 1u);
+                            umma_bf16_pair(d_tmem, a_lo + o, b_hi + o, IDESC, 1u);
+                        }
                     }
                     umma_commit_both(&sh->empty[stage]);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
@@ -365,14 +368,15 @@ size_t pair_sweep_tensor_scratch_bytes(int64_t n, int64_t rows, int dim) {
 }
 size_t merge_tensor_scratch_bytes(const Cache *c) { return pair_sweep_tensor_scratch_bytes(c->capacity, c->rows_alloc, c->dim); }
 
-// Sweep + exact check over the rows of X ([rows, dim] fp32, the first N of them taking part, `valid` [N] saying which
+// Sweep + exact check over the rows of X ([rows, dim] fp32; if the values are in fact bf16 values, `rows_bf16` is the
+// same matrix in bf16 and the sweep needs one MMA per K step instead of three; the first N rows take part, `valid` [N] saying which
 // are live, `seed` [N] or NULL marking the members of C_cur).  `ctl` and `row_count` are zeroed (or carry the two-set
 // insertion's failure flag); on return (in stream order) cand[0 .. min(n_cand, max_cand)) holds the provisional
 // pairs, the confirmed ones with their exact similarity and i >= 0, and row_count[i] (if not NULL) counts the
 // confirmed pairs of row i.
 siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, int64_t N, int64_t rows, const uint8_t *valid,
                                        const uint8_t *seed, float theta_c, void *ctl, void *cand, size_t max_cand,
-                                       uint32_t *row_count, cudaStream_t s) {
+                                       uint32_t *row_count, cudaStream_t s, const void *rows_bf16) {
     static tcm::EncodeTiledFn encode = nullptr;
     if (!encode) {
         void *fn = nullptr;
@@ -382,11 +386,18 @@ siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, i
         encode = reinterpret_cast<tcm::EncodeTiledFn>(fn);
     }
     const size_t elems = static_cast<size_t>(rows) * c->dim;
-    __nv_bfloat16 *hi = scr->take<__nv_bfloat16>(elems);
-    __nv_bfloat16 *lo = scr->take<__nv_bfloat16>(elems);
-    const long long n4 = static_cast<long long>(elems / 4);
-    tcm::split_bf16_kernel<<<static_cast<unsigned>((n4 + 255) / 256), 256, 0, s>>>(X, hi, lo, n4);
-    SISO_LAUNCHED(c);
+    const int split = rows_bf16 ? 0 : 1;           // rows that ARE bf16 values need no second part
+    const __nv_bfloat16 *hi, *lo;
+    if (split) {
+        __nv_bfloat16 *h = scr->take<__nv_bfloat16>(elems), *l = scr->take<__nv_bfloat16>(elems);
+        const long long n4 = static_cast<long long>(elems / 4);
+        tcm::split_bf16_kernel<<<static_cast<unsigned>((n4 + 255) / 256), 256, 0, s>>>(X, h, l, n4);
+        SISO_LAUNCHED(c);
+        hi = h;
+        lo = l;
+    } else {
+        hi = lo = static_cast<const __nv_bfloat16 *>(rows_bf16);
+    }
     CUtensorMap map_hi, map_lo;
     SISO_TRY(tcm::encode_rows_map(encode, &map_hi, hi, static_cast<uint64_t>(rows), static_cast<uint64_t>(c->dim)));
     SISO_TRY(tcm::encode_rows_map(encode, &map_lo, lo, static_cast<uint64_t>(rows), static_cast<uint64_t>(c->dim)));
@@ -410,7 +421,7 @@ siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, i
         c->merge_tensor_attr_set = true;
     }
     tcm::merge_sweep_tensor_kernel<<<static_cast<unsigned>(2 * used), tcm::THREADS, tcm::SMEM_BYTES, s>>>(
-        map_hi, map_lo, valid, seed, N, c->dim, pair_list, n_pairs, theta_c - tcm::FILTER_MARGIN,
+        map_hi, map_lo, valid, seed, N, c->dim, pair_list, n_pairs, theta_c - tcm::FILTER_MARGIN, split,
         static_cast<MergeCtlView *>(ctl), static_cast<MergeCandidate *>(cand), max_cand, c->status);
     SISO_LAUNCHED(c);
     tcm::merge_verify_kernel<<<8 * c->sm_count, 256, 0, s>>>(static_cast<const MergeCtlView *>(ctl), X, c->dim, theta_c,
@@ -422,7 +433,7 @@ siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, i
 siso_status_t launch_merge_sweep_tensor(Cache *c, Scratch *scr, const uint8_t *seed, float theta_c, void *ctl, void *cand,
                                         size_t max_cand, uint32_t *row_count, cudaStream_t s) {
     return launch_pair_sweep_tensor(c, scr, c->master, c->capacity, c->rows_alloc, c->valid, seed, theta_c, ctl, cand, max_cand,
-                                    row_count, s);
+                                    row_count, s, nullptr);
 }
 
 }  // namespace siso

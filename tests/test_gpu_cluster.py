@@ -23,6 +23,7 @@ def near_threshold(vecs, theta, tol):
     ("f32", "P", 0.86, 1500, 136),      # spread clusters: neighbourhoods overlap, founders compete
     ("f32", "T", 0.90, 2300, 64),       # tight clusters
     ("bf16", "P", 0.80, 1300, 200),
+    ("bf16", "T", 0.88, 2900, 768),     # bf16 rows go to the tensor cores as they are (one product per pair of elements)
     ("f32", "L", 0.30, 700, 24),        # loose: long chains of dependent decisions
     ("f32", "P", 0.86, 5, 8),           # smaller than one tile
 ])
