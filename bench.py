@@ -41,7 +41,7 @@ def parse_args():
     ap.add_argument("--queries", type=int, default=8192, help="query batch per step")
     ap.add_argument("--path", default="auto", choices=["auto", "simt", "tensor", "stream"])
     ap.add_argument("--workload", default="config4",
-                    choices=["config4", "config1", "config2", "config3", "config5", "stream_probe", "cluster", "evict", "f32_lookup", "config5_full"],
+                    choices=["config4", "config1", "config2", "config3", "config5", "stream_probe", "cluster", "evict", "f32_lookup", "config5_full", "tiered"],
                     help="config4 (default) is the benchmark contract; the others print one line each for the other "
                          "configurations (single GPU only)")
     ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"], help="vector type of the cluster workload")
@@ -435,6 +435,39 @@ def run_other(args):
                               "frac": fl / ms / 1e9 / tc_peak, "traffic": None,
                               "peak_kind": "measured bf16 burst peak / 3 (split-bf16 emulation of fp32 products)",
                               "fp32_alu_peak": fp32_peak})
+    elif args.workload == "tiered":
+        # locality-ordered exact search (the exact counterpart of the Sec. 4.3 placement): a merged cache of 524,288 x 1024
+        # bf16 centroids (one per cluster, 1 GiB), cluster_size grown by 8 batches of hits, hot tier = the 1/16 of the
+        # entries FilteringCentroids would evict last; batches of 8,192 queries (Zipf 1.0, 20 % out of distribution)
+        N = 524288 if args.rows == (1 << 20) else args.rows
+        B, D, warm_batches = args.queries, 1024, 8
+        w = W.config(4, threads=cores, n_centroids=16, n_queries=B * (warm_batches + 1), dim=D, n_clusters=N)
+        cent = W.f32_to_bf16_bits(W.unit_gaussian_rows(N, D, 0, W._TAG_MEANS, cores))      # the cluster means themselves
+        cache = siso.SisoCache(N, D, "bf16")
+        fill(cache, cent, "bf16")
+        q_all, th_all = to_dev(w.queries, "bf16"), torch.from_numpy(w.theta).to(dev)
+        for t in range(warm_batches):
+            qb, tb = q_all[t * B:(t + 1) * B], th_all[t * B:(t + 1) * B]
+            idx, sim, hit = cache.lookup(qb, tb, 1)
+            cache.update(qb, idx, hit)
+        # MergeCentroids at 0.5 finds nothing to merge: every pair of entries is at most 0.5 similar (checked in fp64)
+        sep = 0.5
+        _, merged = cache.merge(sep, siso.MERGE_WEIGHTED_MEAN)
+        assert merged == 0, merged
+        tiers = siso.TieredCache(cache, N // 16, sep + 4e-3, 2e-3)          # bf16 rounding of the fp32 masters: 4e-3, norms 2e-3
+        q, th = q_all[warm_batches * B:], th_all[warm_batches * B:]
+        ms_full = time_ms(lambda: cache.lookup(q, th, 1), steps, warm)
+        ms = time_ms(lambda: tiers.lookup(q, th), steps, warm)
+        a, b = cache.lookup(q, th, 1), tiers.lookup(q, th)
+        same = bool((a[0][:, 0] == b[0]).all().item() and (a[2] == b[2]).all().item())
+        n_go = B - tiers.settled
+        fl = 2.0 * D * (B * tiers.n_hot + n_go * tiers.n_cold)
+        line.update(metric=f"lookup queries/s, locality-ordered exact search, {N:,} x {D} bf16, hot tier {tiers.n_hot:,}, batch {B:,}, top-1",
+                    value=B / ms * 1e3, unit=UNIT, ms_per_step=ms, whole_cache_ms=ms_full, speedup=ms_full / ms,
+                    ended_in_hot_tier=tiers.settled / B, exit_similarity=tiers.exit_sim, equal_to_whole_cache_lookup=same, dtype="bf16",
+                    roofline={"bound": "tensor", "achieved": fl / ms / 1e9, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
+                              "frac": fl / ms / 1e9 / peaks["bf16_tflops"], "traffic": None,
+                              "note": "products actually computed (all queries x hot tier + remaining queries x cold tier)"})
     elif args.workload == "evict":
         # FilteringCentroids on the configuration-5 cache: the 256 lowest (cluster_size, access_count, last_access, slot)
         # keys of 262,144 entries, then the decay pass; entries are put back between calls

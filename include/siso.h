@@ -219,6 +219,33 @@ siso_status_t siso_lookup_keys(siso_cache_t *c, const void *d_queries, int64_t n
 siso_status_t siso_combine_keys(const uint64_t *d_keys, int64_t n_queries, int32_t n_lists, int32_t k, const float *d_theta,
                                 float theta_scalar, int64_t *d_idx, float *d_sim, uint8_t *d_hit, void *stream);
 
+/* Locality-ordered exact search, k = 1 (the exact-search counterpart of Sec. 4.3, "Searching for vectors in semantic
+ * cache": entries with strong semantic locality are searched first and most queries end there).  The cache is held as
+ * two handles: a small hot tier and the cold rest.  A query whose best hot similarity s exceeds exit_sim needs no cold
+ * search: if every hot/cold pair of entries has similarity <= sep, then by the triangle inequality on angles no cold
+ * entry can reach s once angle(q, hot) < acos(sep) / 2.  The result equals the top-1 over the whole cache.
+ *   siso_tier_exit_sim  (host arithmetic) the exit similarity for a separation bound `sep_sim` when all norms lie in
+ *                       [1 - norm_slack, 1 + norm_slack]; includes 1e-5 for the rounding of computed similarities;
+ *                       +infinity when no exit is possible (sep too close to 1, bad arguments).
+ *   siso_tier_select    d_hot_keys [n_queries] = siso_lookup_keys(hot tier, k = 1, slot_offset 0).  d_rows [n_queries]
+ *                       receives, ascending, the rows whose key is 0 or whose similarity is not above exit_sim;
+ *                       *d_count (device int64) their number; d_cold_queries [n_queries, row_bytes] those rows of
+ *                       d_queries, densely packed (row_bytes = dim * element size, a multiple of 16).
+ *   siso_tier_finish    d_cold_keys [n_cold] = siso_lookup_keys(cold tier, k = 1, slot_offset 0) of the packed rows;
+ *                       d_hot_slot / d_cold_slot (device int32, or NULL for identity) map a tier's slot to the slot
+ *                       reported; per query the better of the two keys (ties to the lower reported slot) gives
+ *                       d_idx [n_queries] (int32, -1 where both tiers are empty), d_sim, and d_hit by the strict
+ *                       threshold test (d_theta per query, or theta_scalar if NULL).  exit_sim as given to select.
+ * All device pointers, no handle, current device, asynchronous on `stream`; the caller reads *d_count (one 8-byte copy)
+ * to size the cold lookup.  SISO_ERR_INVALID_ARG on bad sizes or NULL pointers, nothing written. */
+double siso_tier_exit_sim(double sep_sim, double norm_slack);
+siso_status_t siso_tier_select(const uint64_t *d_hot_keys, int64_t n_queries, float exit_sim, const void *d_queries,
+                               int64_t row_bytes, void *d_cold_queries, int32_t *d_rows, int64_t *d_count, void *stream);
+siso_status_t siso_tier_finish(const uint64_t *d_hot_keys, int64_t n_queries, float exit_sim, const uint64_t *d_cold_keys,
+                               const int32_t *d_rows, int64_t n_cold, const int32_t *d_hot_slot, const int32_t *d_cold_slot,
+                               const float *d_theta, float theta_scalar, int32_t *d_idx, float *d_sim, uint8_t *d_hit,
+                               void *stream);
+
 /* Algorithm 1 as a whole (Sec. 4.2): C_new <- MergeCentroids(C_cur, C_repo, theta_C); C_new <- FilteringCentroids(C_new, M);
  * UpdateCentroids(C_cur, C_new).  With a second handle as C_new the steps are
  *     siso_cache_copy(c_new, cur)                       "C_new <- C_cur", the first line of MergeCentroids

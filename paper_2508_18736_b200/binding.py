@@ -22,7 +22,7 @@ EXPORTS = ["siso_cache_create", "siso_cache_destroy", "siso_set_option", "siso_i
            "siso_lookup_host", "siso_update", "siso_merge", "siso_evict", "siso_make_room", "siso_insert_misses",
            "siso_stream_step", "siso_export", "siso_import", "siso_get_stats", "siso_sync_status",
            "siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_lookup_small_noalloc", "siso_cluster", "siso_cache_copy", "siso_update_centroids", "siso_lookup_keys", "siso_combine_keys", "siso_t2h", "siso_md1_wait",
-           "siso_choose_theta", "siso_correct_theta"]
+           "siso_choose_theta", "siso_correct_theta", "siso_tier_exit_sim", "siso_tier_select", "siso_tier_finish"]
 
 
 class SisoError(RuntimeError):
@@ -79,6 +79,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_cache_copy.argtypes = [vp, vp, vp]
     L.siso_update_centroids.argtypes = [vp, vp, i64, i64, vp]
     L.siso_cluster.argtypes = [vp, vp, i64, f32, vp, vp, vp, vp, ctypes.POINTER(i64), vp]
+    L.siso_tier_exit_sim.argtypes = [ctypes.c_double] * 2
+    L.siso_tier_exit_sim.restype = ctypes.c_double
+    L.siso_tier_select.argtypes = [vp, i64, f32, vp, i64, vp, vp, vp, vp]
+    L.siso_tier_finish.argtypes = [vp, i64, f32, vp, vp, i64, vp, vp, vp, f32, vp, vp, vp, vp]
     L.siso_md1_wait.argtypes = [ctypes.c_double] * 3
     L.siso_md1_wait.restype = ctypes.c_double
     L.siso_choose_theta.argtypes = [vp, vp, i32, ctypes.c_double, ctypes.c_double, ctypes.c_double,
@@ -95,7 +99,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_last_cuda_error.argtypes = []
     L.siso_last_cuda_error.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name not in ("siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_md1_wait"):
+        if name not in ("siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_md1_wait", "siso_tier_exit_sim"):
             getattr(L, name).restype = i32
     if path is None:
         _lib = L
@@ -384,6 +388,48 @@ def combine_keys(keys: torch.Tensor, theta, stream=None) -> Tuple[torch.Tensor, 
                                               _stream(stream))
     if st != 0:
         raise SisoError(st, "siso_combine_keys")
+    return idx, sim, hit
+
+
+def tier_exit_sim(sep_sim: float, norm_slack: float = 0.0) -> float:
+    """Exit similarity of the locality-ordered search for a hot/cold separation bound (see siso_tier_exit_sim)."""
+    return float(load_library().siso_tier_exit_sim(float(sep_sim), float(norm_slack)))
+
+
+def tier_select(hot_keys: torch.Tensor, queries: torch.Tensor, exit_sim: float, stream=None):
+    """hot_keys [n] or [n, 1] packed keys, queries [n, dim] -> (rows [n] int32, packed queries [n, dim], count [1] int64
+    on the device): the queries that must also search the cold tier (see siso_tier_select)."""
+    hk = hot_keys.reshape(-1).contiguous()
+    q = queries.contiguous()
+    n = q.shape[0]
+    assert hk.dtype == torch.int64 and hk.numel() == n and q.is_cuda
+    rows = torch.empty((n,), dtype=torch.int32, device=q.device)
+    packed = torch.empty_like(q)
+    count = torch.empty((1,), dtype=torch.int64, device=q.device)
+    with torch.cuda.device(q.device):
+        st = load_library().siso_tier_select(_ptr(hk), n, float(exit_sim), _ptr(q), q.shape[1] * q.element_size(), _ptr(packed),
+                                             _ptr(rows), _ptr(count), _stream(stream))
+    if st != 0:
+        raise SisoError(st, "siso_tier_select")
+    return rows, packed, count
+
+
+def tier_finish(hot_keys: torch.Tensor, exit_sim: float, cold_keys: Optional[torch.Tensor], rows: torch.Tensor, n_cold: int,
+                hot_slot: Optional[torch.Tensor], cold_slot: Optional[torch.Tensor], theta, stream=None):
+    """-> (idx [n] int32, sim [n] fp32, hit [n] uint8): per query the better of its hot and cold keys (see siso_tier_finish)."""
+    hk = hot_keys.reshape(-1).contiguous()
+    n = hk.numel()
+    ck = None if cold_keys is None else cold_keys.reshape(-1).contiguous()
+    th_t, th_s = (theta.to(device=hk.device, dtype=torch.float32).contiguous(), 0.0) \
+        if isinstance(theta, torch.Tensor) else (None, float(theta))
+    idx = torch.empty((n,), dtype=torch.int32, device=hk.device)
+    sim = torch.empty((n,), dtype=torch.float32, device=hk.device)
+    hit = torch.empty((n,), dtype=torch.uint8, device=hk.device)
+    with torch.cuda.device(hk.device):
+        st = load_library().siso_tier_finish(_ptr(hk), n, float(exit_sim), _ptr(ck), _ptr(rows), int(n_cold), _ptr(hot_slot),
+                                             _ptr(cold_slot), _ptr(th_t), th_s, _ptr(idx), _ptr(sim), _ptr(hit), _stream(stream))
+    if st != 0:
+        raise SisoError(st, "siso_tier_finish")
     return idx, sim, hit
 
 
