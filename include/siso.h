@@ -219,6 +219,33 @@ siso_status_t siso_lookup_keys(siso_cache_t *c, const void *d_queries, int64_t n
 siso_status_t siso_combine_keys(const uint64_t *d_keys, int64_t n_queries, int32_t n_lists, int32_t k, const float *d_theta,
                                 float theta_scalar, int64_t *d_idx, float *d_sim, uint8_t *d_hit, void *stream);
 
+/* Maintenance of a cache partitioned across GPUs: updates, insertions and evictions go to the shard that owns the slot,
+ * and the whole behaves as one cache over the global slots (same victims, same slots for new entries).
+ *   siso_route         no handle.  From the combined result of a batch (d_idx int64 global slots read with stride idx_stride,
+ *                      d_hit [n]) what the shard owning global slots [slot_lo, slot_hi) has to do: d_idx_local [n] (local
+ *                      slot of a hit on its rows, else -1) and d_update_hit [n] (1 there, else 0) are the arguments of
+ *                      siso_update, which every shard calls once per batch so that the clocks agree; d_insert_hit [n] is
+ *                      the d_hit argument of siso_insert_misses: 0 exactly for the misses number miss_skip ..
+ *                      miss_skip + miss_take - 1, counted in ascending row order (the misses that land in this shard's
+ *                      free slots when the shards before it have miss_skip free slots and it has miss_take).
+ *   siso_evict_keys    the n lowest entries of this shard in FilteringCentroids order, ascending, as keys of three
+ *                      64-bit words [n, 3] (order-preserving cluster_size; access_count and last_access; last_access and
+ *                      slot + slot_offset), padded with all-ones words where the shard holds fewer; nothing is evicted.
+ *   siso_select_evict  no handle.  d_keys [n_lists, n, 3], every list as siso_evict_keys wrote it: the n_take lowest of
+ *                      all keys give d_victims [n_take] (int64 global slots in eviction order, -1 padding).  n_take <= n
+ *                      makes the result the exact global selection.
+ *   siso_evict_slots   drops the victims that lie in [slot_offset, slot_offset + capacity) from this shard (others are
+ *                      ignored), then the decay pass if SISO_EVICT_DECAY is set.
+ * All asynchronous on `stream`; device pointers. */
+siso_status_t siso_route(const int64_t *d_idx, int64_t idx_stride, const uint8_t *d_hit, int64_t n, int64_t slot_lo,
+                         int64_t slot_hi, int64_t miss_skip, int64_t miss_take, int32_t *d_idx_local, uint8_t *d_update_hit,
+                         uint8_t *d_insert_hit, void *stream);
+siso_status_t siso_evict_keys(siso_cache_t *c, int64_t n, int64_t slot_offset, uint64_t *d_keys, void *stream);
+siso_status_t siso_select_evict(const uint64_t *d_keys, int32_t n_lists, int64_t n, int64_t n_take, int64_t *d_victims,
+                                void *stream);
+siso_status_t siso_evict_slots(siso_cache_t *c, const int64_t *d_victims, int64_t n, int64_t slot_offset, uint32_t flags,
+                               void *stream);
+
 /* Locality-ordered exact search, k = 1 (the exact-search counterpart of Sec. 4.3, "Searching for vectors in semantic
  * cache": entries with strong semantic locality are searched first and most queries end there).  The cache is held as
  * two handles: a small hot tier and the cold rest.  A query whose best hot similarity s exceeds exit_sim needs no cold

@@ -22,7 +22,8 @@ EXPORTS = ["siso_cache_create", "siso_cache_destroy", "siso_set_option", "siso_i
            "siso_lookup_host", "siso_update", "siso_merge", "siso_evict", "siso_make_room", "siso_insert_misses",
            "siso_stream_step", "siso_export", "siso_import", "siso_get_stats", "siso_sync_status",
            "siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_lookup_small_noalloc", "siso_cluster", "siso_cache_copy", "siso_update_centroids", "siso_lookup_keys", "siso_combine_keys", "siso_t2h", "siso_md1_wait",
-           "siso_choose_theta", "siso_correct_theta", "siso_tier_exit_sim", "siso_tier_select", "siso_tier_finish"]
+           "siso_choose_theta", "siso_correct_theta", "siso_tier_exit_sim", "siso_tier_select", "siso_tier_finish",
+           "siso_route", "siso_evict_keys", "siso_select_evict", "siso_evict_slots"]
 
 
 class SisoError(RuntimeError):
@@ -79,6 +80,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_cache_copy.argtypes = [vp, vp, vp]
     L.siso_update_centroids.argtypes = [vp, vp, i64, i64, vp]
     L.siso_cluster.argtypes = [vp, vp, i64, f32, vp, vp, vp, vp, ctypes.POINTER(i64), vp]
+    L.siso_route.argtypes = [vp, i64, vp, i64, i64, i64, i64, i64, vp, vp, vp, vp]
+    L.siso_evict_keys.argtypes = [vp, i64, i64, vp, vp]
+    L.siso_select_evict.argtypes = [vp, i32, i64, i64, vp, vp]
+    L.siso_evict_slots.argtypes = [vp, vp, i64, i64, u32, vp]
     L.siso_tier_exit_sim.argtypes = [ctypes.c_double] * 2
     L.siso_tier_exit_sim.restype = ctypes.c_double
     L.siso_tier_select.argtypes = [vp, i64, f32, vp, i64, vp, vp, vp, vp]
@@ -282,6 +287,18 @@ class SisoCache:
                     "siso_lookup_keys")
         return keys
 
+    def evict_keys(self, n: int, slot_offset: int = 0, stream=None) -> torch.Tensor:
+        """This shard's n lowest entries in eviction order as keys [n, 3] (int64 tensor of the 64-bit words); see siso_evict_keys."""
+        keys = self._new((max(int(n), 0), 3), torch.int64)
+        self._check(self._lib.siso_evict_keys(self._h, int(n), int(slot_offset), _ptr(keys), _stream(stream)), "siso_evict_keys")
+        return keys
+
+    def evict_slots(self, victims: torch.Tensor, slot_offset: int = 0, flags: int = 0, stream=None) -> None:
+        """Drops the global victims that this shard holds (see siso_evict_slots)."""
+        v = victims.to(device=self._dev, dtype=torch.int64).contiguous()
+        self._check(self._lib.siso_evict_slots(self._h, _ptr(v), v.numel(), int(slot_offset), flags, _stream(stream)),
+                    "siso_evict_slots")
+
     def copy_from(self, src: "SisoCache", stream=None) -> None:
         """C_new <- C_cur (first line of MergeCentroids, Algorithm 1): every slot of `src` into the same slot here."""
         self._check(self._lib.siso_cache_copy(self._h, src._h, _stream(stream)), "siso_cache_copy")
@@ -389,6 +406,35 @@ def combine_keys(keys: torch.Tensor, theta, stream=None) -> Tuple[torch.Tensor, 
     if st != 0:
         raise SisoError(st, "siso_combine_keys")
     return idx, sim, hit
+
+
+def route(idx: torch.Tensor, hit: torch.Tensor, slot_lo: int, slot_hi: int, miss_skip: int, miss_take: int, stream=None):
+    """Combined (idx [n] or [n, k] int64 global slots, hit [n]) -> (idx_local [n] int32, update_hit [n], insert_hit [n]) for
+    the shard that owns [slot_lo, slot_hi) (see siso_route)."""
+    assert idx.dtype == torch.int64 and idx.is_cuda and hit.dtype == torch.uint8
+    idx, hit = idx.contiguous(), hit.contiguous()
+    n = hit.numel()
+    stride = 1 if idx.dim() == 1 else idx.shape[1]
+    idx_local = torch.empty((n,), dtype=torch.int32, device=idx.device)
+    upd, ins = torch.empty_like(hit), torch.empty_like(hit)
+    with torch.cuda.device(idx.device):
+        st = load_library().siso_route(_ptr(idx), stride, _ptr(hit), n, int(slot_lo), int(slot_hi), int(miss_skip), int(miss_take),
+                                       _ptr(idx_local), _ptr(upd), _ptr(ins), _stream(stream))
+    if st != 0:
+        raise SisoError(st, "siso_route")
+    return idx_local, upd, ins
+
+
+def select_evict(keys: torch.Tensor, n_take: int, stream=None) -> torch.Tensor:
+    """keys [n_lists, n, 3] (the shards' siso_evict_keys lists) -> victims [n_take] int64 global slots in eviction order."""
+    assert keys.dtype == torch.int64 and keys.dim() == 3 and keys.shape[2] == 3 and keys.is_cuda
+    keys = keys.contiguous()
+    victims = torch.empty((max(int(n_take), 0),), dtype=torch.int64, device=keys.device)
+    with torch.cuda.device(keys.device):
+        st = load_library().siso_select_evict(_ptr(keys), keys.shape[0], keys.shape[1], int(n_take), _ptr(victims), _stream(stream))
+    if st != 0:
+        raise SisoError(st, "siso_select_evict")
+    return victims
 
 
 def tier_exit_sim(sep_sim: float, norm_slack: float = 0.0) -> float:

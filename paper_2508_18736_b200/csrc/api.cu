@@ -357,6 +357,43 @@ siso_status_t siso_combine_keys(const uint64_t *d_keys, int64_t n_queries, int32
                                 theta_scalar, reinterpret_cast<long long *>(d_idx), d_sim, d_hit, static_cast<cudaStream_t>(stream));
 }
 
+siso_status_t siso_route(const int64_t *d_idx, int64_t idx_stride, const uint8_t *d_hit, int64_t n, int64_t slot_lo,
+                         int64_t slot_hi, int64_t miss_skip, int64_t miss_take, int32_t *d_idx_local, uint8_t *d_update_hit,
+                         uint8_t *d_insert_hit, void *stream) {
+    if (n < 0 || idx_stride < 1 || slot_lo < 0 || slot_hi < slot_lo || miss_skip < 0 || miss_take < 0) return SISO_ERR_INVALID_ARG;
+    if (slot_hi - slot_lo > 0x7FFFFFFFll) return SISO_ERR_UNSUPPORTED;
+    if (n == 0) return SISO_OK;
+    if (!d_idx || !d_hit || !d_idx_local || !d_update_hit || !d_insert_hit) return SISO_ERR_INVALID_ARG;
+    return launch_shard_route(reinterpret_cast<const long long *>(d_idx), idx_stride, d_hit, n, slot_lo, slot_hi, miss_skip,
+                              miss_take, d_idx_local, d_update_hit, d_insert_hit, static_cast<cudaStream_t>(stream));
+}
+
+siso_status_t siso_evict_keys(siso_cache_t *c, int64_t n, int64_t slot_offset, uint64_t *d_keys, void *stream) {
+    if (!c || n < 0 || slot_offset < 0) return SISO_ERR_INVALID_ARG;
+    if (slot_offset + c->capacity > 0xFFFFFFFFll) return SISO_ERR_UNSUPPORTED;
+    if (n == 0) return SISO_OK;
+    if (!d_keys) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    return launch_evict_keys(c, n, slot_offset, reinterpret_cast<unsigned long long *>(d_keys), static_cast<cudaStream_t>(stream));
+}
+
+siso_status_t siso_select_evict(const uint64_t *d_keys, int32_t n_lists, int64_t n, int64_t n_take, int64_t *d_victims,
+                                void *stream) {
+    if (n_lists < 1 || n < 0 || n_take < 0) return SISO_ERR_INVALID_ARG;
+    if (n_take == 0) return SISO_OK;
+    if (!d_victims || (n > 0 && !d_keys)) return SISO_ERR_INVALID_ARG;
+    return launch_evict_select(reinterpret_cast<const unsigned long long *>(d_keys), n_lists, n, n_take,
+                               reinterpret_cast<long long *>(d_victims), static_cast<cudaStream_t>(stream));
+}
+
+siso_status_t siso_evict_slots(siso_cache_t *c, const int64_t *d_victims, int64_t n, int64_t slot_offset, uint32_t flags,
+                               void *stream) {
+    if (!c || n < 0 || slot_offset < 0 || (n > 0 && !d_victims) || (flags & ~SISO_EVICT_DECAY)) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    return launch_evict_slots(c, reinterpret_cast<const long long *>(d_victims), n, slot_offset, flags,
+                              static_cast<cudaStream_t>(stream));
+}
+
 siso_status_t siso_cache_copy(siso_cache_t *dst, siso_cache_t *src, void *stream) {
     if (!dst || !src || dst == src) return SISO_ERR_INVALID_ARG;
     if (dst->dim != src->dim || dst->dtype != src->dtype || dst->device != src->device) return SISO_ERR_INVALID_ARG;

@@ -207,7 +207,8 @@ evict_collect_kernel(long long capacity, const double *__restrict__ size, const 
 // one warp per candidate
 __global__ void __launch_bounds__(256)
 evict_rank_kernel(EvictPlan *plan, const Key3 *__restrict__ cand, uint8_t *__restrict__ valid,
-                  int32_t *__restrict__ victims, long long *counters) {
+                  int32_t *__restrict__ victims, long long *counters, Key3 *__restrict__ keys_out, unsigned long long slot_offset,
+                  int apply) {
     const long long m = plan->m;
     if (m == 0) return;
     const unsigned int n = plan->n_cand;
@@ -222,10 +223,15 @@ evict_rank_kernel(EvictPlan *plan, const Key3 *__restrict__ cand, uint8_t *__res
         if (lane == 0 && rank < m) {
             const int32_t slot = static_cast<int32_t>(mine.w2 & 0xFFFFFFFFull);
             if (victims) victims[rank] = slot;
-            valid[slot] = 0;
+            if (keys_out) {                  // the key with the slot made global (slot + offset < 2^32: no carry into last_access)
+                Key3 k = mine;
+                k.w2 += slot_offset;
+                keys_out[rank] = k;
+            }
+            if (apply) valid[slot] = 0;
         }
     }
-    if (blockIdx.x == 0 && threadIdx.x == 0) {
+    if (apply && blockIdx.x == 0 && threadIdx.x == 0) {
         counters[CNT_OCCUPANCY] -= m;
         counters[CNT_EVICTIONS] += m;
     }
@@ -259,8 +265,104 @@ siso_status_t launch_evict(Cache *c, int64_t n_evict, const uint8_t *hit, int64_
     SISO_LAUNCHED(c);
     evict_collect_kernel<<<grid, 256, 0, s>>>(c->capacity, c->size, c->access, c->last, c->valid, plan, bucket, cand);
     SISO_LAUNCHED(c);
-    evict_rank_kernel<<<grid, 256, 0, s>>>(plan, cand, c->valid, victims, c->counters);
+    evict_rank_kernel<<<grid, 256, 0, s>>>(plan, cand, c->valid, victims, c->counters, nullptr, 0ull, 1);
     SISO_LAUNCHED(c);
+    if (flags & SISO_EVICT_DECAY) {
+        decay_kernel<<<static_cast<unsigned>((c->capacity + 255) / 256), 256, 0, s>>>(c->capacity, c->decay, c->size,
+                                                                                      c->access, c->valid);
+        SISO_LAUNCHED(c);
+    }
+    return SISO_OK;
+}
+
+// ---------------------------------------------------------------------------------------------
+// eviction over a cache partitioned across GPUs: every shard reports its n lowest keys (global slots), the n_take lowest
+// of all reported keys are the victims, every shard drops those it holds
+// ---------------------------------------------------------------------------------------------
+siso_status_t launch_evict_keys(Cache *c, int64_t n, int64_t slot_offset, unsigned long long *keys_out, cudaStream_t s) {
+    Scratch scr;
+    SISO_TRY(scratch_reserve(c, pad256(sizeof(EvictPlan)) + pad256(sizeof(Key3) * EV_SAMPLE) +
+                                    pad256(sizeof(uint16_t) * c->capacity) + pad256(sizeof(Key3) * c->capacity), s, &scr));
+    EvictPlan *plan = scr.take<EvictPlan>(1);
+    Key3 *splitters = scr.take<Key3>(EV_SAMPLE);
+    uint16_t *bucket = scr.take<uint16_t>(c->capacity);
+    Key3 *cand = scr.take<Key3>(c->capacity);
+    SISO_CUDA(cudaMemsetAsync(keys_out, 0xFF, sizeof(Key3) * n, s));           // padding: sorts after every real key
+    evict_sample_kernel<<<1, 1024, 0, s>>>(n, nullptr, 0, c->capacity, c->size, c->access, c->last, c->valid, c->counters, plan,
+                                           splitters, nullptr, 0);
+    SISO_LAUNCHED(c);
+    const int grid = static_cast<int>(std::min<int64_t>((c->capacity + 255) / 256, 4ll * c->sm_count));
+    const int grid_bucket = static_cast<int>(std::min<int64_t>((c->capacity + 255) / 256, 8ll * c->sm_count));
+    evict_bucket_kernel<<<grid_bucket, 256, 0, s>>>(c->capacity, c->size, c->access, c->last, c->valid, plan, splitters, bucket);
+    SISO_LAUNCHED(c);
+    evict_collect_kernel<<<grid, 256, 0, s>>>(c->capacity, c->size, c->access, c->last, c->valid, plan, bucket, cand);
+    SISO_LAUNCHED(c);
+    evict_rank_kernel<<<grid, 256, 0, s>>>(plan, cand, c->valid, nullptr, c->counters, reinterpret_cast<Key3 *>(keys_out),
+                                           static_cast<unsigned long long>(slot_offset), 0);
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
+
+namespace {
+
+// keys [n_lists, n] (Key3), every list ascending with all-ones padding; one thread per key: its rank among all keys is the
+// sum over the lists of the number of smaller keys there (binary search); the n_take lowest give victims[rank] = global slot
+__global__ void __launch_bounds__(256)
+evict_select_kernel(const Key3 *__restrict__ keys, int n_lists, long long n, long long n_take, long long *__restrict__ victims) {
+    const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (t >= n * n_lists) return;
+    const Key3 mine = keys[t];
+    if ((mine.w0 & mine.w1 & mine.w2) == ~0ull) return;
+    long long rank = 0;
+    for (int l = 0; l < n_lists; ++l) {
+        const Key3 *list = keys + static_cast<long long>(l) * n;
+        long long lo = 0, hi = n;                                  // first position whose key is not below mine
+        while (lo < hi) {
+            const long long mid = (lo + hi) >> 1;
+            if (key_less(list[mid], mine)) lo = mid + 1; else hi = mid;
+        }
+        rank += lo;
+    }
+    if (rank < n_take) victims[rank] = static_cast<long long>(mine.w2 & 0xFFFFFFFFull);
+}
+
+// one CTA: drops the victims that fall into [slot_offset, slot_offset + capacity)
+__global__ void __launch_bounds__(1024)
+evict_slots_kernel(const long long *__restrict__ victims, long long n, long long slot_offset, long long capacity,
+                   uint8_t *__restrict__ valid, long long *counters) {
+    __shared__ int warp_sum[32];
+    int dropped = 0;
+    for (long long i = threadIdx.x; i < n; i += 1024) {
+        const long long v = victims[i] - slot_offset;
+        if (victims[i] >= 0 && v >= 0 && v < capacity && valid[v]) {
+            valid[v] = 0;
+            ++dropped;
+        }
+    }
+    int total;
+    block_exclusive_scan_1024(dropped, &total, warp_sum);
+    if (threadIdx.x == 0) {
+        counters[CNT_OCCUPANCY] -= total;
+        counters[CNT_EVICTIONS] += total;
+    }
+}
+
+}  // namespace
+
+siso_status_t launch_evict_select(const unsigned long long *keys, int n_lists, int64_t n, int64_t n_take, long long *victims,
+                                  cudaStream_t s) {
+    SISO_CUDA(cudaMemsetAsync(victims, 0xFF, sizeof(long long) * n_take, s));  // -1: fewer live entries than asked for
+    if (n > 0)
+        evict_select_kernel<<<static_cast<unsigned>((n * n_lists + 255) / 256), 256, 0, s>>>(
+            reinterpret_cast<const Key3 *>(keys), n_lists, n, n_take, victims);
+    return check_cuda(cudaGetLastError(), "evict_select_kernel");
+}
+
+siso_status_t launch_evict_slots(Cache *c, const long long *victims, int64_t n, int64_t slot_offset, uint32_t flags, cudaStream_t s) {
+    if (n > 0) {
+        evict_slots_kernel<<<1, 1024, 0, s>>>(victims, n, slot_offset, c->capacity, c->valid, c->counters);
+        SISO_LAUNCHED(c);
+    }
     if (flags & SISO_EVICT_DECAY) {
         decay_kernel<<<static_cast<unsigned>((c->capacity + 255) / 256), 256, 0, s>>>(c->capacity, c->decay, c->size,
                                                                                       c->access, c->valid);

@@ -5,6 +5,10 @@
 // lower global slot, so that the combined result does not depend on the number of shards or on their order.
 //   pack     a shard's (idx, sim) lists -> keys with the shard's slot offset added
 //   combine  per query the k largest of n_lists * k keys -> global slot (int64), similarity, strict threshold test
+//   route    the combined (global slot, hit) of a batch -> what THIS shard has to do: the hits on its own rows as local
+//            slots (for the running-mean update), and the misses it stores: misses are numbered in ascending row order and
+//            take the free slots of the whole cache in ascending global order, so a shard with `take` free slots after
+//            `skip` free slots on the shards before it stores misses number skip .. skip + take - 1
 #include "common.cuh"
 
 namespace siso {
@@ -53,7 +57,47 @@ shard_combine_kernel(const unsigned long long *__restrict__ keys, long long n, i
     }
 }
 
+// one CTA
+__global__ void __launch_bounds__(1024)
+shard_route_kernel(const long long *__restrict__ idx, long long idx_stride, const uint8_t *__restrict__ hit, long long n,
+                   long long slot_lo, long long slot_hi, long long skip, long long take, int32_t *__restrict__ idx_local,
+                   uint8_t *__restrict__ upd_hit, uint8_t *__restrict__ ins_hit) {
+    __shared__ int warp_cnt[32];
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    long long base = 0;                                          // misses before this round, the same in every thread
+    for (long long b0 = 0; b0 < n; b0 += 1024) {
+        const long long b = b0 + tid;
+        const bool miss = b < n && hit[b] == 0;
+        const unsigned int ballot = __ballot_sync(0xFFFFFFFFu, miss);
+        if (lane == 0) warp_cnt[warp] = __popc(ballot);
+        __syncthreads();
+        int before = 0, total = 0;
+        for (int w = 0; w < 32; ++w) {
+            const int c = warp_cnt[w];
+            before += w < warp ? c : 0;
+            total += c;
+        }
+        if (b < n) {
+            const long long g = idx[b * idx_stride];
+            const bool mine = !miss && g >= slot_lo && g < slot_hi;
+            idx_local[b] = mine ? static_cast<int32_t>(g - slot_lo) : -1;
+            upd_hit[b] = mine ? 1 : 0;
+            const long long number = base + before + __popc(ballot & ((1u << lane) - 1u));
+            ins_hit[b] = (miss && number >= skip && number < skip + take) ? 0 : 1;      // 0 = store this row here
+        }
+        base += total;
+        __syncthreads();
+    }
+}
+
 }  // namespace
+
+siso_status_t launch_shard_route(const long long *idx, long long idx_stride, const uint8_t *hit, int64_t n, int64_t slot_lo,
+                                 int64_t slot_hi, int64_t skip, int64_t take, int32_t *idx_local, uint8_t *upd_hit,
+                                 uint8_t *ins_hit, cudaStream_t s) {
+    shard_route_kernel<<<1, 1024, 0, s>>>(idx, idx_stride, hit, n, slot_lo, slot_hi, skip, take, idx_local, upd_hit, ins_hit);
+    return check_cuda(cudaGetLastError(), "shard_route_kernel");
+}
 
 siso_status_t launch_shard_pack(Cache *c, const int32_t *idx, const float *sim, int64_t n, int64_t slot_offset,
                                 unsigned long long *keys, cudaStream_t s) {

@@ -63,3 +63,82 @@ def test_keys_of_an_empty_or_small_shard_and_bad_arguments():
     with pytest.raises(siso.SisoError):
         c.lookup_keys(to_dev(w.queries, "bf16"), 4, slot_offset=(1 << 32))      # global slots are 32-bit
     c.close()
+
+
+@pytest.mark.parametrize("dtype,total,dim,shards,batch,n_batches", [
+    ("bf16", 301, 72, 3, 96, 14),         # ragged last shard (101 + 101 + 99); the cache fills up and evicts
+    ("f32", 200, 64, 4, 130, 8),
+    ("bf16", 5, 64, 8, 3, 6),             # more ranks than rows: ranks 5-7 hold nothing; one row per rank
+])
+def test_sharded_stream_equals_one_cache(dtype, total, dim, shards, batch, n_batches):
+    """The owner-routed streaming step over several shards (driven in lockstep on one GPU, exchanges = stacks) against the
+    oracle's step over ONE cache of the same global slots: lookup, victims, slots of the stored misses, and the whole state."""
+    sp = W.StreamSpec(capacity=total, dim=dim, n_queries=batch * n_batches, batch=batch, n_clusters=max(8, 2 * total), zipf_s=1.1,
+                      reshuffle_every=batch * 5, theta=0.80, mode="P", dtype=dtype, seed=61)
+    stream = W.QueryStream(sp)
+    parts = [siso.ShardedCache(total, dim, dtype, rank=r, world=shards) for r in range(shards)]
+    ora = oracle.OracleCache(total, dim, dtype)
+    evicted = 0
+    for t in range(n_batches):
+        qn, _ = stream.batch(t)
+        theta = np.full(len(qn), sp.theta, np.float32)
+        q = to_dev(qn, dtype)
+        pre_copy, pre_valid = ora.lookup_copy(), ora.valid.copy()
+        res = siso.run_lockstep([p.stream_steps(q, float(sp.theta)) for p in parts])
+        for r in res[1:]:                                               # every rank holds the same answer
+            assert all((a == b).all().item() for a, b in zip(res[0], r))
+        idx, sim, hit, victims, slots = [x.cpu().numpy() for x in res[0]]
+        o_idx, o_sim, o_hit, o_victims, o_slots = ora.stream_step(qn, theta, forced=(idx[:, None].astype(np.int32), hit))
+        check_lookup((idx[:, None].astype(np.int32), sim[:, None], hit), (o_idx, o_sim, o_hit), pre_copy, qn, theta, TOL[dtype],
+                     valid=pre_valid)
+        assert (victims == o_victims[:len(victims)]).all() and len(victims) == (o_victims >= 0).sum()
+        assert (slots == o_slots).all()
+        evicted += len(victims)
+        # the shards' states, laid side by side, are the one cache's state
+        for p in parts:
+            if p.hi == p.lo:
+                assert p.local.stats()["occupancy"] == 0
+                continue
+            st = p.local.export()
+            sl = slice(p.lo, p.hi)
+            live = ora.valid[sl] == 1
+            assert (st["valid"].cpu().numpy() == ora.valid[sl]).all()
+            assert (st["size"].cpu().numpy()[live] == ora.size[sl][live]).all()
+            assert (st["access"].cpu().numpy().view(np.uint32)[live] == ora.access[sl][live]).all()
+            assert (st["last"].cpu().numpy().view(np.uint64)[live] == ora.last[sl][live]).all()
+            assert np.abs(st["master"].cpu().numpy()[live] - ora.master[sl][live]).max(initial=0) <= 1e-6
+    assert evicted > 0
+    for p in parts:
+        p.close()
+
+
+def test_sharded_eviction_is_the_global_selection():
+    """FilteringCentroids over shards: the victims are those of one cache, in the same order, with ties in cluster_size and
+    access count that only last_access and the global slot break; also asking for more than a shard (or the cache) holds."""
+    rng = np.random.default_rng(7)
+    total, dim, shards = 900, 64, 4
+    rows = rng.standard_normal((total, dim)).astype(np.float32)
+    rows /= np.linalg.norm(rows, axis=1, keepdims=True)
+    sizes = rng.integers(1, 4, total).astype(np.float64)              # many equal cluster sizes
+    parts = [siso.ShardedCache(total, dim, "f32", rank=r, world=shards) for r in range(shards)]
+    ora = oracle.OracleCache(total, dim, "f32")
+    ora.insert(rows, sizes=sizes)
+    for p in parts:
+        p.local.insert(torch.from_numpy(rows[p.lo:p.hi]).cuda(), torch.from_numpy(sizes[p.lo:p.hi]).cuda())
+    for m, decay in ((37, False), (300, True), (0, True), (700, False)):   # 300 > a shard's 225 rows; the last empties the cache
+        res = siso.run_lockstep([p.evict_steps(m, siso.EVICT_DECAY if decay else 0) for p in parts])
+        want = ora.evict(m, decay)
+        got = res[0].cpu().numpy()
+        assert all((r == res[0]).all().item() for r in res)
+        live_before = len(want[want >= 0])
+        assert (got[:live_before] == want[:live_before]).all() and (got[live_before:] == -1).all()
+        for p in parts:
+            st = p.local.export()
+            sl = slice(p.lo, p.hi)
+            live = ora.valid[sl] == 1
+            assert (st["valid"].cpu().numpy() == ora.valid[sl]).all()
+            assert (st["size"].cpu().numpy()[live] == ora.size[sl][live]).all()            # the decay reached every shard
+            assert (st["access"].cpu().numpy().view(np.uint32)[live] == ora.access[sl][live]).all()
+    assert sum(p.local.stats()["occupancy"] for p in parts) == 0 and sum(p.local.stats()["evictions"] for p in parts) == total
+    for p in parts:
+        p.close()

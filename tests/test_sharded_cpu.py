@@ -62,3 +62,44 @@ def test_two_ranks_gather_and_agree_on_the_global_top_k():
     want = np.lexsort((np.broadcast_to(np.arange(37), S.shape), -S), axis=1)[:, :3]
     assert res[0][3] == want.tolist()
     assert res[0][4] == [(int(i) // 19, int(i) % 19) for i in want[:, 0]]
+
+
+def _toy_steps(rank, value):
+    """A sharded operation in the library's form: a generator that yields its exchanges."""
+    all_v = yield ("gather", torch.tensor([value, rank], dtype=torch.int64))
+    top = yield ("max", torch.tensor([value * 2, -rank], dtype=torch.int64))
+    return all_v.tolist(), top.tolist()
+
+
+def _worker_run(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2508_18736_b200 import sharded
+    out[rank] = sharded.run(_toy_steps(rank, 10 + rank))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_the_two_drivers_of_a_sharded_operation_agree():
+    """run() does the exchanges with torch.distributed (two gloo ranks), run_lockstep() by stacking inside one process:
+    both must hand every shard the same gathered and reduced tensors."""
+    world = 2
+    port = 33500 + os.getpid() % 2000
+    with mp.get_context("spawn").Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_worker_run, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    sys.path.insert(0, ROOT)
+    from paper_2508_18736_b200 import sharded
+    want = ([[10, 0], [11, 1]], [22, 0])
+    assert res[0] == want and res[1] == want
+    assert sharded.run_lockstep([_toy_steps(r, 10 + r) for r in range(2)]) == [want, want]
+    # without a process group the world is this process alone
+    assert sharded.run(_toy_steps(0, 5)) == ([[5, 0]], [10, 0])
+
+    def nothing_to_do():
+        return 7
+        yield
+
+    assert sharded.run(nothing_to_do()) == 7 and sharded.run_lockstep([nothing_to_do(), nothing_to_do()]) == [7, 7]
