@@ -183,6 +183,255 @@ update_apply_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restric
     }
 }
 
+// The same work with one WARP per chunk, for dim = 128 * NQ <= 1024.  A first kernel lists the chunks (start, slot,
+// first and past-the-end position of the group) with one thread per position of the sorted hit list; then a grid of
+// resident warps walks that list.  Lane l owns the element quartets l, l + 32, ..., the running sums stay in registers
+// (fp64), the norm is a shuffle tree, nothing needs a CTA-wide barrier and no warp is launched only to find that it has
+// nothing to do.  Chunks, their scratch rows, the arrival counter and every order of addition are those of
+// update_apply_kernel; the order in which chunks are listed does not matter to any sum.
+constexpr int UPW_THREADS = 128;
+constexpr int UPW_SUPER = 16;            // chunks per run of the two-level combination
+
+__global__ void __launch_bounds__(256)
+update_chunks_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restrict__ rows, int64_t B, int64_t capacity, int chunk,
+                     int4 *__restrict__ desc, unsigned int *__restrict__ n_desc) {
+    const int64_t p = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const int lane = threadIdx.x & 31;
+    bool start = false;
+    uint32_t slot = 0xFFFFFFFFu;
+    int64_t head = p, gend = p;
+    if (p < B) {
+        slot = keys[p];
+        if (slot < capacity) {
+            const uint32_t left = p > 0 ? keys[p - 1] : 0xFFFFFFFFu;
+            if (left != slot) {
+                start = true;
+            } else if (p >= chunk && keys[p - chunk] == slot) {
+                // a long group: its first position, and whether this one is a whole number of chunks away from it
+                int64_t lo = 0, hi = p;
+                while (lo < hi) {
+                    const int64_t mid = (lo + hi) >> 1;
+                    if (keys[mid] < slot) lo = mid + 1; else hi = mid;
+                }
+                head = lo;
+                start = (p - head) % chunk == 0;
+            }
+        }
+    }
+    if (start) {
+        int64_t lo = p + 1, hi = B;            // first position past the group
+        while (lo < hi) {
+            const int64_t mid = (lo + hi) >> 1;
+            if (keys[mid] <= slot) lo = mid + 1; else hi = mid;
+        }
+        gend = lo;
+    }
+    // chunks of groups that span several chunks are listed from the front, the others from the back: the warps take
+    // the list front to back, so the long dependent chains (sum, publish, combine) start first and the short ones fill in
+    const bool multi = start && !(head == p && gend <= p + chunk);
+    const unsigned int ballot_m = __ballot_sync(0xFFFFFFFFu, multi), ballot_s = __ballot_sync(0xFFFFFFFFu, start && !multi);
+    if ((ballot_m | ballot_s) == 0u) return;
+    unsigned int base_m = 0, base_s = 0;
+    if (lane == 0) {
+        if (ballot_m) base_m = atomicAdd(&n_desc[0], static_cast<unsigned int>(__popc(ballot_m)));
+        if (ballot_s) base_s = atomicAdd(&n_desc[1], static_cast<unsigned int>(__popc(ballot_s)));
+    }
+    base_m = __shfl_sync(0xFFFFFFFFu, base_m, 0);
+    base_s = __shfl_sync(0xFFFFFFFFu, base_s, 0);
+    if (start) {
+        // two words of 16 bytes per chunk: where it is, and its first four rows (most chunks have no more)
+        const unsigned int below = (1u << lane) - 1u;
+        const unsigned int at = multi ? base_m + __popc(ballot_m & below)
+                                      : static_cast<unsigned int>(B) - 1u - (base_s + __popc(ballot_s & below));
+        int r[4];
+#pragma unroll
+        for (int x = 0; x < 4; ++x) r[x] = static_cast<int>(rows[p + x < gend ? p + x : p]);
+        desc[2 * at] = make_int4(static_cast<int>(p), static_cast<int>(slot), static_cast<int>(head), static_cast<int>(gend));
+        desc[2 * at + 1] = make_int4(r[0], r[1], r[2], r[3]);
+    }
+}
+
+template <typename T> struct Raw4;
+template <> struct Raw4<float> { using type = float4; };
+template <> struct Raw4<__nv_bfloat16> { using type = uint2; };
+__device__ __forceinline__ float4 widen4(float4 v) { return v; }
+__device__ __forceinline__ float4 widen4(uint2 u) {
+    return make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xFFFF0000u), __uint_as_float(u.y << 16),
+                       __uint_as_float(u.y & 0xFFFF0000u));
+}
+
+template <typename T, int NQ>
+__global__ void __launch_bounds__(UPW_THREADS, 4)
+update_apply_warp_kernel(const int4 *__restrict__ desc, unsigned int list_len, const unsigned int *__restrict__ n_desc,
+                         unsigned int *__restrict__ ticket,
+                         const uint32_t *__restrict__ rows,
+                         int chunk, const T *__restrict__ Q, float *__restrict__ master, T *__restrict__ vecs,
+                         double *__restrict__ size, uint32_t *__restrict__ access, unsigned long long *__restrict__ last,
+                         const long long *__restrict__ counters, double *__restrict__ partial,
+                         unsigned int *__restrict__ arrived, unsigned int *__restrict__ arrived_runs) {
+    using raw_t = typename Raw4<T>::type;
+    constexpr int D = 128 * NQ;
+    const int lane = threadIdx.x & 31;
+    const unsigned int n_front = n_desc[0], n = n_front + n_desc[1];
+    auto place = [&](unsigned int t) { return t < n_front ? t : list_len - 1u - (t - n_front); };      // ticket -> list entry
+    // chunks are handed out by a ticket counter (a long chunk delays nobody else); a warp draws its next ticket and
+    // requests that chunk's description before it sums the current one
+    auto draw = [&]() {
+        unsigned int t = 0;
+        if (lane == 0) t = atomicAdd(ticket, 1u);
+        return __shfl_sync(0xFFFFFFFFu, t, 0);
+    };
+    unsigned int i = draw();
+    if (i >= n) return;
+    int4 next = desc[2 * place(i)], next_rows = desc[2 * place(i) + 1];
+    while (i < n) {
+        const int4 d = next, dr = next_rows;
+        i = draw();
+        if (i < n) { next = desc[2 * place(i)]; next_rows = desc[2 * place(i) + 1]; }
+        const int64_t p = d.x, head = d.z, gend = d.w;
+        const uint32_t slot = static_cast<uint32_t>(d.y);
+        const bool is_head = p == head;
+        const bool more = gend > p + chunk;
+        const int64_t e = more ? p + chunk : gend;
+        const double n_old = size[slot];
+        const uint32_t access_old = access[slot];
+        float *m = master + static_cast<int64_t>(slot) * D;
+        double a[NQ][4];
+#pragma unroll
+        for (int j = 0; j < NQ; ++j) {
+            float4 m4 = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (is_head) m4 = *reinterpret_cast<const float4 *>(m + 4 * (lane + 32 * j));
+            a[j][0] = n_old * static_cast<double>(m4.x); a[j][1] = n_old * static_cast<double>(m4.y);
+            a[j][2] = n_old * static_cast<double>(m4.z); a[j][3] = n_old * static_cast<double>(m4.w);
+        }
+        // the rows four at a time: their loads are in flight together, additions stay in ascending row order
+        uint32_t rid[4] = {static_cast<uint32_t>(dr.x), static_cast<uint32_t>(dr.y), static_cast<uint32_t>(dr.z),
+                           static_cast<uint32_t>(dr.w)};
+        for (int64_t t = p; t < e; t += 4) {
+            const int nrow = static_cast<int>(e - t < 4 ? e - t : 4);
+            const raw_t *q[4];
+#pragma unroll
+            for (int r = 0; r < 4; ++r) q[r] = reinterpret_cast<const raw_t *>(Q + static_cast<int64_t>(rid[r]) * D) + lane;
+            if (t + 4 < e) {                                  // the next quartet's row numbers, requested with this one's rows
+#pragma unroll
+                for (int r = 0; r < 4; ++r) rid[r] = rows[t + 4 + r < e ? t + 4 + r : t + 4];
+            }
+#pragma unroll
+            for (int j = 0; j < NQ; ++j) {
+                raw_t v[4];
+#pragma unroll
+                for (int r = 0; r < 4; ++r) v[r] = __ldg(q[r] + 32 * j);
+#pragma unroll
+                for (int r = 0; r < 4; ++r) {
+                    if (r < nrow) {
+                        const float4 f = widen4(v[r]);
+                        a[j][0] += f.x; a[j][1] += f.y; a[j][2] += f.z; a[j][3] += f.w;
+                    }
+                }
+            }
+        }
+        long long count = e - p;
+        if (!(is_head && !more)) {
+            // several chunks: publish this chunk's sum.  Chunks are combined in two levels so that a centroid with thousands
+            // of hits is not one warp's serial work: the warp that arrives last among the UPW_SUPER chunks of a run adds
+            // that run up in chunk order; with several runs it publishes the run's sum (in the scratch row of the run's
+            // first chunk, which only it reads) and the warp that arrives last among the runs adds those up in order.
+            auto chunk_id = [&](int64_t cidx) { return cidx == 0 ? 2 * (head / chunk) + 1 : 2 * ((head + cidx * chunk) / chunk); };
+            auto publish = [&](double *dst_row) {
+#pragma unroll
+                for (int j = 0; j < NQ; ++j) {
+                    double2 *dst = reinterpret_cast<double2 *>(dst_row + 4 * (lane + 32 * j));
+                    dst[0] = make_double2(a[j][0], a[j][1]);
+                    dst[1] = make_double2(a[j][2], a[j][3]);
+                }
+            };
+            auto arrive = [&](unsigned int *counter, int64_t expected) {
+                __threadfence();
+                __syncwarp();
+                int is_last = 0;
+                if (lane == 0) is_last = (atomicAdd(counter, 1u) == static_cast<unsigned int>(expected - 1)) ? 1 : 0;
+                is_last = __shfl_sync(0xFFFFFFFFu, is_last, 0);
+                if (is_last) __threadfence();
+                return is_last != 0;
+            };
+            auto add_up = [&](int64_t first, int64_t stop, int64_t step) {      // rows of chunks first, first + step, ... < stop
+#pragma unroll
+                for (int j = 0; j < NQ; ++j) {
+                    const int64_t off = 4 * (lane + 32 * j);
+#pragma unroll
+                    for (int x = 0; x < 4; ++x) a[j][x] = __ldcg(&partial[chunk_id(first) * D + off + x]);
+                }
+                for (int64_t cidx = first + step; cidx < stop; cidx += step) {
+                    const double *src = partial + chunk_id(cidx) * D;
+#pragma unroll
+                    for (int j = 0; j < NQ; ++j) {
+                        const int64_t off = 4 * (lane + 32 * j);
+#pragma unroll
+                        for (int x = 0; x < 4; ++x) a[j][x] += __ldcg(&src[off + x]);
+                    }
+                }
+            };
+            const int64_t n_chunks = (gend - head + chunk - 1) / chunk;
+            const int64_t my_chunk = (p - head) / chunk;
+            const int64_t run = my_chunk / UPW_SUPER, n_runs = (n_chunks + UPW_SUPER - 1) / UPW_SUPER;
+            const int64_t run_first = run * UPW_SUPER, run_stop = min(n_chunks, run_first + UPW_SUPER);
+            publish(partial + chunk_id(my_chunk) * D);
+            if (!arrive(&arrived[chunk_id(run_first)], run_stop - run_first)) continue;
+            add_up(run_first, run_stop, 1);
+            if (n_runs > 1) {
+                publish(partial + chunk_id(run_first) * D);
+                if (!arrive(&arrived_runs[chunk_id(0)], n_runs)) continue;
+                add_up(0, n_chunks, UPW_SUPER);
+            }
+            count = gend - head;
+        }
+        double ss = 0.0;
+#pragma unroll
+        for (int j = 0; j < NQ; ++j) ss += a[j][0] * a[j][0] + a[j][1] * a[j][1] + a[j][2] * a[j][2] + a[j][3] * a[j][3];
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+        const double norm = sqrt(ss);
+        T *v = vecs + static_cast<int64_t>(slot) * D;
+#pragma unroll
+        for (int j = 0; j < NQ; ++j) {
+            const float4 f = make_float4(static_cast<float>(a[j][0] / norm), static_cast<float>(a[j][1] / norm),
+                                         static_cast<float>(a[j][2] / norm), static_cast<float>(a[j][3] / norm));
+            *reinterpret_cast<float4 *>(m + 4 * (lane + 32 * j)) = f;
+            if constexpr (sizeof(T) == 2) {
+                const __nv_bfloat162 lo = __floats2bfloat162_rn(f.x, f.y), hi = __floats2bfloat162_rn(f.z, f.w);
+                uint2 packed;
+                packed.x = *reinterpret_cast<const uint32_t *>(&lo);
+                packed.y = *reinterpret_cast<const uint32_t *>(&hi);
+                *reinterpret_cast<uint2 *>(v + 4 * (lane + 32 * j)) = packed;
+            }
+        }
+        if (lane == 0) {
+            size[slot] = n_old + static_cast<double>(count);
+            const unsigned long long acc_new = static_cast<unsigned long long>(access_old) + static_cast<unsigned long long>(count);
+            access[slot] = (access_old == SISO_ACCESS_INF || acc_new >= SISO_ACCESS_INF) ? SISO_ACCESS_INF : static_cast<uint32_t>(acc_new);
+            last[slot] = static_cast<unsigned long long>(counters[CNT_CLOCK]);
+        }
+    }
+}
+
+template <typename T>
+static bool launch_update_apply_warp(int nq, unsigned blocks, cudaStream_t s, const int4 *desc, unsigned int list_len,
+                                     const unsigned int *n_desc,
+                                     unsigned int *ticket, const uint32_t *vs, int chunk, const T *q, float *master, T *vecs, double *size,
+                                     uint32_t *access, unsigned long long *last, const long long *counters, double *partial,
+                                     unsigned int *arrived, unsigned int *arrived_runs) {
+#define SISO_UPW(N)                                                                                                          \
+    case N:                                                                                                                  \
+        update_apply_warp_kernel<T, N><<<blocks, UPW_THREADS, 0, s>>>(desc, list_len, n_desc, ticket, vs, chunk, q, master, vecs, size, access,  \
+                                                                     last, counters, partial, arrived, arrived_runs);        \
+        return true;
+    switch (nq) {
+        SISO_UPW(1) SISO_UPW(2) SISO_UPW(3) SISO_UPW(4) SISO_UPW(5) SISO_UPW(6) SISO_UPW(7) SISO_UPW(8)
+        default: return false;
+    }
+#undef SISO_UPW
+}
+
 // Small batches (at most UPS_MAX_B rows): one launch.  CTA b looks at row b; it works only if row b is the first
 // hit of its slot in the batch, then collects the later hits of that slot in ascending order (an ordered
 // compaction in shared memory) and applies them exactly like update_apply_kernel.  Every CTA reads the clock
@@ -307,8 +556,10 @@ siso_status_t launch_update(Cache *c, const void *q, int64_t B, const int32_t *i
     Scratch scr;
     const int chunk = static_cast<int>(std::max<int64_t>(32, (B + 4095) / 4096));
     const size_t n_ids = 2 * static_cast<size_t>(B / chunk + 1);
+    const bool warp_path = c->dim % 128 == 0 && c->dim <= 1024;
     const size_t need = 4 * pad256(sizeof(uint32_t) * B) + sort_pairs_scratch_bytes(B) +
-                        pad256(sizeof(double) * n_ids * c->dim) + pad256(sizeof(unsigned int) * n_ids);
+                        pad256(sizeof(double) * n_ids * c->dim) + pad256(sizeof(unsigned int) * (2 * n_ids + 4)) +
+                        pad256(sizeof(int4) * 2 * B);
     SISO_TRY(scratch_reserve(c, need, s, &scr));
     uint32_t *keys = scr.take<uint32_t>(B), *vals = scr.take<uint32_t>(B);
     uint32_t *keys2 = scr.take<uint32_t>(B), *vals2 = scr.take<uint32_t>(B);
@@ -325,9 +576,26 @@ siso_status_t launch_update(Cache *c, const void *q, int64_t B, const int32_t *i
     SISO_TRY(launch_sort_pairs(c, &scr, keys, vals, keys2, vals2, B, key_bits, &ks, &vs, s));
     const size_t smem = sizeof(double) * c->dim;
     double *partial = scr.take<double>(n_ids * c->dim);
-    unsigned int *arrived = scr.take<unsigned int>(n_ids);
-    SISO_CUDA(cudaMemsetAsync(arrived, 0, sizeof(unsigned int) * n_ids, s));
-    if (c->dtype == SISO_F32) {
+    // arrival counters per chunk id; number of chunks listed from the front and from the back (+ one unused word); the
+    // ticket counter; arrival counters of the runs
+    unsigned int *arrived = scr.take<unsigned int>(2 * n_ids + 4);
+    int4 *desc = scr.take<int4>(2 * B);
+    SISO_CUDA(cudaMemsetAsync(arrived, 0, sizeof(unsigned int) * (2 * n_ids + 4), s));
+    if (warp_path) {
+        // the list of chunks, then resident warps that walk it with the sums in registers
+        update_chunks_kernel<<<static_cast<unsigned>((B + 255) / 256), 256, 0, s>>>(ks, vs, B, c->capacity, chunk, desc, arrived + n_ids);
+        SISO_LAUNCHED(c);
+        const unsigned wblocks = static_cast<unsigned>(std::min<int64_t>((B + UPW_THREADS / 32 - 1) / (UPW_THREADS / 32), 4ll * c->sm_count));
+        if (c->dtype == SISO_F32)
+            launch_update_apply_warp<float>(c->dim / 128, wblocks, s, desc, static_cast<unsigned int>(B), arrived + n_ids, arrived + n_ids + 3, vs, chunk, static_cast<const float *>(q),
+                                            c->master, static_cast<float *>(c->vecs), c->size, c->access, c->last, c->counters,
+                                            partial, arrived, arrived + n_ids + 4);
+        else
+            launch_update_apply_warp<__nv_bfloat16>(c->dim / 128, wblocks, s, desc, static_cast<unsigned int>(B), arrived + n_ids, arrived + n_ids + 3, vs, chunk,
+                                                    static_cast<const __nv_bfloat16 *>(q), c->master,
+                                                    static_cast<__nv_bfloat16 *>(c->vecs), c->size, c->access, c->last,
+                                                    c->counters, partial, arrived, arrived + n_ids + 4);
+    } else if (c->dtype == SISO_F32) {
         update_apply_kernel<float><<<static_cast<unsigned>(B), UP_THREADS, smem, s>>>(
             ks, vs, B, c->capacity, c->dim, chunk, static_cast<const float *>(q), c->master, static_cast<float *>(c->vecs),
             c->size, c->access, c->last, c->counters, partial, arrived);

@@ -61,6 +61,8 @@ def make_pair(w, capacity=None, sizes=None):
     (2, dict(n_centroids=2048, n_queries=4096, dim=768, n_clusters=64), "T"),        # radix-sort grouping, hot rows
     (2, dict(n_centroids=500, n_queries=300, dim=136, n_clusters=40), "P"),          # single-CTA grouping
     (1, dict(n_centroids=700, n_queries=2500, dim=384, n_clusters=32), "T"),         # fp32 cache
+    (4, dict(n_centroids=900, n_queries=3000, dim=1024, n_clusters=24), "T"),        # widest row of the warp-per-position kernel
+    (2, dict(n_centroids=600, n_queries=1500, dim=264, n_clusters=20), "T"),         # dim not a multiple of 128: CTA-per-position kernel
 ])
 def test_update_matches_oracle(cfg, over, mode):
     w = W.config(cfg, mode=mode, **over)
