@@ -130,7 +130,8 @@ def test_config5_full_scale_sampled_batches():
     # start from a nearly full cache so that the sampled batches evict: fill with the stream's own later queries
     filler = stream.block(20000, 20000 + (sp.capacity - 3000) // 256, threads=THREADS)
     fill(cache, filler, "bf16")
-    sampled = {700, 1399}
+    sampled = {150, 400, 700, 900, 1000, 1150, 1300, 1399}     # before the cache is full, while it fills, and evicting
+    n_evicting = 0
     out = None
     for t in range(n_batches):
         q = q_all[t * 256:(t + 1) * 256]
@@ -150,7 +151,7 @@ def test_config5_full_scale_sampled_batches():
             o_idx, o_sim, o_hit, o_victims, o_slots = ora.stream_step(qn, theta, forced=(idx, hit))
             check_lookup((idx, sim, hit), (o_idx, o_sim, o_hit), pre_copy, qn, theta, TOL["bf16"], valid=pre_valid)
             nv = len(o_victims)
-            assert nv > 0, "the sampled batch did not evict"
+            n_evicting += 1 if nv > 0 else 0
             assert (victims[:nv] == o_victims).all() and (victims[nv:] == -1).all()
             assert (slots == o_slots).all()
             post = cache.export()
@@ -162,6 +163,7 @@ def test_config5_full_scale_sampled_batches():
             touched = np.unique(np.concatenate([idx[hit == 1, 0], slots[slots >= 0]]))
             assert np.abs(post["master"].cpu().numpy()[touched] - ora.master[touched]).max() <= 1e-6
     s = cache.stats()
+    assert n_evicting >= 4, "too few of the sampled batches evicted"
     assert s["occupancy"] == sp.capacity and s["evictions"] > 0
     assert s["inserts"] - s["evictions"] == s["occupancy"]
     cache.check_status()
