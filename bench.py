@@ -46,6 +46,8 @@ def parse_args():
                          "configurations (single GPU only)")
     ap.add_argument("--dtype", default="f32", choices=["f32", "bf16"], help="vector type of the cluster workload")
     ap.add_argument("--seed", type=int, default=0, help="seed of the configuration-5 stream (config5_full)")
+    ap.add_argument("--theta-range", type=float, nargs=2, default=None, metavar=("LO", "HI"),
+                    help="config5_full: per-query thresholds uniform in [LO, HI] instead of the fixed 0.86")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -538,6 +540,10 @@ def run_other(args):
         while done < sp.n_batches:
             stop = min(sp.n_batches, done + per_chunk)
             q = to_dev(stream.block(done, stop, threads=cores), "bf16")
+            th_all = None
+            if args.theta_range is not None:                   # theta_b ~ U[lo, hi], seeded per chunk
+                th_all = torch.from_numpy(W.thresholds(q.shape[0], args.theta_range[0], args.theta_range[1],
+                                                       1000 * args.seed + len(epochs))).to(dev)
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
             for t in range(done, stop):
@@ -545,7 +551,7 @@ def run_other(args):
                 qb = q[lo:lo + sp.batch]
                 if qb.shape[0] != sp.batch:
                     out = None                                 # the last batch is short
-                out = cache.stream_step(qb, float(sp.theta), out=out)
+                out = cache.stream_step(qb, float(sp.theta) if th_all is None else th_all[lo:lo + qb.shape[0]], out=out)
             e1.record()
             torch.cuda.synchronize()
             total_ms += e0.elapsed_time(e1)
@@ -564,6 +570,7 @@ def run_other(args):
         gbs = sp.capacity * sp.dim * 2 / (us * 1e-6) / 1e9
         line.update(metric="streaming cache, whole stream: 10,000,000 queries, 262,144 x 768 bf16, micro-batches of 256, from an empty cache",
                     value=sp.n_queries / total_ms * 1e3, unit=UNIT, us_per_batch=us, batches=sp.n_batches, seed=args.seed, dtype="bf16",
+                    theta=float(sp.theta) if args.theta_range is None else f"uniform in [{args.theta_range[0]}, {args.theta_range[1]}] per query",
                     hit_ratio=st["hits"] / sp.n_queries, inserts=st["inserts"], evictions=st["evictions"],
                     cache_full_after_chunk=first_full, chunks=epochs,
                     roofline={"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
