@@ -64,7 +64,7 @@ shard_route_kernel(const long long *__restrict__ idx, long long idx_stride, cons
                    uint8_t *__restrict__ upd_hit, uint8_t *__restrict__ ins_hit) {
     __shared__ int warp_cnt[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    long long base = 0;                                          // misses before this round, the same in every thread
+    long long base = 0;                                          // misses in the rows already visited, the same in every thread
     for (long long b0 = 0; b0 < n; b0 += 1024) {
         const long long b = b0 + tid;
         const bool miss = b < n && hit[b] == 0;
