@@ -2,7 +2,8 @@
 // with the query order kept inside each group, and the merged entries by surviving slot, so that
 // every later floating-point sum is taken in one fixed order (bitwise reproducible results).
 //   n <= SMALL_N : one CTA, rank by counting over packed 64-bit (key, position) words
-//   otherwise    : least-significant-digit radix sort, 8 bits per pass, three kernels per pass
+//   otherwise    : least-significant-digit radix sort, 8 or 9 bits per pass (9 where that saves a pass: 17- and 18-bit
+//                  keys, e.g. the slots of a 65,536-entry cache, sort in two passes), three kernels per pass
 #include "common.cuh"
 
 namespace siso {
@@ -11,6 +12,7 @@ constexpr int SMALL_N = 2048;
 constexpr int RS_THREADS = 256;
 constexpr int RS_ITEMS = 8;                       // rounds per tile
 constexpr int RS_TILE = RS_THREADS * RS_ITEMS;    // items per CTA
+constexpr int RS_MAX_BINS = 512;                  // 9 bits
 
 __global__ void __launch_bounds__(1024)
 sort_small_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restrict__ vals, int n,
@@ -29,21 +31,22 @@ sort_small_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restrict_
 
 // pass 1: per-tile digit histogram, stored digit-major: hist[digit * n_tiles + tile]
 __global__ void __launch_bounds__(RS_THREADS)
-radix_hist_kernel(const uint32_t *__restrict__ keys, int64_t n, int shift, int n_tiles, uint32_t *__restrict__ hist) {
-    __shared__ uint32_t h[256];
-    h[threadIdx.x] = 0;
+radix_hist_kernel(const uint32_t *__restrict__ keys, int64_t n, int shift, int bins, int n_tiles, uint32_t *__restrict__ hist) {
+    __shared__ uint32_t h[RS_MAX_BINS];
+    const uint32_t mask = static_cast<uint32_t>(bins - 1);
+    for (int d = threadIdx.x; d < bins; d += RS_THREADS) h[d] = 0;
     __syncthreads();
     const int64_t base = static_cast<int64_t>(blockIdx.x) * RS_TILE;
 #pragma unroll
     for (int r = 0; r < RS_ITEMS; ++r) {
         const int64_t i = base + r * RS_THREADS + threadIdx.x;
-        if (i < n) atomicAdd(&h[(keys[i] >> shift) & 255u], 1u);
+        if (i < n) atomicAdd(&h[(keys[i] >> shift) & mask], 1u);
     }
     __syncthreads();
-    hist[static_cast<int64_t>(threadIdx.x) * n_tiles + blockIdx.x] = h[threadIdx.x];
+    for (int d = threadIdx.x; d < bins; d += RS_THREADS) hist[static_cast<int64_t>(d) * n_tiles + blockIdx.x] = h[d];
 }
 
-// pass 2: exclusive scan of the histogram in place (one CTA; the array has 256 * n_tiles entries)
+// pass 2: exclusive scan of the histogram in place (one CTA; the array has bins * n_tiles entries)
 __global__ void __launch_bounds__(1024) exclusive_scan_u32_kernel(uint32_t *__restrict__ a, int64_t n) {
     __shared__ uint32_t warp_sum[32];
     __shared__ uint32_t carry_s;
@@ -83,22 +86,25 @@ __global__ void __launch_bounds__(1024) exclusive_scan_u32_kernel(uint32_t *__re
 // pass 3: stable scatter.  Items of a tile are visited in 8 rounds of 256 in index order; inside a
 // round the rank of an item among equal digits is (equal digits in earlier warps) + (in earlier lanes).
 __global__ void __launch_bounds__(RS_THREADS)
-radix_scatter_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restrict__ vals, int64_t n, int shift,
+radix_scatter_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restrict__ vals, int64_t n, int shift, int bins,
                      int n_tiles, const uint32_t *__restrict__ hist_scanned, uint32_t *__restrict__ keys_out,
                      uint32_t *__restrict__ vals_out) {
-    __shared__ uint32_t base_s[256];
-    __shared__ uint32_t cnt_s[RS_THREADS / 32][256];
+    __shared__ uint32_t base_s[RS_MAX_BINS];
+    __shared__ uint32_t cnt_s[RS_THREADS / 32][RS_MAX_BINS];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
-    base_s[tid] = hist_scanned[static_cast<int64_t>(tid) * n_tiles + blockIdx.x];
+    const uint32_t mask = static_cast<uint32_t>(bins - 1);
+    for (int d = tid; d < bins; d += RS_THREADS) base_s[d] = hist_scanned[static_cast<int64_t>(d) * n_tiles + blockIdx.x];
     const int64_t base = static_cast<int64_t>(blockIdx.x) * RS_TILE;
     for (int r = 0; r < RS_ITEMS; ++r) {
+        for (int d = tid; d < bins; d += RS_THREADS) {
 #pragma unroll
-        for (int w = 0; w < RS_THREADS / 32; ++w) cnt_s[w][tid] = 0;
+            for (int w = 0; w < RS_THREADS / 32; ++w) cnt_s[w][d] = 0;
+        }
         __syncthreads();
         const int64_t i = base + r * RS_THREADS + tid;
         const bool live = i < n;
-        uint32_t key = 0, digit = 256 + lane;     // dead lanes never match anything
-        if (live) { key = keys[i]; digit = (key >> shift) & 255u; }
+        uint32_t key = 0, digit = static_cast<uint32_t>(bins + lane);     // dead lanes never match anything
+        if (live) { key = keys[i]; digit = (key >> shift) & mask; }
         const unsigned peers = __match_any_sync(0xFFFFFFFFu, digit);
         const int rank_in_warp = __popc(peers & ((1u << lane) - 1u));
         if (live && rank_in_warp == 0) cnt_s[warp][digit] = __popc(peers);
@@ -110,10 +116,12 @@ radix_scatter_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restri
             vals_out[pos] = vals[i];
         }
         __syncthreads();
-        uint32_t total = 0;
+        for (int d = tid; d < bins; d += RS_THREADS) {
+            uint32_t total = 0;
 #pragma unroll
-        for (int w = 0; w < RS_THREADS / 32; ++w) total += cnt_s[w][tid];
-        base_s[tid] += total;
+            for (int w = 0; w < RS_THREADS / 32; ++w) total += cnt_s[w][d];
+            base_s[d] += total;
+        }
         __syncthreads();
     }
 }
@@ -126,7 +134,7 @@ siso_status_t launch_exclusive_scan_u32(Cache *c, uint32_t *a, int64_t n, cudaSt
 
 size_t sort_pairs_scratch_bytes(int64_t n) {
     const int64_t n_tiles = (n + RS_TILE - 1) / RS_TILE;
-    return pad256(sizeof(uint32_t) * 256 * static_cast<size_t>(n_tiles > 0 ? n_tiles : 1));
+    return pad256(sizeof(uint32_t) * RS_MAX_BINS * static_cast<size_t>(n_tiles > 0 ? n_tiles : 1));
 }
 
 // Sorts n pairs by the low key_bits of the key, stably.  The result lands either in the input
@@ -142,14 +150,17 @@ siso_status_t launch_sort_pairs(Cache *c, Scratch *scr, uint32_t *keys, uint32_t
         return SISO_OK;
     }
     const int n_tiles = static_cast<int>((n + RS_TILE - 1) / RS_TILE);
-    uint32_t *hist = scr->take<uint32_t>(256 * static_cast<size_t>(n_tiles));
+    uint32_t *hist = scr->take<uint32_t>(RS_MAX_BINS * static_cast<size_t>(n_tiles));
     uint32_t *ka = keys, *va = vals, *kb = keys_tmp, *vb = vals_tmp;
-    for (int shift = 0; shift < key_bits; shift += 8) {
-        radix_hist_kernel<<<n_tiles, RS_THREADS, 0, s>>>(ka, n, shift, n_tiles, hist);
+    // 9-bit digits where they save a pass over 8-bit ones
+    const int bits = (key_bits + 8) / 9 < (key_bits + 7) / 8 ? 9 : 8;
+    const int bins = 1 << bits;
+    for (int shift = 0; shift < key_bits; shift += bits) {
+        radix_hist_kernel<<<n_tiles, RS_THREADS, 0, s>>>(ka, n, shift, bins, n_tiles, hist);
         SISO_LAUNCHED(c);
-        exclusive_scan_u32_kernel<<<1, 1024, 0, s>>>(hist, 256 * static_cast<int64_t>(n_tiles));
+        exclusive_scan_u32_kernel<<<1, 1024, 0, s>>>(hist, bins * static_cast<int64_t>(n_tiles));
         SISO_LAUNCHED(c);
-        radix_scatter_kernel<<<n_tiles, RS_THREADS, 0, s>>>(ka, va, n, shift, n_tiles, hist, kb, vb);
+        radix_scatter_kernel<<<n_tiles, RS_THREADS, 0, s>>>(ka, va, n, shift, bins, n_tiles, hist, kb, vb);
         SISO_LAUNCHED(c);
         uint32_t *t = ka; ka = kb; kb = t;
         t = va; va = vb; vb = t;
