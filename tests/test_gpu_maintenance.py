@@ -34,7 +34,15 @@ def assert_state_equal(cache, ora, dtype, what=""):
     gm = g["master"][live].astype(np.float64)
     cosine = np.einsum("ij,ij->i", gm, ora.master[live]) / (np.linalg.norm(gm, axis=1) * np.linalg.norm(ora.master[live], axis=1))
     assert (cosine >= 1 - 1e-6).all(), what
-    assert np.abs(widen64(g["vecs"][live]) - widen64(ora.lookup_copy()[live])).max(initial=0) <= VEC_TOL[dtype], what
+    a, b = widen64(g["vecs"][live]), widen64(ora.lookup_copy()[live])
+    if dtype == "bf16":
+        # the GPU rounds its fp32 master, the oracle its fp64 master: where the master lies within 1e-6 of a rounding
+        # boundary the two copies are neighbours, so the bound is one bf16 ulp of the value (2.5e-4 is that ulp below
+        # 0.125) and such elements are few
+        ulp = 2.0 ** (np.floor(np.log2(np.maximum(np.abs(b), 1e-30))) - 7)
+        assert (np.abs(a - b) <= np.maximum(ulp, VEC_TOL[dtype])).all() and (a != b).sum() <= 0.01 * a.size, what
+    else:
+        assert np.abs(a - b).max(initial=0) <= VEC_TOL[dtype], what
     if dtype == "bf16":   # the lookup copy is the master rounded once
         m = torch.from_numpy(g["master"]).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
         assert (m[live] == g["vecs"][live]).all(), what
