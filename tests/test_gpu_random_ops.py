@@ -25,11 +25,13 @@ def resync(cache, dtype):
     return ora
 
 
-@pytest.mark.parametrize("dtype,dim,seed", [("bf16", 72, 0), ("bf16", 128, 1), ("f32", 72, 2), ("f32", 136, 3), ("bf16", 264, 4),
-                                            ("f32", 384, 5), ("bf16", 1024, 6), ("f32", 8, 7)])
-def test_random_operation_sequences_match_the_oracle(dtype, dim, seed):
+@pytest.mark.parametrize("dtype,dim,seed,cap", [
+    ("bf16", 72, 0, 700), ("bf16", 128, 1, 700), ("f32", 72, 2, 700), ("f32", 136, 3, 700), ("bf16", 264, 4, 700),
+    ("f32", 384, 5, 700), ("bf16", 1024, 6, 700), ("f32", 8, 7, 700),
+    ("f32", 136, 8, 4500), ("bf16", 136, 9, 4500),          # large enough for the tensor-core merge sweep
+])
+def test_random_operation_sequences_match_the_oracle(dtype, dim, seed, cap):
     rng = np.random.default_rng(100 + seed)
-    cap = 700
     pool = W.config(2 if dtype == "bf16" else 1, seed=70 + seed, mode="P", n_centroids=3000, n_queries=3000, dim=dim, n_clusters=150,
                     dtype=dtype, theta=(0.78, 0.93))
     rows = np.concatenate([pool.centroids, pool.queries])              # 6000 vectors around 150 cluster means
@@ -45,7 +47,7 @@ def test_random_operation_sequences_match_the_oracle(dtype, dim, seed):
         op = rng.choice(list(done), p=[0.15, 0.25, 0.25, 0.1, 0.1, 0.15])
         what = f"seed {seed} step {step} {op}"
         if op == "insert":
-            n = int(rng.integers(0, min(cap - occ, 200) + 1))
+            n = int(rng.integers(0, min(cap - occ, max(200, cap // 3)) + 1))
             v = draw(n)
             sizes = rng.integers(1, 20, n).astype(np.float64) if rng.random() < 0.5 else None
             slots = cache.insert(to_dev(v, dtype), None if sizes is None else torch.from_numpy(sizes)) if n else None
