@@ -48,6 +48,9 @@ def parse_args():
     ap.add_argument("--seed", type=int, default=0, help="seed of the configuration-5 stream (config5_full)")
     ap.add_argument("--theta-range", type=float, nargs=2, default=None, metavar=("LO", "HI"),
                     help="config5_full: per-query thresholds uniform in [LO, HI] instead of the fixed 0.86")
+    ap.add_argument("--maintain", action="store_true",
+                    help="config5_full: after every million queries a MergeCentroids pass (theta_C 0.86, weighted mean) and the "
+                         "decay of FilteringCentroids, as the paper re-clusters when enough new queries have arrived")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
     return ap.parse_args()
@@ -536,7 +539,7 @@ def run_other(args):
         cache = siso.SisoCache(sp.capacity, sp.dim, "bf16")
         per_chunk = 3906                                      # batches per chunk (about one popularity epoch)
         total_ms, done, out = 0.0, 0, None
-        epochs, first_full, prev = [], None, cache.stats()
+        epochs, first_full, prev, maintenance = [], None, cache.stats(), []
         while done < sp.n_batches:
             stop = min(sp.n_batches, done + per_chunk)
             q = to_dev(stream.block(done, stop, threads=cores), "bf16")
@@ -563,16 +566,28 @@ def run_other(args):
             if first_full is None and st["occupancy"] == sp.capacity:
                 first_full = len(epochs)
             prev, done = st, stop
+            if args.maintain and done < sp.n_batches:
+                m0, m1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                m0.record()
+                _, n_merged = cache.merge(0.86, siso.MERGE_WEIGHTED_MEAN)
+                cache.evict(0, siso.EVICT_DECAY)
+                m1.record()
+                torch.cuda.synchronize()
+                cache.check_status()
+                maintenance.append({"after_queries": done * sp.batch, "merged": n_merged, "ms": round(m0.elapsed_time(m1), 2),
+                                    "occupancy_after": cache.stats()["occupancy"]})
+                prev = cache.stats()
         cache.check_status()
         st = cache.stats()
-        assert st["lookups"] == sp.n_queries and st["inserts"] - st["evictions"] == st["occupancy"] <= sp.capacity
+        assert st["lookups"] == sp.n_queries and st["inserts"] - st["evictions"] - st["merges"] == st["occupancy"] <= sp.capacity
         us = total_ms / sp.n_batches * 1e3
         gbs = sp.capacity * sp.dim * 2 / (us * 1e-6) / 1e9
         line.update(metric="streaming cache, whole stream: 10,000,000 queries, 262,144 x 768 bf16, micro-batches of 256, from an empty cache",
                     value=sp.n_queries / total_ms * 1e3, unit=UNIT, us_per_batch=us, batches=sp.n_batches, seed=args.seed, dtype="bf16",
                     theta=float(sp.theta) if args.theta_range is None else f"uniform in [{args.theta_range[0]}, {args.theta_range[1]}] per query",
                     hit_ratio=st["hits"] / sp.n_queries, inserts=st["inserts"], evictions=st["evictions"],
-                    cache_full_after_chunk=first_full, chunks=epochs,
+                    cache_full_after_chunk=first_full, chunks=epochs, merges=st["merges"], maintenance=maintenance,
+                    maintenance_ms_total=sum(m["ms"] for m in maintenance),
                     roofline={"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
                               "frac": gbs / peaks["hbm_gbs"], "traffic": None,
                               "note": "384 MiB of centroid slots per batch over the whole step time (the early batches sweep a partly empty cache)"})
