@@ -71,6 +71,8 @@ def make_pair(w, capacity=None, sizes=None):
     (1, dict(n_centroids=700, n_queries=2500, dim=384, n_clusters=32), "T"),         # fp32 cache
     (4, dict(n_centroids=900, n_queries=3000, dim=1024, n_clusters=24), "T"),        # widest row of the warp-per-position kernel
     (2, dict(n_centroids=600, n_queries=1500, dim=264, n_clusters=20), "T"),         # dim not a multiple of 128: CTA-per-position kernel
+    (1, dict(n_centroids=800, n_queries=2000, dim=1024, n_clusters=20), "T"),        # fp32 rows of 4 KiB in the warp kernel
+    (2, dict(n_centroids=40, n_queries=6000, dim=128, n_clusters=4), "T"),           # a few centroids take over a thousand hits each: runs of chunks
 ])
 def test_update_matches_oracle(cfg, over, mode):
     w = W.config(cfg, mode=mode, **over)
