@@ -142,3 +142,33 @@ def test_sharded_eviction_is_the_global_selection():
     assert sum(p.local.stats()["occupancy"] for p in parts) == 0 and sum(p.local.stats()["evictions"] for p in parts) == total
     for p in parts:
         p.close()
+
+
+def test_world_of_one_through_the_distributed_driver():
+    """Without a process group the torch.distributed driver (run) sees a world of one rank: the sharded step and the
+    sharded eviction must then equal the plain cache's, bit for bit."""
+    sp = W.StreamSpec(capacity=400, dim=64, n_queries=100 * 12, batch=100, n_clusters=900, zipf_s=1.1, reshuffle_every=500,
+                      theta=0.80, mode="P", dtype="bf16", seed=62)
+    stream = W.QueryStream(sp)
+    one = siso.ShardedCache(400, 64, "bf16")
+    plain = siso.SisoCache(400, 64, "bf16")
+    for t in range(12):
+        qn, _ = stream.batch(t)
+        q = to_dev(qn, "bf16")
+        idx, sim, hit, victims, slots = one.stream_step(q, float(sp.theta))
+        p_idx, p_sim, p_hit, p_victims, p_slots = plain.stream_step(q, float(sp.theta))
+        assert (idx.to(torch.int32) == p_idx[:, 0]).all().item() and (hit == p_hit).all().item()
+        assert (sim == p_sim[:, 0]).all().item()
+        nv = victims.numel()
+        assert (victims.to(torch.int32) == p_victims[:nv]).all().item() and (p_victims[nv:] == -1).all().item()
+        assert (slots.to(torch.int32) == p_slots).all().item()
+    a, b = one.local.export(), plain.export()
+    assert all((a[k] == b[k]).all().item() for k in ("valid", "size", "access", "last", "master", "vecs"))
+    assert one.local.stats()["evictions"] == plain.stats()["evictions"] > 0
+    v1 = one.evict(37, siso.EVICT_DECAY)
+    v2 = plain.evict(37, siso.EVICT_DECAY)
+    assert (v1.to(torch.int32) == v2).all().item()
+    a, b = one.local.export(), plain.export()
+    assert all((a[k] == b[k]).all().item() for k in ("valid", "size", "access"))
+    one.close()
+    plain.close()
