@@ -91,6 +91,7 @@ static uint16_t round_to_bf16(double x) {
 }
 
 void siso_oracle_round_bf16(const double *in, uint16_t *out, int64_t n) {
+#pragma omp parallel for schedule(static)
     for (int64_t i = 0; i < n; ++i) out[i] = round_to_bf16(in[i]);
 }
 

@@ -8,6 +8,7 @@ import pytest
 
 import oracle
 from gen import workloads as W
+from util import verify_merge_map
 
 INF = oracle.ACCESS_INF
 
@@ -309,6 +310,90 @@ def test_stream_conservation_and_recovery_after_reshuffle():
     assert hits[110:].mean() > hits[60:63].mean()                   # ... and the cache recovers
 
 
+def _run_streaming_example(ex, step):
+    """Feeds the hand-computed two-batch example through `step(cache, queries, theta)` and compares every output and
+    the whole state after each batch with the pencil values.  Returns normally or raises AssertionError."""
+    inf = lambda a: np.array([INF if x == "inf" else x for x in a], dtype=np.uint32)
+    init = ex["initial"]
+    c = oracle.OracleCache(ex["capacity"], ex["dim"], "f32")
+    c.load_state(np.array(init["vectors"], dtype=np.float64), np.array(init["size"], dtype=np.float64),
+                 inf(init["access"]), np.array(init["last"], dtype=np.uint64), np.array(init["valid"], dtype=np.uint8),
+                 ex["clock_before"])
+    for b in ex["batches"]:
+        q = np.array(b["queries"], dtype=np.float64)
+        idx, sim, hit, victims, slots = step(c, q, np.float32(ex["theta"]))
+        assert idx[:, 0].tolist() == b["idx"] and hit.tolist() == b["hit"]
+        np.testing.assert_allclose(sim[:, 0], b["sim"], atol=1e-6)
+        assert victims.tolist() == b["victims"], "victims"
+        assert slots.tolist() == b["slots"], "slots"
+        a = b["after"]
+        assert c.clock == a["clock"] and c.valid.tolist() == a["valid"]
+        np.testing.assert_allclose(c.master, np.array(a["vectors"], dtype=np.float64), atol=1e-6)
+        assert c.size.tolist() == a["size"] and c.access.tolist() == inf(a["access"]).tolist()
+        assert c.last.tolist() == a["last"]
+
+
+@pytest.fixture(scope="module")
+def streaming_example(golden_dir):
+    return json.load(open(os.path.join(golden_dir, "streaming_two_batches.json")))
+
+
+def test_stream_step_worked_example(streaming_example):
+    """lookup -> update -> evict(#miss - free) -> insert on a capacity-4 cache, two batches, every number by hand:
+    Algorithm 1 (MergeCentroids' else-branch, FilteringCentroids' order) and Sec. 5.2.5 (spare-space vectors under LRU)."""
+    _run_streaming_example(streaming_example, lambda c, q, th: c.stream_step(q, th))
+
+
+def _evicts_one_per_miss(c, q, th):
+    idx, sim, hit = c.lookup(q, th, 1)
+    c.update(q, idx, hit)
+    victims = c.evict(int((hit == 0).sum()))                     # forgets the free slots
+    return idx, sim, hit, victims, c.insert(q, hit)
+
+
+def _evicts_before_updating(c, q, th):
+    idx, sim, hit = c.lookup(q, th, 1)
+    n_miss, free = int((hit == 0).sum()), c.capacity - c.occupancy
+    victims = c.evict(n_miss - free) if n_miss > free else np.empty(0, np.int32)
+    c.update(q, idx, hit)                                        # the hit no longer protects its entry
+    return idx, sim, hit, victims, c.insert(q, hit)
+
+
+def _inserts_in_victim_order(c, q, th):
+    idx, sim, hit = c.lookup(q, th, 1)
+    c.update(q, idx, hit)
+    n_miss, free = int((hit == 0).sum()), c.capacity - c.occupancy
+    free_slots = np.flatnonzero(c.valid == 0).tolist()
+    victims = c.evict(n_miss - free) if n_miss > free else np.empty(0, np.int32)
+    order = free_slots + victims.tolist()                        # free slots first, then victims as evicted
+    slots = np.full(len(q), -1, np.int32)
+    for b, s in zip(np.flatnonzero(hit == 0), order):
+        c.master[s], c.size[s], c.access[s], c.last[s], c.valid[s] = q[b], 1.0, INF, c.clock, 1
+        slots[b] = s
+    return idx, sim, hit, victims, slots
+
+
+def _sees_its_own_batch(c, q, th):
+    outs = [c.stream_step(q[b:b + 1], th) for b in range(len(q))]       # one query at a time: not batch-synchronous
+    c.clock -= len(q) - 1
+    cat = lambda j: np.concatenate([o[j] for o in outs])
+    return cat(0), cat(1), cat(2), cat(3), cat(4)
+
+
+def _keeps_the_old_clock(c, q, th):
+    out = c.stream_step(q, th)
+    c.last[c.last == c.clock] = c.clock - 1
+    return out
+
+
+@pytest.mark.parametrize("mistake", [_evicts_one_per_miss, _evicts_before_updating, _inserts_in_victim_order,
+                                     _sees_its_own_batch, _keeps_the_old_clock])
+def test_stream_step_worked_example_catches_planted_mistakes(streaming_example, mistake):
+    """The example is chosen so that each plausible mistake in the composition changes a number in it."""
+    with pytest.raises((AssertionError, RuntimeError)):          # RuntimeError: the oracle refuses an update of an empty slot
+        _run_streaming_example(streaming_example, mistake)
+
+
 def test_two_set_merge_with_interleaved_slots_equals_transcription():
     """C_cur and the repository entries may sit in any slots: seeds are given by a mask."""
     w = W.config(3, n_centroids=180, dim=20, n_clusters=14, mode="P")
@@ -347,6 +432,48 @@ def test_two_set_merge_with_interleaved_slots_equals_transcription():
     c = make_cache(np.array([[1.0, 0], [0, 1.0], [1.0, 0], [1.0, 0]]))
     mm, n = c.merge(0.5, weighted_mean=False, seed_mask=np.array([0, 0, 0, 1]))
     assert mm.tolist() == [3, 1, 3, 3] and n == 2
+
+
+def test_tolerant_merge_verifier_accepts_the_oracle_and_rejects_wrong_maps():
+    """The GPU tests accept a merge map that differs from the oracle's only through `verify_merge_map`; here that
+    verifier is held against the oracle itself (one-set and two-set) and against planted wrong maps."""
+    w = W.config(3, n_centroids=160, dim=20, n_clusters=12, mode="P")
+    rng = np.random.default_rng(3)
+    sizes = rng.integers(1, 6, 160).astype(np.float64)
+    for seeded in (False, True):
+        seed = (rng.random(160) < 0.4).astype(np.uint8) if seeded else np.zeros(160, np.uint8)
+        c = make_cache(w.centroids, sizes=sizes)
+        c.valid[rng.random(160) < 0.1] = 0
+        entry, valid0 = c.master.copy(), c.valid.copy()
+        mm, n = c.merge(0.9, weighted_mean=False, seed_mask=seed if seeded else None, new_access_inf=seeded)
+        assert n > 5
+        size = verify_merge_map(entry, valid0, seed, sizes, mm, 0.9, tol=0.0)
+        live = c.valid == 1
+        np.testing.assert_array_equal(size[live], c.size[live])
+        merged = [i for i in range(160) if mm[i] >= 0 and mm[i] != i]
+        surv = [i for i in range(160) if mm[i] == i and not seed[i]]
+        S = entry @ entry.T
+        bad = mm.copy()
+        bad[merged[0]] = merged[0]                             # a merged entry declared a survivor
+        with pytest.raises(AssertionError):
+            verify_merge_map(entry, valid0, seed, sizes, bad, 0.9)
+        bad = mm.copy()
+        i = merged[-1]
+        other = [s for s in surv if s < i and s != mm[i] and S[i, s] < S[i, mm[i]] - 1e-3]
+        bad[i] = other[0]                                      # merged into a survivor that is not the closest
+        with pytest.raises(AssertionError):
+            verify_merge_map(entry, valid0, seed, sizes, bad, 0.9)
+        bad = mm.copy()
+        lone = [s for s in surv if s > 0 and S[s, [t for t in surv if t < s] or [s]].max() < 0.8]
+        if lone:
+            bad[lone[-1]] = [t for t in surv if t < lone[-1]][0]    # a survivor merged below the threshold
+            with pytest.raises(AssertionError):
+                verify_merge_map(entry, valid0, seed, sizes, bad, 0.9)
+        bad = mm.copy()
+        later = [(i, s) for i in merged for s in surv if s > i]
+        bad[later[0][0]] = later[0][1]                         # merged into a LATER survivor
+        with pytest.raises(AssertionError):
+            verify_merge_map(entry, valid0, seed, sizes, bad, 0.9)
 
 
 # ---------------------------------------------------------------------------- Algorithm 1 as a whole
