@@ -53,6 +53,8 @@ def parse_args():
                          "decay of FilteringCentroids, as the paper re-clusters when enough new queries have arrived")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--no-secondary", action="store_true",
+                    help="skip the extra measurements of the default line (streaming step, small-batch sweeps, hit update)")
     return ap.parse_args()
 
 
@@ -135,6 +137,8 @@ def run_reference(args):
 
 # ------------------------------------------------------------------------------ clocks
 class ClockSampler:
+    """nvidia-smi sampled every 50 ms between start and stop(): SM clock (plain median, min and max of ALL samples of
+    the window), power and the throttle reasons that were active in any sample."""
     FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
               "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
               "clocks_event_reasons.sw_power_cap")
@@ -143,10 +147,11 @@ class ClockSampler:
         self.proc = None
         try:
             self.proc = subprocess.Popen(["nvidia-smi", f"--id={index}", f"--query-gpu={self.FIELDS}",
-                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                          "--format=csv,noheader,nounits", "-lms", "50"],
                                          stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.proc.stdout.readline()          # the first sample: the sampler is running before the timed region starts
         except OSError:
-            pass
+            self.proc = None
 
     def stop(self):
         if self.proc is None:
@@ -157,7 +162,7 @@ class ClockSampler:
         except subprocess.TimeoutExpired:
             self.proc.kill()
             out, _ = self.proc.communicate()
-        sm, mx, reasons = [], [], set()
+        sm, mx, pw, reasons = [], [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         for ln in out.splitlines():
             f = [x.strip() for x in ln.split(",")]
@@ -166,14 +171,46 @@ class ClockSampler:
             try:
                 sm.append(float(f[0]))
                 mx.append(float(f[1]))
+                pw.append(float(f[2]))
             except ValueError:
                 continue
             for name, v in zip(names, f[3:7]):
                 if v.lower().startswith("active"):
                     reasons.add(name)
-        hi = sorted(sm)[len(sm) // 2:] if sm else []     # the upper half of the samples: those under load
-        return {"sm_mhz": statistics.median(hi) if hi else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        if not sm:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["no sample inside the timed region"], "samples": 0}
+        return {"sm_mhz": statistics.median(sm), "sm_mhz_min": min(sm), "sm_mhz_max": max(sm), "sm_max_mhz": max(mx),
+                "power_w_max": max(pw), "reasons": sorted(reasons), "samples": len(sm)}
+
+
+# ------------------------------------------------------------------------------ DRAM traffic from the committed profile
+TRAFFIC_PROFILE = os.path.join(ROOT, "profiles", "lookup_tensor_config4_launches.txt")
+
+
+def kernel_sources_sha(paths) -> str:
+    import hashlib
+    h = hashlib.sha256()
+    for rel in paths:
+        with open(os.path.join(ROOT, rel), "rb") as f:
+            h.update(f.read())
+    return h.hexdigest()
+
+
+def committed_traffic():
+    """DRAM bytes per launch of the sweep kernel from the committed ncu capture, or None when the kernel's sources
+    have changed since that capture (the profile records their hash): a stale counter is not reported."""
+    try:
+        fields = {}
+        with open(TRAFFIC_PROFILE) as f:
+            for ln in f:
+                if ln.startswith(("traffic_bytes_per_launch:", "kernel_sources:", "kernel_sources_sha256:")):
+                    key, val = ln.split(":", 1)
+                    fields[key] = val.strip()
+        if kernel_sources_sha(fields["kernel_sources"].split()) != fields["kernel_sources_sha256"]:
+            return None
+        return float(fields["traffic_bytes_per_launch"])
+    except (OSError, KeyError, ValueError):
+        return None
 
 
 # ------------------------------------------------------------------------------ GPU arm
@@ -253,16 +290,21 @@ def run_ours(args):
 
     for _ in range(max(3, args.warmup)):
         step_device()
-    sampler = ClockSampler(local_rank) if rank == 0 else None
+    torch.cuda.synchronize()
+    sampler = ClockSampler(local_rank) if rank == 0 else None        # started after the warm-up
     ms, per_step, launches = timed(step_device, args.steps)
     clocks = sampler.stop() if sampler else None
     cache.check_status()
+    legs = {"device": {"ms_per_step": ms, "clocks": clocks}}
 
     e2e = None
     if not args.no_e2e:
         for _ in range(3):
             step_host()
+        torch.cuda.synchronize()
+        sampler = ClockSampler(local_rank) if rank == 0 else None
         ms_e2e, _, _ = timed(step_host, args.steps)
+        legs["e2e"] = {"ms_per_step": ms_e2e, "clocks": sampler.stop() if sampler else None}
         cache.check_status()
         e2e = {"value": whole_job_value(B, world, ms_e2e), "unit": UNIT,
                "h2d_bytes_per_step": int(w.queries.nbytes + w.theta.nbytes),
@@ -270,6 +312,37 @@ def run_ours(args):
                "ms_per_step": ms_e2e}
         # the host-buffer call must return what the device call returns
         assert torch.equal(h_idx, out[0].cpu()) and torch.equal(h_hit, out[2].cpu())
+        # where the end-to-end step's time goes: the same three stages issued one by one with an event after each
+        # (host -> device copies of queries and thresholds, the lookup, device -> host copies of the three results)
+        ev = [[torch.cuda.Event(enable_timing=True) for _ in range(4)] for _ in range(args.steps)]
+        q_stage, th_stage = torch.empty_like(q_dev), torch.empty_like(th_dev)
+        barrier()
+        for e in ev:
+            e[0].record(stream)
+            q_stage.view(torch.int16).copy_(h_q, non_blocking=True)
+            th_stage.copy_(h_th, non_blocking=True)
+            e[1].record(stream)
+            cache.lookup(q_stage, th_stage, k, out=out)
+            e[2].record(stream)
+            h_idx.copy_(out[0], non_blocking=True)
+            h_sim.copy_(out[1], non_blocking=True)
+            h_hit.copy_(out[2], non_blocking=True)
+            e[3].record(stream)
+        barrier()
+        e2e["stages_ms"] = {name: statistics.median(e[a].elapsed_time(e[a + 1]) for e in ev)
+                            for a, name in enumerate(("h2d_copy", "lookup", "d2h_copy"))}
+
+    # the same device-resident step back to back for at least two seconds: the clock the power cap settles at, and the
+    # step time x clock product that makes runs at different clocks comparable
+    sustained = None
+    if rank == 0 and world == 1:
+        n_sus = max(args.steps, int(2200.0 / ms) + 1)
+        sampler = ClockSampler(local_rank)
+        ms_sus, per_sus, _ = timed(step_device, n_sus)
+        ck = sampler.stop()
+        sustained = {"steps": n_sus, "ms_per_step": ms_sus, "median_step_ms": statistics.median(per_sus), "clocks": ck,
+                     "ms_x_mhz": ms_sus * ck["sm_mhz"] if ck.get("sm_mhz") else None}
+        cache.check_status()
 
     if rank != 0:
         if world > 1:
@@ -280,26 +353,34 @@ def run_ours(args):
     flops = 2.0 * B * args.rows * 1024
     kernel_ms = statistics.median(per_step)           # the sweep kernel plus its small finalize kernel
     achieved = flops / (kernel_ms * 1e-3) / 1e12
-    # DRAM bytes per launch of the dominant kernel, from the committed one-pass ncu capture of this very command
-    # (profiles/lookup_tensor_config4_launches.txt: 2.888e9 read, 5.5e6 / 2.4e6 written in two launches);
-    # only known for the full-size workload on the tensor-core kernel as profiled
+    # DRAM bytes per launch of the dominant kernel come from the committed one-pass ncu capture of this very command;
+    # they are only known for the full-size workload on the tensor-core kernel, and only while the kernel's sources
+    # are the ones that were profiled
     traffic = None
     if args.path in ("auto", "tensor") and args.rows == (1 << 20) and B == 8192:
-        traffic = 0.5 * (2892656384 + 2893686784) + 0.5 * (5250560 + 1996544)
+        traffic = committed_traffic()
     roofline = {"bound": "tensor", "achieved": achieved, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
-                "frac": achieved / peaks["bf16_tflops"], "traffic": traffic, "peak_kind": f"{peak_kind}, burst",
+                "frac": achieved / peaks["bf16_tflops"], "traffic": traffic,
+                "traffic_source": "committed ncu capture (profiles/), not this run" if traffic else None,
+                "peak_kind": f"{peak_kind}, burst",
                 "frac_of_sustained": achieved / peaks["bf16_tflops_sustained"],
                 "hbm_floor_ms": (args.rows * 1024 * 2 + B * 1024 * 2) / (peaks["hbm_gbs"] * 1e9) * 1e3,
                 "kernel": {"auto": "tensor-core sweep (auto)", "tensor": "tensor-core sweep", "simt": "CUDA-core sweep",
                            "stream": "streaming sweep"}[args.path],
                 "flops_per_launch": flops, "median_launch_ms": kernel_ms}
+    if sustained:
+        sustained["frac_of_sustained_peak"] = flops / (sustained["ms_per_step"] * 1e-3) / 1e12 / peaks["bf16_tflops_sustained"]
     line = {"metric": METRIC, "value": whole_job_value(B, world, ms), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "weak",
             "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
             "config": {"workload": workload_name(args), "parallelism": f"replica x{world}, queries sharded",
                        "l2": "inputs larger than L2: the 2 GiB centroid matrix is swept on every step",
                        "lookup_path": args.path},
-            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline}
+            "clocks": clocks, "e2e": e2e, "gpu_launches": launches, "roofline": roofline, "legs": legs,
+            "sustained": sustained}
+
+    if world == 1 and not args.no_secondary:
+        line["secondary"] = secondary_measurements(args, siso, cache, w, peaks, cores, dev)
 
     if not args.no_cpu_baseline and world == 1:
         import oracle
@@ -311,16 +392,140 @@ def run_ours(args):
         sample = f"first {n_sample} of {B} queries against all {args.rows} centroids, top-{k}"
         line["cpu_baseline"] = {"value": n_sample / t, "unit": UNIT, "cores": cores, "kind": "oracle", "sample": sample,
                                 "seconds": t}
-        # the sampled rows double as a full-size parity check of the timed configuration
+        # the sampled rows double as a full-size parity check of the timed configuration: decisions that differ from
+        # the oracle's outside the stated band (2e-3 for bf16), inside it, and outside a band of 1e-5
+        g_idx, g_hit = out[0][:n_sample].cpu().numpy(), out[2][:n_sample].cpu().numpy()
         g_sim = out[1][:n_sample].cpu().numpy().astype(np.float64)
+        diff = g_idx != o_idx
+        short = np.where(diff, np.abs(o_sim - g_sim), 0.0)       # how far the differing slot falls short of the rank's best
+        margin = np.abs(o_sim[:, 0] - w.theta[:n_sample].astype(np.float64))
+        hit_diff = g_hit != o_hit
         line["parity_sample"] = {"rows": n_sample, "max_sim_err": float(np.abs(g_sim - o_sim).max()),
-                                 "top1_equal": int((out[0][:n_sample, 0].cpu().numpy() == o_idx[:, 0]).sum()),
-                                 "hit_equal": int((out[2][:n_sample].cpu().numpy() == o_hit).sum())}
+                                 "top1_equal": int((g_idx[:, 0] == o_idx[:, 0]).sum()), "hit_equal": int((~hit_diff).sum()),
+                                 "outside_band": int((short > 2e-3).sum() + (hit_diff & (margin >= 2e-3)).sum()),
+                                 "excused": int(diff.sum() + hit_diff.sum()),
+                                 "strict_mismatch": int((short > 1e-5).sum() + (hit_diff & (margin >= 1e-5)).sum())}
     print(json.dumps(line), flush=True)
     cache.close()
     if world > 1:
         dist.destroy_process_group()
     return 0
+
+
+# ------------------------------------------------------------------------------ the rest of the target, in the default line
+def _time_ms(torch, fn, steps, warm):
+    for _ in range(warm):
+        fn()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / steps
+
+
+def small_batch_sweep(torch, cache, queries_dev, rows, dim, peaks, batches=(1, 8, 128, 256), steps=20, warm=3):
+    """Top-1 lookups of a few queries: the centroid matrix is streamed from HBM once per call."""
+    out = []
+    for b in batches:
+        q = queries_dev[:b].contiguous()
+        ms = _time_ms(torch, lambda: cache.lookup(q, 0.86, 1), steps, warm)
+        gbs = rows * dim * 2 / ms / 1e6
+        out.append({"batch": b, "us": round(ms * 1e3, 2), "GB/s": round(gbs, 1), "frac": round(gbs / peaks["hbm_gbs"], 4)})
+    return out
+
+
+def config5_steady_state(torch, siso, W, peaks, cores, dev, n_warm=400, n_timed=1200):
+    """The streaming step on a full cache (262,144 x 768 bf16, micro-batches of 256): lookup, hit update, eviction of
+    what the misses lack, insertion of the misses.  Returns (result dict, cache, one batch of queries on the device)."""
+    sp = W.StreamSpec()
+    stream = W.QueryStream(sp, threads=cores)
+
+    def to_dev(a):
+        return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    q_all = to_dev(stream.block(0, n_warm + n_timed, threads=cores))
+    cache = siso.SisoCache(sp.capacity, sp.dim, "bf16")
+    # the stream starts on an empty cache; to time the steady state (full cache, evicting every batch) the cache is
+    # first filled with later queries of the same stream
+    filler = stream.block(20000, 20000 + (sp.capacity - 2048) // sp.batch, threads=cores)
+    for lo in range(0, filler.shape[0], 1 << 16):
+        cache.insert(to_dev(filler[lo:lo + (1 << 16)]))
+    cache.check_status()
+    out = None
+    for t in range(n_warm):
+        out = cache.stream_step(q_all[t * 256:(t + 1) * 256], float(sp.theta), out=out)
+    torch.cuda.synchronize()
+    s0, l0 = cache.stats(), cache.launch_count
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for t in range(n_warm, n_warm + n_timed):
+        out = cache.stream_step(q_all[t * 256:(t + 1) * 256], float(sp.theta), out=out)
+    e1.record()
+    torch.cuda.synchronize()
+    cache.check_status()
+    s1 = cache.stats()
+    us = e0.elapsed_time(e1) / n_timed * 1e3
+    gbs = sp.capacity * sp.dim * 2 / (us * 1e-6) / 1e9
+    res = {"workload": "config 5 steady state: 262,144 x 768 bf16 cache, full; micro-batches of 256 (lookup, hit update, "
+                       "eviction, insertion of the misses)",
+           "us_per_batch": us, "queries_per_s": 256 / us * 1e6, "batches_timed": n_timed,
+           "hit_ratio": (s1["hits"] - s0["hits"]) / (256.0 * n_timed), "evictions": s1["evictions"] - s0["evictions"],
+           "inserts": s1["inserts"] - s0["inserts"], "launches_per_batch": (cache.launch_count - l0) / n_timed,
+           "roofline": {"bound": "hbm", "achieved": gbs, "peak": peaks["hbm_gbs"], "unit": "GB/s",
+                        "frac": gbs / peaks["hbm_gbs"],
+                        "note": "384 MiB of centroids per micro-batch over the whole step time; at 256 queries the step "
+                                "also sits on the tensor roof (flop per centroid byte = 256 against a ridge near 250)"}}
+    return res, cache, q_all[:256]
+
+
+def secondary_measurements(args, siso, cache4, w4, peaks, cores, dev):
+    """What the target names besides the headline: the streaming paths against the HBM roof (small-batch sweeps of both
+    stated matrices, the whole streaming step of configuration 5) and the hit update of configuration 2."""
+    import torch
+    from gen import workloads as W
+    t_start = time.perf_counter()
+    sec = {}
+
+    def to_dev(a):
+        return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    cache4.set_lookup_path(siso.PATH_AUTO)
+    sec["small_batch_1048576x1024"] = small_batch_sweep(torch, cache4, to_dev(w4.queries[:256]), args.rows, 1024, peaks)
+    c5, cache5, q5 = config5_steady_state(torch, siso, W, peaks, cores, dev)
+    sec["config5"] = c5
+    sec["small_batch_262144x768"] = small_batch_sweep(torch, cache5, q5, 262144, 768, peaks)
+    cache5.close()
+    # configuration 2: lookup, then the running-mean update of the hit centroids (65,536 queries into 65,536 rows)
+    w2 = W.config(2, threads=cores)
+    cache2 = siso.SisoCache(65536, 768, "bf16")
+    cache2.insert(to_dev(w2.centroids))
+    q, th = to_dev(w2.queries), torch.from_numpy(w2.theta).to(dev)
+    ms_l = _time_ms(torch, lambda: cache2.lookup(q, th, 1), 10, 3)
+    idx, sim, hit = cache2.lookup(q, th, 1)
+    times = []
+    for _ in range(7):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        cache2.update(q, idx, hit)
+        e1.record()
+        torch.cuda.synchronize()
+        times.append(e0.elapsed_time(e1))
+    cache2.check_status()
+    n_hit = int(hit.sum().item())
+    touched = int(torch.unique(idx[hit.bool(), 0]).numel())
+    upd_bytes = n_hit * 768 * 2 + touched * 768 * (4 + 4 + 2)        # hit queries read; master read + written, copy written
+    ms_u = statistics.median(times[2:])
+    sec["config2"] = {"workload": "config 2: 65,536 x 768 bf16, batch 65,536, Zipf 1.1, theta in [0.80, 0.92]",
+                      "lookup_ms": ms_l, "update_ms": ms_u, "hits": n_hit, "centroids_touched": touched,
+                      "lookup_frac_of_bf16_peak": 2.0 * 65536 * 65536 * 768 / ms_l / 1e9 / peaks["bf16_tflops"],
+                      "update_roofline": {"bound": "hbm", "achieved": upd_bytes / ms_u / 1e6, "peak": peaks["hbm_gbs"],
+                                          "unit": "GB/s", "frac": upd_bytes / ms_u / 1e6 / peaks["hbm_gbs"]}}
+    cache2.close()
+    sec["seconds"] = time.perf_counter() - t_start
+    return sec
 
 
 # ------------------------------------------------------------------------------ the other configurations
@@ -361,7 +566,24 @@ def run_other(args):
     steps, warm = args.steps, max(3, args.warmup)
     line = {"workload": args.workload, "n_gpus": 1, "steps": steps, "warmup": warm, "data": "synthetic",
             "peaks": peak_kind}
-    fp32_peak = 148 * 128 * 2 * 1.965e9 / 1e12            # FFMA lanes x 2 flop x max SM clock
+    props = torch.cuda.get_device_properties(0)
+    # nominal: SMs x 128 FP32 lanes x 2 flop x max SM clock; measured: the library's register-only FMA kernel
+    fp32_nominal = props.multi_processor_count * 128 * 2 * (getattr(props, "clock_rate", 1965000) * 1e3) / 1e12
+    probe = siso.SisoCache(64, 64, "f32")
+    fp32_peak = {"measured_tflops": probe.measure_fp32_fma(), "nominal_tflops": fp32_nominal,
+                 "sm_count": props.multi_processor_count}
+    probe.close()
+
+    def oracle_baseline(fn, value_of, unit, sample):
+        """The CPU oracle as it stands, timed once on the host cores beside the GPU number."""
+        if args.no_cpu_baseline:
+            return None
+        import oracle
+        oracle.build()
+        t0 = time.perf_counter()
+        res = fn(oracle)
+        t = time.perf_counter() - t0
+        return {"value": value_of(t), "unit": unit, "cores": cores, "kind": "oracle", "sample": sample, "seconds": t}, res
     if args.workload == "config1":
         w = W.config(1)
         cache = siso.SisoCache(1024, 384, "f32")
@@ -377,6 +599,10 @@ def run_other(args):
                               "peak_kind": "measured bf16 burst peak / 3 (split-bf16 emulation of fp32 products)",
                               "note": "3.2 GFLOP in six launches: a launch-latency-sized problem (one tile per CTA)",
                               "fp32_alu_peak": fp32_peak})
+        cb = oracle_baseline(lambda o: o.lookup(w.centroids, w.queries, w.theta, 1), lambda t: 4096 / t, UNIT,
+                             "the whole batch: 4,096 queries against 1,024 centroids")
+        if cb:
+            line["cpu_baseline"] = cb[0]
     elif args.workload == "config2":
         w = W.config(2, threads=cores)
         cache = siso.SisoCache(65536, 768, "bf16")
@@ -391,6 +617,19 @@ def run_other(args):
                     hit_ratio=float(hit.float().mean().item()),
                     roofline={"bound": "tensor", "achieved": fl / ms_l / 1e9, "peak": peaks["bf16_tflops"], "unit": "TFLOP/s",
                               "frac": fl / ms_l / 1e9 / peaks["bf16_tflops"], "kernel": "lookup only"})
+        n_s = min(65536, 64 * cores)
+        cb = oracle_baseline(lambda o: o.lookup(w.centroids, w.queries[:n_s], w.theta[:n_s], 1), lambda t: n_s / t, UNIT,
+                             f"lookup of the first {n_s} of 65,536 queries against all 65,536 centroids")
+        if cb:
+            line["cpu_baseline"] = cb[0]
+            import oracle
+            oc = oracle.OracleCache(65536, 768, "bf16")
+            oc.insert(w.centroids)
+            i_np, h_np = idx.cpu().numpy(), hit.cpu().numpy()
+            t0 = time.perf_counter()
+            oc.update(w.queries, i_np, h_np)
+            line["cpu_baseline"]["update_seconds"] = time.perf_counter() - t0
+            line["cpu_baseline"]["update_sample"] = "the whole batch of 65,536 queries with the GPU's decisions"
     elif args.workload == "config3":
         w = W.config(3, threads=cores)
         cache = siso.SisoCache(32768, 768, "f32")
@@ -418,6 +657,16 @@ def run_other(args):
                               "note": "whole pass (split, sweep, exact check, grouping, resolution, apply) over the "
                                       "lower-triangle flops N(N-1)/2 x 2D; the sweep kernel is about three quarters of it",
                               "fp32_alu_peak": fp32_peak})
+
+        def whole_merge(o):
+            oc = o.OracleCache(32768, 768, "f32")
+            oc.insert(w.centroids)
+            return oc.merge(W.MERGE_THRESHOLD_CONFIG3, True)
+
+        cb = oracle_baseline(whole_merge, lambda t: 32768 / t, "centroids/s", "the whole pass over all 32,768 centroids")
+        if cb:
+            line["cpu_baseline"] = cb[0]
+            line["cpu_baseline"]["merged_equal"] = bool(cb[1][1] == merged)
     elif args.workload == "f32_lookup":
         # an fp32 cache at scale: 262,144 x 1024 fp32 centroids (1 GiB), batch 4,096, top-4; clusters as in configuration 4
         N = 262144 if args.rows == (1 << 20) else args.rows

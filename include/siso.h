@@ -352,6 +352,20 @@ siso_status_t siso_import(siso_cache_t *c, const float *d_master, const double *
 siso_status_t siso_get_stats(siso_cache_t *c, int64_t *h_counts, void *stream);
 /* Synchronise `stream`, return the device status word (SISO_OK if clear) and clear it. */
 siso_status_t siso_sync_status(siso_cache_t *c, void *stream);
+/* Diagnostics (no passage of the paper: they serve the error model and the measurements of this library).
+ *   siso_selftest_wait_timeout  Every device-side wait of the tensor-core kernels is bounded; when one runs out the
+ *                      kernel records SISO_ERR_TIMEOUT in the status word and returns normally.  This call exercises
+ *                      exactly that path without touching a real sweep: one warp waits, with the kernels' own wait
+ *                      routine, at most poll_limit polls (1 .. 2^20) on a barrier that nothing arrives on and with no
+ *                      copy or tensor-core operation in flight.  Afterwards siso_sync_status returns SISO_ERR_TIMEOUT
+ *                      once and the handle is usable as before.  d_gave_up (device int32, may be NULL) receives 1 if
+ *                      the wait gave up.  Asynchronous on `stream`.
+ *   siso_measure_fp32_fma       FP32 fused multiply-add throughput of the device's CUDA cores in TFLOP/s (2 flop per
+ *                      FMA; best of three timed launches of a register-only kernel): the roof of the CUDA-core
+ *                      sweeps.  Synchronises `stream`. */
+siso_status_t siso_selftest_wait_timeout(siso_cache_t *c, uint32_t poll_limit, int32_t *d_gave_up, void *stream);
+siso_status_t siso_measure_fp32_fma(siso_cache_t *c, double *h_tflops, void *stream);
+
 /* Number of kernels this handle has launched so far (host-side count). */
 int64_t siso_launch_count(const siso_cache_t *c);
 const char *siso_status_string(siso_status_t s);

@@ -23,7 +23,8 @@ EXPORTS = ["siso_cache_create", "siso_cache_destroy", "siso_set_option", "siso_i
            "siso_stream_step", "siso_export", "siso_import", "siso_get_stats", "siso_sync_status",
            "siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_lookup_small_noalloc", "siso_cluster", "siso_cache_copy", "siso_update_centroids", "siso_lookup_keys", "siso_combine_keys", "siso_t2h", "siso_md1_wait",
            "siso_choose_theta", "siso_correct_theta", "siso_tier_exit_sim", "siso_tier_select", "siso_tier_finish",
-           "siso_route", "siso_evict_keys", "siso_select_evict", "siso_evict_slots"]
+           "siso_route", "siso_evict_keys", "siso_select_evict", "siso_evict_slots", "siso_selftest_wait_timeout",
+           "siso_measure_fp32_fma"]
 
 
 class SisoError(RuntimeError):
@@ -97,6 +98,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_import.argtypes = [vp, vp, vp, vp, vp, vp, ctypes.c_uint64, vp]
     L.siso_get_stats.argtypes = [vp, ctypes.POINTER(i64), vp]
     L.siso_sync_status.argtypes = [vp, vp]
+    L.siso_selftest_wait_timeout.argtypes = [vp, u32, vp, vp]
+    L.siso_measure_fp32_fma.argtypes = [vp, ctypes.POINTER(ctypes.c_double), vp]
     L.siso_launch_count.argtypes = [vp]
     L.siso_launch_count.restype = i64
     L.siso_status_string.argtypes = [i32]
@@ -139,9 +142,16 @@ class SisoCache:
         if use_torch_allocator:
             # the cache's own state and scratch live in torch's caching allocator
             def _alloc(nbytes, stream, ctx):
+                # the block is taken from the pool of the stream the library will first use it on (torch keeps one pool
+                # per stream and orders a block's reuse only against that stream); the library waits for the device before
+                # it hands a block back, so the release below needs no stream
                 try:
                     with torch.cuda.device(self._dev):
-                        t = torch.empty(int(nbytes), dtype=torch.uint8, device=self._dev)
+                        if stream:
+                            with torch.cuda.stream(torch.cuda.ExternalStream(int(stream), device=self._dev)):
+                                t = torch.empty(int(nbytes), dtype=torch.uint8, device=self._dev)
+                        else:
+                            t = torch.empty(int(nbytes), dtype=torch.uint8, device=self._dev)
                 except Exception:       # out of memory -> NULL -> SISO_ERR_OOM
                     return None
                 self._blocks[t.data_ptr()] = t
@@ -357,6 +367,19 @@ class SisoCache:
         self._check(self._lib.siso_get_stats(self._h, buf, _stream(stream)), "siso_get_stats")
         names = ["occupancy", "lookups", "hits", "inserts", "evictions", "merges", "clock", "rescans"]
         return {n: int(buf[i]) for i, n in enumerate(names)}
+
+    def selftest_wait_timeout(self, poll_limit: int = 4096, stream=None) -> torch.Tensor:
+        """Lets one bounded device-side wait run out (see siso_selftest_wait_timeout); returns the device flag."""
+        flag = torch.zeros(1, dtype=torch.int32, device=self._dev)
+        self._check(self._lib.siso_selftest_wait_timeout(self._h, int(poll_limit), _ptr(flag), _stream(stream)),
+                    "siso_selftest_wait_timeout")
+        return flag
+
+    def measure_fp32_fma(self, stream=None) -> float:
+        """Measured FP32 FMA throughput of the CUDA cores in TFLOP/s."""
+        v = ctypes.c_double(0.0)
+        self._check(self._lib.siso_measure_fp32_fma(self._h, ctypes.byref(v), _stream(stream)), "siso_measure_fp32_fma")
+        return float(v.value)
 
     def sync_status(self, stream=None) -> int:
         """Synchronise and return the device status word (0 = clear); it is cleared by the call."""

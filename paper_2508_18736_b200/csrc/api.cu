@@ -37,12 +37,24 @@ void *cache_alloc_zeroed(Cache *c, size_t bytes) {
     return p;
 }
 
+// A block that an earlier call handed to kernels is released only once the device is idle: the kernels of earlier
+// calls (on this stream or, for a handle used on several streams, on another one) may still be reading or writing it,
+// and an allocator with per-stream pools (torch's) would otherwise hand the block to someone else at once.  Regrowth is
+// rare (the buffers grow by a quarter more than asked and never shrink), so the wait costs nothing in the steady state.
+static siso_status_t retire_block(Cache *c, void *p) {
+    if (!p) return SISO_OK;
+    SISO_CUDA(cudaDeviceSynchronize());
+    c->alloc.free(p, c->alloc.ctx);
+    return SISO_OK;
+}
+
 siso_status_t scratch_reserve(Cache *c, size_t bytes, cudaStream_t s, Scratch *out) {
     bytes += 4096;
     if (bytes > c->ws_bytes) {
-        if (c->ws) c->alloc.free(c->ws, c->alloc.ctx);
+        void *old = c->ws;
         c->ws = nullptr;
         c->ws_bytes = 0;
+        SISO_TRY(retire_block(c, old));
         const size_t want = bytes + bytes / 4;
         c->ws = cache_alloc(c, want, s);
         if (!c->ws) return SISO_ERR_OOM;
@@ -51,6 +63,19 @@ siso_status_t scratch_reserve(Cache *c, size_t bytes, cudaStream_t s, Scratch *o
     out->base = static_cast<char *>(c->ws);
     out->off = 0;
     out->cap = c->ws_bytes;
+    return SISO_OK;
+}
+
+siso_status_t stage_reserve(Cache *c, size_t bytes, cudaStream_t s) {
+    if (bytes > c->stage_bytes) {
+        void *old = c->stage;
+        c->stage = nullptr;
+        c->stage_bytes = 0;
+        SISO_TRY(retire_block(c, old));
+        c->stage = cache_alloc(c, bytes, s);
+        if (!c->stage) return SISO_ERR_OOM;
+        c->stage_bytes = bytes;
+    }
     return SISO_OK;
 }
 
@@ -268,14 +293,7 @@ siso_status_t siso_lookup_host(siso_cache_t *c, const void *h_queries, int64_t n
     const size_t ib = pad256(sizeof(int32_t) * n_queries * k), sb = pad256(sizeof(float) * n_queries * k);
     const size_t hb = pad256(static_cast<size_t>(n_queries));
     const size_t need = qb + tb + ib + sb + hb;
-    if (need > c->stage_bytes) {
-        if (c->stage) c->alloc.free(c->stage, c->alloc.ctx);
-        c->stage = nullptr;
-        c->stage_bytes = 0;
-        c->stage = cache_alloc(c, need, s);
-        if (!c->stage) return SISO_ERR_OOM;
-        c->stage_bytes = need;
-    }
+    SISO_TRY(stage_reserve(c, need, s));
     char *p = static_cast<char *>(c->stage);
     void *dq = p; float *dt = reinterpret_cast<float *>(p + qb);
     int32_t *di = reinterpret_cast<int32_t *>(p + qb + tb);
@@ -331,14 +349,7 @@ siso_status_t siso_lookup_keys(siso_cache_t *c, const void *d_queries, int64_t n
     const size_t ib = pad256(sizeof(int32_t) * n_queries * k), sb = pad256(sizeof(float) * n_queries * k);
     const size_t hb = pad256(static_cast<size_t>(n_queries));
     const size_t need = ib + sb + hb;
-    if (need > c->stage_bytes) {
-        if (c->stage) c->alloc.free(c->stage, c->alloc.ctx);
-        c->stage = nullptr;
-        c->stage_bytes = 0;
-        c->stage = cache_alloc(c, need, s);
-        if (!c->stage) return SISO_ERR_OOM;
-        c->stage_bytes = need;
-    }
+    SISO_TRY(stage_reserve(c, need, s));
     char *p = static_cast<char *>(c->stage);
     int32_t *di = reinterpret_cast<int32_t *>(p);
     float *ds = reinterpret_cast<float *>(p + ib);

@@ -80,6 +80,7 @@ struct Scratch {
 };
 inline size_t pad256(size_t b) { return (b + 255) & ~size_t(255); }
 siso_status_t scratch_reserve(Cache *c, size_t bytes, cudaStream_t s, Scratch *out);
+siso_status_t stage_reserve(Cache *c, size_t bytes, cudaStream_t s);   // c->stage of at least `bytes`
 // memory that lives as long as the cache, set to zero; NULL if the allocator fails
 void *cache_alloc_zeroed(Cache *c, size_t bytes);
 siso_status_t check_cuda(cudaError_t e, const char *what);

@@ -45,14 +45,7 @@ siso_status_t siso_t2h(siso_cache_t *c, const void *d_queries, int64_t n_queries
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     // results of the test lookups live in the staging buffer (the lookup itself uses the scratch buffer)
     const size_t ib = pad256(sizeof(int32_t) * n_queries), sb = pad256(sizeof(float) * n_queries), hb = pad256(n_queries);
-    if (ib + sb + hb > cc->stage_bytes) {
-        if (cc->stage) cc->alloc.free(cc->stage, cc->alloc.ctx);
-        cc->stage = nullptr;
-        cc->stage_bytes = 0;
-        cc->stage = cc->alloc.alloc(ib + sb + hb, s, cc->alloc.ctx);
-        if (!cc->stage) return SISO_ERR_OOM;
-        cc->stage_bytes = ib + sb + hb;
-    }
+    SISO_TRY(stage_reserve(cc, ib + sb + hb, s));
     char *p = static_cast<char *>(cc->stage);
     int32_t *idx = reinterpret_cast<int32_t *>(p);
     float *best = reinterpret_cast<float *>(p + ib);

@@ -159,6 +159,55 @@ def test_fp32_tensor_path_sees_every_change_of_the_vectors():
     cache.close()
 
 
+def test_scratch_regrowth_on_a_side_stream_matches_oracle():
+    """Lookups of growing size on a stream that is not torch's current one: every growth replaces the handle's scratch
+    and staging buffers while kernels of the earlier calls are still queued.  Tensors allocated and overwritten on the
+    current stream right after each call would land in a block that was handed back too early."""
+    w = W.config(2, n_centroids=6000, n_queries=1500, dim=768, n_clusters=128, mode="P")
+    cache = siso.SisoCache(6000, 768, "bf16")
+    cache.insert(to_dev(w.centroids, "bf16"))
+    torch.cuda.synchronize()
+    q_all, th_all = to_dev(w.queries, "bf16"), torch.from_numpy(w.theta).cuda()
+    side = torch.cuda.Stream()
+    results, junk = [], []
+    for n in (4, 130, 700, 1500, 9):
+        side.wait_stream(torch.cuda.current_stream())
+        results.append((n, cache.lookup(q_all[:n], th_all[:n], 4, stream=side)))
+        junk.append([torch.full((1 << 22,), 255, dtype=torch.uint8, device="cuda") for _ in range(6)])
+    side.synchronize()
+    torch.cuda.synchronize()
+    assert cache.sync_status(side) == 0
+    for n, (idx, sim, hit) in results:
+        ora = oracle.lookup(w.centroids, w.queries[:n], w.theta[:n], 4)
+        check_lookup((idx.cpu().numpy(), sim.cpu().numpy(), hit.cpu().numpy()), ora, w.centroids, w.queries[:n],
+                     w.theta[:n], TOL["bf16"])
+    cache.close()
+
+
+def test_a_device_wait_that_runs_out_reports_timeout_and_the_handle_stays_usable():
+    """Every wait inside the tensor-core kernels is bounded.  Here the kernels' own wait routine polls a barrier that
+    nothing arrives on (no copy, no tensor-core operation in flight) until its limit runs out: the status word must say
+    SISO_ERR_TIMEOUT once, the kernel must have returned normally, and the next lookup must be right."""
+    w = W.config(2, n_centroids=1500, n_queries=200, dim=768, n_clusters=64, mode="P")
+    cache = siso.SisoCache(1500, 768, "bf16")
+    cache.insert(to_dev(w.centroids, "bf16"))
+    cache.check_status()
+    flag = cache.selftest_wait_timeout(2048)
+    assert cache.sync_status() == 6                      # SISO_ERR_TIMEOUT
+    assert flag.item() == 1
+    assert cache.sync_status() == 0                      # reported once, then clear
+    with pytest.raises(siso.SisoError):
+        cache.selftest_wait_timeout(0)
+    cache.set_lookup_path(siso.PATH_TENSOR)
+    idx, sim, hit = cache.lookup(to_dev(w.queries, "bf16"), torch.from_numpy(w.theta).cuda(), 4)
+    check_lookup((idx.cpu().numpy(), sim.cpu().numpy(), hit.cpu().numpy()),
+                 oracle.lookup(w.centroids, w.queries, w.theta, 4), w.centroids, w.queries, w.theta, TOL["bf16"])
+    cache.check_status()
+    tf = cache.measure_fp32_fma()
+    assert 20.0 < tf < 120.0, tf                         # 148 SMs x 128 lanes x 2 flop x 1.0-2.0 GHz
+    cache.close()
+
+
 def test_bad_arguments_return_status_and_touch_nothing():
     cache = siso.SisoCache(64, 64, "bf16")
     q = torch.zeros(4, 64, dtype=torch.bfloat16, device="cuda")

@@ -5,7 +5,7 @@ import torch
 
 import oracle
 from gen import workloads as W
-from util import TOL, check_lookup, to_dev, widen64
+from util import TOL, check_lookup, to_dev, verify_merge_map, widen64
 
 pytestmark = pytest.mark.gpu
 
@@ -47,6 +47,26 @@ def assert_state_equal(cache, ora, dtype, what=""):
         m = torch.from_numpy(g["master"]).to(torch.bfloat16).view(torch.int16).numpy().view(np.uint16)
         assert (m[live] == g["vecs"][live]).all(), what
     assert cache.stats()["occupancy"] == int(live.sum()) and cache.stats()["clock"] == ora.clock, what
+
+
+def adopt_gpu_merge(cache, ora, mm, entry, valid0, seed, sizes0, theta_c, weighted, what):
+    """The GPU's merge map differs from the oracle's.  That is accepted only if the map is a valid outcome of
+    Algorithm 1 with every comparison within 1e-5 of the oracle's (a decision at the threshold or between two
+    equally close survivors, and what follows from it); the applied state is then checked against that map's own
+    closed form, and the oracle carries on from the GPU's state."""
+    size = verify_merge_map(entry, valid0, seed, sizes0, mm, theta_c, tol=1e-5)
+    g = state_np(cache)
+    surv = (mm == np.arange(len(mm)))
+    assert (g["valid"] == surv).all(), what
+    np.testing.assert_array_equal(g["size"][surv], size[surv], err_msg=what)
+    for s in np.flatnonzero(surv):
+        members = np.flatnonzero(mm == s)
+        if weighted and len(members) > 1:
+            v = (sizes0[members, None] * entry[members]).sum(0)
+            assert np.abs(g["master"][s] - v / np.linalg.norm(v)).max() <= 1e-6, what
+        else:
+            assert np.abs(g["master"][s] - entry[s]).max() <= 1e-6, what
+    ora.load_state(g["master"], g["size"], g["access"], g["last"], g["valid"], ora.clock)
 
 
 def dataclass_slice(w, lo, hi):
@@ -131,15 +151,9 @@ def test_self_merge_matches_oracle(dtype, mode, theta_c, weighted, sweep):
         o_mm, o_n = ora.merge(theta_c, weighted)
         mm = mm.cpu().numpy()
         if not (mm == o_mm).all():
-            # a differing target is allowed only where the deciding similarity is within tolerance of theta_c
-            # or of the runner-up; check validity and adopt the GPU's state
-            bad = np.flatnonzero(mm != o_mm)
-            S = before["master"].astype(np.float64)
-            for i in bad:
-                cand = [int(t) for t in (mm[i], o_mm[i]) if t != i]
-                sims = [float(S[i] @ S[t]) for t in cand]
-                assert min(abs(s - theta_c) for s in sims) < 1e-5 or (len(sims) == 2 and abs(sims[0] - sims[1]) < 1e-5)
-            pytest.skip("near-threshold merge decision: lock-step comparison ends here")
+            adopt_gpu_merge(cache, ora, mm, before["master"].astype(np.float64), before["valid"],
+                            np.zeros(len(mm), np.uint8), before["size"], theta_c, weighted, f"merge pass {rounds}")
+            o_n = int((mm[mm >= 0] != np.flatnonzero(mm >= 0)).sum())
         assert n == o_n
         assert_state_equal(cache, ora, dtype, f"merge pass {rounds}")
         if rounds == 0:
@@ -221,12 +235,12 @@ def test_two_set_merge_matches_oracle(dtype, weighted, sweep):
     cache.set_option(2, 200000)
     mm, n = cache.merge(0.9, flags, repo=to_dev(repo, dtype), repo_sizes=torch.from_numpy(repo_sizes))
     ora.insert(repo, sizes=repo_sizes)
+    entry, valid0, sizes0 = ora.master.copy(), ora.valid.copy(), ora.size.copy()
     o_mm, o_n = ora.merge(0.9, weighted, seed_mask=seed, new_access_inf=True)
     mm = mm.cpu().numpy()
     if not (mm == o_mm).all():
-        bad = np.flatnonzero(mm != o_mm)
-        S = state_np(cache)["master"].astype(np.float64)
-        pytest.skip(f"near-threshold merge decision on {len(bad)} rows")
+        adopt_gpu_merge(cache, ora, mm, entry, valid0, seed, sizes0, 0.9, weighted, "two-set merge")
+        o_n = int((mm[mm >= 0] != np.flatnonzero(mm >= 0)).sum())
     assert n == o_n and n > 100
     assert_state_equal(cache, ora, dtype, "two-set merge")
     live = ora.valid == 1
@@ -295,11 +309,16 @@ def test_insert_misses_and_capacity_error():
     assert all((before[k] == after[k]).all() for k in before)
 
 
-@pytest.mark.parametrize("theta_mode,dtype,batch", [("fixed", "bf16", 256), ("per_query", "bf16", 256), ("fixed", "f32", 256),
-                                                    ("fixed", "bf16", 100)])      # 100: a batch that is padded to a query tile
-def test_streaming_step_lockstep_on_a_scaled_twin(theta_mode, dtype, batch):
-    sp = W.StreamSpec(capacity=1024, dim=128, n_queries=batch * 60, batch=batch, n_clusters=400, zipf_s=1.2,
-                      reshuffle_every=batch * 30, theta=0.86, mode="P", dtype=dtype)
+@pytest.mark.parametrize("theta_mode,dtype,batch,capacity,dim,n_batches,n_clusters", [
+    ("fixed", "bf16", 256, 1024, 128, 60, 400), ("per_query", "bf16", 256, 1024, 128, 60, 400),
+    ("fixed", "f32", 256, 1024, 128, 60, 400),
+    ("fixed", "bf16", 100, 1024, 128, 60, 400),           # 100: a batch that is padded to a query tile
+    ("fixed", "bf16", 256, 4096, 768, 782, 1024),         # the scaled twin of the streaming configuration: 200,000 queries
+])
+def test_streaming_step_lockstep_on_a_scaled_twin(theta_mode, dtype, batch, capacity, dim, n_batches, n_clusters):
+    n_queries = 200_000 if n_batches == 782 else batch * n_batches
+    sp = W.StreamSpec(capacity=capacity, dim=dim, n_queries=n_queries, batch=batch, n_clusters=n_clusters, zipf_s=1.2,
+                      reshuffle_every=n_queries // 2, theta=0.86, mode="P", dtype=dtype)
     st = W.QueryStream(sp)
     cache = siso.SisoCache(sp.capacity, sp.dim, dtype)
     ora = oracle.OracleCache(sp.capacity, sp.dim, dtype)
@@ -325,6 +344,38 @@ def test_streaming_step_lockstep_on_a_scaled_twin(theta_mode, dtype, batch):
     s = cache.stats()
     assert s["inserts"] - s["evictions"] == s["occupancy"] and s["lookups"] == sp.n_queries
     cache.check_status()
+
+
+@pytest.mark.parametrize("fused", [1, 0])
+def test_streaming_step_reproduces_the_hand_computed_example(golden_dir, fused):
+    """The two pencil-computed batches of tests/golden/streaming_two_batches.json (capacity 4; one hit and two misses
+    each; one free slot, then none) through siso_stream_step itself, not through the oracle: outputs and the whole
+    state after each batch.  The vectors are padded with zeros from dim 4 to dim 8 (rows must be multiples of 8)."""
+    import json, os
+    ex = json.load(open(os.path.join(golden_dir, "streaming_two_batches.json")))
+    inf = lambda a: np.array([siso.ACCESS_INF if x == "inf" else x for x in a], dtype=np.uint32)
+    pad = lambda v: np.pad(np.array(v, dtype=np.float32), ((0, 0), (0, 4)))
+    cache = siso.SisoCache(ex["capacity"], 8, "f32")
+    cache.set_option(siso.OPT_STREAM_FUSED, fused)
+    init = ex["initial"]
+    cache.import_(torch.from_numpy(pad(init["vectors"])), torch.tensor(init["size"], dtype=torch.float64),
+                  torch.from_numpy(inf(init["access"]).view(np.int32)), torch.tensor(init["last"], dtype=torch.int64),
+                  torch.tensor(init["valid"], dtype=torch.uint8), ex["clock_before"])
+    for b in ex["batches"]:
+        out = [x.cpu().numpy() for x in cache.stream_step(torch.from_numpy(pad(b["queries"])).cuda(), float(ex["theta"]))]
+        idx, sim, hit, victims, slots = out
+        assert idx[:, 0].tolist() == b["idx"] and hit.tolist() == b["hit"]
+        assert np.abs(sim[:, 0] - np.array(b["sim"])).max() <= 1e-6
+        nv = len(b["victims"])
+        assert victims[:nv].tolist() == b["victims"] and (victims[nv:] == -1).all()
+        assert slots.tolist() == b["slots"]
+        g, a = state_np(cache), b["after"]
+        assert g["valid"].tolist() == a["valid"] and cache.stats()["clock"] == a["clock"]
+        assert np.abs(g["master"][:, :4] - np.array(a["vectors"])).max() <= 1e-6 and (g["master"][:, 4:] == 0).all()
+        assert g["size"].tolist() == a["size"] and g["access"].tolist() == inf(a["access"]).tolist()
+        assert g["last"].tolist() == a["last"]
+    cache.check_status()
+    cache.close()
 
 
 def test_fused_streaming_maintenance_equals_separate_kernels_bit_for_bit():
@@ -400,9 +451,10 @@ def test_algorithm1_with_progressive_update_matches_oracle(dtype):
     seed = o_new.valid.copy()
     mm, n_merged = new.merge(0.9, siso.MERGE_SIZES_ONLY, repo=to_dev(repo, dtype), repo_sizes=torch.from_numpy(repo_sizes))
     o_new.insert(repo, sizes=repo_sizes)
+    entry, valid0, sizes0 = o_new.master.copy(), o_new.valid.copy(), o_new.size.copy()
     o_mm, o_n = o_new.merge(0.9, False, seed_mask=seed, new_access_inf=True)
     if not (mm.cpu().numpy() == o_mm).all():
-        pytest.skip("near-threshold merge decision")
+        adopt_gpu_merge(new, o_new, mm.cpu().numpy(), entry, valid0, seed, sizes0, 0.9, False, "C_new after the merge")
     over = o_new.occupancy - M
     assert over > 0 and (new.evict(over, siso.EVICT_DECAY).cpu().numpy() == o_new.evict(over, decay=True)).all()
     assert_state_equal(new, o_new, dtype, "C_new after filtering")

@@ -4,14 +4,16 @@ Some users of the library call it from places where the CUDA allocator is off li
 with all device memory handed out at start-up, a callback under an allocator lock).  For them the
 library has one entry point whose scratch is a fixed array inside the library image.  This test calls
 it through the C ABI twice in a row on different inputs - the shared scratch still holds the first
-call's partial results when the second runs - and checks both results against siso_lookup, then checks
+call's partial results when the second runs - and checks both results against siso_lookup and against
+the CPU oracle, checks that the calls leave the amount of allocated device memory unchanged, then checks
 that sizes beyond the fixed limits are refused.  It is collected last on purpose."""
 import numpy as np
 import pytest
 import torch
 
 from gen import workloads as W
-from util import TOL, to_dev
+import oracle
+from util import TOL, check_lookup, to_dev
 
 pytestmark = pytest.mark.gpu
 
@@ -40,8 +42,16 @@ def test_no_alloc_lookup_matches_ordinary_lookup_twice_in_a_row(dtype, dim):
         idx = torch.full((n, k), -7, dtype=torch.int32, device="cuda")
         sim = torch.zeros((n, k), dtype=torch.float32, device="cuda")
         hit = torch.full((n,), 9, dtype=torch.uint8, device="cuda")
+        torch.cuda.synchronize()
+        free_before, held_before = torch.cuda.mem_get_info()[0], torch.cuda.memory_allocated()
         siso.lookup_small_noalloc(cent, q, theta, k, idx, sim, hit, valid=valid)
         torch.cuda.synchronize()
+        if lo > 0:        # the first call on a device may still load the library's kernels; the second changes nothing
+            assert torch.cuda.mem_get_info()[0] == free_before and torch.cuda.memory_allocated() == held_before
+        th_np = w.theta[lo:lo + n] if use_vec else np.full(n, 0.86, np.float32)
+        ora = oracle.lookup(w.centroids, w.queries[lo:lo + n], th_np, k, valid.cpu().numpy())
+        check_lookup((idx.cpu().numpy(), sim.cpu().numpy(), hit.cpu().numpy()), ora, w.centroids, w.queries[lo:lo + n],
+                     th_np, tol, valid=valid.cpu().numpy())
         assert (sim - want_sim).abs().max().item() <= tol
         gap_ok = (want_sim[:, :-1] - want_sim[:, 1:]).min(dim=1).values >= tol     # rows without near-ties
         assert torch.equal(idx[gap_ok], want_idx[gap_ok])
