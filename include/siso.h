@@ -64,6 +64,10 @@ typedef enum { SISO_F32 = 0, SISO_BF16 = 1 } siso_dtype_t;
                                            of at most 1024 rows into one cooperative launch; 0: separate kernels */
 #define SISO_OPT_MERGE_PATH 5           /* pairwise sweep of siso_merge: SISO_PATH_AUTO (default: tensor cores from 4096
                                            entries), SISO_PATH_SIMT or SISO_PATH_TENSOR; the results are the same */
+#define SISO_OPT_SWEEP_FINALIZE 6       /* 0 (default): a top-1 tensor-core lookup of at most 256 queries picks its results inside the
+                                         * sweep kernel; 1: always by a separate finalisation launch */
+#define SISO_OPT_STREAM_LIST 7          /* 0 (default): on a full cache the fused streaming step takes its victims from an
+                                         * eviction-order list kept across batches (no grid-wide barrier); 1: never */
 #define SISO_OPT_TENSOR_CTA_PAIR 3      /* 0 (default): tensor-core lookup runs CTA pairs for >= 2 query tiles; 1: never */
 #define SISO_PATH_AUTO 0
 #define SISO_PATH_SIMT 1   /* CUDA-core tiled sweep (fp32 accumulate of exact products)        */

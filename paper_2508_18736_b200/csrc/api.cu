@@ -167,6 +167,7 @@ siso_status_t siso_cache_create(siso_cache_t **out, const siso_config_t *cfg) {
     else { c->alloc.alloc = default_alloc; c->alloc.free = default_free; c->alloc.ctx = nullptr; c->own_alloc = true; }
     c->lookup_path = SISO_PATH_AUTO;
     c->stream_fused = 1;
+    c->low_dirty = true;
     c->merge_max_cand = 16 * c->capacity + (1ll << 20);
 
     const size_t rows = static_cast<size_t>(c->rows_alloc), D = static_cast<size_t>(c->dim);
@@ -204,7 +205,7 @@ siso_status_t siso_cache_destroy(siso_cache_t *c) {
     cudaDeviceSynchronize();
     tensor_state_destroy(c);
     void *ptrs[] = {c->dtype == SISO_F32 ? nullptr : c->vecs, c->master, c->size, c->access, c->last, c->valid,
-                    c->counters, c->status, c->ws, c->stage, c->swap_plan, c->split_hi, c->split_lo};
+                    c->counters, c->status, c->ws, c->stage, c->swap_plan, c->split_hi, c->split_lo, c->low_list};
     for (void *p : ptrs)
         if (p) c->alloc.free(p, c->alloc.ctx);
     delete c;
@@ -226,6 +227,15 @@ siso_status_t siso_set_option(siso_cache_t *c, int32_t key, int64_t value) {
             if (value != 0 && value != 1) return SISO_ERR_INVALID_ARG;
             c->stream_fused = static_cast<int32_t>(value);
             return SISO_OK;
+        case SISO_OPT_SWEEP_FINALIZE:
+            if (value != 0 && value != 1) return SISO_ERR_INVALID_ARG;
+            c->sweep_finalize_separate = static_cast<int32_t>(value);
+            return SISO_OK;
+        case SISO_OPT_STREAM_LIST:
+            if (value != 0 && value != 1) return SISO_ERR_INVALID_ARG;
+            c->stream_list_off = static_cast<int32_t>(value);
+            c->low_dirty = true;
+            return SISO_OK;
         case SISO_OPT_MERGE_PATH:
             if (value != SISO_PATH_AUTO && value != SISO_PATH_SIMT && value != SISO_PATH_TENSOR) return SISO_ERR_INVALID_ARG;
             c->merge_path = static_cast<int32_t>(value);
@@ -243,6 +253,7 @@ siso_status_t siso_insert(siso_cache_t *c, const void *d_vecs, const double *d_s
     if (!c || n < 0 || (n > 0 && !d_vecs)) return SISO_ERR_INVALID_ARG;
     if (n > 0 && !aligned16(d_vecs)) return SISO_ERR_INVALID_ARG;
     SISO_CUDA(cudaSetDevice(c->device));
+    c->low_dirty = true;        // entries or their metadata change outside the streaming maintenance kernel
     return launch_insert(c, d_vecs, d_sizes, nullptr, n, d_slots_out, static_cast<cudaStream_t>(stream));
 }
 
@@ -313,6 +324,7 @@ siso_status_t siso_update(siso_cache_t *c, const void *d_queries, int64_t n_quer
     if (!c || n_queries < 0 || idx_stride < 1) return SISO_ERR_INVALID_ARG;
     if (n_queries > 0 && (!d_queries || !d_idx || !d_hit || !aligned16(d_queries))) return SISO_ERR_INVALID_ARG;
     SISO_CUDA(cudaSetDevice(c->device));
+    c->low_dirty = true;        // entries or their metadata change outside the streaming maintenance kernel
     return launch_update(c, d_queries, n_queries, d_idx, idx_stride, d_hit, static_cast<cudaStream_t>(stream));
 }
 
@@ -323,6 +335,7 @@ siso_status_t siso_merge(siso_cache_t *c, const void *d_repo, const double *d_re
         return SISO_ERR_INVALID_ARG;
     if (n_repo >= (1ll << 31)) return SISO_ERR_UNSUPPORTED;
     SISO_CUDA(cudaSetDevice(c->device));
+    c->low_dirty = true;        // entries or their metadata change outside the streaming maintenance kernel
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     long long *d_n = nullptr;
     if (h_n_merged) d_n = c->counters + CNT_SPARE;
@@ -401,6 +414,7 @@ siso_status_t siso_evict_slots(siso_cache_t *c, const int64_t *d_victims, int64_
                                void *stream) {
     if (!c || n < 0 || slot_offset < 0 || (n > 0 && !d_victims) || (flags & ~SISO_EVICT_DECAY)) return SISO_ERR_INVALID_ARG;
     SISO_CUDA(cudaSetDevice(c->device));
+    c->low_dirty = true;        // entries or their metadata change outside the streaming maintenance kernel
     return launch_evict_slots(c, reinterpret_cast<const long long *>(d_victims), n, slot_offset, flags,
                               static_cast<cudaStream_t>(stream));
 }
@@ -410,6 +424,7 @@ siso_status_t siso_cache_copy(siso_cache_t *dst, siso_cache_t *src, void *stream
     if (dst->dim != src->dim || dst->dtype != src->dtype || dst->device != src->device) return SISO_ERR_INVALID_ARG;
     if (dst->capacity < src->capacity) return SISO_ERR_CAPACITY;
     SISO_CUDA(cudaSetDevice(dst->device));
+    dst->low_dirty = true;
     return launch_cache_copy(dst, src, static_cast<cudaStream_t>(stream));
 }
 
@@ -418,6 +433,7 @@ siso_status_t siso_update_centroids(siso_cache_t *cur, siso_cache_t *c_new, int6
     if (cur->dim != c_new->dim || cur->dtype != c_new->dtype || cur->device != c_new->device) return SISO_ERR_INVALID_ARG;
     if (first_slot > cur->capacity) return SISO_ERR_INVALID_ARG;
     SISO_CUDA(cudaSetDevice(cur->device));
+    cur->low_dirty = true;
     return launch_update_centroids(cur, c_new, first_slot, n_slots, static_cast<cudaStream_t>(stream));
 }
 
@@ -446,6 +462,7 @@ siso_status_t siso_cluster(siso_cache_t *c, const void *d_vecs, int64_t n, float
 siso_status_t siso_evict(siso_cache_t *c, int64_t n_evict, uint32_t flags, int32_t *d_victims, void *stream) {
     if (!c || n_evict < 0 || (flags & ~SISO_EVICT_DECAY)) return SISO_ERR_INVALID_ARG;
     SISO_CUDA(cudaSetDevice(c->device));
+    c->low_dirty = true;        // entries or their metadata change outside the streaming maintenance kernel
     return launch_evict(c, n_evict, nullptr, 0, flags, d_victims, n_evict, static_cast<cudaStream_t>(stream));
 }
 
@@ -453,6 +470,7 @@ siso_status_t siso_make_room(siso_cache_t *c, const uint8_t *d_hit, int64_t n, u
                              void *stream) {
     if (!c || n < 0 || (n > 0 && !d_hit) || (flags & ~SISO_EVICT_DECAY)) return SISO_ERR_INVALID_ARG;
     SISO_CUDA(cudaSetDevice(c->device));
+    c->low_dirty = true;        // entries or their metadata change outside the streaming maintenance kernel
     return launch_evict(c, -1, d_hit, n, flags, d_victims, n, static_cast<cudaStream_t>(stream));
 }
 
@@ -460,6 +478,7 @@ siso_status_t siso_insert_misses(siso_cache_t *c, const void *d_queries, int64_t
                                  int32_t *d_slots_out, void *stream) {
     if (!c || n < 0 || (n > 0 && (!d_queries || !d_hit || !aligned16(d_queries)))) return SISO_ERR_INVALID_ARG;
     SISO_CUDA(cudaSetDevice(c->device));
+    c->low_dirty = true;        // entries or their metadata change outside the streaming maintenance kernel
     return launch_insert(c, d_queries, nullptr, d_hit, n, d_slots_out, static_cast<cudaStream_t>(stream));
 }
 
@@ -511,6 +530,7 @@ siso_status_t siso_import(siso_cache_t *c, const float *d_master, const double *
     if (!c || !d_master || !d_sizes || !d_access || !d_last || !d_valid) return SISO_ERR_INVALID_ARG;
     c->vec_epoch += 1;          // the vectors may change: derived copies (the split-bf16 parts) are stale
     SISO_CUDA(cudaSetDevice(c->device));
+    c->low_dirty = true;        // entries or their metadata change outside the streaming maintenance kernel
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t n = static_cast<size_t>(c->capacity), D = static_cast<size_t>(c->dim);
     SISO_CUDA(cudaMemcpyAsync(c->master, d_master, n * D * 4, cudaMemcpyDeviceToDevice, s));

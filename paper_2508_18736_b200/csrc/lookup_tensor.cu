@@ -323,6 +323,7 @@ struct TensorState {
     CUtensorMap map_c_half;   // box of 128 centroid rows (CTA-pair kernel: each CTA stages half a tile)
     bool attr_set[3];
     bool attr_set_pair[3];
+    unsigned int *tail_counter;   // ticket counters of the in-sweep finalisation (one per query tile of a pair), zero between launches
 };
 
 static siso_status_t encode_map(EncodeTiledFn fn, CUtensorMap *map, const void *base, uint64_t rows, uint64_t dim,
@@ -342,10 +343,14 @@ static siso_status_t encode_map(EncodeTiledFn fn, CUtensorMap *map, const void *
 
 siso_status_t launch_lookup_tensor_pair(Cache *c, bool *attr_set3, const CUtensorMap &map_q, const CUtensorMap &map_c_half,
                                         int64_t B, int kmax, int tiles_per_split, int n_tiles, int splits, int m_tiles_even,
-                                        unsigned long long *partial, cudaStream_t s);
+                                        unsigned long long *partial, unsigned int *tail_counter, const float *theta,
+                                        float theta_s, int32_t *idx, float *sim, uint8_t *hit, long long *counters,
+                                        cudaStream_t s);
 
 void tensor_state_destroy(Cache *c) {
-    delete static_cast<tc::TensorState *>(c->tensor_state);
+    auto *ts = static_cast<tc::TensorState *>(c->tensor_state);
+    if (ts && ts->tail_counter) c->alloc.free(ts->tail_counter, c->alloc.ctx);
+    delete ts;
     c->tensor_state = nullptr;
 }
 
@@ -385,6 +390,10 @@ siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const flo
         if (st == SISO_OK)
             st = tc::encode_map(ts->encode, &ts->map_c_half, c->vecs, static_cast<uint64_t>(c->rows_alloc),
                                 static_cast<uint64_t>(c->dim), tc::TN / 2);
+        if (st == SISO_OK) {
+            ts->tail_counter = static_cast<unsigned int *>(cache_alloc_zeroed(c, 256 + 256 * sizeof(unsigned long long)));   // tickets, then one word per row
+            if (!ts->tail_counter) st = SISO_ERR_OOM;
+        }
         if (st != SISO_OK) { delete ts; return st; }
         c->tensor_state = ts;
     }
@@ -438,16 +447,19 @@ siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const flo
     CUtensorMap map_q;
     SISO_TRY(tc::encode_map(ts->encode, &map_q, q_rows, q_row_count, static_cast<uint64_t>(c->dim), tc::TM));
     siso_status_t st;
+    // a top-1 lookup of one CTA pair's worth of queries is finished by the sweep itself (no finalisation launch)
+    const bool in_sweep = pair && kmax == 1 && m_ctas == 2 && !c->sweep_finalize_separate;
     if (pair)
         st = launch_lookup_tensor_pair(c, ts->attr_set_pair, map_q, ts->map_c_half, B, kmax, tiles_per_split, n_tiles, splits,
-                                       m_ctas, partial, s);
+                                       m_ctas, partial, in_sweep ? ts->tail_counter : nullptr, theta, theta_s, idx, sim, hit,
+                                       defer ? nullptr : c->counters, s);
     else
         st = kmax == 1 ? run_tensor<1>(c, ts, 0, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s)
            : kmax == 4 ? run_tensor<4>(c, ts, 1, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s)
                        : run_tensor<8>(c, ts, 2, map_q, B, tiles_per_split, n_tiles, splits, m_tiles, partial, s);
     SISO_TRY(st);
     if (defer) {
-        defer->partial = partial;
+        defer->partial = in_sweep ? nullptr : partial;       // NULL: idx / sim / hit are already final
         defer->splits = splits;
         defer->theta = theta;
         defer->theta_s = theta_s;
@@ -455,6 +467,7 @@ siso_status_t launch_lookup_tensor(Cache *c, const void *q, int64_t B, const flo
         *tail = scr.base + scr.off;
         return SISO_OK;
     }
+    if (in_sweep) return SISO_OK;
     return launch_topk_finalize(c, partial, B, splits, kmax, k, theta, theta_s, idx, sim, hit, s);
 }
 

@@ -43,13 +43,30 @@ struct Barriers {
     uint64_t full[STAGES], empty[STAGES], acc_full[ACC_STAGES], acc_empty[ACC_STAGES];
     uint32_t tmem_base;
     int abort_flag;
+    int is_last;
+};
+
+// Top-1 lookups of at most two query tiles (a streaming micro-batch) are finished inside the sweep: every CTA folds
+// the best key of each of its rows into a per-row word with an atomic maximum, and the CTA that is the last of its
+// query tile to have done so (a ticket counter per query tile, no waiting) reads the words out and applies the threshold.  That saves a kernel launch, or a phase and
+// a grid-wide barrier of the streaming maintenance kernel.  counter == NULL: the partial results are all there is.
+struct TailFinal {
+    unsigned int *counter;     // [query tiles], zero between launches
+    unsigned long long *best;  // [256] best key of every row so far, zero between launches
+    const float *theta;
+    float theta_s;
+    int32_t *idx;              // [B]
+    float *sim;                // [B]
+    uint8_t *hit;              // [B]
+    long long *counters;       // lookups and hits are counted here unless NULL (the caller then counts them itself)
 };
 
 template <int KMAX>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 lookup_tensor_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_constant__ CUtensorMap map_c_half,
                           const uint8_t *__restrict__ valid, int64_t B, int D, int tiles_per_split, int n_tiles,
-                          unsigned long long *__restrict__ partial, int splits, int stream_c, int *status) {
+                          unsigned long long *__restrict__ partial, int splits, int stream_c, int *status,
+                          const TailFinal tail) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *tiles = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     Barriers *bars = reinterpret_cast<Barriers *>(tiles + STAGES * STAGE_BYTES);
@@ -192,6 +209,10 @@ lookup_tensor_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
             unsigned long long *dst = partial + ((static_cast<int64_t>(q0) + row) * splits + split) * KMAX;
 #pragma unroll
             for (int j = 0; j < KMAX; ++j) dst[j] = top.key(j);
+            if (KMAX == 1 && tail.counter) {
+                atomicMax(tail.best + static_cast<int64_t>(q0) + row, top.key(0));
+                __threadfence();                                  // folded in before this CTA takes its ticket
+            }
         }
     }
 
@@ -208,6 +229,41 @@ lookup_tensor_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
         tcgen05_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::2.sync.aligned.b32 %0, %1;" ::"r"(tmem_base), "r"(TMEM_COLS) : "memory");
     }
+    if constexpr (KMAX == 1) {
+        if (tail.counter) {
+            if (threadIdx.x == 0) {
+                __threadfence();
+                const unsigned int ticket = atomicAdd(&tail.counter[blockIdx.x], 1u);
+                bars->is_last = ticket == static_cast<unsigned int>(splits) - 1u ? 1 : 0;
+            }
+            __syncthreads();
+            if (bars->is_last) {
+                __threadfence();
+                // every CTA has folded its rows' best keys into tail.best with an atomic maximum: read them out,
+                // one thread per row (little code: this runs once per launch, from a cold instruction cache)
+                const int n_rows = static_cast<int>(min(static_cast<int64_t>(TM), B - q0));
+                int is_hit = 0;
+                if (static_cast<int>(threadIdx.x) < n_rows) {
+                    const int64_t b = static_cast<int64_t>(q0) + threadIdx.x;
+                    const unsigned long long key = __ldcg(tail.best + b);
+                    tail.best[b] = 0ull;                                   // ready for the next launch
+                    tail.idx[b] = key ? key_slot(key) : -1;
+                    tail.sim[b] = key ? key_sim(key) : -INFINITY;
+                    const float th = tail.theta ? tail.theta[b] : tail.theta_s;
+                    is_hit = (key != 0ull && key_sim(key) > th) ? 1 : 0;
+                    tail.hit[b] = static_cast<uint8_t>(is_hit);
+                }
+                if (tail.counters) {
+                    const int n_hit = __syncthreads_count(is_hit);
+                    if (threadIdx.x == 0 && n_rows > 0) {
+                        if (n_hit) atomicAdd(reinterpret_cast<unsigned long long *>(tail.counters + CNT_HITS), static_cast<unsigned long long>(n_hit));
+                        atomicAdd(reinterpret_cast<unsigned long long *>(tail.counters + CNT_LOOKUPS), static_cast<unsigned long long>(n_rows));
+                    }
+                }
+                if (threadIdx.x == 0) tail.counter[blockIdx.x] = 0u;      // ready for the next launch
+            }
+        }
+    }
 }
 
 }  // namespace tc2
@@ -215,7 +271,7 @@ lookup_tensor_pair_kernel(const __grid_constant__ CUtensorMap map_q, const __gri
 template <int KMAX>
 static siso_status_t run_pair(Cache *c, bool *attr_set, const CUtensorMap &map_q, const CUtensorMap &map_c_half, int64_t B,
                               int tiles_per_split, int n_tiles, int splits, int m_tiles_even, unsigned long long *partial,
-                              cudaStream_t s) {
+                              const tc2::TailFinal &tail, cudaStream_t s) {
     auto kern = tc2::lookup_tensor_pair_kernel<KMAX>;
     if (!*attr_set) {
         SISO_CUDA(cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, tc2::SMEM_BYTES));
@@ -224,18 +280,25 @@ static siso_status_t run_pair(Cache *c, bool *attr_set, const CUtensorMap &map_q
     dim3 grid(m_tiles_even, splits);
     // one pair covers the whole batch: every centroid tile is read by exactly one cluster, so it need not stay in L2
     kern<<<grid, tc2::THREADS, tc2::SMEM_BYTES, s>>>(map_q, map_c_half, c->valid, B, c->dim, tiles_per_split, n_tiles,
-                                                     partial, splits, m_tiles_even == 2 ? 1 : 0, c->status);
+                                                     partial, splits, m_tiles_even == 2 ? 1 : 0, c->status, tail);
     SISO_LAUNCHED(c);
     return SISO_OK;
 }
 
-// Called by launch_lookup_tensor when the batch spans at least two query tiles.
+// Called by launch_lookup_tensor when the batch spans at least two query tiles.  With `tail_counter` (k = 1 only) the
+// kernel also writes idx / sim / hit itself (see TailFinal).
 siso_status_t launch_lookup_tensor_pair(Cache *c, bool *attr_set3, const CUtensorMap &map_q, const CUtensorMap &map_c_half,
                                         int64_t B, int kmax, int tiles_per_split, int n_tiles, int splits, int m_tiles_even,
-                                        unsigned long long *partial, cudaStream_t s) {
-    return kmax == 1 ? run_pair<1>(c, attr_set3 + 0, map_q, map_c_half, B, tiles_per_split, n_tiles, splits, m_tiles_even, partial, s)
-         : kmax == 4 ? run_pair<4>(c, attr_set3 + 1, map_q, map_c_half, B, tiles_per_split, n_tiles, splits, m_tiles_even, partial, s)
-                     : run_pair<8>(c, attr_set3 + 2, map_q, map_c_half, B, tiles_per_split, n_tiles, splits, m_tiles_even, partial, s);
+                                        unsigned long long *partial, unsigned int *tail_counter, const float *theta,
+                                        float theta_s, int32_t *idx, float *sim, uint8_t *hit, long long *counters,
+                                        cudaStream_t s) {
+    tc2::TailFinal tail;
+    tail.counter = kmax == 1 ? tail_counter : nullptr;
+    tail.best = tail_counter ? reinterpret_cast<unsigned long long *>(tail_counter + 64) : nullptr;     // 256 bytes in
+    tail.theta = theta; tail.theta_s = theta_s; tail.idx = idx; tail.sim = sim; tail.hit = hit; tail.counters = counters;
+    return kmax == 1 ? run_pair<1>(c, attr_set3 + 0, map_q, map_c_half, B, tiles_per_split, n_tiles, splits, m_tiles_even, partial, tail, s)
+         : kmax == 4 ? run_pair<4>(c, attr_set3 + 1, map_q, map_c_half, B, tiles_per_split, n_tiles, splits, m_tiles_even, partial, tail, s)
+                     : run_pair<8>(c, attr_set3 + 2, map_q, map_c_half, B, tiles_per_split, n_tiles, splits, m_tiles_even, partial, tail, s);
 }
 
 }  // namespace siso

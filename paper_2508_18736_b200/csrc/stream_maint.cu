@@ -19,6 +19,19 @@
 // histogram pass and a collection pass, as evict.cu does.  Whatever the splitters are, the victims are the m
 // smallest keys exactly.
 // Used by siso_stream_step for batches of at most 1024 rows; larger batches take the separate kernels.
+//
+// Steady state of a full cache (every batch evicts exactly its misses): phases S and R and all barriers are
+// replaced by a list that lives across batches.  The list holds, in eviction order, EVERY live entry whose key is
+// at most a bound (about 3,000 entries after a rebuild).  The victims of a batch are the m lowest keys AFTER the
+// hit update; a hit only raises a key, so with at least 2B entries in the list the m lowest are found among its
+// first 2B entries (at most B of them were hit, so at least B >= m keep their key and stay below everything
+// outside).  Every CTA derives the same victims from that prefix on its own (mark the hit entries with a hash of
+// the batch's hit slots, give them their new keys, rank by position), so update and insertion run without a
+// grid-wide barrier; a hit entry that is evicted in the same batch is not updated (its slot is overwritten by a
+// miss).  The last CTA then takes the victims and the hit entries out of the list; an entry whose new key would
+// still lie below the bound, or a new entry that does, cuts the list (and the bound) off just below that key, so
+// the list always holds ALL live entries up to its bound.  When fewer than 2B entries are left, or another entry
+// point has changed the cache, the batch takes the phases above and the list is rebuilt from a sample-chosen bound.
 #include <cooperative_groups.h>
 
 #include "evict_keys.cuh"
@@ -35,6 +48,34 @@ constexpr int SM_STAGE = 2048;      // candidates a CTA can hold in shared memor
 constexpr int SM_SELECT = 16;       // up to this many splitters are extracted one by one instead of sorting the sample
 constexpr int SM_RANK_STRIDE = 4;   // every fourth CTA ranks candidates
 constexpr int SM_DENSE = 4;         // entries per sampler thread in the fine sample (4 x 256 entries)
+
+constexpr int LOW_K = 4096;         // capacity of the eviction-order list kept across batches
+constexpr int LOW_TARGET = 3072;    // entries a rebuild aims at
+constexpr int LOW_UPD = 256;        // hit entries inside the examined prefix that the barrier-free path handles
+constexpr int LOW_MAP_BITS = 13;
+constexpr int LOW_MAP = 1 << LOW_MAP_BITS;   // open-addressing table slot -> position in the list (load at most 1/2)
+constexpr int LOW_PER_THREAD = LOW_K / SM_THREADS;
+constexpr unsigned int LOW_SPIN_LIMIT = 1u << 18;
+
+// Every live entry with key <= bound (all live entries if has_bound == 0) is among k[head .. n), ascending.  An entry
+// that was hit leaves the list by a mark (dead[i] = 1: its key has risen above the bound); the victims of a batch are
+// the first entries that are neither marked nor hit, so evicting them moves `head` forward and nothing is copied.
+// Written only by the streaming maintenance kernel; the host flag Cache::low_dirty says whether any other entry point
+// has touched the cache since.
+struct LowList {
+    int n;                    // end of the list
+    int head;                 // first entry still in it
+    int n_dead;               // marked entries in [head, n), or more (it only sizes the prefix that is examined)
+    int valid;
+    int has_bound;
+    int pad;
+    Key3 bound;
+    unsigned int started;     // CTAs of the running kernel that no longer read the list (reset by the writer)
+    unsigned int n_cand;      // rebuild: candidates collected
+    unsigned long long k0[LOW_K], k1[LOW_K], k2[LOW_K];
+    uint8_t dead[LOW_K];
+    unsigned long long map[LOW_MAP];   // (slot + 1) << 32 | position, 0 = empty; written by the rebuild only
+};
 
 struct MaintCtl {
     unsigned int n_cand;                 // candidates appended in phase S
@@ -61,6 +102,7 @@ struct MaintArgs {
     int32_t *victims;                  // [B] or NULL
     int32_t *slots_out;                // [B] or NULL
     // phase F (partial == NULL: idx and hit are inputs)
+    int count_lookup;                  // the lookup of this batch has not been counted yet (lookups, hits)
     const unsigned long long *partial; // [B, splits] packed (similarity, slot) keys
     int splits;
     const float *theta;
@@ -74,6 +116,8 @@ struct MaintArgs {
     int32_t *victim_buf;               // [B] victims in key order (always present, unlike `victims`)
     int *cta_free;                     // [grid]
     int32_t *free_list;                // [B]
+    LowList *low;                      // eviction-order list kept across batches
+    int low_ok;                        // host: nothing but this kernel has changed the cache since the list was written
 };
 
 // fixed part of the shared memory; it follows the 48 KiB that hold the fp64 row accumulator during the update and
@@ -89,6 +133,17 @@ struct MaintSmem {
     uint8_t hit[SM_MAX_B];
     int n_stage;
     int p;
+    // barrier-free path
+    int32_t vict[SM_MAX_B];            // victims in eviction order
+    int32_t by_slot[SM_MAX_B];         // victims in slot order
+    uint32_t pcnt[2 * SM_MAX_B];       // hits of this batch on entry i of the prefix
+    uint16_t hb[2 * SM_MAX_B + 1];     // hit entries of the list before position i
+    uint8_t lflag[2 * SM_MAX_B];       // entry i of the prefix: 1 = hit in this batch, 2 = marked earlier
+    unsigned long long u0[LOW_UPD], u1[LOW_UPD], u2[LOW_UPD];    // new keys of the hit entries of the prefix
+    uint16_t upos[LOW_UPD];            // their positions in the list
+    uint8_t uvict[LOW_UPD];            // evicted all the same
+    int n_upd;
+    int v_end;                         // prefix position just behind the last victim that was not hit in this batch
 };
 constexpr size_t SM_UNION_BYTES = 3 * sizeof(unsigned long long) * SM_STAGE;      // 48 KiB >= 8 * kMaxDim
 constexpr size_t SM_SMEM_BYTES = SM_UNION_BYTES + sizeof(MaintSmem);
@@ -651,6 +706,295 @@ __device__ __forceinline__ void maint_insert_row(const MaintArgs &a, int b, int3
     }
 }
 
+// ==== barrier-free path: the victims from the list kept across batches ============================================
+__device__ __forceinline__ uint32_t low_hash(uint32_t slot) { return (slot * 2654435761u) >> (32 - LOW_MAP_BITS); }
+
+// position of `slot` in the list as the last rebuild wrote it, or -1.  (The caller checks that the position still
+// lies in [head, n) and is not marked: the table keeps entries that have left the list since.)
+__device__ __forceinline__ int low_pos_of(const LowList *low, uint32_t slot) {
+    uint32_t h = low_hash(slot);
+    for (int probe = 0; probe < LOW_MAP; ++probe) {
+        const unsigned long long e = __ldcg(&low->map[h]);
+        if (e == 0ull) return -1;
+        if (static_cast<uint32_t>(e >> 32) == slot + 1u) return static_cast<int>(e & 0xFFFFFFFFull);
+        h = (h + 1u) & (LOW_MAP - 1u);
+    }
+    return -1;
+}
+
+// the key of a list entry after `cnt` hits in the batch that ends at clock_new (what the update writes: cluster_size
+// + cnt, access_count + cnt saturating at infinity, last_access = clock_new); cluster_size and access_count are
+// read back from the key, because other CTAs may be updating the arrays right now
+__device__ __forceinline__ Key3 low_key_after_hits(const Key3 &k, uint32_t cnt, long long clock_new) {
+    const unsigned long long u = (k.w0 >> 63) ? (k.w0 & 0x7FFFFFFFFFFFFFFFull) : ~k.w0;
+    const double size = __longlong_as_double(static_cast<long long>(u)) + static_cast<double>(cnt);
+    const uint32_t ac_old = static_cast<uint32_t>(k.w1 >> 32);
+    const unsigned long long ac = static_cast<unsigned long long>(ac_old) + cnt;
+    const uint32_t ac_new = (ac_old == SISO_ACCESS_INF || ac >= SISO_ACCESS_INF) ? SISO_ACCESS_INF : static_cast<uint32_t>(ac);
+    return make_key(size, ac_new, static_cast<unsigned long long>(clock_new), static_cast<uint32_t>(k.w2 & 0xFFFFFFFFull));
+}
+
+// Loads the L entries of the list from `head` on into `stage`, finds the ones hit in this batch (through the table
+// slot -> position) and ranks all of them by their keys after the update; entries marked earlier take no part.  At most B <= LOW_UPD entries can have
+// been hit.  sm.vict[0..m) receives the victims in eviction order.
+__device__ void maint_low_select(const MaintArgs &a, int head, int L, int m, long long clock_new, unsigned long long *stage,
+                                 MaintSmem &sm) {
+    const int tid = threadIdx.x;
+    unsigned long long *s0 = stage, *s1 = stage + SM_STAGE, *s2 = stage + 2 * SM_STAGE;
+    const LowList *low = a.low;
+    for (int i = tid; i < L; i += SM_THREADS) {
+        s0[i] = __ldcg(&low->k0[head + i]); s1[i] = __ldcg(&low->k1[head + i]); s2[i] = __ldcg(&low->k2[head + i]);
+        sm.lflag[i] = __ldcg(&low->dead[head + i]) ? 2 : 0;
+    }
+    for (int i = tid; i < L; i += SM_THREADS) sm.pcnt[i] = 0u;
+    if (tid == 0) { sm.n_upd = 0; sm.v_end = 0; }
+    __syncthreads();
+    // every hit row looks its slot up in the table: a hit on an unmarked entry of the prefix is counted there
+    for (int b = tid; b < a.B; b += SM_THREADS) {
+        if (!sm.hit[b]) continue;
+        const int32_t slot = sm.idx[b];
+        if (slot < 0 || slot >= a.capacity) continue;          // reported by the update of that row
+        const int pos = low_pos_of(low, static_cast<uint32_t>(slot)) - head;
+        if (pos >= 0 && pos < L && sm.lflag[pos] != 2) atomicAdd(&sm.pcnt[pos], 1u);
+    }
+    __syncthreads();
+    // hb[i] = entries before position i that were hit or marked (thread t owns a contiguous run)
+    const int per = (L + SM_THREADS - 1) / SM_THREADS;
+    const int lo = min(L, tid * per), hi = min(L, lo + per);
+    int c = 0, c_upd = 0;
+    for (int i = lo; i < hi; ++i) {
+        if (sm.pcnt[i]) sm.lflag[i] = 1;
+        c += sm.lflag[i] ? 1 : 0;
+        c_upd += sm.lflag[i] == 1 ? 1 : 0;
+    }
+    int n_gone, n_upd, run, run_u;
+    {
+        int both;                                               // the two counts share one scan (each is at most 2048)
+        const int r = block_exclusive_scan_256(c | (c_upd << 16), &both, sm.warp_sum);
+        run = r & 0xFFFF; run_u = r >> 16;
+        n_gone = both & 0xFFFF; n_upd = both >> 16;
+    }
+    for (int i = lo; i < hi; ++i) {
+        sm.hb[i] = static_cast<uint16_t>(run);
+        run += sm.lflag[i] ? 1 : 0;
+        if (sm.lflag[i] == 1) {
+            Key3 k;
+            k.w0 = s0[i]; k.w1 = s1[i]; k.w2 = s2[i];
+            const Key3 nk = low_key_after_hits(k, sm.pcnt[i], clock_new);
+            sm.u0[run_u] = nk.w0; sm.u1[run_u] = nk.w1; sm.u2[run_u] = nk.w2;
+            sm.upos[run_u] = static_cast<uint16_t>(i);
+            ++run_u;
+        }
+    }
+    if (tid == 0) { sm.hb[L] = static_cast<uint16_t>(n_gone); sm.n_upd = n_upd; }
+    __syncthreads();
+    // ranks after the update.  An entry that was neither hit nor marked: its position among such entries, plus the hit
+    // entries whose new key is smaller.  A hit entry: the entries of the first kind below its new key (binary search
+    // in the old order, minus the hit and marked entries there), plus the hit entries with a smaller new key.
+    for (int i = tid; i < L; i += SM_THREADS) {
+        if (sm.lflag[i]) continue;
+        Key3 k;
+        k.w0 = s0[i]; k.w1 = s1[i]; k.w2 = s2[i];
+        int rank = i - sm.hb[i];
+        for (int u = 0; u < n_upd; ++u) {
+            Key3 nk;
+            nk.w0 = sm.u0[u]; nk.w1 = sm.u1[u]; nk.w2 = sm.u2[u];
+            rank += key_less(nk, k) ? 1 : 0;
+        }
+        if (rank < m) {
+            sm.vict[rank] = static_cast<int32_t>(k.w2 & 0xFFFFFFFFull);
+            atomicMax(&sm.v_end, i + 1);
+        }
+    }
+    for (int u = tid; u < n_upd; u += SM_THREADS) {
+        Key3 nk;
+        nk.w0 = sm.u0[u]; nk.w1 = sm.u1[u]; nk.w2 = sm.u2[u];
+        int lo_i = 0, hi_i = L;
+        while (lo_i < hi_i) {
+            const int mid = (lo_i + hi_i) >> 1;
+            Key3 k;
+            k.w0 = s0[mid]; k.w1 = s1[mid]; k.w2 = s2[mid];
+            if (key_less(k, nk)) lo_i = mid + 1; else hi_i = mid;
+        }
+        int rank = lo_i - sm.hb[lo_i];
+        for (int v = 0; v < n_upd; ++v) {
+            Key3 ok;
+            ok.w0 = sm.u0[v]; ok.w1 = sm.u1[v]; ok.w2 = sm.u2[v];
+            rank += key_less(ok, nk) ? 1 : 0;
+        }
+        sm.uvict[u] = rank < m ? 1 : 0;
+        if (rank < m) sm.vict[rank] = static_cast<int32_t>(nk.w2 & 0xFFFFFFFFull);
+    }
+    __syncthreads();
+}
+
+// The last CTA brings the list up to date for the next batch (see the head of the file).  It first waits, with a
+// limit, until every other CTA has said that it no longer reads the list; in a cooperative launch all CTAs are
+// resident and they say so a few microseconds into the kernel.  Nothing is moved: the victims that were not hit
+// are the first unmarked entries, so `head` steps behind the last of them; hit entries are marked; and only if a
+// moved or new key lies below the bound is the end of the list pulled in to just below that key.
+__device__ void maint_low_advance(const MaintArgs &a, int head, int L, int m, long long clock_new, MaintSmem &sm) {
+    const int tid = threadIdx.x;
+    LowList *low = a.low;
+    const int n = low->n;
+    const int has_bound = low->has_bound;
+    const Key3 bound = low->bound;
+    const int n_dead_old = low->n_dead;
+    if (tid == 0) {
+        unsigned int it = 0;
+        while (atomicAdd(&low->started, 0u) < gridDim.x - 1u && it < LOW_SPIN_LIMIT) { __nanosleep(100); ++it; }
+        if (it >= LOW_SPIN_LIMIT) set_status(a.status, SISO_ERR_TIMEOUT);
+        __threadfence();
+    }
+    __syncthreads();
+    // the smallest key that moved or arrived: the new entries (the lowest slot gives the lowest key) ...
+    Key3 cut;
+    cut.w0 = cut.w1 = cut.w2 = ~0ull;
+    if (m > 0) {
+        int32_t lowest = sm.vict[0];
+        for (int r = 1; r < m; ++r) lowest = min(lowest, sm.vict[r]);
+        cut = make_key(1.0, SISO_ACCESS_INF, static_cast<unsigned long long>(clock_new), static_cast<uint32_t>(lowest));
+    }
+    // ... and the hit entries that stay in the cache; every hit entry of the list is marked on the way.  The first
+    // row of each hit slot looks the slot up in the table (the list itself is not scanned).
+    const int new_head = head + sm.v_end;
+    int newly_dead = 0;
+    for (int b = tid; b < a.B; b += SM_THREADS) {
+        if (!sm.hit[b]) continue;
+        const int32_t slot = sm.idx[b];
+        if (slot < 0 || slot >= a.capacity) continue;
+        const int pos = low_pos_of(low, static_cast<uint32_t>(slot));
+        if (pos < new_head || pos >= n || low->dead[pos]) continue;
+        int cnt = 0;
+        bool first = true;
+        for (int r = 0; r < a.B; ++r) {
+            const bool same = sm.hit[r] && sm.idx[r] == slot;
+            cnt += same ? 1 : 0;
+            first = first && !(same && r < b);
+        }
+        if (!first) continue;
+        low->dead[pos] = 1;
+        ++newly_dead;
+        bool evicted = false;
+        if (pos - head < L) {
+            for (int v = 0; v < sm.n_upd; ++v)
+                if (sm.upos[v] == pos - head) evicted = sm.uvict[v] != 0;
+        }
+        if (!evicted) {
+            Key3 k;
+            k.w0 = low->k0[pos]; k.w1 = low->k1[pos]; k.w2 = low->k2[pos];
+            const Key3 nk = low_key_after_hits(k, static_cast<uint32_t>(cnt), clock_new);
+            if (key_less(nk, cut)) cut = nk;
+        }
+    }
+    // hit entries in front of the new head leave with it, but one of them that stays in the cache still counts for the cut
+    for (int v = tid; v < sm.n_upd; v += SM_THREADS) {
+        if (sm.upos[v] < sm.v_end && !sm.uvict[v]) {
+            Key3 nk;
+            nk.w0 = sm.u0[v]; nk.w1 = sm.u1[v]; nk.w2 = sm.u2[v];
+            if (key_less(nk, cut)) cut = nk;
+        }
+    }
+    cut = block_min_key(cut, sm);
+    int dead_total;
+    block_exclusive_scan_256(newly_dead, &dead_total, sm.warp_sum);
+    if (tid == 0) {
+        const bool moved = (cut.w0 & cut.w1 & cut.w2) != ~0ull;
+        const bool cut_off = moved && (!has_bound || key_less(cut, bound));
+        int n_new = n;
+        if (cut_off) {
+            // first entry that is not below the cut (the list is in ascending order, marks or not)
+            int lo_i = new_head, hi_i = n;
+            while (lo_i < hi_i) {
+                const int mid = (lo_i + hi_i) >> 1;
+                Key3 k;
+                k.w0 = low->k0[mid]; k.w1 = low->k1[mid]; k.w2 = low->k2[mid];
+                if (key_less(k, cut)) lo_i = mid + 1; else hi_i = mid;
+            }
+            n_new = lo_i;
+            if (n_new > new_head) {
+                Key3 k;
+                k.w0 = low->k0[n_new - 1]; k.w1 = low->k1[n_new - 1]; k.w2 = low->k2[n_new - 1];
+                low->bound = k;
+            }
+            low->has_bound = 1;
+        }
+        low->head = new_head;
+        low->n = n_new;
+        // marked entries that the head has passed no longer count (hb counts hit and marked entries alike); the hit
+        // entries behind the new head have just been marked (dead_total).  Entries beyond a pulled-in end stay
+        // counted: too large a number only makes the next prefix longer than it has to be.
+        int hit_front = 0;
+        for (int v = 0; v < sm.n_upd; ++v) hit_front += sm.upos[v] < sm.v_end ? 1 : 0;
+        low->n_dead = n_dead_old - (static_cast<int>(sm.hb[sm.v_end]) - hit_front) + dead_total;
+        low->valid = (cut_off && n_new <= new_head) ? 0 : 1;
+        low->started = 0u;
+    }
+}
+
+// ==== rebuild of the list (all CTAs; the cache's state is final) ====================================================
+// Collect every live entry up to the sample-chosen bound, rank all of them, store the LOW_K lowest in order.
+__device__ void maint_low_collect(const MaintArgs &a, bool has_bound, const Key3 &bound) {
+    const int tid = threadIdx.x, lane = tid & 31;
+    for (long long base = static_cast<long long>(blockIdx.x) * SM_THREADS; base < a.capacity;
+         base += static_cast<long long>(gridDim.x) * SM_THREADS) {
+        const long long sl = base + tid;
+        bool take = false;
+        Key3 k;
+        k.w0 = k.w1 = k.w2 = 0ull;
+        if (sl < a.capacity && a.valid[sl]) {
+            k = make_key(a.size[sl], a.access[sl], a.last[sl], static_cast<uint32_t>(sl));
+            take = !has_bound || !key_less(bound, k);
+        }
+        const unsigned ballot = __ballot_sync(0xFFFFFFFFu, take);
+        if (ballot) {
+            unsigned int warp_base = 0;
+            if (lane == 0) warp_base = atomicAdd(&a.low->n_cand, static_cast<unsigned int>(__popc(ballot)));
+            warp_base = __shfl_sync(0xFFFFFFFFu, warp_base, 0);
+            if (take) {
+                const unsigned int at = warp_base + __popc(ballot & ((1u << lane) - 1u));
+                a.cand0[at] = k.w0; a.cand1[at] = k.w1; a.cand2[at] = k.w2;
+            }
+        }
+    }
+}
+
+__device__ void maint_low_rank(const MaintArgs &a, unsigned int n) {
+    const int lane = threadIdx.x & 31;
+    const unsigned int warps = gridDim.x * SM_WARPS;
+    const unsigned int keep = n < static_cast<unsigned int>(LOW_K) ? n : static_cast<unsigned int>(LOW_K);
+#pragma unroll 1
+    for (unsigned int i = blockIdx.x * SM_WARPS + (threadIdx.x >> 5); i < n; i += warps) {
+        const Key3 mine = cand_key(a, i);
+        unsigned int rank = 0;
+        for (unsigned int j0 = 0; j0 < n; j0 += 128) {
+            Key3 o[4];
+#pragma unroll
+            for (int u = 0; u < 4; ++u) {
+                const unsigned int j = j0 + u * 32 + lane;
+                o[u].w0 = o[u].w1 = o[u].w2 = ~0ull;
+                if (j < n) o[u] = cand_key(a, j);
+            }
+#pragma unroll
+            for (int u = 0; u < 4; ++u) rank += key_less(o[u], mine) ? 1u : 0u;
+        }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) rank += __shfl_xor_sync(0xFFFFFFFFu, rank, o);
+        if (lane == 0 && rank < keep) {
+            a.low->k0[rank] = mine.w0; a.low->k1[rank] = mine.w1; a.low->k2[rank] = mine.w2;
+            a.low->dead[rank] = 0;
+            const uint32_t slot = static_cast<uint32_t>(mine.w2 & 0xFFFFFFFFull);
+            const unsigned long long entry = (static_cast<unsigned long long>(slot + 1u) << 32) | rank;
+            uint32_t h = low_hash(slot);
+            for (int probe = 0; probe < LOW_MAP; ++probe) {
+                if (atomicCAS(&a.low->map[h], 0ull, entry) == 0ull) break;
+                h = (h + 1u) & (LOW_MAP - 1u);
+            }
+            if (n > keep && rank == keep - 1) a.low->bound = mine;        // the list was cut at LOW_K entries
+        }
+    }
+}
+
 template <typename T>
 __global__ void __launch_bounds__(SM_THREADS, 2)
 stream_maint_kernel(const MaintArgs a) {
@@ -691,6 +1035,83 @@ stream_maint_kernel(const MaintArgs a) {
     m = m > 0 ? m : 0;
     m = m < occupancy ? m : occupancy;
     __syncthreads();
+
+    // ---- a full cache whose eviction-order list is long enough: no barrier from here on
+    int L = 0, head = 0;
+    bool fast = false;
+    if (a.low) {
+        head = a.low->head;
+        const int avail = a.low->n - head, n_dead = a.low->n_dead;
+        L = min(avail, 2 * a.B + n_dead);          // at least 2B unmarked entries, or all there are
+        fast = a.low_ok && a.low->valid && free0 == 0 && n_miss <= occupancy && L <= 2 * SM_MAX_B && a.B <= LOW_UPD &&
+               (avail - n_dead >= 2 * a.B || !a.low->has_bound);
+    }
+    if (fast) {
+        const int G = static_cast<int>(gridDim.x);
+        const bool last_cta = static_cast<int>(blockIdx.x) == G - 1;
+        const int from_end = G - 2 - static_cast<int>(blockIdx.x);
+        const bool ins_cta = from_end >= 0 && from_end * SM_WARPS < n_miss;
+        const bool out_cta = static_cast<int>(blockIdx.x) == (a.B < G - 1 ? a.B : 0);      // a CTA without a row to update, if there is one
+        // A CTA that only updates the entry of row blockIdx.x needs the victims only if that entry could be one of
+        // them, i.e. if it is an unmarked entry of the examined prefix (rare: the prefix holds the coldest entries).
+        bool need = last_cta || ins_cta || out_cta || a.B > G;
+        if (!need) {
+            int in_prefix = 0;
+            const int b = blockIdx.x;
+            if (tid == 0 && b < a.B && sm.hit[b] && sm.idx[b] >= 0 && sm.idx[b] < a.capacity) {
+                const int pos = low_pos_of(a.low, static_cast<uint32_t>(sm.idx[b])) - head;
+                in_prefix = (pos >= 0 && pos < L && !__ldcg(&a.low->dead[head + pos])) ? 1 : 0;
+            }
+            need = __syncthreads_or(in_prefix) != 0;
+        }
+        if (need) maint_low_select(a, head, L, static_cast<int>(m), clock_new, stage, sm);
+        if (tid == 0 && !last_cta) atomicAdd(&a.low->started, 1u);      // this CTA has read what it needs of the list
+        if (out_cta) {
+            if (a.victims)
+                for (int r = tid; r < a.B; r += SM_THREADS) a.victims[r] = r < m ? sm.vict[r] : -1;
+            if (a.slots_out)
+                for (int b = tid; b < a.B; b += SM_THREADS)
+                    if (sm.hit[b]) a.slots_out[b] = -1;
+        }
+        // U: a hit entry that is evicted in this very batch is not updated (a miss overwrites its slot)
+        for (int b = blockIdx.x; b < a.B; b += gridDim.x) {
+            if (need) {
+                int evicted = 0;
+                if (sm.hit[b])
+                    for (int r = tid; r < m; r += SM_THREADS) evicted |= sm.vict[r] == sm.idx[b] ? 1 : 0;
+                if (__syncthreads_or(evicted)) continue;
+            }
+            maint_update_row<T>(a, b, clock_new, acc, sm);
+        }
+        // I: the victims' slots in ascending order take the misses in ascending row order
+        // (by the CTAs counted from the far end, the last one excepted: the first ones are busy with the updates)
+        const int ins_ctas = G - 1;
+        if (ins_cta) {
+            for (int r = tid; r < n_miss; r += SM_THREADS) {
+                const int32_t mine = sm.vict[r];
+                int rank = 0;
+                for (int j = 0; j < n_miss; ++j) rank += sm.vict[j] < mine ? 1 : 0;
+                sm.by_slot[rank] = mine;
+            }
+            __syncthreads();
+            for (int r = from_end * SM_WARPS + warp; r < n_miss; r += ins_ctas * SM_WARPS)
+                maint_insert_row<T>(a, sm.miss_list[r], sm.by_slot[r], clock_new);
+        }
+        if (last_cta) {
+            __syncthreads();
+            maint_low_advance(a, head, L, static_cast<int>(m), clock_new, sm);
+            if (tid == 0) {
+                a.counters[CNT_CLOCK] = clock_new;
+                a.counters[CNT_EVICTIONS] += m;
+                a.counters[CNT_INSERTS] += n_miss;
+                if (a.count_lookup) {
+                    a.counters[CNT_LOOKUPS] += a.B;
+                    a.counters[CNT_HITS] += a.B - n_miss;
+                }
+            }
+        }
+        return;
+    }
 
     // ---- U (+ sampler)
     if (blockIdx.x == 0) {
@@ -814,9 +1235,46 @@ stream_maint_kernel(const MaintArgs a) {
         a.counters[CNT_OCCUPANCY] = occupancy - m + (insert_ok ? n_miss : 0);
         a.counters[CNT_EVICTIONS] += m;
         if (insert_ok) a.counters[CNT_INSERTS] += n_miss;
-        if (a.partial) {
+        if (a.count_lookup) {
             a.counters[CNT_LOOKUPS] += a.B;
             a.counters[CNT_HITS] += a.B - n_miss;
+        }
+    }
+
+    // ---- the eviction-order list for the batches to come: rebuilt once the cache is full, dropped otherwise
+    if (a.low) {
+        const long long occupancy_after = occupancy - m + (insert_ok ? n_miss : 0);
+        if (occupancy_after != a.capacity) {
+            // every CTA read the list's header before the first barrier of this launch
+            if (blockIdx.x == 0 && tid == 0) { a.low->valid = 0; a.low->n = 0; }
+            return;
+        }
+        grid.sync();                                             // the cache's state is final
+        const long long m_equiv = LOW_TARGET / 3;                // the sampler aims at about 3 m entries below its last splitter
+        if (blockIdx.x == 0) {
+            if (tid == 0) a.low->n_cand = 0u;
+            maint_evict_sample(a, clock_new, m_equiv, occupancy_after, false, sm);
+        }
+        grid.sync();
+        const int n_sample = a.ctl->n_sample;
+        const int P = maint_spec_buckets(m_equiv, n_sample, occupancy_after);
+        const bool has_bound = P < n_sample;
+        Key3 bound;
+        bound.w0 = bound.w1 = bound.w2 = ~0ull;
+        if (has_bound) bound = a.splitters[P];
+        for (int i = blockIdx.x * SM_THREADS + tid; i < LOW_MAP; i += gridDim.x * SM_THREADS) a.low->map[i] = 0ull;
+        maint_low_collect(a, has_bound, bound);
+        grid.sync();
+        const unsigned int n_c = a.low->n_cand;
+        maint_low_rank(a, n_c);
+        if (blockIdx.x == 0 && tid == 0) {
+            a.low->n = static_cast<int>(n_c < static_cast<unsigned int>(LOW_K) ? n_c : static_cast<unsigned int>(LOW_K));
+            a.low->head = 0;
+            a.low->n_dead = 0;
+            a.low->valid = n_c > 0u ? 1 : 0;
+            a.low->has_bound = (has_bound || n_c > static_cast<unsigned int>(LOW_K)) ? 1 : 0;
+            if (has_bound && n_c <= static_cast<unsigned int>(LOW_K)) a.low->bound = bound;
+            a.low->started = 0u;
         }
     }
 }
@@ -867,6 +1325,7 @@ siso_status_t launch_stream_maint(Cache *c, const void *q, int64_t B, int32_t *i
     a.Q = q; a.idx = idx; a.hit = hit; a.B = static_cast<int>(B); a.D = c->dim; a.capacity = c->capacity;
     a.vecs = c->vecs; a.master = c->master; a.size = c->size; a.access = c->access; a.last = c->last; a.valid = c->valid;
     a.counters = c->counters; a.status = c->status; a.victims = victims; a.slots_out = slots_out;
+    a.count_lookup = deferred ? 1 : 0;
     a.partial = deferred ? deferred->partial : nullptr;
     a.splits = deferred ? deferred->splits : 0;
     a.theta = deferred ? deferred->theta : nullptr;
@@ -881,11 +1340,19 @@ siso_status_t launch_stream_maint(Cache *c, const void *q, int64_t B, int32_t *i
     a.victim_buf = scr.take<int32_t>(B);
     a.cta_free = scr.take<int>(grid);
     a.free_list = scr.take<int32_t>(B);
+    a.low = nullptr;
+    if (!c->stream_list_off) {
+        if (!c->low_list) c->low_list = cache_alloc_zeroed(c, sizeof(LowList));      // all zero: an empty, invalid list
+        if (!c->low_list) return SISO_ERR_OOM;
+        a.low = static_cast<LowList *>(c->low_list);
+    }
+    a.low_ok = c->low_dirty ? 0 : 1;
     void *args[] = {&a};
     const void *fn = c->dtype == SISO_F32 ? reinterpret_cast<const void *>(stream_maint_kernel<float>)
                                           : reinterpret_cast<const void *>(stream_maint_kernel<__nv_bfloat16>);
     SISO_CUDA(cudaLaunchCooperativeKernel(fn, dim3(grid), dim3(SM_THREADS), args, SM_SMEM_BYTES, s));
     c->launches += 1;
+    c->low_dirty = false;       // from here on the list on the device matches the cache, or says that it does not
     return SISO_OK;
 }
 
