@@ -209,7 +209,7 @@ siso_status_t siso_lookup_small_noalloc(const void *d_centroids, const uint8_t *
 /* Lookup over a cache whose rows are partitioned across several GPUs (one handle per GPU, each holding a contiguous
  * range of the global slots).  FindClosestCentroid over the whole cache = the best of the shards' best, so every GPU
  * scores the full query batch against its own rows and the shards' top-k lists are combined after one exchange.
- * siso_lookup_keys is a1-a2 on one shard: d_keys [n_queries, k] receives packed 64-bit keys,
+ * siso_lookup_keys is the similarity sweep and the top-k selection on one shard: d_keys [n_queries, k] receives packed 64-bit keys,
  * (order-preserving similarity bits << 32) | (2^32 - 1 - (slot + slot_offset)), 0 where the shard has fewer than k
  * entries; a larger key is a better match, ties go to the lower global slot.  The shard's hit statistics are not
  * touched.  slot_offset + capacity must stay below 2^32.

@@ -16,7 +16,7 @@
 
 #include <cstring>
 
-#include "common.cuh"
+#include "umma_pair.cuh"
 
 namespace siso {
 namespace tc {
@@ -32,105 +32,9 @@ constexpr uint32_t B_BYTES = TN * TK * 2;     // 32 KiB
 constexpr uint32_t STAGE_BYTES = A_BYTES + B_BYTES;
 constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 constexpr uint32_t TMEM_COLS = ACC_STAGES * TN;   // 512: the whole tensor memory of the SM
-constexpr uint32_t SPIN_LIMIT = 4u << 20;
 
-// ---- PTX wrappers -------------------------------------------------------------------------------
-__device__ __forceinline__ uint32_t smem_u32(const void *p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+using namespace umma2;      // PTX wrappers and the epilogue scan shared with the CTA-pair kernels
 
-__device__ __forceinline__ void mbar_init(uint64_t *bar, uint32_t count) {
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_u32(bar)), "r"(count) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive_expect_tx(uint64_t *bar, uint32_t bytes) {
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_u32(bar)), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
-    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
-    return ok != 0;
-}
-// Bounded wait.  Returns false if the limit ran out or another role has already given up.
-__device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag) {
-    for (uint32_t it = 0; it < SPIN_LIMIT; ++it) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((it & 63u) == 63u) {
-            if (*abort_flag) return false;
-            __nanosleep(64);
-        }
-    }
-    *abort_flag = 1;
-    return false;
-}
-__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
-                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar))
-                 : "memory");
-}
-// the same load with an L2 eviction policy: used for centroid tiles that no other CTA will read again, so that the
-// one-pass stream does not push the queries, the cache's metadata and the kernels' code out of L2
-__device__ __forceinline__ void tma_load_2d_hint(void *dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar, uint64_t policy) {
-    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
-                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar)), "l"(policy)
-                 : "memory");
-}
-__device__ __forceinline__ uint64_t l2_evict_first_policy() {
-    uint64_t p;
-    asm volatile("createpolicy.fractional.L2::evict_first.b64 %0, 1.0;" : "=l"(p));
-    return p;
-}
-__device__ __forceinline__ void tcgen05_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tcgen05_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void umma_commit(uint64_t *bar) {
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
-}
-__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
-        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
-}
-// 32 lanes x 32 consecutive 32-bit columns: thread i of the warp receives row (lane base + i).  The load is
-// asynchronous: the registers hold the data only after tmem_ld_fence() on the same array.
-__device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32]) {
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]),
-          "=r"(r[8]), "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15]),
-          "=r"(r[16]), "=r"(r[17]), "=r"(r[18]), "=r"(r[19]), "=r"(r[20]), "=r"(r[21]), "=r"(r[22]), "=r"(r[23]),
-          "=r"(r[24]), "=r"(r[25]), "=r"(r[26]), "=r"(r[27]), "=r"(r[28]), "=r"(r[29]), "=r"(r[30]), "=r"(r[31])
-        : "r"(taddr) : "memory");
-}
-// Wait for all tensor-memory loads issued so far.  The registers pass through the statement as in/out operands,
-// so the compiler cannot schedule any use of them before the wait.
-__device__ __forceinline__ void tmem_ld_fence(uint32_t (&r)[32]) {
-    asm volatile("tcgen05.wait::ld.sync.aligned;"
-        : "+r"(r[0]), "+r"(r[1]), "+r"(r[2]), "+r"(r[3]), "+r"(r[4]), "+r"(r[5]), "+r"(r[6]), "+r"(r[7]),
-          "+r"(r[8]), "+r"(r[9]), "+r"(r[10]), "+r"(r[11]), "+r"(r[12]), "+r"(r[13]), "+r"(r[14]), "+r"(r[15]),
-          "+r"(r[16]), "+r"(r[17]), "+r"(r[18]), "+r"(r[19]), "+r"(r[20]), "+r"(r[21]), "+r"(r[22]), "+r"(r[23]),
-          "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
-        :: "memory");
-}
-
-// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes and 128-byte swizzled
-// (what the TMA writes): 8-row groups 1024 bytes apart; descriptor version 1; layout type 2 = 128B swizzle.
-__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
-    uint64_t d = 0;
-    d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);          // start address, 16-byte units
-    d |= static_cast<uint64_t>(1) << 16;                         // leading byte offset (unused for swizzled K-major)
-    d |= static_cast<uint64_t>(1024 >> 4) << 32;                 // stride byte offset: 8 rows x 128 B
-    d |= static_cast<uint64_t>(1) << 46;                         // descriptor version
-    d |= static_cast<uint64_t>(2) << 61;                         // SWIZZLE_128B
-    return d;
-}
 // Instruction descriptor: D fp32, A and B bf16, both K-major, N = 256, M = 128.
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(TN >> 3) << 17) |
                            (static_cast<uint32_t>(TM >> 4) << 24);
@@ -243,42 +147,7 @@ lookup_tensor_kernel(const __grid_constant__ CUtensorMap map_q, const __grid_con
             if (!mbar_wait(&bars->acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
             tcgen05_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * TN;
-            // two register buffers: while one chunk of 32 columns is scanned the next is in flight from tensor
-            // memory.  The loop stays rolled (two chunks per trip): unrolled eight times the scan code no longer
-            // fits the instruction cache.
-            uint32_t ra[32], rb[32];
-            auto scan = [&](uint32_t (&r)[32], int ch) {
-                const uint32_t live = __ballot_sync(0xFFFFFFFFu, ((vflags >> ch) & 1ull) != 0ull);
-                if (live == 0u) return;
-                if (live != 0xFFFFFFFFu) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (!((live >> j) & 1u)) r[j] = 0xFF800000u;      // -inf: never enters a list
-                }
-                // Groups of 8 columns: a group is looked at value by value only if its maximum beats the row's
-                // k-th best.  A warp pays for that path when ANY of its 32 rows takes it, so small groups keep
-                // the common case (nothing to insert) down to 7 max operations and one comparison per group.
-#pragma unroll
-                for (int g8 = 0; g8 < 8; ++g8) {
-                    float m = __uint_as_float(r[g8 * 4]);
-#pragma unroll
-                    for (int j = 1; j < 4; ++j) m = fmaxf(m, __uint_as_float(r[g8 * 4 + j]));
-                    if (m > top.s[KMAX - 1]) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) top.push(__uint_as_float(r[g8 * 4 + j]), n0 + ch * 32 + g8 * 4 + j);
-                    }
-                }
-            };
-            tmem_ld_32x32(taddr, ra);
-#pragma unroll 1
-            for (int ch = 0; ch < TN / 32; ch += 2) {
-                tmem_ld_fence(ra);
-                tmem_ld_32x32(taddr + (ch + 1) * 32, rb);
-                scan(ra, ch);
-                tmem_ld_fence(rb);
-                if (ch + 2 < TN / 32) tmem_ld_32x32(taddr + (ch + 2) * 32, ra);
-                scan(rb, ch + 1);
-            }
+            drain_accumulator<KMAX, TN>(taddr, vflags, n0, top);
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive(&bars->acc_empty[acc]);

@@ -151,42 +151,7 @@ lookup_tensor_split_kernel(const __grid_constant__ CUtensorMap map_q_hi, const _
             if (!mbar_wait(&bars->acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
             tcgen05_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * TN;
-            // two register buffers: while one chunk of 32 columns is scanned the next is in flight from tensor
-            // memory.  The loop stays rolled (two chunks per trip): unrolled eight times the scan code no longer
-            // fits the instruction cache.
-            uint32_t ra[32], rb[32];
-            auto scan = [&](uint32_t (&r)[32], int ch) {
-                const uint32_t live = __ballot_sync(0xFFFFFFFFu, ((vflags >> ch) & 1ull) != 0ull);
-                if (live == 0u) return;
-                if (live != 0xFFFFFFFFu) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j)
-                        if (!((live >> j) & 1u)) r[j] = 0xFF800000u;      // -inf: never enters a list
-                }
-                // Groups of 8 columns: a group is looked at value by value only if its maximum beats the row's
-                // k-th best.  A warp pays for that path when ANY of its 32 rows takes it, so small groups keep
-                // the common case (nothing to insert) down to 7 max operations and one comparison per group.
-#pragma unroll
-                for (int g8 = 0; g8 < 8; ++g8) {
-                    float m = __uint_as_float(r[g8 * 4]);
-#pragma unroll
-                    for (int j = 1; j < 4; ++j) m = fmaxf(m, __uint_as_float(r[g8 * 4 + j]));
-                    if (m > top.s[KMAX - 1]) {
-#pragma unroll
-                        for (int j = 0; j < 4; ++j) top.push(__uint_as_float(r[g8 * 4 + j]), n0 + ch * 32 + g8 * 4 + j);
-                    }
-                }
-            };
-            tmem_ld_32x32(taddr, ra);
-#pragma unroll 1
-            for (int ch = 0; ch < TN / 32; ch += 2) {
-                tmem_ld_fence(ra);
-                tmem_ld_32x32(taddr + (ch + 1) * 32, rb);
-                scan(ra, ch);
-                tmem_ld_fence(rb);
-                if (ch + 2 < TN / 32) tmem_ld_32x32(taddr + (ch + 2) * 32, ra);
-                scan(rb, ch + 1);
-            }
+            drain_accumulator<KMAX, TN>(taddr, vflags, n0, top);
             tcgen05_fence_before();
             __syncwarp();
             if (lane == 0) mbar_arrive_cluster(cluster_addr(smem_u32(&bars->acc_empty[acc]), 0));

@@ -1,7 +1,8 @@
-// PTX wrappers for kernels in which two CTAs of a cluster drive one tcgen05 tensor-core tile (cta_group::2):
-// cluster addressing, mbarriers with bounded waits, TMA tile loads that report to the leader CTA's barrier,
-// commits that signal both CTAs, the M=256 MMA, tensor-memory loads and the shared-memory operand descriptor.
-// Shared by the CTA-pair lookup kernel and the CTA-pair merge sweep.
+// PTX wrappers of the tensor-core kernels: mbarriers with bounded waits, TMA tile loads, tcgen05 MMA and commit,
+// tensor-memory loads, the shared-memory operand descriptor, and the epilogue's scan of one chunk of accumulator
+// columns.  Two forms where they differ: one CTA drives a tile (cta_group::1), or two CTAs of a cluster drive one
+// tile (cta_group::2: cluster addressing, loads that report to the leader CTA's barrier, commits that signal both
+// CTAs, the M=256 MMA).  Shared by the lookup kernels (single CTA, CTA pair, fp32 split) and the merge sweep.
 #pragma once
 
 #include <cuda.h>
@@ -116,14 +117,88 @@ __device__ __forceinline__ void tmem_ld_fence(uint32_t (&r)[32]) {
           "+r"(r[24]), "+r"(r[25]), "+r"(r[26]), "+r"(r[27]), "+r"(r[28]), "+r"(r[29]), "+r"(r[30]), "+r"(r[31])
         :: "memory");
 }
+// Shared-memory matrix descriptor of a K-major bf16 tile whose rows are 128 bytes and 128-byte swizzled
+// (what the TMA writes): 8-row groups 1024 bytes apart; descriptor version 1; layout type 2 = 128B swizzle.
 __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t saddr) {
     uint64_t d = 0;
-    d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);
-    d |= static_cast<uint64_t>(1) << 16;
-    d |= static_cast<uint64_t>(1024 >> 4) << 32;
-    d |= static_cast<uint64_t>(1) << 46;
-    d |= static_cast<uint64_t>(2) << 61;
+    d |= static_cast<uint64_t>((saddr & 0x3FFFFu) >> 4);          // start address, 16-byte units
+    d |= static_cast<uint64_t>(1) << 16;                         // leading byte offset (unused for swizzled K-major)
+    d |= static_cast<uint64_t>(1024 >> 4) << 32;                 // stride byte offset: 8 rows x 128 B
+    d |= static_cast<uint64_t>(1) << 46;                         // descriptor version
+    d |= static_cast<uint64_t>(2) << 61;                         // SWIZZLE_128B
     return d;
+}
+
+// ---- one CTA per tile ----------------------------------------------------------------------------------------
+__device__ __forceinline__ void mbar_arrive(uint64_t *bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void tma_load_2d(void *dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar))
+                 : "memory");
+}
+// the same load with an L2 eviction policy: used for centroid tiles that no other CTA will read again, so that the
+// one-pass stream does not push the queries, the cache's metadata and the kernels' code out of L2
+__device__ __forceinline__ void tma_load_2d_hint(void *dst, const CUtensorMap *map, int c0, int c1, uint64_t *bar, uint64_t policy) {
+    asm volatile("cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes.L2::cache_hint [%0], [%1, {%2, %3}], [%4], %5;"
+                 ::"r"(smem_u32(dst)), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(smem_u32(bar)), "l"(policy)
+                 : "memory");
+}
+__device__ __forceinline__ void umma_commit(uint64_t *bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(smem_u32(bar)) : "memory");
+}
+__device__ __forceinline__ void umma_bf16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+
+// ---- epilogue of the lookup kernels ----------------------------------------------------------------------------
+// One thread owns one query row: r holds 32 consecutive accumulator columns of that row (similarities of slots
+// first_slot .. first_slot + 31), `live` says which of those slots hold an entry (the same for the whole warp).
+// The columns are taken in groups of 4: a group is looked at value by value only if its maximum beats the row's
+// k-th best.  A warp pays for that path when ANY of its 32 rows takes it, so small groups keep the common case
+// (nothing to insert) down to 3 max operations and one comparison per group.  Insertion is in ascending slot order.
+template <int KMAX>
+__device__ __forceinline__ void scan_chunk32(uint32_t (&r)[32], uint32_t live, int first_slot, TopK<KMAX> &top) {
+    if (live == 0u) return;
+    if (live != 0xFFFFFFFFu) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j)
+            if (!((live >> j) & 1u)) r[j] = 0xFF800000u;      // -inf: never enters a list
+    }
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+        float m = __uint_as_float(r[g * 4]);
+#pragma unroll
+        for (int j = 1; j < 4; ++j) m = fmaxf(m, __uint_as_float(r[g * 4 + j]));
+        if (m > top.s[KMAX - 1]) {
+#pragma unroll
+            for (int j = 0; j < 4; ++j) top.push(__uint_as_float(r[g * 4 + j]), first_slot + g * 4 + j);
+        }
+    }
+}
+
+// Drains one finished accumulator of TN columns for this thread's row (tensor-memory address `taddr`): vflags bit ch
+// says whether slot first_slot + 32 ch + lane holds an entry.  Two register buffers: while one chunk of 32 columns
+// is scanned the next is in flight from tensor memory.  The loop stays rolled (two chunks per trip): unrolled eight
+// times the scan code no longer fits the instruction cache.
+template <int KMAX, int TN>
+__device__ __forceinline__ void drain_accumulator(uint32_t taddr, unsigned long long vflags, int first_slot, TopK<KMAX> &top) {
+    uint32_t ra[32], rb[32];
+    tmem_ld_32x32(taddr, ra);
+#pragma unroll 1
+    for (int ch = 0; ch < TN / 32; ch += 2) {
+        tmem_ld_fence(ra);
+        tmem_ld_32x32(taddr + (ch + 1) * 32, rb);
+        scan_chunk32<KMAX>(ra, __ballot_sync(0xFFFFFFFFu, ((vflags >> ch) & 1ull) != 0ull), first_slot + ch * 32, top);
+        tmem_ld_fence(rb);
+        if (ch + 2 < TN / 32) tmem_ld_32x32(taddr + (ch + 2) * 32, ra);
+        scan_chunk32<KMAX>(rb, __ballot_sync(0xFFFFFFFFu, ((vflags >> (ch + 1)) & 1ull) != 0ull), first_slot + (ch + 1) * 32, top);
+    }
 }
 }  // namespace umma2
 }  // namespace siso
