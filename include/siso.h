@@ -356,6 +356,42 @@ siso_status_t siso_import(siso_cache_t *c, const float *d_master, const double *
 siso_status_t siso_get_stats(siso_cache_t *c, int64_t *h_counts, void *stream);
 /* Synchronise `stream`, return the device status word (SISO_OK if clear) and clear it. */
 siso_status_t siso_sync_status(siso_cache_t *c, void *stream);
+/* MergeCentroids (Algorithm 1, Sec. 4.2 merge step) over a cache whose rows are partitioned across several GPUs: one
+ * handle per GPU holds a contiguous block of the global slots [own_offset, own_offset + capacity).  The double loop of
+ * MergeCentroids is a pairwise sweep over the whole cache; by blocks it falls into one sweep of every block with itself
+ * and one sweep of every unordered pair of blocks, done on one of the two owners after the other block's rows have been
+ * copied into that GPU's own memory (the caller moves them: NCCL send/recv or a peer copy; the library reads local
+ * memory only).  Every GPU then holds the same candidates and runs the same resolution, so all merge maps agree.
+ *   siso_pair_sweep_block   Pairs with similarity > theta_c (exact: fp64 over the fp32 vectors) between the rows of this
+ *                           block and (d_peer_master == NULL) the earlier rows of the same block, or the rows of a peer
+ *                           block d_peer_master [n_peer, dim] fp32 with live flags d_peer_valid [n_peer] at global slots
+ *                           peer_offset + row.  Records (i, j, similarity) of three 32-bit words, global slots, j < i,
+ *                           are APPENDED to d_cand [max_cand][3] at *d_n_cand (a device counter the caller zeroes once);
+ *                           more than max_cand records: SISO_ERR_OVERFLOW in the status word.
+ *   siso_merge_resolve      d_cand [n_cand][3] (records of all GPUs in any order; i = -1 marks an unused place), d_valid
+ *                           [n_total] live flags of all global slots -> d_merge_map [n_total]: the survivor every slot
+ *                           joins (itself for survivors, -1 for empty slots), exactly as siso_merge over one cache would
+ *                           resolve it (closest earlier survivor, ties to the lower slot); *d_n_merged (device) = slots
+ *                           merged away.  The handle only lends its scratch memory.
+ *   siso_merge_pack         This block's merged rows in ascending slot: d_meta [pack_capacity][2] int32 (global slot,
+ *                           survivor; slot -1 in unused places), d_sizes [pack_capacity] cluster_size, d_rows
+ *                           [pack_capacity, dim] fp32 vectors (NULL in sizes-only mode), *d_n_pack (device) their number.
+ *   siso_merge_apply_shard  d_meta / d_sizes / d_rows [n_places]: the packs of all GPUs one after the other in rank order
+ *                           (so ascending global slot, unused places skipped).  Every survivor of this block takes its
+ *                           members: cluster_size added, and with SISO_MERGE_WEIGHTED_MEAN the vector becomes
+ *                           normalise(cluster_size_s c_s + sum of cluster_size_m c_m), vectors as at the start of the
+ *                           merge; this block's merged rows leave the cache.
+ * All asynchronous on `stream`; device pointers. */
+siso_status_t siso_pair_sweep_block(siso_cache_t *c, int64_t own_offset, const float *d_peer_master, const uint8_t *d_peer_valid,
+                                    int64_t n_peer, int64_t peer_offset, float theta_c, int32_t *d_cand, int64_t max_cand,
+                                    int64_t *d_n_cand, void *stream);
+siso_status_t siso_merge_resolve(siso_cache_t *c, const int32_t *d_cand, int64_t n_cand, const uint8_t *d_valid, int64_t n_total,
+                                 int32_t *d_merge_map, int64_t *d_n_merged, void *stream);
+siso_status_t siso_merge_pack(siso_cache_t *c, const int32_t *d_merge_map, int64_t own_offset, int64_t pack_capacity,
+                              int32_t *d_meta, double *d_sizes, float *d_rows, int64_t *d_n_pack, void *stream);
+siso_status_t siso_merge_apply_shard(siso_cache_t *c, const int32_t *d_merge_map, int64_t own_offset, const int32_t *d_meta,
+                                     const double *d_sizes, const float *d_rows, int64_t n_places, uint32_t flags, void *stream);
+
 /* Diagnostics (no passage of the paper: they serve the error model and the measurements of this library).
  *   siso_selftest_wait_timeout  Every device-side wait of the tensor-core kernels is bounded; when one runs out the
  *                      kernel records SISO_ERR_TIMEOUT in the status word and returns normally.  This call exercises

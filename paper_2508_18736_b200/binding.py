@@ -25,7 +25,8 @@ EXPORTS = ["siso_cache_create", "siso_cache_destroy", "siso_set_option", "siso_i
            "siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_lookup_small_noalloc", "siso_cluster", "siso_cache_copy", "siso_update_centroids", "siso_lookup_keys", "siso_combine_keys", "siso_t2h", "siso_md1_wait",
            "siso_choose_theta", "siso_correct_theta", "siso_tier_exit_sim", "siso_tier_select", "siso_tier_finish",
            "siso_route", "siso_evict_keys", "siso_select_evict", "siso_evict_slots", "siso_selftest_wait_timeout",
-           "siso_measure_fp32_fma"]
+           "siso_measure_fp32_fma", "siso_pair_sweep_block", "siso_merge_resolve", "siso_merge_pack",
+           "siso_merge_apply_shard"]
 
 
 class SisoError(RuntimeError):
@@ -101,6 +102,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_sync_status.argtypes = [vp, vp]
     L.siso_selftest_wait_timeout.argtypes = [vp, u32, vp, vp]
     L.siso_measure_fp32_fma.argtypes = [vp, ctypes.POINTER(ctypes.c_double), vp]
+    L.siso_pair_sweep_block.argtypes = [vp, i64, vp, vp, i64, i64, f32, vp, i64, vp, vp]
+    L.siso_merge_resolve.argtypes = [vp, vp, i64, vp, i64, vp, vp, vp]
+    L.siso_merge_pack.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp]
+    L.siso_merge_apply_shard.argtypes = [vp, vp, i64, vp, vp, vp, i64, u32, vp]
     L.siso_launch_count.argtypes = [vp]
     L.siso_launch_count.restype = i64
     L.siso_status_string.argtypes = [i32]
@@ -368,6 +373,50 @@ class SisoCache:
         self._check(self._lib.siso_get_stats(self._h, buf, _stream(stream)), "siso_get_stats")
         names = ["occupancy", "lookups", "hits", "inserts", "evictions", "merges", "clock", "rescans"]
         return {n: int(buf[i]) for i, n in enumerate(names)}
+
+    # ---- MergeCentroids over a cache partitioned across GPUs (see siso_pair_sweep_block ... in siso.h) ----
+    def pair_sweep_block(self, own_offset: int, theta_c: float, cand: torch.Tensor, n_cand: torch.Tensor,
+                         peer_master: Optional[torch.Tensor] = None, peer_valid: Optional[torch.Tensor] = None,
+                         peer_offset: int = 0, stream=None) -> None:
+        """Appends the pairs of this block with itself (no peer) or with a peer block to cand [max, 3] int32 at n_cand."""
+        assert cand.dtype == torch.int32 and cand.dim() == 2 and cand.shape[1] == 3 and cand.is_contiguous()
+        assert n_cand.dtype == torch.int64 and n_cand.numel() == 1
+        n_peer = 0
+        if peer_master is not None:
+            peer_master = peer_master.to(self._dev, torch.float32).contiguous()
+            peer_valid = peer_valid.to(self._dev, torch.uint8).contiguous()
+            n_peer = peer_master.shape[0]
+            assert peer_master.shape[1] == self.dim and peer_valid.numel() == n_peer
+        self._check(self._lib.siso_pair_sweep_block(self._h, int(own_offset), _ptr(peer_master) if n_peer else None,
+                                                    _ptr(peer_valid) if n_peer else None, n_peer, int(peer_offset), float(theta_c),
+                                                    _ptr(cand), cand.shape[0], _ptr(n_cand), _stream(stream)), "siso_pair_sweep_block")
+
+    def merge_resolve(self, cand: torch.Tensor, valid: torch.Tensor, stream=None):
+        """Candidates of all shards [n, 3] int32 + live flags of all global slots -> (merge_map int32 [n_total], n_merged int64 [1])."""
+        cand = cand.to(self._dev, torch.int32).contiguous()
+        valid = valid.to(self._dev, torch.uint8).contiguous()
+        mm = self._new((valid.numel(),), torch.int32)
+        n = self._new((1,), torch.int64)
+        self._check(self._lib.siso_merge_resolve(self._h, _ptr(cand) if cand.shape[0] else None, cand.shape[0], _ptr(valid),
+                                                 valid.numel(), _ptr(mm), _ptr(n), _stream(stream)), "siso_merge_resolve")
+        return mm, n
+
+    def merge_pack(self, merge_map: torch.Tensor, own_offset: int, capacity: int, with_rows: bool, stream=None):
+        """This shard's merged rows: (meta int32 [capacity, 2], sizes f64 [capacity], rows f32 [capacity, dim] or None, n int64 [1])."""
+        cap = max(1, int(capacity))
+        meta, sizes = self._new((cap, 2), torch.int32), self._new((cap,), torch.float64)
+        rows = self._new((cap, self.dim), torch.float32) if with_rows else None
+        n = self._new((1,), torch.int64)
+        self._check(self._lib.siso_merge_pack(self._h, _ptr(merge_map), int(own_offset), cap, _ptr(meta), _ptr(sizes), _ptr(rows),
+                                              _ptr(n), _stream(stream)), "siso_merge_pack")
+        return meta, sizes, rows, n
+
+    def merge_apply_shard(self, merge_map: torch.Tensor, own_offset: int, meta: torch.Tensor, sizes: torch.Tensor,
+                          rows: Optional[torch.Tensor], flags: int, stream=None) -> None:
+        meta, sizes = meta.contiguous(), sizes.contiguous()
+        rows = None if rows is None else rows.contiguous()
+        self._check(self._lib.siso_merge_apply_shard(self._h, _ptr(merge_map), int(own_offset), _ptr(meta), _ptr(sizes), _ptr(rows),
+                                                     meta.shape[0], int(flags), _stream(stream)), "siso_merge_apply_shard")
 
     def selftest_wait_timeout(self, poll_limit: int = 4096, stream=None) -> torch.Tensor:
         """Lets one bounded device-side wait run out (see siso_selftest_wait_timeout); returns the device flag."""

@@ -9,7 +9,7 @@ HERE = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(HERE, "csrc")
 LIB = os.path.join(HERE, "libsiso.so")
 SOURCES = ["api.cu", "lookup_simt.cu", "lookup_stream.cu", "lookup_tensor.cu", "lookup_tensor_pair.cu", "lookup_tensor_split.cu", "lookup_noalloc.cu", "sort.cu", "update.cu", "evict.cu",
-           "merge.cu", "merge_tensor.cu", "cluster.cu", "swap.cu", "shard.cu", "tier.cu", "t2h.cu", "stream_maint.cu", "selftest.cu"]
+           "merge.cu", "merge_tensor.cu", "cluster.cu", "swap.cu", "shard.cu", "tier.cu", "t2h.cu", "stream_maint.cu", "selftest.cu", "shard_merge.cu"]
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17", "--use_fast_math=false",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-O2"]
 

@@ -134,11 +134,13 @@ siso_status_t launch_update(Cache *c, const void *q, int64_t B, const int32_t *i
                             cudaStream_t s);
 siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes, int64_t n_repo, float theta_c,
                            uint32_t flags, int32_t *merge_map, long long *d_n_merged, cudaStream_t s);
+siso_status_t launch_merge_resolve_global(Cache *c, const void *cand, int64_t n_cand, const uint8_t *valid, int64_t N,
+                                          int32_t *merge_map, long long *d_n_merged, cudaStream_t s);
 size_t merge_tensor_scratch_bytes(const Cache *c);
 size_t pair_sweep_tensor_scratch_bytes(int64_t n, int64_t rows, int dim);
 siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, int64_t N, int64_t rows, const uint8_t *valid,
                                        const uint8_t *seed, float theta_c, void *ctl, void *cand, size_t max_cand,
-                                       uint32_t *row_count, cudaStream_t s, const void *rows_bf16);
+                                       uint32_t *row_count, cudaStream_t s, const void *rows_bf16, int64_t cross_rows = 0);
 siso_status_t launch_merge_resolve(Cache *c, void *ctl, int64_t N, const uint8_t *valid, const uint8_t *seed,
                                    const uint32_t *row_off, const uint32_t *row_count, const int32_t *csr_j,
                                    const float *csr_sim, uint8_t *state, int32_t *target, unsigned int *undecided,

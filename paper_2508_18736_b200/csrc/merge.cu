@@ -358,6 +358,71 @@ siso_status_t launch_merge_resolve(Cache *c, void *ctl_v, int64_t N, const uint8
     return SISO_OK;
 }
 
+// ---- resolution over candidates that were found elsewhere (a cache partitioned over several GPUs) ----------------
+__global__ void merge_count_rows_kernel(const Candidate *__restrict__ cand, unsigned long long n, int64_t N,
+                                        uint32_t *__restrict__ row_count, int *status) {
+    for (unsigned long long e = static_cast<unsigned long long>(blockIdx.x) * blockDim.x + threadIdx.x; e < n;
+         e += static_cast<unsigned long long>(gridDim.x) * blockDim.x) {
+        const Candidate cd = cand[e];
+        if (cd.i < 0) continue;
+        if (cd.i >= N || cd.j < 0 || cd.j >= cd.i) { set_status(status, SISO_ERR_INVALID_ARG); continue; }
+        atomicAdd(&row_count[cd.i], 1u);
+    }
+}
+
+__global__ void merge_map_out_kernel(int64_t N, const volatile uint8_t *state, const int32_t *__restrict__ target,
+                                     int32_t *__restrict__ merge_map, unsigned long long *n_merged) {
+    const int64_t i = static_cast<int64_t>(blockIdx.x) * blockDim.x + threadIdx.x;
+    const bool merged = i < N && state[i] == 2;
+    if (i < N) merge_map[i] = target[i];
+    const unsigned ballot = __ballot_sync(0xFFFFFFFFu, merged);
+    if (ballot && (threadIdx.x & 31) == 0) atomicAdd(n_merged, static_cast<unsigned long long>(__popc(ballot)));
+}
+
+// cand [n_cand]: records (i, j, similarity) with j < i over rows 0..N-1, i = -1 for unused places; valid [N].
+// merge_map [N] receives, for every row, the survivor it joins (itself for survivors, -1 for empty rows), as the
+// resolution inside siso_merge would give it; *d_n_merged the number of rows merged away.
+siso_status_t launch_merge_resolve_global(Cache *c, const void *cand_v, int64_t n_cand, const uint8_t *valid, int64_t N,
+                                          int32_t *merge_map, long long *d_n_merged, cudaStream_t s) {
+    if (N >= (1ll << 31) - 1 || n_cand < 0) return SISO_ERR_UNSUPPORTED;
+    const Candidate *cand = static_cast<const Candidate *>(cand_v);
+    const size_t nc = static_cast<size_t>(std::max<int64_t>(n_cand, 1));
+    Scratch scr;
+    const size_t need = pad256(sizeof(MergeCtl)) + 3 * pad256(sizeof(uint32_t) * (N + 1)) + pad256(sizeof(int32_t) * nc) +
+                        pad256(sizeof(float) * nc) + pad256(N) + pad256(sizeof(int32_t) * N) + 256 + 256;
+    SISO_TRY(scratch_reserve(c, need, s, &scr));
+    MergeCtl *ctl = scr.take<MergeCtl>(1);
+    uint32_t *row_count = scr.take<uint32_t>(N + 1);
+    uint32_t *row_off = scr.take<uint32_t>(N + 1);
+    uint32_t *row_cursor = scr.take<uint32_t>(N + 1);
+    int32_t *csr_j = scr.take<int32_t>(nc);
+    float *csr_sim = scr.take<float>(nc);
+    uint8_t *state = scr.take<uint8_t>(N);
+    int32_t *target = scr.take<int32_t>(N);
+    unsigned int *undecided = scr.take<unsigned int>(3);
+    MergeCtl h = {};
+    h.n_cand = static_cast<unsigned long long>(n_cand);
+    SISO_CUDA(cudaMemcpyAsync(ctl, &h, sizeof(h), cudaMemcpyHostToDevice, s));      // pageable source: copied before the call returns
+    SISO_CUDA(cudaMemsetAsync(row_count, 0, sizeof(uint32_t) * (N + 1), s));
+    SISO_CUDA(cudaMemsetAsync(row_cursor, 0, sizeof(uint32_t) * (N + 1), s));
+    SISO_CUDA(cudaMemsetAsync(d_n_merged, 0, sizeof(long long), s));
+    if (n_cand > 0) {
+        merge_count_rows_kernel<<<4 * c->sm_count, 256, 0, s>>>(cand, static_cast<unsigned long long>(n_cand), N, row_count, c->status);
+        SISO_LAUNCHED(c);
+    }
+    SISO_CUDA(cudaMemcpyAsync(row_off, row_count, sizeof(uint32_t) * (N + 1), cudaMemcpyDeviceToDevice, s));
+    SISO_TRY(launch_exclusive_scan_u32(c, row_off, N + 1, s));
+    if (n_cand > 0) {
+        merge_scatter_kernel<<<4 * c->sm_count, 256, 0, s>>>(ctl, cand, row_off, row_cursor, csr_j, csr_sim);
+        SISO_LAUNCHED(c);
+    }
+    SISO_TRY(launch_merge_resolve(c, ctl, N, valid, nullptr, row_off, row_count, csr_j, csr_sim, state, target, undecided, s));
+    merge_map_out_kernel<<<static_cast<unsigned>((N + 255) / 256), 256, 0, s>>>(N, state, target, merge_map,
+                                                                               reinterpret_cast<unsigned long long *>(d_n_merged));
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
+
 siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes, int64_t n_repo, float theta_c,
                            uint32_t flags, int32_t *merge_map, long long *d_n_merged, cudaStream_t s) {
     c->vec_epoch += 1;          // the vectors may change: derived copies (the split-bf16 parts) are stale

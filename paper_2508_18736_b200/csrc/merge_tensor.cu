@@ -374,9 +374,11 @@ size_t merge_tensor_scratch_bytes(const Cache *c) { return pair_sweep_tensor_scr
 // insertion's failure flag); on return (in stream order) cand[0 .. min(n_cand, max_cand)) holds the provisional
 // pairs, the confirmed ones with their exact similarity and i >= 0, and row_count[i] (if not NULL) counts the
 // confirmed pairs of row i.
+// `cross_rows` > 0 (a multiple of 256, with `seed` marking exactly the rows below it): only the pairs of a row at or
+// beyond cross_rows with a row below it are swept, i.e. one block of rows against another block.
 siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, int64_t N, int64_t rows, const uint8_t *valid,
                                        const uint8_t *seed, float theta_c, void *ctl, void *cand, size_t max_cand,
-                                       uint32_t *row_count, cudaStream_t s, const void *rows_bf16) {
+                                       uint32_t *row_count, cudaStream_t s, const void *rows_bf16, int64_t cross_rows) {
     static tcm::EncodeTiledFn encode = nullptr;
     if (!encode) {
         void *fn = nullptr;
@@ -407,11 +409,21 @@ siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, i
     constexpr int SB = 9;
     std::vector<uint32_t> list;
     list.reserve(static_cast<size_t>(tiles) * (tiles + 1) / (seed ? 1 : 2));
-    for (int bi = 0; bi < tiles; bi += SB)
-        for (int bt = 0; bt < (seed ? tiles : bi + 1); bt += SB)
-            for (int I = bi; I < std::min(tiles, bi + SB); ++I)
-                for (int t = bt; t < std::min(seed ? tiles : I + 1, bt + SB); ++t)
-                    list.push_back((static_cast<uint32_t>(I) << 16) | static_cast<uint32_t>(t));
+    const int cross_tiles = static_cast<int>(cross_rows / (2 * tcm::TM));
+    if (cross_rows > 0) {
+        if (!seed || cross_rows % (2 * tcm::TM) != 0 || cross_tiles >= tiles) return SISO_ERR_INVALID_ARG;
+        for (int bi = cross_tiles; bi < tiles; bi += SB)
+            for (int bt = 0; bt < cross_tiles; bt += SB)
+                for (int I = bi; I < std::min(tiles, bi + SB); ++I)
+                    for (int t = bt; t < std::min(cross_tiles, bt + SB); ++t)
+                        list.push_back((static_cast<uint32_t>(I) << 16) | static_cast<uint32_t>(t));
+    } else {
+        for (int bi = 0; bi < tiles; bi += SB)
+            for (int bt = 0; bt < (seed ? tiles : bi + 1); bt += SB)
+                for (int I = bi; I < std::min(tiles, bi + SB); ++I)
+                    for (int t = bt; t < std::min(seed ? tiles : I + 1, bt + SB); ++t)
+                        list.push_back((static_cast<uint32_t>(I) << 16) | static_cast<uint32_t>(t));
+    }
     const long long n_pairs = static_cast<long long>(list.size());
     uint32_t *pair_list = scr->take<uint32_t>(list.size());
     SISO_CUDA(cudaMemcpyAsync(pair_list, list.data(), sizeof(uint32_t) * list.size(), cudaMemcpyHostToDevice, s));
@@ -433,7 +445,7 @@ siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, i
 siso_status_t launch_merge_sweep_tensor(Cache *c, Scratch *scr, const uint8_t *seed, float theta_c, void *ctl, void *cand,
                                         size_t max_cand, uint32_t *row_count, cudaStream_t s) {
     return launch_pair_sweep_tensor(c, scr, c->master, c->capacity, c->rows_alloc, c->valid, seed, theta_c, ctl, cand, max_cand,
-                                    row_count, s, nullptr);
+                                    row_count, s, nullptr, 0);
 }
 
 }  // namespace siso

@@ -11,8 +11,10 @@ calls the update once per batch, so the clocks agree), FilteringCentroids become
 the m lowest of all reported keys go" (one all-gather of 24 bytes per key), and the misses of a batch, in ascending row
 order, take the free slots of the whole cache in ascending global order (one all-gather of the free counts, one
 all-reduce(max) of the slots).  Each of these operations is written once, as a generator that yields its exchanges
-(`("gather", tensor)` -> [world, ...], `("max", tensor)` -> elementwise maximum over ranks) and is driven either by
-torch.distributed (`run`) or, on one GPU, by `run_lockstep` over several shards of the same process.
+(`("gather", tensor)` -> [world, ...], `("max", tensor)` -> elementwise maximum over ranks, `("ring", tensor, shift)` ->
+the tensor of the rank `shift` places back, copied into this rank's memory) and is driven either by torch.distributed
+(`run`) or, on one GPU, by `run_lockstep` over several shards of the same process.  MergeCentroids over the partitioned
+cache (`merge_steps`) cuts its pairwise sweep into block products along such a ring.
 
 Global slot g lives on rank g // rows_per_rank at local slot g % rows_per_rank.
 """
@@ -53,9 +55,25 @@ def gather_keys(keys: torch.Tensor, group=None) -> torch.Tensor:
     return out.view(world, n, k).permute(1, 0, 2).contiguous()
 
 
-def exchange(kind: str, t: torch.Tensor, group=None) -> torch.Tensor:
-    """One exchange of a sharded operation over torch.distributed: "gather" -> [world, *t.shape], "max" -> t's shape."""
+def exchange(kind: str, t: torch.Tensor, group=None, shift: int = 0) -> torch.Tensor:
+    """One exchange of a sharded operation over torch.distributed: "gather" -> [world, *t.shape], "max" -> t's shape,
+    "ring" -> the tensor that rank (own rank - shift) mod world passed, received into this rank's own memory (every
+    rank passes the same shape)."""
     inited = dist.is_available() and dist.is_initialized()
+    if kind == "ring":
+        world = dist.get_world_size(group) if inited else 1
+        shift %= world
+        if shift == 0:
+            return t.clone()
+        rank = dist.get_rank(group)
+        src, dst = (rank - shift) % world, (rank + shift) % world
+        if group is not None:
+            src, dst = dist.get_global_rank(group, src), dist.get_global_rank(group, dst)
+        t = t.contiguous()
+        out = torch.empty_like(t)
+        for req in dist.batch_isend_irecv([dist.P2POp(dist.isend, t, dst, group), dist.P2POp(dist.irecv, out, src, group)]):
+            req.wait()
+        return out
     if kind == "gather":
         if not inited:
             return t.unsqueeze(0).contiguous()
@@ -77,7 +95,7 @@ def run(steps: Generator, group=None):
     try:
         req = next(steps)
         while True:
-            req = steps.send(exchange(req[0], req[1], group))
+            req = steps.send(exchange(req[0], req[1], group, *req[2:]))
     except StopIteration as done:
         return done.value
 
@@ -101,9 +119,16 @@ def run_lockstep(all_steps: Sequence[Generator]) -> List:
         kinds = {q[0] for q in reqs.values()}
         assert len(kinds) == 1, "shards disagree on the next exchange"
         stacked = torch.stack([reqs[r][1] for r in range(len(all_steps))])
-        answer = stacked if kinds == {"gather"} else stacked.max(dim=0).values
+        if kinds == {"ring"}:
+            shifts = {q[2] for q in reqs.values()}
+            assert len(shifts) == 1, "shards disagree on the ring step"
+            shift = shifts.pop() % len(all_steps)
+            answers = [stacked[(r - shift) % len(all_steps)].clone() for r in range(len(all_steps))]
+        else:
+            answer = stacked if kinds == {"gather"} else stacked.max(dim=0).values
+            answers = [answer.clone() for _ in range(len(all_steps))]
         for r in range(len(all_steps)):
-            advance(r, answer.clone(), False)
+            advance(r, answers[r], False)
     return results
 
 
@@ -194,6 +219,65 @@ class ShardedCache:
             slots.fill_(-1)
         slots = yield ("max", slots)
         return idx, sim, hit, victims, slots
+
+    def merge_steps(self, theta_c: float, flags: int, cand_capacity: Optional[int] = None):
+        """MergeCentroids over the whole cache (one pass, like siso_merge with no repository): -> (merge_map int32
+        [total_rows] over the global slots, number of entries merged away), the same on every rank and equal to one
+        unsharded cache's pass.  The pairwise sweep is cut into block products: every rank sweeps its own block, and
+        every unordered pair of blocks is swept once, on one of its owners, after the other block has travelled round
+        the ring into that rank's own memory (about world / 2 ring steps).  Candidates, live flags and the merged rows
+        are then gathered; the resolution runs identically on every rank."""
+        from .binding import MERGE_WEIGHTED_MEAN
+        G, r, rpr = self.world, self.rank, self.rows_per_rank
+        dev, D = self.local._dev, self.local.dim
+        n_own = self.hi - self.lo
+        st = self.local.export()
+        block = torch.zeros((rpr, D), dtype=torch.float32, device=dev)
+        valid = torch.zeros((rpr,), dtype=torch.uint8, device=dev)
+        if n_own:
+            block[:n_own] = st["master"][:n_own]
+            valid[:n_own] = st["valid"][:n_own]
+        del st
+        cap = int(cand_capacity) if cand_capacity else 32 * rpr + 65536
+        cand = torch.full((cap, 3), -1, dtype=torch.int32, device=dev)
+        n_cand = torch.zeros((1,), dtype=torch.int64, device=dev)
+        if n_own:
+            self.local.pair_sweep_block(self.lo, theta_c, cand, n_cand)
+        for t in range(1, G // 2 + 1):
+            peer_block = yield ("ring", block, t)
+            peer_valid = yield ("ring", valid, t)
+            s = (r - t) % G
+            s_lo, s_hi = local_range(s, self.total_rows, rpr)
+            mine = (2 * t < G) or (2 * t == G and r < s)          # each unordered pair of blocks on exactly one owner
+            if mine and n_own and s_hi > s_lo:
+                self.local.pair_sweep_block(self.lo, theta_c, cand, n_cand, peer_block[:s_hi - s_lo], peer_valid[:s_hi - s_lo], s_lo)
+        self.local.check_status()
+        counts = yield ("gather", n_cand)                        # [world, 1]
+        pad = max(1, int(counts.max().item()))
+        all_cand = yield ("gather", cand[:pad].contiguous())     # [world, pad, 3]; places beyond a rank's count hold i = -1
+        all_valid = yield ("gather", valid)                      # [world, rows_per_rank] = live flags by global slot
+        mm, n_merged = self.local.merge_resolve(all_cand.reshape(-1, 3), all_valid.reshape(-1))
+        weighted = bool(flags & MERGE_WEIGHTED_MEAN)
+        own_map = mm[self.lo:self.lo + max(n_own, 1)]
+        n_gone = 0
+        if n_own:
+            slots = torch.arange(self.lo, self.hi, dtype=torch.int32, device=dev)
+            n_gone = int(((own_map[:n_own] >= 0) & (own_map[:n_own] != slots) & (valid[:n_own] != 0)).sum().item())
+        gone = yield ("gather", torch.tensor([n_gone], dtype=torch.int64, device=dev))
+        P = max(1, int(gone.max().item()))
+        meta, sizes, rows, _ = self.local.merge_pack(mm, self.lo, P, weighted)
+        if not n_own:
+            meta.fill_(-1)
+        all_meta = yield ("gather", meta)                        # [world, P, 2]: rank order = ascending global slot
+        all_sizes = yield ("gather", sizes)
+        all_rows = (yield ("gather", rows)) if weighted else None
+        self.local.merge_apply_shard(mm, self.lo, all_meta.reshape(-1, 2), all_sizes.reshape(-1),
+                                     None if all_rows is None else all_rows.reshape(-1, D), flags)
+        self.local.check_status()
+        return mm[:self.total_rows], int(n_merged.item())
+
+    def merge(self, theta_c: float, flags: int):
+        return run(self.merge_steps(theta_c, flags), self.group)
 
     def evict(self, n_evict: int, flags: int = 0) -> torch.Tensor:
         return run(self.evict_steps(n_evict, flags), self.group)

@@ -7,7 +7,7 @@ import torch
 
 import oracle
 from gen import workloads as W
-from util import TOL, check_lookup, to_dev
+from util import TOL, check_lookup, to_dev, verify_merge_map
 
 pytestmark = pytest.mark.gpu
 
@@ -172,3 +172,71 @@ def test_world_of_one_through_the_distributed_driver():
     assert all((a[k] == b[k]).all().item() for k in ("valid", "size", "access"))
     one.close()
     plain.close()
+
+
+@pytest.mark.parametrize("dtype,n,dim,shards,weighted,theta_c", [
+    ("f32", 1500, 136, 3, True, 0.90),        # ragged last shard; an odd number of blocks
+    ("f32", 1400, 72, 4, False, 0.86),        # an even number: the opposite blocks are swept by the lower rank only
+    ("bf16", 2100, 264, 2, True, 0.90),
+    ("f32", 900, 64, 8, True, 0.90),          # shards smaller than a tile of the sweep
+    ("f32", 40, 64, 6, True, 0.90),           # more ranks than rows can fill: empty shards at the end
+])
+def test_sharded_merge_equals_one_cache(dtype, n, dim, shards, weighted, theta_c):
+    """MergeCentroids over a partitioned cache, the blocks travelling round a ring: merge map, cluster sizes, live flags
+    and vectors of every shard against the oracle's pass over the whole cache, pass after pass until nothing merges."""
+    w = W.config(3, seed=17, mode="P", n_centroids=n, dim=dim, n_clusters=max(2, n // 18), sigma=0.06, dtype=dtype)
+    sizes = np.random.default_rng(3).integers(1, 9, n).astype(np.float64)
+    parts = [siso.ShardedCache(n, dim, dtype, rank=r, world=shards) for r in range(shards)]
+    all_rows = to_dev(w.centroids, dtype)
+    for p in parts:
+        if p.hi > p.lo:
+            p.local.insert(all_rows[p.lo:p.hi], torch.from_numpy(sizes[p.lo:p.hi]))
+    ora = oracle.OracleCache(n, dim, dtype)
+    ora.insert(w.centroids, sizes=sizes)
+    flags = siso.MERGE_WEIGHTED_MEAN if weighted else siso.MERGE_SIZES_ONLY
+    total_merged = 0
+    for rounds in range(40):
+        entry, valid0, sizes0 = ora.master.copy(), ora.valid.copy(), ora.size.copy()
+        results = siso.run_lockstep([p.merge_steps(theta_c, flags) for p in parts])
+        mm, n_merged = results[0][0].cpu().numpy(), results[0][1]
+        for other, cnt in results[1:]:
+            assert (other.cpu().numpy() == mm).all() and cnt == n_merged           # every rank holds the same map
+        o_mm, o_n = ora.merge(theta_c, weighted)
+        same = (mm == o_mm).all()
+        if not same:       # only a decision within 1e-5 of the threshold or of the runner-up may differ
+            verify_merge_map(entry, valid0, np.zeros(n, np.uint8), sizes0, mm, theta_c, tol=1e-5)
+        else:
+            assert n_merged == o_n
+        total_merged += n_merged
+        for p in parts:
+            if p.hi == p.lo:
+                continue
+            st = p.local.export()
+            torch.cuda.synchronize()
+            lo, hi = p.lo, p.hi
+            surv = mm[lo:hi] == np.arange(lo, hi)
+            assert (st["valid"].cpu().numpy() == surv).all()
+            if same:
+                live = ora.valid[lo:hi] == 1
+                assert (st["size"].cpu().numpy()[live] == ora.size[lo:hi][live]).all()
+                assert np.abs(st["master"].cpu().numpy()[live] - ora.master[lo:hi][live]).max(initial=0) <= 1e-6
+            assert p.local.stats()["occupancy"] == int(surv.sum())
+            p.local.check_status()
+        if not same or n_merged == 0:
+            break
+    assert total_merged > (n // 3 if n > 100 else 0)
+    if same:
+        assert n_merged == 0, "no fixed point within 40 passes"
+    # the candidate buffer of a shard that is too small is reported, not overrun
+    if n >= 900:
+        fresh = [siso.ShardedCache(n, dim, dtype, rank=r, world=shards) for r in range(shards)]
+        for p in fresh:
+            if p.hi > p.lo:
+                p.local.insert(all_rows[p.lo:p.hi])
+        with pytest.raises(siso.SisoError) as e:
+            siso.run_lockstep([p.merge_steps(theta_c, flags, cand_capacity=8) for p in fresh])
+        assert e.value.status == 5
+        for p in fresh:
+            p.close()
+    for p in parts:
+        p.close()

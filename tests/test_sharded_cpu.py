@@ -103,3 +103,46 @@ def test_the_two_drivers_of_a_sharded_operation_agree():
         yield
 
     assert sharded.run(nothing_to_do()) == 7 and sharded.run_lockstep([nothing_to_do(), nothing_to_do()]) == [7, 7]
+
+
+def _ring_steps(rank, world):
+    """The exchange pattern of the sharded MergeCentroids: about world / 2 ring steps, each unordered pair of blocks
+    assigned to exactly one of its owners."""
+    block = torch.full((3,), float(rank))
+    swept = []
+    for t in range(1, world // 2 + 1):
+        peer = yield ("ring", block, t)
+        s = (rank - t) % world
+        assert peer.tolist() == [float(s)] * 3, "the ring delivered another rank's block"
+        if (2 * t < world) or (2 * t == world and rank < s):
+            swept.append((rank, s))
+    pairs = yield ("gather", torch.tensor(swept + [(-1, -1)] * (world - len(swept)), dtype=torch.int64))
+    return pairs.reshape(-1, 2).tolist()
+
+
+def _worker_ring(rank, world, port, out):
+    sys.path.insert(0, ROOT)
+    os.environ.update(MASTER_ADDR="127.0.0.1", MASTER_PORT=str(port), RANK=str(rank), WORLD_SIZE=str(world))
+    dist.init_process_group("gloo", rank=rank, world_size=world)
+    from paper_2508_18736_b200 import sharded
+    out[rank] = sharded.run(_ring_steps(rank, world))
+    dist.barrier()
+    dist.destroy_process_group()
+
+
+def test_ring_exchange_delivers_every_pair_of_blocks_to_exactly_one_owner():
+    sys.path.insert(0, ROOT)
+    from paper_2508_18736_b200 import sharded
+    for world in (2, 3, 4, 5, 8):                       # in one process
+        res = sharded.run_lockstep([_ring_steps(r, world) for r in range(world)])
+        pairs = sorted(tuple(sorted(p)) for p in res[0] if p[0] >= 0)
+        assert pairs == [(a, b) for a in range(world) for b in range(a + 1, world)], world
+        assert all(r == res[0] for r in res)
+    world = 3                                           # and over torch.distributed (gloo, three processes)
+    port = 35500 + os.getpid() % 2000
+    with mp.get_context("spawn").Manager() as mgr:
+        out = mgr.dict()
+        mp.spawn(_worker_ring, args=(world, port, out), nprocs=world, join=True)
+        res = dict(out)
+    pairs = sorted(tuple(sorted(p)) for p in res[0] if p[0] >= 0)
+    assert pairs == [(0, 1), (0, 2), (1, 2)] and res[0] == res[1] == res[2]
