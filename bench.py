@@ -53,6 +53,10 @@ def parse_args():
                          "decay of FilteringCentroids, as the paper re-clusters when enough new queries have arrived")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-e2e", action="store_true")
+    ap.add_argument("--sharded", action="store_true",
+                    help="time the CENTROID-SHARDED cache instead of replicas: the rows of the workload are partitioned over the "
+                         "--gpus ranks, every rank scores the same query batch against its rows, one all-gather of packed keys "
+                         "(strong scaling); also times the sharded streaming step on the configuration-5 cache")
     ap.add_argument("--no-secondary", action="store_true",
                     help="skip the extra measurements of the default line (streaming step, small-batch sweeps, hit update)")
     return ap.parse_args()
@@ -528,6 +532,110 @@ def secondary_measurements(args, siso, cache4, w4, peaks, cores, dev):
     return sec
 
 
+# ------------------------------------------------------------------------------ the centroid-sharded cache
+def run_sharded(args):
+    """One JSON line for the cache partitioned over the ranks (sharded.py): config-4 lookup with the rows split N ways
+    and the sharded streaming step of configuration 5.  Launched like the default arm (torchrun for N > 1)."""
+    import torch
+    import torch.distributed as dist
+    from paper_2508_18736_b200 import build as _b
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if world != args.gpus:
+        raise SystemExit(f"--gpus {args.gpus} needs WORLD_SIZE={args.gpus} (launch with torch.distributed.run); got {world}")
+    torch.cuda.set_device(local_rank)
+    dev = torch.device("cuda", local_rank)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=dev)
+    if local_rank == 0:
+        _b.build()
+    if world > 1:
+        dist.barrier()
+    import paper_2508_18736_b200 as siso
+    from gen import workloads as W
+    cores = max(1, (os.cpu_count() or 1) // world)
+    peaks, peak_kind = load_peaks()
+
+    def to_dev(a):
+        return torch.from_numpy(a.view(np.int16)).to(dev).view(torch.bfloat16)
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(step, steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        e0.record()
+        for _ in range(steps):
+            step()
+        e1.record()
+        barrier()
+        return max_over_ranks(e0.elapsed_time(e1), world, dev) / steps
+
+    # ---- lookup: the same centroids and the same batch on every rank (seeded), each rank keeps its rows
+    w = workload(args, 0, cores)
+    B, k = args.queries, w.k
+    shard = siso.ShardedCache(args.rows, 1024, "bf16", device=local_rank)
+    for lo in range(shard.lo, shard.hi, 1 << 16):
+        hi = min(shard.hi, lo + (1 << 16))
+        shard.local.insert(to_dev(w.centroids[lo:hi]))
+    shard.local.check_status()
+    q, th = to_dev(w.queries), torch.from_numpy(w.theta).to(dev)
+    for _ in range(max(3, args.warmup)):
+        shard.lookup(q, th, k)
+    sampler = ClockSampler(local_rank) if rank == 0 else None
+    ms = timed(lambda: shard.lookup(q, th, k), args.steps)
+    clocks = sampler.stop() if sampler else None
+    idx, sim, hit = shard.lookup(q, th, k)
+    shard.local.check_status()
+    flops = 2.0 * B * args.rows * 1024
+    line = {"metric": METRIC + " (centroid-sharded cache)", "value": B / (ms * 1e-3), "unit": UNIT, "n_gpus": world,
+            "steps": args.steps, "warmup": max(3, args.warmup), "ms_per_step": ms, "higher_is_better": True, "scaling": "strong",
+            "vs_baseline": None, "dtype": "bf16", "data": "synthetic",
+            "config": {"workload": workload_name(args), "parallelism": f"centroid rows sharded x{world}: {shard.hi - shard.lo} rows per rank, "
+                       "every rank scores the whole batch, one all-gather of packed top-k keys",
+                       "l2": "inputs larger than L2 while rows / ranks x 2 KiB exceeds it"},
+            "clocks": clocks, "hits": int(hit.sum().item()),
+            "roofline": {"bound": "tensor", "achieved": flops / (ms * 1e-3) / 1e12, "peak": peaks["bf16_tflops"] * world, "unit": "TFLOP/s",
+                         "frac": flops / (ms * 1e-3) / 1e12 / (peaks["bf16_tflops"] * world), "traffic": None,
+                         "peak_kind": f"{peak_kind}, burst, x{world} GPUs"}}
+    shard.close()
+    # ---- the sharded streaming step (configuration 5's cache split over the ranks, steady state)
+    sp = W.StreamSpec()
+    stream = W.QueryStream(sp, threads=cores)
+    n_warm, n_timed = 100, 300
+    q_all = to_dev(stream.block(0, n_warm + n_timed, threads=cores))
+    sc = siso.ShardedCache(sp.capacity, sp.dim, "bf16", device=local_rank)
+    first = 20000 + sc.lo // sp.batch
+    filler = stream.block(first, first + (sc.hi - sc.lo) // sp.batch, threads=cores)
+    for lo in range(0, filler.shape[0], 1 << 16):
+        sc.local.insert(to_dev(filler[lo:lo + (1 << 16)]))
+    sc.local.check_status()
+    t = [0]
+
+    def stream_step():
+        sc.stream_step(q_all[t[0] * 256:(t[0] + 1) * 256], float(sp.theta))
+        t[0] += 1
+
+    for _ in range(n_warm):
+        stream_step()
+    us = timed(stream_step, n_timed) * 1e3
+    st = sc.local.stats()
+    line["stream_step"] = {"workload": f"config 5 cache ({sp.capacity} x {sp.dim} bf16) sharded x{world}, micro-batches of 256",
+                           "us_per_batch": us, "queries_per_s": 256 / us * 1e6, "evictions_this_rank": st["evictions"],
+                           "note": "lookup keys, free counts, eviction keys and slots are exchanged every batch; this version reads "
+                                   "a few counts on the host between phases"}
+    sc.close()
+    if rank == 0:
+        print(json.dumps(line), flush=True)
+    if world > 1:
+        dist.destroy_process_group()
+    return 0
+
+
 # ------------------------------------------------------------------------------ the other configurations
 def run_other(args):
     """One JSON line for configuration 1, 2, 3, 5 or the small-batch streaming probe (single GPU, device-resident)."""
@@ -896,6 +1004,8 @@ def main():
     args = parse_args()
     if args.impl == "reference":
         return run_reference(args)
+    if args.sharded:
+        return run_sharded(args)
     if args.workload != "config4":
         return run_other(args)
     return run_ours(args)

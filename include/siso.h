@@ -277,6 +277,30 @@ siso_status_t siso_tier_finish(const uint64_t *d_hot_keys, int64_t n_queries, fl
                                const float *d_theta, float theta_scalar, int32_t *d_idx, float *d_sim, uint8_t *d_hit,
                                void *stream);
 
+/* The locality-ordered search as two calls (Sec. 4.3, "Searching for vectors in semantic cache", exact counterpart).
+ *   siso_tier_build   Splits `cache` (left untouched) into the HOT tier - the hot_rows entries FilteringCentroids would
+ *                     evict last - and the COLD rest, written into the handles `hot` and `cold` (same dim, dtype and
+ *                     device; capacities at least hot_rows and occupancy - hot_rows, else SISO_ERR_CAPACITY; what they
+ *                     held is dropped).  Entries keep their vectors and metadata and are laid out in ascending slot of
+ *                     `cache`; d_hot_slot / d_cold_slot [capacity of the tier] receive the slot of `cache` each place
+ *                     came from.  h_counts[0], [1] = entries in the hot and the cold tier.  If sep_sim is not NaN, every
+ *                     hot/cold pair is also checked against it (tensor-core sweep + exact fp64 check) and h_counts[2]
+ *                     receives the number of pairs MORE similar than sep_sim (at least 65 if there are more than 64):
+ *                     the exit rule of siso_tier_exit_sim(sep_sim, ...) is only valid if that is 0.  h_counts[2] = -1 if
+ *                     the check was not asked for.  Synchronises `stream`.
+ *   siso_tier_lookup  Top-1 over both tiers, equal to siso_lookup(k = 1) on the cache the tiers were built from: the
+ *                     whole batch against the hot tier, the queries whose best hot similarity does not exceed exit_sim
+ *                     packed and scored against the cold tier, the better of the two per query (ties to the lower slot),
+ *                     strict threshold.  d_idx are slots of the original cache.  d_work: siso_tier_work_bytes() bytes of
+ *                     device memory, 256-byte aligned.  *h_settled (may be NULL) = queries that ended in the hot tier.
+ *                     Synchronises `stream` once in the middle (one 8-byte read sizes the cold sweep). */
+siso_status_t siso_tier_build(siso_cache_t *cache, int64_t hot_rows, double sep_sim, siso_cache_t *hot, siso_cache_t *cold,
+                              int32_t *d_hot_slot, int32_t *d_cold_slot, int64_t *h_counts, void *stream);
+int64_t siso_tier_work_bytes(int64_t n_queries, int32_t dim, int32_t dtype);
+siso_status_t siso_tier_lookup(siso_cache_t *hot, siso_cache_t *cold, const int32_t *d_hot_slot, const int32_t *d_cold_slot,
+                               const void *d_queries, int64_t n_queries, float exit_sim, const float *d_theta, float theta_scalar,
+                               void *d_work, int32_t *d_idx, float *d_sim, uint8_t *d_hit, int64_t *h_settled, void *stream);
+
 /* Algorithm 1 as a whole (Sec. 4.2): C_new <- MergeCentroids(C_cur, C_repo, theta_C); C_new <- FilteringCentroids(C_new, M);
  * UpdateCentroids(C_cur, C_new).  With a second handle as C_new the steps are
  *     siso_cache_copy(c_new, cur)                       "C_new <- C_cur", the first line of MergeCentroids

@@ -26,7 +26,7 @@ EXPORTS = ["siso_cache_create", "siso_cache_destroy", "siso_set_option", "siso_i
            "siso_choose_theta", "siso_correct_theta", "siso_tier_exit_sim", "siso_tier_select", "siso_tier_finish",
            "siso_route", "siso_evict_keys", "siso_select_evict", "siso_evict_slots", "siso_selftest_wait_timeout",
            "siso_measure_fp32_fma", "siso_pair_sweep_block", "siso_merge_resolve", "siso_merge_pack",
-           "siso_merge_apply_shard"]
+           "siso_merge_apply_shard", "siso_tier_build", "siso_tier_work_bytes", "siso_tier_lookup"]
 
 
 class SisoError(RuntimeError):
@@ -106,6 +106,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_merge_resolve.argtypes = [vp, vp, i64, vp, i64, vp, vp, vp]
     L.siso_merge_pack.argtypes = [vp, vp, i64, i64, vp, vp, vp, vp, vp]
     L.siso_merge_apply_shard.argtypes = [vp, vp, i64, vp, vp, vp, i64, u32, vp]
+    L.siso_tier_build.argtypes = [vp, i64, ctypes.c_double, vp, vp, vp, vp, ctypes.POINTER(i64), vp]
+    L.siso_tier_work_bytes.argtypes = [i64, i32, i32]
+    L.siso_tier_work_bytes.restype = i64
+    L.siso_tier_lookup.argtypes = [vp, vp, vp, vp, vp, i64, f32, vp, f32, vp, vp, vp, vp, ctypes.POINTER(i64), vp]
     L.siso_launch_count.argtypes = [vp]
     L.siso_launch_count.restype = i64
     L.siso_status_string.argtypes = [i32]
@@ -113,7 +117,8 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_last_cuda_error.argtypes = []
     L.siso_last_cuda_error.restype = ctypes.c_char_p
     for name in EXPORTS:
-        if name not in ("siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_md1_wait", "siso_tier_exit_sim"):
+        if name not in ("siso_launch_count", "siso_status_string", "siso_last_cuda_error", "siso_md1_wait", "siso_tier_exit_sim",
+                        "siso_tier_work_bytes"):
             getattr(L, name).restype = i32
     if path is None:
         _lib = L

@@ -136,6 +136,9 @@ siso_status_t launch_merge(Cache *c, const void *repo, const double *repo_sizes,
                            uint32_t flags, int32_t *merge_map, long long *d_n_merged, cudaStream_t s);
 siso_status_t launch_merge_resolve_global(Cache *c, const void *cand, int64_t n_cand, const uint8_t *valid, int64_t N,
                                           int32_t *merge_map, long long *d_n_merged, cudaStream_t s);
+siso_status_t launch_pair_sweep_block(Cache *c, int64_t own_offset, const void *d_peer_rows, const uint8_t *d_peer_valid, int64_t n_peer,
+                                      int64_t peer_offset, float theta_c, int32_t *d_cand, int64_t max_cand, int64_t *d_n_cand,
+                                      bool lookup_copies, cudaStream_t s);
 size_t merge_tensor_scratch_bytes(const Cache *c);
 size_t pair_sweep_tensor_scratch_bytes(int64_t n, int64_t rows, int dim);
 siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, int64_t N, int64_t rows, const uint8_t *valid,

@@ -80,6 +80,17 @@ __global__ void block_flags_kernel(const uint8_t *__restrict__ peer_valid, long 
     }
 }
 
+// bf16 rows -> fp32, eight elements per thread
+__global__ void widen_rows_kernel(const uint4 *__restrict__ src, float4 *__restrict__ dst, long long n8) {
+    const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n8) return;
+    const uint4 u = __ldg(src + i);
+    dst[2 * i] = make_float4(__uint_as_float(u.x << 16), __uint_as_float(u.x & 0xFFFF0000u), __uint_as_float(u.y << 16),
+                             __uint_as_float(u.y & 0xFFFF0000u));
+    dst[2 * i + 1] = make_float4(__uint_as_float(u.z << 16), __uint_as_float(u.z & 0xFFFF0000u), __uint_as_float(u.w << 16),
+                                 __uint_as_float(u.w & 0xFFFF0000u));
+}
+
 // flag[i] = 1 if local row i is live and merged away (merge_map names another slot)
 __global__ void pack_flags_kernel(const int32_t *__restrict__ merge_map, long long own_offset, long long n_own,
                                   const uint8_t *__restrict__ valid, uint32_t *__restrict__ flag) {
@@ -190,18 +201,21 @@ __global__ void shard_drop_kernel(const int32_t *__restrict__ merge_map, long lo
 
 using namespace siso;
 
-extern "C" siso_status_t siso_pair_sweep_block(siso_cache_t *h, int64_t own_offset, const float *d_peer_master,
-                                               const uint8_t *d_peer_valid, int64_t n_peer, int64_t peer_offset, float theta_c,
-                                               int32_t *d_cand, int64_t max_cand, int64_t *d_n_cand, void *stream) {
-    Cache *c = reinterpret_cast<Cache *>(h);
+// `lookup_copies`: compare the vectors that lookups read (for a bf16 cache its bf16 copies, widened; d_peer_rows is
+// then a bf16 array too) instead of the fp32 masters.  Used to certify the separation of the two tiers of the
+// locality-ordered search, whose exit rule is about the vectors that lookups see.
+siso_status_t siso::launch_pair_sweep_block(Cache *c, int64_t own_offset, const void *d_peer_rows, const uint8_t *d_peer_valid,
+                                            int64_t n_peer, int64_t peer_offset, float theta_c, int32_t *d_cand, int64_t max_cand,
+                                            int64_t *d_n_cand, bool lookup_copies, cudaStream_t s) {
     if (!c || own_offset < 0 || !d_cand || max_cand < 1 || !d_n_cand || !(theta_c == theta_c)) return SISO_ERR_INVALID_ARG;
-    if ((d_peer_master != nullptr) != (n_peer > 0) || (n_peer > 0 && (!d_peer_valid || peer_offset < 0))) return SISO_ERR_INVALID_ARG;
-    if (n_peer > 0 && (reinterpret_cast<uintptr_t>(d_peer_master) & 15u)) return SISO_ERR_INVALID_ARG;
+    if ((d_peer_rows != nullptr) != (n_peer > 0) || (n_peer > 0 && (!d_peer_valid || peer_offset < 0))) return SISO_ERR_INVALID_ARG;
+    if (n_peer > 0 && (reinterpret_cast<uintptr_t>(d_peer_rows) & 15u)) return SISO_ERR_INVALID_ARG;
+    const bool widen = lookup_copies && c->dtype == SISO_BF16;
+    if (widen && n_peer == 0) return SISO_ERR_UNSUPPORTED;
     const int64_t n_own = c->capacity;
     const int64_t peer_pad = (n_peer + 255) / 256 * 256;
     if (own_offset + n_own >= (1ll << 31) || peer_offset + n_peer >= (1ll << 31) || peer_pad + c->rows_alloc >= (1ll << 24)) return SISO_ERR_UNSUPPORTED;
     SISO_CUDA(cudaSetDevice(c->device));
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
     const size_t tmp_cand = static_cast<size_t>(c->merge_max_cand);
     const int64_t rows = peer_pad + c->rows_alloc, N = peer_pad + n_own;
     const size_t D = static_cast<size_t>(c->dim);
@@ -220,11 +234,20 @@ extern "C" siso_status_t siso_pair_sweep_block(siso_cache_t *h, int64_t own_offs
         // one array in this GPU's memory; the peer rows play the part of C_cur: they are compared with, never merged
         float *X = scr.take<float>(static_cast<size_t>(rows) * D);
         uint8_t *valid = scr.take<uint8_t>(static_cast<size_t>(N)), *seed = scr.take<uint8_t>(static_cast<size_t>(N));
-        SISO_CUDA(cudaMemcpyAsync(X, d_peer_master, static_cast<size_t>(n_peer) * D * sizeof(float), cudaMemcpyDeviceToDevice, s));
+        if (widen) {
+            const long long p8 = static_cast<long long>(n_peer) * D / 8, o8 = static_cast<long long>(c->rows_alloc) * D / 8;
+            widen_rows_kernel<<<static_cast<unsigned>((p8 + 255) / 256), 256, 0, s>>>(static_cast<const uint4 *>(d_peer_rows),
+                                                                                      reinterpret_cast<float4 *>(X), p8);
+            widen_rows_kernel<<<static_cast<unsigned>((o8 + 255) / 256), 256, 0, s>>>(static_cast<const uint4 *>(c->vecs),
+                                                                                      reinterpret_cast<float4 *>(X + static_cast<size_t>(peer_pad) * D), o8);
+            c->launches += 2;
+        } else {
+            SISO_CUDA(cudaMemcpyAsync(X, d_peer_rows, static_cast<size_t>(n_peer) * D * sizeof(float), cudaMemcpyDeviceToDevice, s));
+            SISO_CUDA(cudaMemcpyAsync(X + static_cast<size_t>(peer_pad) * D, c->master, static_cast<size_t>(c->rows_alloc) * D * sizeof(float),
+                                      cudaMemcpyDeviceToDevice, s));
+        }
         if (peer_pad > n_peer)
             SISO_CUDA(cudaMemsetAsync(X + static_cast<size_t>(n_peer) * D, 0, static_cast<size_t>(peer_pad - n_peer) * D * sizeof(float), s));
-        SISO_CUDA(cudaMemcpyAsync(X + static_cast<size_t>(peer_pad) * D, c->master, static_cast<size_t>(c->rows_alloc) * D * sizeof(float),
-                                  cudaMemcpyDeviceToDevice, s));
         block_flags_kernel<<<static_cast<unsigned>((N + 255) / 256), 256, 0, s>>>(d_peer_valid, n_peer, peer_pad, c->valid, n_own, valid, seed);
         SISO_LAUNCHED(c);
         SISO_TRY(launch_pair_sweep_tensor(c, &scr, X, N, rows, valid, seed, theta_c, ctl, cand, tmp_cand, nullptr, s, nullptr, peer_pad));
@@ -234,6 +257,13 @@ extern "C" siso_status_t siso_pair_sweep_block(siso_cache_t *h, int64_t own_offs
                                                            reinterpret_cast<unsigned long long *>(d_n_cand), c->status);
     SISO_LAUNCHED(c);
     return SISO_OK;
+}
+
+extern "C" siso_status_t siso_pair_sweep_block(siso_cache_t *h, int64_t own_offset, const float *d_peer_master,
+                                               const uint8_t *d_peer_valid, int64_t n_peer, int64_t peer_offset, float theta_c,
+                                               int32_t *d_cand, int64_t max_cand, int64_t *d_n_cand, void *stream) {
+    return launch_pair_sweep_block(reinterpret_cast<Cache *>(h), own_offset, d_peer_master, d_peer_valid, n_peer, peer_offset, theta_c,
+                                   d_cand, max_cand, d_n_cand, false, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" siso_status_t siso_merge_resolve(siso_cache_t *h, const int32_t *d_cand, int64_t n_cand, const uint8_t *d_valid,

@@ -109,6 +109,68 @@ tier_finish_settled_kernel(const unsigned long long *__restrict__ hot_keys, long
     hit[b] = s > (theta ? theta[b] : theta_s) ? 1 : 0;
 }
 
+// ---- building the tiers ------------------------------------------------------------------------------------------
+// cold[slot] = 1 for the slots named by the eviction keys (low 32 bits of a key's third word)
+__global__ void tier_mark_cold_kernel(const unsigned long long *__restrict__ keys, long long n, long long capacity,
+                                      uint32_t *__restrict__ cold) {
+    const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i >= n) return;
+    const unsigned long long w2 = keys[3 * i + 2];
+    if (keys[3 * i] == ~0ull && w2 == ~0ull) return;              // padding: fewer live entries than asked for
+    const long long slot = static_cast<long long>(w2 & 0xFFFFFFFFull);
+    if (slot < capacity) cold[slot] = 1u;
+}
+
+// hot[slot] = live and not cold; both arrays have capacity + 1 places (the last one 0) for the scans that follow
+__global__ void tier_flags_kernel(const uint8_t *__restrict__ valid, long long capacity, const uint32_t *__restrict__ cold,
+                                  uint32_t *__restrict__ hot) {
+    const long long i = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (i > capacity) return;
+    hot[i] = (i < capacity && valid[i] && !cold[i]) ? 1u : 0u;
+}
+
+// One CTA per slot of the source cache: the entry goes to place pos[slot] of its tier (ascending slot order), with its
+// vectors (lookup copy and fp32 master) and its metadata; `list` receives the source slot of every place.
+template <typename T>
+__global__ void __launch_bounds__(128)
+tier_copy_kernel(const uint32_t *__restrict__ flag_pos, const uint8_t *__restrict__ valid, const uint32_t *__restrict__ cold,
+                 int want_cold, int D, const T *__restrict__ src_vecs, const float *__restrict__ src_master,
+                 const double *__restrict__ src_size, const uint32_t *__restrict__ src_access,
+                 const unsigned long long *__restrict__ src_last, T *__restrict__ dst_vecs, float *__restrict__ dst_master,
+                 double *__restrict__ dst_size, uint32_t *__restrict__ dst_access, unsigned long long *__restrict__ dst_last,
+                 uint8_t *__restrict__ dst_valid, int32_t *__restrict__ list) {
+    const long long slot = blockIdx.x;
+    const bool is_cold = cold[slot] != 0u;
+    if (!valid[slot] || is_cold != (want_cold != 0)) return;
+    const long long at = flag_pos[slot];
+    const float4 *sm = reinterpret_cast<const float4 *>(src_master + slot * D);
+    float4 *dm = reinterpret_cast<float4 *>(dst_master + at * D);
+    for (int q = threadIdx.x; q < D / 4; q += blockDim.x) dm[q] = sm[q];
+    if constexpr (sizeof(T) == 2) {
+        const uint4 *sv = reinterpret_cast<const uint4 *>(src_vecs + slot * D);
+        uint4 *dv = reinterpret_cast<uint4 *>(dst_vecs + at * D);
+        for (int q = threadIdx.x; q < D / 8; q += blockDim.x) dv[q] = sv[q];
+    }
+    if (threadIdx.x == 0) {
+        dst_size[at] = src_size[slot];
+        dst_access[at] = src_access[slot];
+        dst_last[at] = src_last[slot];
+        dst_valid[at] = 1;
+        list[at] = static_cast<int32_t>(slot);
+    }
+}
+
+__global__ void tier_counters_kernel(const uint32_t *__restrict__ hot_pos, const uint32_t *__restrict__ cold_pos, long long capacity,
+                                     const long long *__restrict__ src_counters, long long *hot_counters, long long *cold_counters,
+                                     long long *out2) {
+    const long long n_hot = hot_pos[capacity], n_cold = cold_pos[capacity];
+    hot_counters[CNT_OCCUPANCY] = n_hot;
+    cold_counters[CNT_OCCUPANCY] = n_cold;
+    hot_counters[CNT_CLOCK] = cold_counters[CNT_CLOCK] = src_counters[CNT_CLOCK];
+    out2[0] = n_hot;
+    out2[1] = n_cold;
+}
+
 }  // namespace
 
 }  // namespace siso
@@ -116,6 +178,135 @@ tier_finish_settled_kernel(const unsigned long long *__restrict__ hot_keys, long
 using namespace siso;
 
 extern "C" {
+
+siso_status_t siso_tier_build(siso_cache_t *cache_h, int64_t hot_rows, double sep_sim, siso_cache_t *hot_h, siso_cache_t *cold_h,
+                              int32_t *d_hot_slot, int32_t *d_cold_slot, int64_t *h_counts, void *stream) {
+    Cache *c = reinterpret_cast<Cache *>(cache_h), *hot = reinterpret_cast<Cache *>(hot_h), *cold = reinterpret_cast<Cache *>(cold_h);
+    if (!c || !hot || !cold || hot == cold || hot == c || cold == c || hot_rows < 0 || !d_hot_slot || !d_cold_slot || !h_counts)
+        return SISO_ERR_INVALID_ARG;
+    if (hot->dim != c->dim || cold->dim != c->dim || hot->dtype != c->dtype || cold->dtype != c->dtype ||
+        hot->device != c->device || cold->device != c->device)
+        return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    long long occ = 0;
+    SISO_CUDA(cudaMemcpyAsync(&occ, c->counters + CNT_OCCUPANCY, sizeof(occ), cudaMemcpyDeviceToHost, s));
+    SISO_CUDA(cudaStreamSynchronize(s));
+    const int64_t n_hot = std::min<int64_t>(hot_rows, occ), n_cold = occ - n_hot;
+    if (n_hot > hot->capacity || n_cold > cold->capacity) return SISO_ERR_CAPACITY;
+    const int64_t cap = c->capacity;
+    // the lists and flags live in the HOT tier's scratch (the source cache's own scratch serves its eviction-order selection)
+    Scratch scr;
+    SISO_TRY(scratch_reserve(hot, 2 * pad256(sizeof(uint32_t) * (cap + 1)) + pad256(sizeof(unsigned long long) * 3 * std::max<int64_t>(n_cold, 1)) +
+                                      pad256(2 * sizeof(long long)) + 256, s, &scr));
+    uint32_t *cold_pos = scr.take<uint32_t>(cap + 1), *hot_pos = scr.take<uint32_t>(cap + 1);
+    unsigned long long *keys = scr.take<unsigned long long>(3 * std::max<int64_t>(n_cold, 1));
+    long long *d_out2 = scr.take<long long>(2);
+    SISO_CUDA(cudaMemsetAsync(cold_pos, 0, sizeof(uint32_t) * (cap + 1), s));
+    if (n_cold > 0) {
+        // the cold tier = what FilteringCentroids would remove to leave n_hot entries (nothing is removed here)
+        SISO_TRY(launch_evict_keys(c, n_cold, 0, keys, s));
+        tier_mark_cold_kernel<<<static_cast<unsigned>((n_cold + 255) / 256), 256, 0, s>>>(keys, n_cold, cap, cold_pos);
+        SISO_LAUNCHED(c);
+    }
+    const unsigned nblk = static_cast<unsigned>((cap + 1 + 255) / 256);
+    tier_flags_kernel<<<nblk, 256, 0, s>>>(c->valid, cap, cold_pos, hot_pos);
+    SISO_LAUNCHED(c);
+    // cold flags are still needed as flags by the copy: scan a copy of them
+    uint32_t *cold_flag = cold_pos;
+    Scratch scr2;
+    SISO_TRY(scratch_reserve(cold, pad256(sizeof(uint32_t) * (cap + 1)) + 256, s, &scr2));
+    uint32_t *cold_scan = scr2.take<uint32_t>(cap + 1);
+    SISO_CUDA(cudaMemcpyAsync(cold_scan, cold_flag, sizeof(uint32_t) * (cap + 1), cudaMemcpyDeviceToDevice, s));
+    SISO_TRY(launch_exclusive_scan_u32(c, cold_scan, cap + 1, s));
+    SISO_TRY(launch_exclusive_scan_u32(c, hot_pos, cap + 1, s));
+    for (Cache *t : {hot, cold}) {
+        SISO_CUDA(cudaMemsetAsync(t->valid, 0, static_cast<size_t>(t->rows_alloc), s));
+        SISO_CUDA(cudaMemsetAsync(t->counters, 0, sizeof(long long) * CNT_N, s));
+        t->vec_epoch += 1;
+        t->low_dirty = true;
+    }
+    for (int want_cold = 0; want_cold < 2; ++want_cold) {
+        Cache *t = want_cold ? cold : hot;
+        const uint32_t *pos = want_cold ? cold_scan : hot_pos;
+        int32_t *list = want_cold ? d_cold_slot : d_hot_slot;
+        if (c->dtype == SISO_F32)
+            tier_copy_kernel<float><<<static_cast<unsigned>(cap), 128, 0, s>>>(
+                pos, c->valid, cold_flag, want_cold, c->dim, static_cast<const float *>(c->vecs), c->master, c->size, c->access, c->last,
+                static_cast<float *>(t->vecs), t->master, t->size, t->access, t->last, t->valid, list);
+        else
+            tier_copy_kernel<__nv_bfloat16><<<static_cast<unsigned>(cap), 128, 0, s>>>(
+                pos, c->valid, cold_flag, want_cold, c->dim, static_cast<const __nv_bfloat16 *>(c->vecs), c->master, c->size, c->access,
+                c->last, static_cast<__nv_bfloat16 *>(t->vecs), t->master, t->size, t->access, t->last, t->valid, list);
+        SISO_LAUNCHED(c);
+    }
+    tier_counters_kernel<<<1, 1, 0, s>>>(hot_pos, cold_scan, cap, c->counters, hot->counters, cold->counters, d_out2);
+    SISO_LAUNCHED(c);
+    long long out2[2] = {0, 0};
+    SISO_CUDA(cudaMemcpyAsync(out2, d_out2, sizeof(out2), cudaMemcpyDeviceToHost, s));
+    SISO_CUDA(cudaStreamSynchronize(s));
+    h_counts[0] = out2[0];
+    h_counts[1] = out2[1];
+    h_counts[2] = -1;
+    // the exit rule rests on every hot/cold pair being at most sep_sim similar: count the pairs above it (exact fp64
+    // similarities of the vectors that lookups read) with the block sweep of the sharded MergeCentroids, hot tier as the peer block
+    if (sep_sim == sep_sim && out2[0] > 0 && out2[1] > 0) {
+        Scratch scr3;
+        SISO_TRY(scratch_reserve(hot, pad256(12 * 64) + pad256(sizeof(long long)) + 256, s, &scr3));
+        int32_t *cand = scr3.take<int32_t>(3 * 64);
+        long long *n_cand = scr3.take<long long>(1);
+        SISO_CUDA(cudaMemsetAsync(n_cand, 0, sizeof(long long), s));
+        SISO_TRY(launch_pair_sweep_block(cold, 0, hot->vecs, hot->valid, out2[0], cold->capacity, static_cast<float>(sep_sim), cand, 64,
+                                         reinterpret_cast<int64_t *>(n_cand), true, s));
+        long long above = 0;
+        SISO_CUDA(cudaMemcpyAsync(&above, n_cand, sizeof(above), cudaMemcpyDeviceToHost, s));
+        SISO_CUDA(cudaStreamSynchronize(s));
+        // more than 64 such pairs leave SISO_ERR_OVERFLOW in the cold tier's status word: the count is what matters here
+        int discard = 0;
+        SISO_CUDA(cudaMemcpyAsync(&discard, cold->status, sizeof(int), cudaMemcpyDeviceToHost, s));
+        SISO_CUDA(cudaMemsetAsync(cold->status, 0, sizeof(int), s));
+        SISO_CUDA(cudaStreamSynchronize(s));
+        if (discard != 0 && discard != SISO_ERR_OVERFLOW) return static_cast<siso_status_t>(discard);
+        h_counts[2] = discard == SISO_ERR_OVERFLOW ? std::max<long long>(above, 65) : above;
+    }
+    return SISO_OK;
+}
+
+int64_t siso_tier_work_bytes(int64_t n_queries, int32_t dim, int32_t dtype) {
+    if (n_queries < 0 || dim < 1) return 0;
+    const size_t row = static_cast<size_t>(dim) * (dtype == SISO_F32 ? 4 : 2);
+    return static_cast<int64_t>(2 * pad256(sizeof(uint64_t) * n_queries) + pad256(sizeof(int32_t) * n_queries) +
+                                pad256(row * n_queries) + 256);
+}
+
+siso_status_t siso_tier_lookup(siso_cache_t *hot, siso_cache_t *cold, const int32_t *d_hot_slot, const int32_t *d_cold_slot,
+                               const void *d_queries, int64_t n_queries, float exit_sim, const float *d_theta, float theta_scalar,
+                               void *d_work, int32_t *d_idx, float *d_sim, uint8_t *d_hit, int64_t *h_settled, void *stream) {
+    if (!hot || !cold || n_queries < 0) return SISO_ERR_INVALID_ARG;
+    if (n_queries == 0) { if (h_settled) *h_settled = 0; return SISO_OK; }
+    if (!d_queries || !d_work || !d_idx || !d_sim || !d_hit || (reinterpret_cast<uintptr_t>(d_work) & 255u)) return SISO_ERR_INVALID_ARG;
+    Cache *h = reinterpret_cast<Cache *>(hot), *c = reinterpret_cast<Cache *>(cold);
+    if (h->dim != c->dim || h->dtype != c->dtype || h->device != c->device) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(h->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t row = static_cast<size_t>(h->dim) * (h->dtype == SISO_F32 ? 4 : 2);
+    char *p = static_cast<char *>(d_work);
+    uint64_t *hk = reinterpret_cast<uint64_t *>(p); p += pad256(sizeof(uint64_t) * n_queries);
+    uint64_t *ck = reinterpret_cast<uint64_t *>(p); p += pad256(sizeof(uint64_t) * n_queries);
+    int32_t *rows = reinterpret_cast<int32_t *>(p); p += pad256(sizeof(int32_t) * n_queries);
+    void *packed = p; p += pad256(row * n_queries);
+    int64_t *count = reinterpret_cast<int64_t *>(p);
+    // the whole batch against the hot tier; the queries that may still find something better go on, packed
+    SISO_TRY(siso_lookup_keys(hot, d_queries, n_queries, 1, 0, hk, stream));
+    SISO_TRY(siso_tier_select(hk, n_queries, exit_sim, d_queries, static_cast<int64_t>(row), packed, rows, count, stream));
+    long long n_go = 0;                              // one 8-byte read sizes the cold tier's sweep
+    SISO_CUDA(cudaMemcpyAsync(&n_go, count, sizeof(n_go), cudaMemcpyDeviceToHost, s));
+    SISO_CUDA(cudaStreamSynchronize(s));
+    if (n_go > 0) SISO_TRY(siso_lookup_keys(cold, packed, n_go, 1, 0, ck, stream));
+    if (h_settled) *h_settled = n_queries - n_go;
+    return siso_tier_finish(hk, n_queries, exit_sim, ck, rows, n_go, d_hot_slot, d_cold_slot, d_theta, theta_scalar, d_idx, d_sim,
+                            d_hit, stream);
+}
 
 double siso_tier_exit_sim(double sep_sim, double norm_slack) {
     // Vectors (queries and entries) have norms in [1 - d, 1 + d]; every hot/cold pair has dot product <= sep.

@@ -7,62 +7,70 @@ best hot similarity exceeds the exit similarity stop there (no cold entry can be
 the remaining queries into a dense batch and scores only those against the cold tier.  The answer is the top-1 over the
 whole cache, with the slots of the cache the tiers were built from.
 
-The tiers are a snapshot: build them after maintenance (MergeCentroids at theta_C makes every pair of entries at most
-theta_C similar, which is the separation bound the exit needs) and rebuild after the next one.
+The tiers are a snapshot: build them after maintenance and rebuild after the next one.  Both the split and the lookup's
+control flow are entry points of the library (siso_tier_build, siso_tier_lookup); this class only marshals.
 """
 from __future__ import annotations
 
+import ctypes
+import math
 from typing import Optional
 
 import torch
 
-from .binding import SisoCache, tier_exit_sim, tier_finish, tier_select
+from .binding import SisoCache, SisoError, _ptr, _stream, tier_exit_sim
 
 
 class TieredCache:
-    def __init__(self, cache: SisoCache, hot_rows: int, sep_sim: float, norm_slack: float = 0.0):
+    def __init__(self, cache: SisoCache, hot_rows: int, sep_sim: float, norm_slack: float = 0.0, certify: bool = True):
         """cache: the cache to split (left untouched).  hot_rows: size of the hot tier.  sep_sim: an upper bound on the
-        similarity of any hot entry to any cold entry (e.g. theta_C right after a merge).  norm_slack: how far the norms
-        of entries and queries may be from 1 (bf16 rounding of unit vectors: about 1e-3)."""
+        similarity of any hot entry to any cold entry; norm_slack: how far the norms of entries and queries may be from 1
+        (bf16 rounding of unit vectors: about 1e-3).  The exit rule is only exact if the bound holds, and nothing in the
+        cache's history guarantees it for good (a weighted merge recentres survivors, a two-set merge never compares
+        the old entries with each other, later inserts and updates move vectors), so by default the build CHECKS it:
+        every hot/cold pair is swept (tensor cores + exact fp64 check) and a pair above sep_sim raises ValueError.
+        certify=False skips the check for a caller that has just established the bound some other way."""
         occ = int(cache.stats()["occupancy"])
         hot_rows = max(0, min(int(hot_rows), occ))
-        dev = cache._dev
-        # the cold tier = what FilteringCentroids would evict to leave hot_rows entries: run it on a copy
-        tmp = SisoCache(cache.capacity, cache.dim, cache.dtype, device=dev.index)
-        tmp.copy_from(cache)
-        victims = tmp.evict(occ - hot_rows) if occ > hot_rows else torch.empty((0,), dtype=torch.int32, device=dev)
-        st = cache.export()
-        torch.cuda.synchronize(dev)
-        tmp.close()
-        cold_slots = torch.sort(victims.to(torch.int64)).values
-        keep = st["valid"].to(torch.bool).clone()
-        keep[cold_slots] = False
-        hot_slots = torch.nonzero(keep).reshape(-1)
-        clock = int(cache.stats()["clock"])
-        self.hot, self.hot_slot = self._tier(cache, st, hot_slots, clock)
-        self.cold, self.cold_slot = self._tier(cache, st, cold_slots, clock)
-        self.n_hot, self.n_cold = int(hot_slots.numel()), int(cold_slots.numel())
+        dev = cache._dev.index
+        self.hot = SisoCache(max(1, hot_rows), cache.dim, cache.dtype, device=dev)
+        self.cold = SisoCache(max(1, occ - hot_rows), cache.dim, cache.dtype, device=dev)
+        self.hot_slot = torch.full((self.hot.capacity,), -1, dtype=torch.int32, device=cache._dev)
+        self.cold_slot = torch.full((self.cold.capacity,), -1, dtype=torch.int32, device=cache._dev)
+        counts = (ctypes.c_int64 * 3)()
+        st = cache._lib.siso_tier_build(cache._h, hot_rows, float(sep_sim) if certify else math.nan, self.hot._h, self.cold._h,
+                                        _ptr(self.hot_slot), _ptr(self.cold_slot), counts, _stream(None))
+        if st != 0:
+            raise SisoError(st, "siso_tier_build")
+        self.n_hot, self.n_cold, self.pairs_above_sep = int(counts[0]), int(counts[1]), int(counts[2])
+        if self.pairs_above_sep > 0:
+            self.close()
+            raise ValueError(f"{self.pairs_above_sep} hot/cold pairs are more similar than sep_sim = {sep_sim}: "
+                             "the early exit would not be exact")
         self.exit_sim = tier_exit_sim(sep_sim, norm_slack)
         self.settled = 0            # queries of the last lookup that ended in the hot tier
-
-    @staticmethod
-    def _tier(cache: SisoCache, st: dict, slots: torch.Tensor, clock: int):
-        n = int(slots.numel())
-        t = SisoCache(max(1, n), cache.dim, cache.dtype, device=cache._dev.index)
-        if n:
-            t.import_(st["master"][slots], st["size"][slots], st["access"][slots], st["last"][slots],
-                      torch.ones(n, dtype=torch.uint8, device=slots.device), clock)
-        return t, slots.to(torch.int32).contiguous()
+        self._work = None
 
     def lookup(self, queries: torch.Tensor, theta, stream=None):
         """-> (idx [n] int32 slots of the original cache, sim [n], hit [n]); equal to cache.lookup(queries, theta, 1)."""
         q = self.hot._vec(queries, "queries")
-        hk = self.hot.lookup_keys(q, 1, stream=stream)
-        rows, packed, count = tier_select(hk, q, self.exit_sim, stream=stream)
-        n_go = int(count.item())                             # one 8-byte read: sizes the cold lookup
-        self.settled = q.shape[0] - n_go
-        ck = self.cold.lookup_keys(packed[:n_go], 1, stream=stream) if n_go else None
-        return tier_finish(hk, self.exit_sim, ck, rows, n_go, self.hot_slot, self.cold_slot, theta, stream=stream)
+        n = q.shape[0]
+        lib, dev = self.hot._lib, q.device
+        need = int(lib.siso_tier_work_bytes(n, self.hot.dim, 0 if self.hot.dtype == "f32" else 1))
+        if self._work is None or self._work.numel() < need:
+            self._work = torch.empty(need, dtype=torch.uint8, device=dev)
+        th_t, th_s = (theta.to(device=dev, dtype=torch.float32).contiguous(), 0.0) if isinstance(theta, torch.Tensor) else (None, float(theta))
+        idx = torch.empty((n,), dtype=torch.int32, device=dev)
+        sim = torch.empty((n,), dtype=torch.float32, device=dev)
+        hit = torch.empty((n,), dtype=torch.uint8, device=dev)
+        settled = ctypes.c_int64(0)
+        st = lib.siso_tier_lookup(self.hot._h, self.cold._h, _ptr(self.hot_slot), _ptr(self.cold_slot), _ptr(q), n, float(self.exit_sim),
+                                  _ptr(th_t), th_s, _ptr(self._work), _ptr(idx), _ptr(sim), _ptr(hit), ctypes.byref(settled),
+                                  _stream(stream))
+        if st != 0:
+            raise SisoError(st, "siso_tier_lookup")
+        self.settled = int(settled.value)
+        return idx, sim, hit
 
     def close(self) -> None:
         self.hot.close()
