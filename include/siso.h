@@ -68,6 +68,12 @@ typedef enum { SISO_F32 = 0, SISO_BF16 = 1 } siso_dtype_t;
                                          * sweep kernel; 1: always by a separate finalisation launch */
 #define SISO_OPT_STREAM_LIST 7          /* 0 (default): on a full cache the fused streaming step takes its victims from an
                                          * eviction-order list kept across batches (no grid-wide barrier); 1: never */
+#define SISO_OPT_CHECKED 9              /* 1: checked mode.  What the library otherwise takes on trust is verified on the device before
+                                         * the call's own kernels run: query, insert and repository rows must be unit vectors
+                                         * (| |x| - 1 | < 1e-2) with finite elements, thresholds must be numbers, hit flags 0 or 1,
+                                         * slots of hits inside the cache.  A violation sets SISO_ERR_INVALID_ARG in the status
+                                         * word (read it with siso_sync_status); nothing traps and the call still runs.  0
+                                         * (default) unless the library was built with -DSISO_CHECKED. */
 #define SISO_OPT_TENSOR_CTA_PAIR 3      /* 0 (default): tensor-core lookup runs CTA pairs for >= 2 query tiles; 1: never */
 #define SISO_PATH_AUTO 0
 #define SISO_PATH_SIMT 1   /* CUDA-core tiled sweep (fp32 accumulate of exact products)        */

@@ -109,6 +109,59 @@ __global__ void normalise_valid_kernel(uint8_t *valid, long long n) {
 
 static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// ---- checked mode (SISO_OPT_CHECKED): what the library otherwise takes on trust is verified on the device ----------
+// One warp per row: the row must be a unit vector (| |x| - 1 | < 1e-2; bf16 rounding of a unit vector stays within
+// 2e-3) with finite elements.  A row that is not sets SISO_ERR_INVALID_ARG in the status word; nothing traps.
+template <typename T>
+__global__ void __launch_bounds__(256)
+check_unit_rows_kernel(const T *__restrict__ rows, long long n, int D, const uint8_t *__restrict__ skip_if_set, int *status) {
+    const int lane = threadIdx.x & 31;
+    const long long warps = static_cast<long long>(gridDim.x) * (blockDim.x >> 5);
+    for (long long r = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); r < n; r += warps) {
+        if (skip_if_set && skip_if_set[r]) continue;           // rows the call will not store (hits of siso_insert_misses)
+        double ss = 0.0;
+        for (int d = lane; d < D; d += 32) {
+            float v;
+            if constexpr (sizeof(T) == 2) v = __bfloat162float(rows[r * D + d]); else v = rows[r * D + d];
+            ss += static_cast<double>(v) * static_cast<double>(v);
+        }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+        if (lane == 0 && !(fabs(sqrt(ss) - 1.0) < 1e-2)) set_status(status, SISO_ERR_INVALID_ARG);      // NaN fails too
+    }
+}
+
+// thresholds must be numbers; hit flags 0 or 1; slots of hits inside the cache
+__global__ void check_batch_args_kernel(const float *__restrict__ theta, const uint8_t *__restrict__ hit, const int32_t *__restrict__ idx,
+                                        int idx_stride, long long n, long long capacity, int *status) {
+    const long long b = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
+    if (b >= n) return;
+    bool ok = true;
+    if (theta && !(theta[b] == theta[b])) ok = false;
+    if (hit && hit[b] > 1) ok = false;
+    if (hit && idx && hit[b] == 1 && (idx[b * idx_stride] < 0 || idx[b * idx_stride] >= capacity)) ok = false;
+    if (!ok) set_status(status, SISO_ERR_INVALID_ARG);
+}
+
+static siso_status_t checked_rows(Cache *c, const void *rows, int64_t n, const uint8_t *skip_if_set, cudaStream_t s) {
+    if (!c->checked || n <= 0) return SISO_OK;
+    const unsigned blocks = static_cast<unsigned>(std::min<int64_t>((n + 7) / 8, 8ll * c->sm_count));
+    if (c->dtype == SISO_F32)
+        check_unit_rows_kernel<float><<<blocks, 256, 0, s>>>(static_cast<const float *>(rows), n, c->dim, skip_if_set, c->status);
+    else
+        check_unit_rows_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(rows), n, c->dim, skip_if_set, c->status);
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
+
+static siso_status_t checked_batch(Cache *c, const float *theta, const uint8_t *hit, const int32_t *idx, int idx_stride, int64_t n,
+                                   cudaStream_t s) {
+    if (!c->checked || n <= 0 || (!theta && !hit)) return SISO_OK;
+    check_batch_args_kernel<<<static_cast<unsigned>((n + 255) / 256), 256, 0, s>>>(theta, hit, idx, idx_stride, n, c->capacity, c->status);
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
+
 }  // namespace siso
 
 using namespace siso;
@@ -168,6 +221,9 @@ siso_status_t siso_cache_create(siso_cache_t **out, const siso_config_t *cfg) {
     c->lookup_path = SISO_PATH_AUTO;
     c->stream_fused = 1;
     c->low_dirty = true;
+#ifdef SISO_CHECKED
+    c->checked = 1;            // a library built with -DSISO_CHECKED checks by default
+#endif
     c->merge_max_cand = 16 * c->capacity + (1ll << 20);
 
     const size_t rows = static_cast<size_t>(c->rows_alloc), D = static_cast<size_t>(c->dim);
@@ -231,6 +287,10 @@ siso_status_t siso_set_option(siso_cache_t *c, int32_t key, int64_t value) {
             if (value != 0 && value != 1) return SISO_ERR_INVALID_ARG;
             c->sweep_finalize_separate = static_cast<int32_t>(value);
             return SISO_OK;
+        case SISO_OPT_CHECKED:
+            if (value != 0 && value != 1) return SISO_ERR_INVALID_ARG;
+            c->checked = static_cast<int32_t>(value);
+            return SISO_OK;
         case SISO_OPT_STREAM_LIST:
             if (value != 0 && value != 1) return SISO_ERR_INVALID_ARG;
             c->stream_list_off = static_cast<int32_t>(value);
@@ -254,6 +314,7 @@ siso_status_t siso_insert(siso_cache_t *c, const void *d_vecs, const double *d_s
     if (n > 0 && !aligned16(d_vecs)) return SISO_ERR_INVALID_ARG;
     SISO_CUDA(cudaSetDevice(c->device));
     c->low_dirty = true;        // entries or their metadata change outside the streaming maintenance kernel
+    SISO_TRY(checked_rows(c, d_vecs, n, nullptr, static_cast<cudaStream_t>(stream)));
     return launch_insert(c, d_vecs, d_sizes, nullptr, n, d_slots_out, static_cast<cudaStream_t>(stream));
 }
 
@@ -278,6 +339,8 @@ siso_status_t siso_lookup(siso_cache_t *c, const void *d_queries, int64_t n_quer
     if (!d_queries || !d_idx || !d_sim || !d_hit || !aligned16(d_queries)) return SISO_ERR_INVALID_ARG;
     SISO_CUDA(cudaSetDevice(c->device));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    SISO_TRY(checked_rows(c, d_queries, n_queries, nullptr, s));
+    SISO_TRY(checked_batch(c, d_theta, nullptr, nullptr, 1, n_queries, s));
     switch (resolve_lookup_path(c, n_queries)) {
         case SISO_PATH_STREAM: return launch_lookup_stream(c, d_queries, n_queries, d_theta, theta_scalar, k, d_idx, d_sim, d_hit, s);
         case SISO_PATH_TENSOR:
@@ -325,6 +388,8 @@ siso_status_t siso_update(siso_cache_t *c, const void *d_queries, int64_t n_quer
     if (n_queries > 0 && (!d_queries || !d_idx || !d_hit || !aligned16(d_queries))) return SISO_ERR_INVALID_ARG;
     SISO_CUDA(cudaSetDevice(c->device));
     c->low_dirty = true;        // entries or their metadata change outside the streaming maintenance kernel
+    SISO_TRY(checked_rows(c, d_queries, n_queries, nullptr, static_cast<cudaStream_t>(stream)));
+    SISO_TRY(checked_batch(c, nullptr, d_hit, d_idx, idx_stride, n_queries, static_cast<cudaStream_t>(stream)));
     return launch_update(c, d_queries, n_queries, d_idx, idx_stride, d_hit, static_cast<cudaStream_t>(stream));
 }
 
@@ -337,6 +402,7 @@ siso_status_t siso_merge(siso_cache_t *c, const void *d_repo, const double *d_re
     SISO_CUDA(cudaSetDevice(c->device));
     c->low_dirty = true;        // entries or their metadata change outside the streaming maintenance kernel
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    SISO_TRY(checked_rows(c, d_repo, n_repo, nullptr, s));
     long long *d_n = nullptr;
     if (h_n_merged) d_n = c->counters + CNT_SPARE;
     SISO_TRY(launch_merge(c, d_repo, d_repo_sizes, n_repo, theta_c, flags, d_merge_map, d_n, s));
@@ -479,6 +545,8 @@ siso_status_t siso_insert_misses(siso_cache_t *c, const void *d_queries, int64_t
     if (!c || n < 0 || (n > 0 && (!d_queries || !d_hit || !aligned16(d_queries)))) return SISO_ERR_INVALID_ARG;
     SISO_CUDA(cudaSetDevice(c->device));
     c->low_dirty = true;        // entries or their metadata change outside the streaming maintenance kernel
+    SISO_TRY(checked_rows(c, d_queries, n, d_hit, static_cast<cudaStream_t>(stream)));
+    SISO_TRY(checked_batch(c, nullptr, d_hit, nullptr, 1, n, static_cast<cudaStream_t>(stream)));
     return launch_insert(c, d_queries, nullptr, d_hit, n, d_slots_out, static_cast<cudaStream_t>(stream));
 }
 
@@ -490,6 +558,10 @@ siso_status_t siso_stream_step(siso_cache_t *c, const void *d_queries, int64_t n
     if (!d_queries || !d_idx || !d_sim || !d_hit || !aligned16(d_queries)) return SISO_ERR_INVALID_ARG;
     SISO_CUDA(cudaSetDevice(c->device));
     cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (c->checked && c->stream_fused && c->dtype == SISO_BF16) {      // (the other branches go through siso_lookup, which checks)
+        SISO_TRY(checked_rows(c, d_queries, n, nullptr, s));
+        SISO_TRY(checked_batch(c, d_theta, nullptr, nullptr, 1, n, s));
+    }
     // small batches: update, make-room and insertion in one cooperative launch, which also finishes the lookup
     // (best key over the splits, threshold test) when the tensor-core kernel produced it
     if (c->stream_fused && stream_maint_supported(c, n)) {

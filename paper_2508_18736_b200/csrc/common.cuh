@@ -66,6 +66,7 @@ struct Cache {
     void *swap_plan;            // UpdateCentroids: slot of the d-th live entry, when this cache serves as C_new
     int maint_grid;             // CTAs of the fused streaming maintenance kernel (0: not yet asked, -1: unavailable)
     int32_t sweep_finalize_separate;   // 1: never finish a top-1 lookup inside the sweep kernel
+    int32_t checked;                   // 1: inputs are verified on the device (SISO_OPT_CHECKED)
     int32_t stream_list_off;           // 1: the streaming maintenance kernel never uses the list below
     void *low_list;             // eviction-order list that the streaming maintenance kernel keeps across batches
     bool low_dirty;             // an entry point other than that kernel has changed entries or their metadata since
