@@ -38,9 +38,11 @@
  * Pins: tests/test_oracle_*.py check every routine against closed forms, the
  * hand-computed four-centroid example under tests/golden/, brute force written
  * independently in numpy, and invariants.  The streaming composition (lookup,
- * update, evict, insert per micro-batch) has no value in the paper to compare
- * with and is pinned by conservation invariants only: "parity unpinned" for the
- * stream as a whole.
+ * update, evict what the misses lack, insert per micro-batch) is pinned by a second
+ * hand-computed example (two batches on a cache of four slots, every output and the
+ * whole state after each batch) that five planted mistakes in the composition each
+ * fail.  What no pin can fix are the hit ratios of a synthetic stream: the paper
+ * prints none for such data ("parity unpinned" for those numbers only).
  */
 #include <math.h>
 #include <stdint.h>
