@@ -260,8 +260,27 @@ __device__ __forceinline__ float4 widen4(uint2 u) {
                        __uint_as_float(u.y & 0xFFFF0000u));
 }
 
+// rows of a chunk in flight at a time (after the first four): 12-16 KiB per warp
+template <typename T> __host__ __device__ constexpr int upw_stage_rows() { return sizeof(T) == 2 ? 8 : 4; }
+
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+// BYTES (a multiple of 16) from global to shared memory by one warp, 16 bytes per lane and step
+template <int BYTES>
+__device__ __forceinline__ void warp_copy_async(void *dst_smem, const void *src, int lane) {
+    const uint32_t d = static_cast<uint32_t>(__cvta_generic_to_shared(dst_smem));
+    const char *g = static_cast<const char *>(src);
+#pragma unroll
+    for (int o = 0; o < BYTES; o += 512) {
+        const int at = o + lane * 16;
+        if (at < BYTES) asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(d + at), "l"(g + at) : "memory");
+    }
+}
+// shared memory of one warp: the master row as fp32, then the query rows of one stage
+template <typename T> __host__ __device__ constexpr size_t upw_warp_smem(int D) { return sizeof(float) * D + upw_stage_rows<T>() * sizeof(T) * D; }
+
 template <typename T, int NQ>
-__global__ void __launch_bounds__(UPW_THREADS, 4)
+__global__ void __launch_bounds__(UPW_THREADS, 3)
 update_apply_warp_kernel(const int4 *__restrict__ desc, unsigned int list_len, const unsigned int *__restrict__ n_desc,
                          unsigned int *__restrict__ ticket,
                          const uint32_t *__restrict__ rows,
@@ -271,7 +290,11 @@ update_apply_warp_kernel(const int4 *__restrict__ desc, unsigned int list_len, c
                          unsigned int *__restrict__ arrived, unsigned int *__restrict__ arrived_runs) {
     using raw_t = typename Raw4<T>::type;
     constexpr int D = 128 * NQ;
+    constexpr int ROW_M_BYTES = D * 4, ROW_Q_BYTES = D * static_cast<int>(sizeof(T)), UPW_STAGE_ROWS = upw_stage_rows<T>();
+    extern __shared__ __align__(16) unsigned char upw_smem[];
     const int lane = threadIdx.x & 31;
+    float *m_s = reinterpret_cast<float *>(upw_smem + (threadIdx.x >> 5) * upw_warp_smem<T>(D));
+    T *q_s = reinterpret_cast<T *>(m_s + D);
     const unsigned int n_front = n_desc[0], n = n_front + n_desc[1];
     auto place = [&](unsigned int t) { return t < n_front ? t : list_len - 1u - (t - n_front); };      // ticket -> list entry
     // chunks are handed out by a ticket counter (a long chunk delays nobody else); a warp draws its next ticket and
@@ -293,43 +316,60 @@ update_apply_warp_kernel(const int4 *__restrict__ desc, unsigned int list_len, c
         const bool is_head = p == head;
         const bool more = gend > p + chunk;
         const int64_t e = more ? p + chunk : gend;
+        float *m = master + static_cast<int64_t>(slot) * D;
+        // Everything the chunk reads travels to this warp's shared-memory buffer with asynchronous 16-byte copies, so
+        // that all of a stage's bytes are in flight at once whatever the registers allow: first the master row (head
+        // chunks) and the chunk's first four rows, whose numbers come with the description, then the remaining rows
+        // UPW_STAGE_ROWS at a time (their numbers: one coalesced load of the whole chunk's list).  The additions run
+        // from shared memory in ascending row order, as before.
+        const int n_rows = static_cast<int>(e - p);
+        const int first = n_rows < 4 ? n_rows : 4;
+        uint32_t rid_lane = 0;
+        if (n_rows > 4 && lane < n_rows) rid_lane = rows[p + lane];
+        if (is_head) warp_copy_async<ROW_M_BYTES>(m_s, m, lane);
+        {
+            const int r4[4] = {dr.x, dr.y, dr.z, dr.w};
+#pragma unroll
+            for (int r = 0; r < 4; ++r)
+                if (r < first) warp_copy_async<ROW_Q_BYTES>(q_s + r * D, Q + static_cast<int64_t>(r4[r]) * D, lane);
+        }
+        cp_async_commit();
         const double n_old = size[slot];
         const uint32_t access_old = access[slot];
-        float *m = master + static_cast<int64_t>(slot) * D;
         double a[NQ][4];
+        cp_async_wait_all();
+        __syncwarp();
 #pragma unroll
         for (int j = 0; j < NQ; ++j) {
             float4 m4 = make_float4(0.f, 0.f, 0.f, 0.f);
-            if (is_head) m4 = *reinterpret_cast<const float4 *>(m + 4 * (lane + 32 * j));
+            if (is_head) m4 = *reinterpret_cast<const float4 *>(m_s + 4 * (lane + 32 * j));
             a[j][0] = n_old * static_cast<double>(m4.x); a[j][1] = n_old * static_cast<double>(m4.y);
             a[j][2] = n_old * static_cast<double>(m4.z); a[j][3] = n_old * static_cast<double>(m4.w);
         }
-        // the rows four at a time: their loads are in flight together, additions stay in ascending row order
-        uint32_t rid[4] = {static_cast<uint32_t>(dr.x), static_cast<uint32_t>(dr.y), static_cast<uint32_t>(dr.z),
-                           static_cast<uint32_t>(dr.w)};
-        for (int64_t t = p; t < e; t += 4) {
-            const int nrow = static_cast<int>(e - t < 4 ? e - t : 4);
-            const raw_t *q[4];
+        auto add_rows = [&](int n_stage) {
+            for (int r = 0; r < n_stage; ++r) {
+                const raw_t *src = reinterpret_cast<const raw_t *>(q_s + r * D) + lane;
 #pragma unroll
-            for (int r = 0; r < 4; ++r) q[r] = reinterpret_cast<const raw_t *>(Q + static_cast<int64_t>(rid[r]) * D) + lane;
-            if (t + 4 < e) {                                  // the next quartet's row numbers, requested with this one's rows
-#pragma unroll
-                for (int r = 0; r < 4; ++r) rid[r] = rows[t + 4 + r < e ? t + 4 + r : t + 4];
-            }
-#pragma unroll
-            for (int j = 0; j < NQ; ++j) {
-                raw_t v[4];
-#pragma unroll
-                for (int r = 0; r < 4; ++r) v[r] = __ldg(q[r] + 32 * j);
-#pragma unroll
-                for (int r = 0; r < 4; ++r) {
-                    if (r < nrow) {
-                        const float4 f = widen4(v[r]);
-                        a[j][0] += f.x; a[j][1] += f.y; a[j][2] += f.z; a[j][3] += f.w;
-                    }
+                for (int j = 0; j < NQ; ++j) {
+                    const float4 f = widen4(src[32 * j]);
+                    a[j][0] += f.x; a[j][1] += f.y; a[j][2] += f.z; a[j][3] += f.w;
                 }
             }
+        };
+        add_rows(first);
+        for (int t = 4; t < n_rows; t += UPW_STAGE_ROWS) {
+            const int n_stage = n_rows - t < UPW_STAGE_ROWS ? n_rows - t : UPW_STAGE_ROWS;
+            __syncwarp();                                     // the buffer's rows have been added
+            for (int r = 0; r < n_stage; ++r) {
+                const uint32_t rid = __shfl_sync(0xFFFFFFFFu, rid_lane, t + r);
+                warp_copy_async<ROW_Q_BYTES>(q_s + r * D, Q + static_cast<int64_t>(rid) * D, lane);
+            }
+            cp_async_commit();
+            cp_async_wait_all();
+            __syncwarp();
+            add_rows(n_stage);
         }
+        __syncwarp();                                         // before the next chunk's copies overwrite the buffer
         long long count = e - p;
         if (!(is_head && !more)) {
             // several chunks: publish this chunk's sum.  Chunks are combined in two levels so that a centroid with thousands
@@ -421,10 +461,18 @@ static bool launch_update_apply_warp(int nq, unsigned blocks, cudaStream_t s, co
                                      uint32_t *access, unsigned long long *last, const long long *counters, double *partial,
                                      unsigned int *arrived, unsigned int *arrived_runs) {
 #define SISO_UPW(N)                                                                                                          \
-    case N:                                                                                                                  \
-        update_apply_warp_kernel<T, N><<<blocks, UPW_THREADS, 0, s>>>(desc, list_len, n_desc, ticket, vs, chunk, q, master, vecs, size, access,  \
-                                                                     last, counters, partial, arrived, arrived_runs);        \
-        return true;
+    case N: {                                                                                                                \
+        const size_t smem = (UPW_THREADS / 32) * upw_warp_smem<T>(128 * N);                                                  \
+        if (smem > 48 * 1024 &&                                                                                              \
+            cudaFuncSetAttribute(update_apply_warp_kernel<T, N>, cudaFuncAttributeMaxDynamicSharedMemorySize,                \
+                                 static_cast<int>(smem)) != cudaSuccess) {                                                   \
+            cudaGetLastError();                                                                                              \
+            return false;                                                                                                    \
+        }                                                                                                                    \
+        update_apply_warp_kernel<T, N><<<blocks, UPW_THREADS, smem, s>>>(desc, list_len, n_desc, ticket, vs, chunk, q, master, vecs, size, \
+                                                                        access, last, counters, partial, arrived, arrived_runs); \
+        return true;                                                                                                         \
+    }
     switch (nq) {
         SISO_UPW(1) SISO_UPW(2) SISO_UPW(3) SISO_UPW(4) SISO_UPW(5) SISO_UPW(6) SISO_UPW(7) SISO_UPW(8)
         default: return false;
