@@ -256,6 +256,22 @@ siso_status_t siso_select_evict(const uint64_t *d_keys, int32_t n_lists, int64_t
 siso_status_t siso_evict_slots(siso_cache_t *c, const int64_t *d_victims, int64_t n, int64_t slot_offset, uint32_t flags,
                                void *stream);
 
+/* The same steps with every count kept on the device, so that a streaming step of the partitioned cache needs no host read:
+ *   siso_free_slots           d_free[0] = free slots of this shard (capacity - occupancy).
+ *   siso_shard_plan           d_hit [n] of the combined result and d_free_all [world] (the gathered free counts) ->
+ *                             d_plan[4] = { misses of the batch, entries to evict over the whole cache (misses - all free
+ *                             slots, at least 0), free slots on the shards before `rank`, free slots on this shard }.
+ *   siso_route_planned        siso_route with miss_skip / miss_take taken from d_plan[2], d_plan[3].
+ *   siso_select_evict_planned siso_select_evict with n_take = min(d_plan[1], n); d_victims [n], -1 beyond the victims. */
+siso_status_t siso_free_slots(siso_cache_t *c, int64_t *d_free, void *stream);
+siso_status_t siso_shard_plan(const uint8_t *d_hit, int64_t n, const int64_t *d_free_all, int32_t world, int32_t rank,
+                              int64_t *d_plan, void *stream);
+siso_status_t siso_route_planned(const int64_t *d_idx, int64_t idx_stride, const uint8_t *d_hit, int64_t n, int64_t slot_lo,
+                                 int64_t slot_hi, const int64_t *d_plan, int32_t *d_idx_local, uint8_t *d_update_hit,
+                                 uint8_t *d_insert_hit, void *stream);
+siso_status_t siso_select_evict_planned(const uint64_t *d_keys, int32_t n_lists, int64_t n, const int64_t *d_plan,
+                                        int64_t *d_victims, void *stream);
+
 /* Locality-ordered exact search, k = 1 (the exact-search counterpart of Sec. 4.3, "Searching for vectors in semantic
  * cache": entries with strong semantic locality are searched first and most queries end there).  The cache is held as
  * two handles: a small hot tier and the cold rest.  A query whose best hot similarity s exceeds exit_sim needs no cold

@@ -26,7 +26,8 @@ EXPORTS = ["siso_cache_create", "siso_cache_destroy", "siso_set_option", "siso_i
            "siso_choose_theta", "siso_correct_theta", "siso_tier_exit_sim", "siso_tier_select", "siso_tier_finish",
            "siso_route", "siso_evict_keys", "siso_select_evict", "siso_evict_slots", "siso_selftest_wait_timeout",
            "siso_measure_fp32_fma", "siso_pair_sweep_block", "siso_merge_resolve", "siso_merge_pack",
-           "siso_merge_apply_shard", "siso_tier_build", "siso_tier_work_bytes", "siso_tier_lookup"]
+           "siso_merge_apply_shard", "siso_tier_build", "siso_tier_work_bytes", "siso_tier_lookup", "siso_free_slots",
+           "siso_shard_plan", "siso_route_planned", "siso_select_evict_planned"]
 
 
 class SisoError(RuntimeError):
@@ -87,6 +88,10 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_evict_keys.argtypes = [vp, i64, i64, vp, vp]
     L.siso_select_evict.argtypes = [vp, i32, i64, i64, vp, vp]
     L.siso_evict_slots.argtypes = [vp, vp, i64, i64, u32, vp]
+    L.siso_free_slots.argtypes = [vp, vp, vp]
+    L.siso_shard_plan.argtypes = [vp, i64, vp, i32, i32, vp, vp]
+    L.siso_route_planned.argtypes = [vp, i64, vp, i64, i64, i64, vp, vp, vp, vp, vp]
+    L.siso_select_evict_planned.argtypes = [vp, i32, i64, vp, vp, vp]
     L.siso_tier_exit_sim.argtypes = [ctypes.c_double] * 2
     L.siso_tier_exit_sim.restype = ctypes.c_double
     L.siso_tier_select.argtypes = [vp, i64, f32, vp, i64, vp, vp, vp, vp]
@@ -320,6 +325,12 @@ class SisoCache:
         self._check(self._lib.siso_evict_slots(self._h, _ptr(v), v.numel(), int(slot_offset), flags, _stream(stream)),
                     "siso_evict_slots")
 
+    def free_slots(self, stream=None) -> torch.Tensor:
+        """[1] int64 on the device: capacity - occupancy, without a host read (see siso_free_slots)."""
+        out = self._new((1,), torch.int64)
+        self._check(self._lib.siso_free_slots(self._h, _ptr(out), _stream(stream)), "siso_free_slots")
+        return out
+
     def copy_from(self, src: "SisoCache", stream=None) -> None:
         """C_new <- C_cur (first line of MergeCentroids, Algorithm 1): every slot of `src` into the same slot here."""
         self._check(self._lib.siso_cache_copy(self._h, src._h, _stream(stream)), "siso_cache_copy")
@@ -486,9 +497,11 @@ def combine_keys(keys: torch.Tensor, theta, stream=None) -> Tuple[torch.Tensor, 
     return idx, sim, hit
 
 
-def route(idx: torch.Tensor, hit: torch.Tensor, slot_lo: int, slot_hi: int, miss_skip: int, miss_take: int, stream=None):
+def route(idx: torch.Tensor, hit: torch.Tensor, slot_lo: int, slot_hi: int, miss_skip: int = 0, miss_take: int = 0, stream=None,
+          plan: Optional[torch.Tensor] = None):
     """Combined (idx [n] or [n, k] int64 global slots, hit [n]) -> (idx_local [n] int32, update_hit [n], insert_hit [n]) for
-    the shard that owns [slot_lo, slot_hi) (see siso_route)."""
+    the shard that owns [slot_lo, slot_hi) (see siso_route).  With `plan` (the device tensor shard_plan wrote) the two miss
+    counts are read from it on the device (siso_route_planned)."""
     assert idx.dtype == torch.int64 and idx.is_cuda and hit.dtype == torch.uint8
     idx, hit = idx.contiguous(), hit.contiguous()
     n = hit.numel()
@@ -496,11 +509,44 @@ def route(idx: torch.Tensor, hit: torch.Tensor, slot_lo: int, slot_hi: int, miss
     idx_local = torch.empty((n,), dtype=torch.int32, device=idx.device)
     upd, ins = torch.empty_like(hit), torch.empty_like(hit)
     with torch.cuda.device(idx.device):
-        st = load_library().siso_route(_ptr(idx), stride, _ptr(hit), n, int(slot_lo), int(slot_hi), int(miss_skip), int(miss_take),
-                                       _ptr(idx_local), _ptr(upd), _ptr(ins), _stream(stream))
+        if plan is None:
+            st = load_library().siso_route(_ptr(idx), stride, _ptr(hit), n, int(slot_lo), int(slot_hi), int(miss_skip),
+                                           int(miss_take), _ptr(idx_local), _ptr(upd), _ptr(ins), _stream(stream))
+        else:
+            assert plan.dtype == torch.int64 and plan.numel() == 4 and plan.device == idx.device
+            st = load_library().siso_route_planned(_ptr(idx), stride, _ptr(hit), n, int(slot_lo), int(slot_hi), _ptr(plan),
+                                                   _ptr(idx_local), _ptr(upd), _ptr(ins), _stream(stream))
     if st != 0:
         raise SisoError(st, "siso_route")
     return idx_local, upd, ins
+
+
+def shard_plan(hit: torch.Tensor, free_all: torch.Tensor, rank: int, stream=None) -> torch.Tensor:
+    """hit [n] of a combined lookup and free_all [world] int64 (every shard's free slots) -> plan [4] int64 on the device:
+    misses, entries to evict over the whole cache, free slots before `rank`, free slots on `rank` (see siso_shard_plan)."""
+    assert hit.dtype == torch.uint8 and hit.is_cuda and free_all.dtype == torch.int64 and free_all.device == hit.device
+    hit, free_all = hit.contiguous(), free_all.reshape(-1).contiguous()
+    plan = torch.empty((4,), dtype=torch.int64, device=hit.device)
+    with torch.cuda.device(hit.device):
+        st = load_library().siso_shard_plan(_ptr(hit), hit.numel(), _ptr(free_all), free_all.numel(), int(rank), _ptr(plan),
+                                            _stream(stream))
+    if st != 0:
+        raise SisoError(st, "siso_shard_plan")
+    return plan
+
+
+def select_evict_planned(keys: torch.Tensor, plan: torch.Tensor, stream=None) -> torch.Tensor:
+    """keys [n_lists, n, 3] -> victims [n] int64: the plan[1] lowest of all keys in eviction order, then -1."""
+    assert keys.dtype == torch.int64 and keys.dim() == 3 and keys.shape[2] == 3 and keys.is_cuda
+    assert plan.dtype == torch.int64 and plan.numel() == 4 and plan.device == keys.device
+    keys = keys.contiguous()
+    victims = torch.empty((keys.shape[1],), dtype=torch.int64, device=keys.device)
+    with torch.cuda.device(keys.device):
+        st = load_library().siso_select_evict_planned(_ptr(keys), keys.shape[0], keys.shape[1], _ptr(plan), _ptr(victims),
+                                                      _stream(stream))
+    if st != 0:
+        raise SisoError(st, "siso_select_evict_planned")
+    return victims
 
 
 def select_evict(keys: torch.Tensor, n_take: int, stream=None) -> torch.Tensor:

@@ -476,6 +476,39 @@ siso_status_t siso_select_evict(const uint64_t *d_keys, int32_t n_lists, int64_t
                                reinterpret_cast<long long *>(d_victims), static_cast<cudaStream_t>(stream));
 }
 
+siso_status_t siso_free_slots(siso_cache_t *c, int64_t *d_free, void *stream) {
+    if (!c || !d_free) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    return launch_free_slots(c, reinterpret_cast<long long *>(d_free), static_cast<cudaStream_t>(stream));
+}
+
+siso_status_t siso_shard_plan(const uint8_t *d_hit, int64_t n, const int64_t *d_free_all, int32_t world, int32_t rank,
+                              int64_t *d_plan, void *stream) {
+    if (n < 0 || (n > 0 && !d_hit) || !d_free_all || world < 1 || rank < 0 || rank >= world || !d_plan) return SISO_ERR_INVALID_ARG;
+    return launch_shard_plan(d_hit, n, reinterpret_cast<const long long *>(d_free_all), world, rank,
+                             reinterpret_cast<long long *>(d_plan), static_cast<cudaStream_t>(stream));
+}
+
+siso_status_t siso_route_planned(const int64_t *d_idx, int64_t idx_stride, const uint8_t *d_hit, int64_t n, int64_t slot_lo,
+                                 int64_t slot_hi, const int64_t *d_plan, int32_t *d_idx_local, uint8_t *d_update_hit,
+                                 uint8_t *d_insert_hit, void *stream) {
+    if (n < 0 || idx_stride < 1 || slot_lo < 0 || slot_hi < slot_lo || !d_plan) return SISO_ERR_INVALID_ARG;
+    if (slot_hi - slot_lo > 0x7FFFFFFFll) return SISO_ERR_UNSUPPORTED;
+    if (n == 0) return SISO_OK;
+    if (!d_idx || !d_hit || !d_idx_local || !d_update_hit || !d_insert_hit) return SISO_ERR_INVALID_ARG;
+    return launch_shard_route(reinterpret_cast<const long long *>(d_idx), idx_stride, d_hit, n, slot_lo, slot_hi, 0, 0, d_idx_local,
+                              d_update_hit, d_insert_hit, static_cast<cudaStream_t>(stream), reinterpret_cast<const long long *>(d_plan));
+}
+
+siso_status_t siso_select_evict_planned(const uint64_t *d_keys, int32_t n_lists, int64_t n, const int64_t *d_plan,
+                                        int64_t *d_victims, void *stream) {
+    if (n_lists < 1 || n < 0 || !d_plan) return SISO_ERR_INVALID_ARG;
+    if (n == 0) return SISO_OK;
+    if (!d_victims || !d_keys) return SISO_ERR_INVALID_ARG;
+    return launch_evict_select(reinterpret_cast<const unsigned long long *>(d_keys), n_lists, n, n, reinterpret_cast<long long *>(d_victims),
+                               static_cast<cudaStream_t>(stream), reinterpret_cast<const long long *>(d_plan));
+}
+
 siso_status_t siso_evict_slots(siso_cache_t *c, const int64_t *d_victims, int64_t n, int64_t slot_offset, uint32_t flags,
                                void *stream) {
     if (!c || n < 0 || slot_offset < 0 || (n > 0 && !d_victims) || (flags & ~SISO_EVICT_DECAY)) return SISO_ERR_INVALID_ARG;

@@ -165,11 +165,14 @@ siso_status_t launch_insert(Cache *c, const void *vecs, const double *sizes, con
                             int32_t *slots_out, cudaStream_t s);
 siso_status_t launch_evict_keys(Cache *c, int64_t n, int64_t slot_offset, unsigned long long *keys_out, cudaStream_t s);
 siso_status_t launch_evict_select(const unsigned long long *keys, int n_lists, int64_t n, int64_t n_take, long long *victims,
-                                  cudaStream_t s);
+                                  cudaStream_t s, const long long *plan = nullptr);
+siso_status_t launch_shard_plan(const uint8_t *hit, int64_t n, const long long *free_all, int world, int rank, long long *plan,
+                                cudaStream_t s);
+siso_status_t launch_free_slots(Cache *c, long long *out, cudaStream_t s);
 siso_status_t launch_evict_slots(Cache *c, const long long *victims, int64_t n, int64_t slot_offset, uint32_t flags, cudaStream_t s);
 siso_status_t launch_shard_route(const long long *idx, long long idx_stride, const uint8_t *hit, int64_t n, int64_t slot_lo,
                                  int64_t slot_hi, int64_t skip, int64_t take, int32_t *idx_local, uint8_t *upd_hit,
-                                 uint8_t *ins_hit, cudaStream_t s);
+                                 uint8_t *ins_hit, cudaStream_t s, const long long *plan = nullptr);
 siso_status_t launch_sort_pairs(Cache *c, Scratch *scr, uint32_t *keys, uint32_t *vals, uint32_t *keys_tmp,
                                 uint32_t *vals_tmp, int64_t n, int key_bits, uint32_t **keys_out, uint32_t **vals_out,
                                 cudaStream_t s);

@@ -308,9 +308,11 @@ namespace {
 // keys [n_lists, n] (Key3), every list ascending with all-ones padding; one thread per key: its rank among all keys is the
 // sum over the lists of the number of smaller keys there (binary search); the n_take lowest give victims[rank] = global slot
 __global__ void __launch_bounds__(256)
-evict_select_kernel(const Key3 *__restrict__ keys, int n_lists, long long n, long long n_take, long long *__restrict__ victims) {
+evict_select_kernel(const Key3 *__restrict__ keys, int n_lists, long long n, long long n_take, const long long *__restrict__ plan,
+                    long long *__restrict__ victims) {
     const long long t = static_cast<long long>(blockIdx.x) * blockDim.x + threadIdx.x;
     if (t >= n * n_lists) return;
+    if (plan) n_take = plan[1] < n ? plan[1] : n;               // decided on the device (siso_shard_plan)
     const Key3 mine = keys[t];
     if ((mine.w0 & mine.w1 & mine.w2) == ~0ull) return;
     long long rank = 0;
@@ -350,11 +352,11 @@ evict_slots_kernel(const long long *__restrict__ victims, long long n, long long
 }  // namespace
 
 siso_status_t launch_evict_select(const unsigned long long *keys, int n_lists, int64_t n, int64_t n_take, long long *victims,
-                                  cudaStream_t s) {
+                                  cudaStream_t s, const long long *plan) {
     SISO_CUDA(cudaMemsetAsync(victims, 0xFF, sizeof(long long) * n_take, s));  // -1: fewer live entries than asked for
     if (n > 0)
         evict_select_kernel<<<static_cast<unsigned>((n * n_lists + 255) / 256), 256, 0, s>>>(
-            reinterpret_cast<const Key3 *>(keys), n_lists, n, n_take, victims);
+            reinterpret_cast<const Key3 *>(keys), n_lists, n, n_take, plan, victims);
     return check_cuda(cudaGetLastError(), "evict_select_kernel");
 }
 

@@ -60,10 +60,11 @@ shard_combine_kernel(const unsigned long long *__restrict__ keys, long long n, i
 // one CTA
 __global__ void __launch_bounds__(1024)
 shard_route_kernel(const long long *__restrict__ idx, long long idx_stride, const uint8_t *__restrict__ hit, long long n,
-                   long long slot_lo, long long slot_hi, long long skip, long long take, int32_t *__restrict__ idx_local,
-                   uint8_t *__restrict__ upd_hit, uint8_t *__restrict__ ins_hit) {
+                   long long slot_lo, long long slot_hi, long long skip, long long take, const long long *__restrict__ plan,
+                   int32_t *__restrict__ idx_local, uint8_t *__restrict__ upd_hit, uint8_t *__restrict__ ins_hit) {
     __shared__ int warp_cnt[32];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
+    if (plan) { skip = plan[2]; take = plan[3]; }              // decided on the device (siso_shard_plan)
     long long base = 0;                                          // misses in the rows already visited, the same in every thread
     for (long long b0 = 0; b0 < n; b0 += 1024) {
         const long long b = b0 + tid;
@@ -90,12 +91,52 @@ shard_route_kernel(const long long *__restrict__ idx, long long idx_stride, cons
     }
 }
 
+// one CTA: what the batch's misses need, from the hit flags and the free slots of every shard
+//   plan[0] misses   plan[1] entries to evict over the whole cache (misses - free slots, at least 0)
+//   plan[2] free slots on the shards before this one   plan[3] free slots on this shard
+__global__ void __launch_bounds__(1024)
+shard_plan_kernel(const uint8_t *__restrict__ hit, long long n, const long long *__restrict__ free_all, int world, int rank,
+                  long long *__restrict__ plan) {
+    __shared__ int warp_cnt[32];
+    int miss = 0;
+    for (long long b = threadIdx.x; b < n; b += 1024) miss += hit[b] == 0 ? 1 : 0;
+#pragma unroll
+    for (int o = 16; o >= 1; o >>= 1) miss += __shfl_xor_sync(0xFFFFFFFFu, miss, o);
+    if ((threadIdx.x & 31) == 0) warp_cnt[threadIdx.x >> 5] = miss;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        long long n_miss = 0, total = 0, before = 0;
+        for (int w = 0; w < 32; ++w) n_miss += warp_cnt[w];
+        for (int r = 0; r < world; ++r) { total += free_all[r]; before += r < rank ? free_all[r] : 0; }
+        plan[0] = n_miss;
+        plan[1] = n_miss > total ? n_miss - total : 0;
+        plan[2] = before;
+        plan[3] = free_all[rank];
+    }
+}
+
+__global__ void free_slots_kernel(const long long *__restrict__ counters, long long capacity, long long *__restrict__ out) {
+    out[0] = capacity - counters[CNT_OCCUPANCY];
+}
+
 }  // namespace
+
+siso_status_t launch_shard_plan(const uint8_t *hit, int64_t n, const long long *free_all, int world, int rank, long long *plan,
+                                cudaStream_t s) {
+    shard_plan_kernel<<<1, 1024, 0, s>>>(hit, n, free_all, world, rank, plan);
+    return check_cuda(cudaGetLastError(), "shard_plan_kernel");
+}
+
+siso_status_t launch_free_slots(Cache *c, long long *out, cudaStream_t s) {
+    free_slots_kernel<<<1, 1, 0, s>>>(c->counters, c->capacity, out);
+    SISO_LAUNCHED(c);
+    return SISO_OK;
+}
 
 siso_status_t launch_shard_route(const long long *idx, long long idx_stride, const uint8_t *hit, int64_t n, int64_t slot_lo,
                                  int64_t slot_hi, int64_t skip, int64_t take, int32_t *idx_local, uint8_t *upd_hit,
-                                 uint8_t *ins_hit, cudaStream_t s) {
-    shard_route_kernel<<<1, 1024, 0, s>>>(idx, idx_stride, hit, n, slot_lo, slot_hi, skip, take, idx_local, upd_hit, ins_hit);
+                                 uint8_t *ins_hit, cudaStream_t s, const long long *plan) {
+    shard_route_kernel<<<1, 1024, 0, s>>>(idx, idx_stride, hit, n, slot_lo, slot_hi, skip, take, plan, idx_local, upd_hit, ins_hit);
     return check_cuda(cudaGetLastError(), "shard_route_kernel");
 }
 

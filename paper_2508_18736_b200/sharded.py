@@ -163,9 +163,6 @@ class ShardedCache:
         return combine_keys(gather_keys(keys, self.group), theta, stream=stream)
 
     # ---- maintenance: generators that yield their exchanges; drive them with run() or run_lockstep() ----
-    def _free(self) -> int:
-        return (self.hi - self.lo) - int(self.local.stats()["occupancy"])
-
     def evict_steps(self, n_evict: int, flags: int = 0):
         """FilteringCentroids over the whole cache: -> victims [n_evict] int64 global slots in eviction order (-1 padding),
         the same on every rank."""
@@ -184,16 +181,24 @@ class ShardedCache:
             self.local.evict_slots(victims, self.lo, flags)
         return victims
 
+    def _free_dev(self) -> torch.Tensor:
+        """[1] int64 on the device: this shard's free slots (0 for a rank without rows)."""
+        if self.hi == self.lo:
+            return torch.zeros((1,), dtype=torch.int64, device=self.local._dev)
+        return self.local.free_slots()
+
     def stream_steps(self, queries: torch.Tensor, theta):
         """One micro-batch of the streaming step over the whole cache (lookup, running-mean update of the hits, room for
-        the misses, insertion): -> (idx [n] int64 global slot, sim [n], hit [n], victims int64 [#evicted], slots [n] int64
-        global slot of each stored miss or -1), the same on every rank and equal to one unsharded cache's step."""
-        from .binding import combine_keys, route
+        the misses, insertion): -> (idx [n] int64 global slot, sim [n], hit [n], victims int64 [n]: the evicted global
+        slots in eviction order, then -1, slots [n] int64 global slot of each stored miss or -1), the same on every rank
+        and equal to one unsharded cache's step.  Every count the step depends on (misses, free slots, entries to evict)
+        stays on the device, so the host issues the same launches and exchanges for every batch and never waits."""
+        from .binding import combine_keys, route, select_evict_planned, shard_plan
         q = self.local._vec(queries, "queries")
         n = q.shape[0]
-        dev = q.device
+        empty = self.hi == self.lo
         keys = self.local.lookup_keys(q, 1, slot_offset=self.lo)
-        if self.hi == self.lo:
+        if empty:
             keys.zero_()
         all_keys = yield ("gather", keys)                     # [world, n, 1]
         idx, sim, hit = combine_keys(all_keys.permute(1, 0, 2).contiguous(), theta)
@@ -201,21 +206,23 @@ class ShardedCache:
         # hits: the owner updates; every rank calls the update so that every clock advances
         idx_local, upd_hit, _ = route(idx, hit, self.lo, self.hi, 0, 0)
         self.local.update(q, idx_local, upd_hit)
-        # room: the misses need free slots somewhere in the cache
-        n_miss = n - int(hit.sum().item())
-        free = yield ("gather", torch.tensor([self._free()], dtype=torch.int64, device=dev))       # [world, 1]
-        lack = n_miss - int(free.sum().item())
-        victims = torch.empty((0,), dtype=torch.int64, device=dev)
-        if lack > 0:
-            victims = yield from self.evict_steps(lack)
-            free = yield ("gather", torch.tensor([self._free()], dtype=torch.int64, device=dev))
+        # room: the misses that find no free slot anywhere in the cache evict (plan[1] of them, possibly none)
+        free = yield ("gather", self._free_dev())             # [world, 1]
+        plan = shard_plan(hit, free, self.rank)
+        ekeys = self.local.evict_keys(n, slot_offset=self.lo)
+        if empty:
+            ekeys.fill_(-1)                                   # a rank without rows reports nothing
+        all_ekeys = yield ("gather", ekeys)                   # [world, n, 3]
+        victims = select_evict_planned(all_ekeys, plan)
+        if not empty:
+            self.local.evict_slots(victims, self.lo, 0)
         # insertion: misses in row order take the free slots in global order
-        skip = int(free[:self.rank].sum().item())
-        take = int(free[self.rank].item())
-        _, _, ins_hit = route(idx, hit, self.lo, self.hi, skip, take)
+        free = yield ("gather", self._free_dev())
+        plan = shard_plan(hit, free, self.rank)
+        _, _, ins_hit = route(idx, hit, self.lo, self.hi, plan=plan)
         slots = self.local.insert_misses(q, ins_hit).to(torch.int64)
         slots = torch.where(slots >= 0, slots + self.lo, slots)
-        if self.hi == self.lo:
+        if empty:
             slots.fill_(-1)
         slots = yield ("max", slots)
         return idx, sim, hit, victims, slots

@@ -91,9 +91,11 @@ def test_sharded_stream_equals_one_cache(dtype, total, dim, shards, batch, n_bat
         o_idx, o_sim, o_hit, o_victims, o_slots = ora.stream_step(qn, theta, forced=(idx[:, None].astype(np.int32), hit))
         check_lookup((idx[:, None].astype(np.int32), sim[:, None], hit), (o_idx, o_sim, o_hit), pre_copy, qn, theta, TOL[dtype],
                      valid=pre_valid)
-        assert (victims == o_victims[:len(victims)]).all() and len(victims) == (o_victims >= 0).sum()
+        nv = int((victims >= 0).sum())                                   # [batch]: eviction order, then -1
+        assert len(victims) == len(qn) and (victims[nv:] == -1).all()
+        assert (victims[:nv] == o_victims[:nv]).all() and nv == (o_victims >= 0).sum()
         assert (slots == o_slots).all()
-        evicted += len(victims)
+        evicted += nv
         # the shards' states, laid side by side, are the one cache's state
         for p in parts:
             if p.hi == p.lo:
@@ -147,7 +149,7 @@ def test_sharded_eviction_is_the_global_selection():
 def test_world_of_one_through_the_distributed_driver():
     """Without a process group the torch.distributed driver (run) sees a world of one rank: the sharded step and the
     sharded eviction must then equal the plain cache's, bit for bit."""
-    sp = W.StreamSpec(capacity=400, dim=64, n_queries=100 * 12, batch=100, n_clusters=900, zipf_s=1.1, reshuffle_every=500,
+    sp = W.StreamSpec(capacity=400, dim=64, n_queries=100 * 13, batch=100, n_clusters=900, zipf_s=1.1, reshuffle_every=500,
                       theta=0.80, mode="P", dtype="bf16", seed=62)
     stream = W.QueryStream(sp)
     one = siso.ShardedCache(400, 64, "bf16")
@@ -159,12 +161,20 @@ def test_world_of_one_through_the_distributed_driver():
         p_idx, p_sim, p_hit, p_victims, p_slots = plain.stream_step(q, float(sp.theta))
         assert (idx.to(torch.int32) == p_idx[:, 0]).all().item() and (hit == p_hit).all().item()
         assert (sim == p_sim[:, 0]).all().item()
-        nv = victims.numel()
-        assert (victims.to(torch.int32) == p_victims[:nv]).all().item() and (p_victims[nv:] == -1).all().item()
+        assert victims.numel() == p_victims.numel() and (victims.to(torch.int32) == p_victims).all().item()
         assert (slots.to(torch.int32) == p_slots).all().item()
     a, b = one.local.export(), plain.export()
     assert all((a[k] == b[k]).all().item() for k in ("valid", "size", "access", "last", "master", "vecs"))
     assert one.local.stats()["evictions"] == plain.stats()["evictions"] > 0
+    # the binding layer of a sharded step reads nothing back: misses, free slots and the eviction count stay on the device
+    q = to_dev(stream.batch(12)[0], "bf16")
+    torch.cuda.set_sync_debug_mode("error")
+    try:
+        res = one.stream_step(q, float(sp.theta))
+    finally:
+        torch.cuda.set_sync_debug_mode("default")
+    p_res = plain.stream_step(q, float(sp.theta))
+    assert (res[0].to(torch.int32) == p_res[0][:, 0]).all().item() and (res[3].to(torch.int32) == p_res[3]).all().item()
     v1 = one.evict(37, siso.EVICT_DECAY)
     v2 = plain.evict(37, siso.EVICT_DECAY)
     assert (v1.to(torch.int32) == v2).all().item()
