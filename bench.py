@@ -626,8 +626,8 @@ def run_sharded(args):
     st = sc.local.stats()
     line["stream_step"] = {"workload": f"config 5 cache ({sp.capacity} x {sp.dim} bf16) sharded x{world}, micro-batches of 256",
                            "us_per_batch": us, "queries_per_s": 256 / us * 1e6, "evictions_this_rank": st["evictions"],
-                           "note": "lookup keys, free counts, eviction keys and slots are exchanged every batch; this version reads "
-                                   "a few counts on the host between phases"}
+                           "note": "lookup keys, free counts, eviction keys and slots are exchanged every batch; the miss count, "
+                                   "the free slots and the number of entries to evict stay on the device (no host read in the step)"}
     sc.close()
     if rank == 0:
         print(json.dumps(line), flush=True)
