@@ -5,7 +5,7 @@ MergeCentroids / FilteringCentroids and spare-space insertion, behind the C ABI 
 pointers and calls ``libsiso.so``; every step runs in the library's own CUDA kernels."""
 from .binding import (ACCESS_INF, EVICT_DECAY, MERGE_SIZES_ONLY, MERGE_WEIGHTED_MEAN, OPT_LOOKUP_PATH,
                       OPT_MERGE_MAX_CANDIDATES, OPT_MERGE_PATH, OPT_STREAM_FUSED, OPT_TENSOR_CTA_PAIR, OPT_SWEEP_FINALIZE,
-                      OPT_STREAM_LIST, OPT_CHECKED, PATH_AUTO, PATH_SIMT,
+                      OPT_STREAM_LIST, OPT_MERGE_SWEEP_PARTS, OPT_CHECKED, PATH_AUTO, PATH_SIMT,
                       PATH_STREAM, PATH_TENSOR, SisoCache, SisoError, combine_keys, load_library, lookup_small_noalloc, md1_wait,
                       choose_theta, correct_theta, tier_exit_sim, tier_finish, tier_select, route, select_evict)
 from .tiered import TieredCache
@@ -13,4 +13,4 @@ from .sharded import ShardedCache, exchange, gather_keys, local_range, owner_of,
 
 __all__ = ["SisoCache", "ShardedCache", "TieredCache", "tier_exit_sim", "tier_select", "tier_finish", "route", "select_evict", "combine_keys", "gather_keys", "exchange", "run", "run_lockstep", "shard_rows", "owner_of", "local_range", "SisoError", "load_library", "lookup_small_noalloc", "md1_wait", "choose_theta", "correct_theta", "ACCESS_INF", "EVICT_DECAY", "MERGE_SIZES_ONLY",
            "MERGE_WEIGHTED_MEAN", "OPT_LOOKUP_PATH", "OPT_MERGE_MAX_CANDIDATES", "OPT_MERGE_PATH", "OPT_STREAM_FUSED",
-           "OPT_TENSOR_CTA_PAIR", "OPT_SWEEP_FINALIZE", "OPT_STREAM_LIST", "OPT_CHECKED", "PATH_AUTO", "PATH_SIMT", "PATH_STREAM", "PATH_TENSOR"]
+           "OPT_TENSOR_CTA_PAIR", "OPT_SWEEP_FINALIZE", "OPT_STREAM_LIST", "OPT_MERGE_SWEEP_PARTS", "OPT_CHECKED", "PATH_AUTO", "PATH_SIMT", "PATH_STREAM", "PATH_TENSOR"]

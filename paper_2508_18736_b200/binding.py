@@ -14,7 +14,7 @@ ACCESS_INF = 0xFFFFFFFF
 MERGE_SIZES_ONLY, MERGE_WEIGHTED_MEAN = 0, 1
 EVICT_DECAY = 1
 OPT_LOOKUP_PATH, OPT_MERGE_MAX_CANDIDATES, OPT_TENSOR_CTA_PAIR, OPT_STREAM_FUSED, OPT_MERGE_PATH = 1, 2, 3, 4, 5
-OPT_SWEEP_FINALIZE, OPT_STREAM_LIST, OPT_CHECKED = 6, 7, 9
+OPT_SWEEP_FINALIZE, OPT_STREAM_LIST, OPT_MERGE_SWEEP_PARTS, OPT_CHECKED = 6, 7, 8, 9
 PATH_AUTO, PATH_SIMT, PATH_TENSOR, PATH_STREAM = 0, 1, 2, 3
 _STATUS_NAMES = {0: "SISO_OK", 1: "SISO_ERR_INVALID_ARG", 2: "SISO_ERR_UNSUPPORTED", 3: "SISO_ERR_OOM",
                  4: "SISO_ERR_CAPACITY", 5: "SISO_ERR_OVERFLOW", 6: "SISO_ERR_TIMEOUT", 7: "SISO_ERR_CUDA"}

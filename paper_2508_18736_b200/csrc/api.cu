@@ -300,6 +300,10 @@ siso_status_t siso_set_option(siso_cache_t *c, int32_t key, int64_t value) {
             if (value != SISO_PATH_AUTO && value != SISO_PATH_SIMT && value != SISO_PATH_TENSOR) return SISO_ERR_INVALID_ARG;
             c->merge_path = static_cast<int32_t>(value);
             return SISO_OK;
+        case SISO_OPT_MERGE_SWEEP_PARTS:
+            if (value != 1 && value != 3) return SISO_ERR_INVALID_ARG;
+            c->merge_sweep_parts = static_cast<int32_t>(value);
+            return SISO_OK;
         case SISO_OPT_MERGE_MAX_CANDIDATES:
             if (value < 1 || value > (1ll << 31)) return SISO_ERR_INVALID_ARG;
             c->merge_max_cand = value;

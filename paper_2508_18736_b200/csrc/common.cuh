@@ -63,6 +63,7 @@ struct Cache {
     bool merge_tensor_attr_set;
     int merge_resolve_grid;     // CTAs of the grid-wide merge resolution (0: not yet asked, -1: unavailable)
     int32_t merge_path;         // SISO_PATH_AUTO, SISO_PATH_SIMT or SISO_PATH_TENSOR for the pairwise sweep of siso_merge
+    int32_t merge_sweep_parts;  // 3: the tensor-core sweep of fp32 rows multiplies three bf16 parts; otherwise one part as a filter
     void *swap_plan;            // UpdateCentroids: slot of the d-th live entry, when this cache serves as C_new
     int maint_grid;             // CTAs of the fused streaming maintenance kernel (0: not yet asked, -1: unavailable)
     int32_t sweep_finalize_separate;   // 1: never finish a top-1 lookup inside the sweep kernel

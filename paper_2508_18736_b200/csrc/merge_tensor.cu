@@ -9,10 +9,15 @@
 // in fp64 and keeps those whose exact similarity exceeds theta_C.  The decisions are therefore those of an exact
 // fp64 sweep; the tensor cores do the 2 N^2 D flops, the exact arithmetic touches the few candidates only.
 //
+// By default even less is asked of the tensor cores: the rows rounded to bf16 are multiplied ONCE (one MMA per 16
+// K-elements, half the operand bytes) and the filter margin is widened to the bound of that rounding (one_part_margin);
+// a few more pairs reach the exact check, the decisions stay the same.
+//
 // Kernel layout (CTA pairs, cta_group::2, as in the large-batch lookup): a cluster works on 256 rows i x 256 rows j
-// at a time; each CTA stages its own 128 rows i (hi and lo) and half of the rows j (hi and lo), 64 KiB per stage,
-// three stages; warp 0 = TMA producer, warp 1 = MMA issuer (leader CTA), warps 2-5 = epilogue (thread = row i)
-// over two TMEM accumulators.  The tile pairs of the lower triangle (one set) or of the whole matrix (two sets) are
+// at a time; each CTA stages its own 128 rows i and half of the rows j: 32 KiB per stage and six stages with one
+// part, 64 KiB (hi and lo of both) and three stages with three parts; warp 0 = TMA producer, warp 1 = MMA issuer
+// (leader CTA), warps 2-9 = epilogue (thread = row i, two warps per 32 rows, 128 columns each) over two TMEM
+// accumulators.  The tile pairs of the lower triangle (one set) or of the whole matrix (two sets) are
 // listed block by block (9 x 9 tiles) and dealt to the clusters round robin, so the clusters that run at the same
 // time work inside one block and share its rows through L2.  No load is multicast; every wait is bounded.
 #include <cstring>
@@ -39,21 +44,25 @@ using namespace umma2;
 constexpr int TM = 128;             // rows i per CTA
 constexpr int TN = 256;             // rows j per tile (128 staged by each CTA)
 constexpr int TK = 64;
-constexpr int STAGES = 3;
+constexpr int MAX_STAGES = 6;
 constexpr int ACC_STAGES = 2;
-constexpr int THREADS = 192;
+constexpr int EPI_WARPS = 8;
+constexpr int THREADS = 64 + 32 * EPI_WARPS;
 constexpr uint32_t OPER_BYTES = TM * TK * 2;              // 16 KiB: 128 rows x 64 bf16
-constexpr uint32_t STAGE_BYTES = 4 * OPER_BYTES;          // hi_i, lo_i, hi_j (half), lo_j (half)
-constexpr uint32_t SMEM_BYTES = STAGES * STAGE_BYTES + 1024 + 4096;
+constexpr uint32_t RING_BYTES = 12 * OPER_BYTES;          // six stages of (hi_i, hi_j half) or three of (hi_i, lo_i, hi_j half, lo_j half)
+constexpr uint32_t SMEM_BYTES = RING_BYTES + 1024 + 4096;
 constexpr uint32_t TMEM_COLS = ACC_STAGES * TN;
-constexpr float FILTER_MARGIN = 1e-4f;
+constexpr float FILTER_MARGIN = 1e-4f;             // three-part products (or rows that are bf16 values): rounding of the fp32 sums
+// One-part filter on fp32 rows: with x^ = bf16(x), |x.y - x^.y^| <= (2u + u^2) |x| |y| for u = 2^-9 (round to nearest),
+// 3.93e-3 for norms up to 1.002; the fp32 accumulation adds at most dim * 2^-23.
+__host__ inline float one_part_margin(int dim) { return 4.0e-3f + 1.2e-7f * static_cast<float>(dim); }
 
 // D fp32, A and B bf16, K-major, N = 256, M = 256 (128 rows per CTA of the pair)
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(TN >> 3) << 17) |
                            (static_cast<uint32_t>((2 * TM) >> 4) << 24);
 
 struct Shared {
-    uint64_t full[STAGES], empty[STAGES], acc_full[ACC_STAGES], acc_empty[ACC_STAGES];
+    uint64_t full[MAX_STAGES], empty[MAX_STAGES], acc_full[ACC_STAGES], acc_empty[ACC_STAGES];
     uint32_t tmem_base;
     int abort_flag;
 };
@@ -72,7 +81,10 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
                           MergeCandidate *__restrict__ cand, unsigned long long max_cand, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *stage_mem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
-    Shared *sh = reinterpret_cast<Shared *>(stage_mem + STAGES * STAGE_BYTES);
+    Shared *sh = reinterpret_cast<Shared *>(stage_mem + RING_BYTES);
+    const uint32_t STAGES = split ? 3u : 6u;
+    const uint32_t STAGE_BYTES = split ? 4 * OPER_BYTES : 2 * OPER_BYTES;
+    const uint32_t OFF_J = split ? 2 * OPER_BYTES : OPER_BYTES;       // where the rows j start inside a stage
     volatile int *abort_flag = &sh->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -85,8 +97,8 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
     const bool skip = ctl->overflow != 0;           // set before the launch (two sets: the insertion failed)
 
     if (threadIdx.x == 0) {
-        for (int s = 0; s < STAGES; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
-        for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(&sh->acc_full[a], 1); mbar_init(&sh->acc_empty[a], 8); }
+        for (int s = 0; s < MAX_STAGES; ++s) { mbar_init(&sh->full[s], 1); mbar_init(&sh->empty[s], 1); }
+        for (int a = 0; a < ACC_STAGES; ++a) { mbar_init(&sh->acc_full[a], 1); mbar_init(&sh->acc_empty[a], 2 * EPI_WARPS); }
         sh->abort_flag = 0;
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         asm volatile("fence.proxy.async.shared::cta;" ::: "memory");
@@ -119,11 +131,11 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
                     uint8_t *dst = stage_mem + stage * STAGE_BYTES;
                     const uint32_t full_leader = cluster_addr(smem_u32(&sh->full[stage]), 0);
                     // bf16 inputs have no second part: only the hi tiles are loaded and one MMA per K step is issued
-                    if (rank == 0) mbar_arrive_expect_tx(&sh->full[stage], split ? 2 * STAGE_BYTES : STAGE_BYTES);
+                    if (rank == 0) mbar_arrive_expect_tx(&sh->full[stage], 2 * STAGE_BYTES);   // both CTAs' loads of the stage
                     tma_load_2d_pair(dst, &map_hi, ks * TK, i0, full_leader);
                     if (split) tma_load_2d_pair(dst + OPER_BYTES, &map_lo, ks * TK, i0, full_leader);
-                    tma_load_2d_pair(dst + 2 * OPER_BYTES, &map_hi, ks * TK, n0, full_leader);
-                    if (split) tma_load_2d_pair(dst + 3 * OPER_BYTES, &map_lo, ks * TK, n0, full_leader);
+                    tma_load_2d_pair(dst + OFF_J, &map_hi, ks * TK, n0, full_leader);
+                    if (split) tma_load_2d_pair(dst + OFF_J + OPER_BYTES, &map_lo, ks * TK, n0, full_leader);
                     if (++stage == STAGES) { stage = 0; phase ^= 1u; }
                 }
             }
@@ -142,7 +154,7 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
                     tcgen05_fence_after();
                     const uint32_t base = smem_u32(stage_mem + stage * STAGE_BYTES);
                     const uint64_t a_hi = smem_desc_sw128(base), a_lo = smem_desc_sw128(base + OPER_BYTES);
-                    const uint64_t b_hi = smem_desc_sw128(base + 2 * OPER_BYTES), b_lo = smem_desc_sw128(base + 3 * OPER_BYTES);
+                    const uint64_t b_hi = smem_desc_sw128(base + OFF_J), b_lo = smem_desc_sw128(base + OFF_J + OPER_BYTES);
 #pragma unroll
                     for (int kk = 0; kk < TK / 16; ++kk) {
                         const uint64_t o = static_cast<uint64_t>(2 * kk);
@@ -161,11 +173,14 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
             }
         }
     } else {
-        // ------------------------------------------------------------------ epilogue (warps 2..5 of both CTAs)
+        // ------------------------------------------------------------------ epilogue (warps 2..9 of both CTAs)
+        // a warp reads the 32 TMEM lanes of its quarter (warp % 4) and one half of the tile's 256 columns
         const int quarter = warp & 3;
+        const int half = (warp - 2) >> 2;
+        constexpr int CHUNKS = TN / 64;          // chunks of 32 columns per warp
         uint32_t acc = 0, acc_phase = 0;
         bool ok = true;
-        constexpr int RUN = 256;                 // places of the candidate list a warp reserves at a time
+        constexpr int RUN = 128;                 // places of the candidate list a warp reserves at a time
         unsigned long long run_base = 0;         // the warp's current run (the same in all lanes)
         int run_left = 0;
         int last_I = -1;
@@ -174,31 +189,37 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
         for (long long p = p_begin; p < p_end && ok; p += p_step) {
             int I, t;
             pair_to_tiles(pair_list, p, &I, &t);
-            const long long n0 = static_cast<long long>(t) * TN;
+            const long long n0 = static_cast<long long>(t) * TN + half * (TN / 2);
             if (I != last_I) {
                 last_I = I;
                 gi = static_cast<long long>(I) * (2 * TM) + static_cast<long long>(rank) * TM + quarter * 32 + lane;
                 // a row takes part if it is live and not a member of C_cur (those are never merged into others)
                 row_ok = gi < N && valid[gi] != 0 && !(two_sets && seed[gi] != 0);
             }
-            // the tile's 256 rows j as bit masks per chunk of 32 (the same in all lanes): live, member of C_cur
-            uint32_t live_mask[TN / 32], seed_mask[TN / 32];
+            // the warp's 128 rows j as bit masks per chunk of 32 (the same in all lanes): live, member of C_cur
+            uint32_t live_mask[CHUNKS], seed_mask[CHUNKS];
 #pragma unroll
-            for (int h = 0; h < TN / 32; ++h) {
+            for (int h = 0; h < CHUNKS; ++h) {
                 const long long gj = n0 + h * 32 + lane;
                 const bool lv = gj < N && valid[gj] != 0;
                 live_mask[h] = __ballot_sync(0xFFFFFFFFu, lv);
                 seed_mask[h] = two_sets ? __ballot_sync(0xFFFFFFFFu, lv && seed[gj] != 0) : 0u;
             }
-            if (!mbar_wait(&sh->acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+            if (!mbar_wait_idle(&sh->acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
             tcgen05_fence_after();
-            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * TN;
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * TN + half * (TN / 2);
             uint32_t ra[32], rb[32];
             auto scan = [&](uint32_t (&r)[32], int ch) {
-                float m = __uint_as_float(r[0]);
+                // the largest of the row's 32 values, by four independent chains
+                float m0 = __uint_as_float(r[0]), m1 = __uint_as_float(r[1]), m2 = __uint_as_float(r[2]), m3 = __uint_as_float(r[3]);
 #pragma unroll
-                for (int j = 1; j < 32; ++j) m = fmaxf(m, __uint_as_float(r[j]));
-                const bool look = row_ok && m > theta_filter;
+                for (int j = 4; j < 32; j += 4) {
+                    m0 = fmaxf(m0, __uint_as_float(r[j]));
+                    m1 = fmaxf(m1, __uint_as_float(r[j + 1]));
+                    m2 = fmaxf(m2, __uint_as_float(r[j + 2]));
+                    m3 = fmaxf(m3, __uint_as_float(r[j + 3]));
+                }
+                const bool look = row_ok && fmaxf(fmaxf(m0, m1), fmaxf(m2, m3)) > theta_filter;
                 if (!__any_sync(0xFFFFFFFFu, look)) return;            // the common case: nothing above the filter
                 // which values of this row are pairs of the sweep
                 uint32_t take = 0;
@@ -213,17 +234,20 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
                         if (__uint_as_float(r[j]) > theta_filter) take |= 1u << j;
                     take &= ok_mask;
                 }
-                // places in the warp's reserved run of the candidate list: one global atomic per RUN places
-                // instead of one per row (a single counter that every warp hits would serialise them)
+                // places in the warp's reserved run of the candidate list (one global atomic per RUN places: a single
+                // counter that every row hits would serialise them).  Few rows of a chunk hold pairs, so their places
+                // are dealt by walking the lanes that have some.
+                uint32_t holders = __ballot_sync(0xFFFFFFFFu, take != 0u);
+                if (holders == 0u) return;
                 const int mine = __popc(take);
-                int incl = mine;
-#pragma unroll
-                for (int o = 1; o < 32; o <<= 1) {
-                    const int y = __shfl_up_sync(0xFFFFFFFFu, incl, o);
-                    if (lane >= o) incl += y;
+                int before = 0, total = 0;
+                while (holders) {
+                    const int src = __ffs(holders) - 1;
+                    holders &= holders - 1u;
+                    const int cnt = __shfl_sync(0xFFFFFFFFu, mine, src);
+                    if (src < lane) before += cnt;
+                    total += cnt;
                 }
-                const int total = __shfl_sync(0xFFFFFFFFu, incl, 31);
-                if (total == 0) return;
                 if (total > run_left) {
                     // give the rest of the old run back as empty records and take a new one
                     for (int t = lane; t < run_left; t += 32)
@@ -235,31 +259,31 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
                     run_left = want;
                     if (run_base + want > max_cand && lane == 0) ctl->overflow = 1;
                 }
-                unsigned long long pos = run_base + static_cast<unsigned long long>(incl - mine);
-#pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    if ((take >> j) & 1u) {
-                        if (pos < max_cand) {
-                            MergeCandidate cd;
-                            cd.i = static_cast<int32_t>(gi);
-                            cd.j = static_cast<int32_t>(n0 + ch * 32 + j);
-                            cd.sim = __uint_as_float(r[j]);
-                            cand[pos] = cd;
-                        }
-                        ++pos;
+                // the exact check writes the similarity of the pairs it confirms; the filter's value is not kept
+                unsigned long long pos = run_base + static_cast<unsigned long long>(before);
+                while (take) {
+                    const int j = __ffs(take) - 1;
+                    take &= take - 1u;
+                    if (pos < max_cand) {
+                        MergeCandidate cd;
+                        cd.i = static_cast<int32_t>(gi);
+                        cd.j = static_cast<int32_t>(n0 + ch * 32 + j);
+                        cd.sim = 0.0f;
+                        cand[pos] = cd;
                     }
+                    ++pos;
                 }
                 run_base += static_cast<unsigned long long>(total);
                 run_left -= total;
             };
             tmem_ld_32x32(taddr, ra);
 #pragma unroll 1
-            for (int ch = 0; ch < TN / 32; ch += 2) {
+            for (int ch = 0; ch < CHUNKS; ch += 2) {
                 tmem_ld_fence(ra);
                 tmem_ld_32x32(taddr + (ch + 1) * 32, rb);
                 scan(ra, ch);
                 tmem_ld_fence(rb);
-                if (ch + 2 < TN / 32) tmem_ld_32x32(taddr + (ch + 2) * 32, ra);
+                if (ch + 2 < CHUNKS) tmem_ld_32x32(taddr + (ch + 2) * 32, ra);
                 scan(rb, ch + 1);
             }
             tcgen05_fence_before();
@@ -301,7 +325,7 @@ __global__ void split_bf16_kernel(const float *__restrict__ x, __nv_bfloat16 *__
         l[k] = __float2bfloat16_rn(f[k] - __bfloat162float(h[k]));
     }
     *reinterpret_cast<uint2 *>(hi + 4 * i) = *reinterpret_cast<const uint2 *>(h);
-    *reinterpret_cast<uint2 *>(lo + 4 * i) = *reinterpret_cast<const uint2 *>(l);
+    if (lo) *reinterpret_cast<uint2 *>(lo + 4 * i) = *reinterpret_cast<const uint2 *>(l);
 }
 
 // One warp per provisional candidate: exact similarity of the fp32 vectors (products and sums in fp64).  The pair
@@ -388,15 +412,19 @@ siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, i
         encode = reinterpret_cast<tcm::EncodeTiledFn>(fn);
     }
     const size_t elems = static_cast<size_t>(rows) * c->dim;
-    const int split = rows_bf16 ? 0 : 1;           // rows that ARE bf16 values need no second part
+    // rows that ARE bf16 values need no second part.  fp32 rows: by default the sweep is a FILTER on the rounded rows
+    // alone (one MMA per K step, half the operand bytes) with a margin that covers the rounding, and the exact check
+    // below decides; with three parts the margin is the one of the fp32 sums and fewer pairs reach the check.
+    const int split = (!rows_bf16 && c->merge_sweep_parts == 3) ? 1 : 0;
+    const float margin = (rows_bf16 || split) ? tcm::FILTER_MARGIN : tcm::one_part_margin(c->dim);
     const __nv_bfloat16 *hi, *lo;
-    if (split) {
-        __nv_bfloat16 *h = scr->take<__nv_bfloat16>(elems), *l = scr->take<__nv_bfloat16>(elems);
+    if (!rows_bf16) {
+        __nv_bfloat16 *h = scr->take<__nv_bfloat16>(elems), *l = split ? scr->take<__nv_bfloat16>(elems) : nullptr;
         const long long n4 = static_cast<long long>(elems / 4);
         tcm::split_bf16_kernel<<<static_cast<unsigned>((n4 + 255) / 256), 256, 0, s>>>(X, h, l, n4);
         SISO_LAUNCHED(c);
         hi = h;
-        lo = l;
+        lo = split ? l : h;
     } else {
         hi = lo = static_cast<const __nv_bfloat16 *>(rows_bf16);
     }
@@ -433,7 +461,7 @@ siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, i
         c->merge_tensor_attr_set = true;
     }
     tcm::merge_sweep_tensor_kernel<<<static_cast<unsigned>(2 * used), tcm::THREADS, tcm::SMEM_BYTES, s>>>(
-        map_hi, map_lo, valid, seed, N, c->dim, pair_list, n_pairs, theta_c - tcm::FILTER_MARGIN, split,
+        map_hi, map_lo, valid, seed, N, c->dim, pair_list, n_pairs, theta_c - margin, split,
         static_cast<MergeCtlView *>(ctl), static_cast<MergeCandidate *>(cand), max_cand, c->status);
     SISO_LAUNCHED(c);
     tcm::merge_verify_kernel<<<8 * c->sm_count, 256, 0, s>>>(static_cast<const MergeCtlView *>(ctl), X, c->dim, theta_c,

@@ -47,6 +47,17 @@ __device__ __forceinline__ bool mbar_try_wait(uint64_t *bar, uint32_t parity) {
         : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
     return ok != 0;
 }
+// the same test with the default (CTA-scope) acquire: for barriers completed by this CTA's own asynchronous work
+// (TMA bytes, tcgen05.commit), whose results the waiting thread does not read through generic loads of a peer's memory
+__device__ __forceinline__ bool mbar_try_wait_cta(uint64_t *bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(smem_u32(bar)), "r"(parity) : "memory");
+    return ok != 0;
+}
 // Bounded wait: false if `limit` polls ran out (the flag is then set) or another role has already given up.
 __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t limit = SPIN_LIMIT) {
     for (uint32_t it = 0; it < limit; ++it) {
@@ -55,6 +66,17 @@ __device__ __forceinline__ bool mbar_wait(uint64_t *bar, uint32_t parity, volati
             if (*abort_flag) return false;
             __nanosleep(64);
         }
+    }
+    *abort_flag = 1;
+    return false;
+}
+// Bounded wait of a role that expects to wait long (an epilogue warp waiting for a whole tile): it sleeps between polls,
+// so that it takes no issue slots from the MMA-issuing warp that shares its scheduler.  At most limit / 16 polls.
+__device__ __forceinline__ bool mbar_wait_idle(uint64_t *bar, uint32_t parity, volatile int *abort_flag, uint32_t limit = SPIN_LIMIT) {
+    for (uint32_t it = 0; it < limit / 16u; ++it) {
+        if (mbar_try_wait_cta(bar, parity)) return true;
+        __nanosleep(96);
+        if ((it & 63u) == 63u && *abort_flag) return false;
     }
     *abort_flag = 1;
     return false;
