@@ -1,16 +1,16 @@
 // Pairwise similarity sweep of MergeCentroids (Algorithm 1: every entry against the earlier entries of C_new) as a
 // dense contraction on the tensor cores, for fp32 vectors.
 //
-// An fp32 value x is split as x = hi + lo + r with hi = bf16(x), lo = bf16(x - hi), |r| <= 2^-18 |x|.  The sweep
+// An fp32 value x is split as x = hi + lo + r with hi = bf16(x), lo = bf16(x - hi), |r| <= 2^-16 |x|.  The sweep
 // accumulates hi_i.hi_j + hi_i.lo_j + lo_i.hi_j in fp32 on tcgen05 (three MMAs per 16 K-elements, one TMEM
-// accumulator); what it leaves out (lo.lo, the r terms) and the fp32 accumulation stay below 3e-5 for unit
+// accumulator); what it leaves out (lo.lo, the r terms) and the fp32 accumulation stay below 6e-5 for unit
 // vectors.  So the tensor cores only FILTER: every pair whose approximate similarity exceeds theta_C - 1e-4
 // becomes a provisional candidate, and merge_verify_kernel recomputes exactly these pairs from the fp32 vectors
 // in fp64 and keeps those whose exact similarity exceeds theta_C.  The decisions are therefore those of an exact
 // fp64 sweep; the tensor cores do the 2 N^2 D flops, the exact arithmetic touches the few candidates only.
 //
 // By default even less is asked of the tensor cores: the rows rounded to bf16 are multiplied ONCE (one MMA per 16
-// K-elements, half the operand bytes) and the filter margin is widened to the bound of that rounding (one_part_margin);
+// K-elements, half the operand bytes) and the filter margin is widened to the bound of that rounding (one_part_margin, 7.9e-3);
 // a few more pairs reach the exact check, the decisions stay the same.
 //
 // Kernel layout (CTA pairs, cta_group::2, as in the large-batch lookup): a cluster works on 256 rows i x 256 rows j
@@ -52,10 +52,11 @@ constexpr uint32_t OPER_BYTES = TM * TK * 2;              // 16 KiB: 128 rows x 
 constexpr uint32_t RING_BYTES = 12 * OPER_BYTES;          // six stages of (hi_i, hi_j half) or three of (hi_i, lo_i, hi_j half, lo_j half)
 constexpr uint32_t SMEM_BYTES = RING_BYTES + 1024 + 4096;
 constexpr uint32_t TMEM_COLS = ACC_STAGES * TN;
-constexpr float FILTER_MARGIN = 1e-4f;             // three-part products (or rows that are bf16 values): rounding of the fp32 sums
-// One-part filter on fp32 rows: with x^ = bf16(x), |x.y - x^.y^| <= (2u + u^2) |x| |y| for u = 2^-9 (round to nearest),
-// 3.93e-3 for norms up to 1.002; the fp32 accumulation adds at most dim * 2^-23.
-__host__ inline float one_part_margin(int dim) { return 4.0e-3f + 1.2e-7f * static_cast<float>(dim); }
+constexpr float FILTER_MARGIN = 1e-4f;             // three-part products (or rows that are bf16 values): left-out terms and fp32 sums
+// One-part filter on fp32 rows.  bf16 keeps 8 significant bits: with x^ = bf16(x), |x - x^| <= u |x| for u = 2^-8 (round
+// to nearest), so |x.y - x^.y^| <= (2u + u^2) |x| |y| = 7.86e-3 for norms up to 1.002; the fp32 accumulator is rounded
+// once per 16 K-elements (dim / 16 roundings of 2^-23 of a sum below 1).
+__host__ inline float one_part_margin(int dim) { return 7.9e-3f + 1.0e-8f * static_cast<float>(dim); }
 
 // D fp32, A and B bf16, K-major, N = 256, M = 256 (128 rows per CTA of the pair)
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(TN >> 3) << 17) |
@@ -74,17 +75,21 @@ __device__ __forceinline__ void pair_to_tiles(const uint32_t *__restrict__ pair_
     *t = static_cast<int>(v & 0xFFFFu);
 }
 
+// SPLIT: three products of bf16 parts per pair and K step (false: one product of the rounded rows); a template
+// parameter so that the MMA-issuing thread runs straight-line code
+template <bool SPLIT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(THREADS, 1)
 merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __grid_constant__ CUtensorMap map_lo,
                           const uint8_t *__restrict__ valid, const uint8_t *__restrict__ seed, int64_t N, int D,
-                          const uint32_t *__restrict__ pair_list, long long n_pairs, float theta_filter, int split, MergeCtlView *ctl,
+                          const uint32_t *__restrict__ pair_list, long long n_pairs, float theta_filter, MergeCtlView *ctl,
                           MergeCandidate *__restrict__ cand, unsigned long long max_cand, int *status) {
     extern __shared__ uint8_t smem_raw[];
     uint8_t *stage_mem = reinterpret_cast<uint8_t *>((reinterpret_cast<uintptr_t>(smem_raw) + 1023) & ~static_cast<uintptr_t>(1023));
     Shared *sh = reinterpret_cast<Shared *>(stage_mem + RING_BYTES);
-    const uint32_t STAGES = split ? 3u : 6u;
-    const uint32_t STAGE_BYTES = split ? 4 * OPER_BYTES : 2 * OPER_BYTES;
-    const uint32_t OFF_J = split ? 2 * OPER_BYTES : OPER_BYTES;       // where the rows j start inside a stage
+    constexpr bool split = SPLIT;
+    constexpr uint32_t STAGES = split ? 3u : 6u;
+    constexpr uint32_t STAGE_BYTES = split ? 4 * OPER_BYTES : 2 * OPER_BYTES;
+    constexpr uint32_t OFF_J = split ? 2 * OPER_BYTES : OPER_BYTES;       // where the rows j start inside a stage
     volatile int *abort_flag = &sh->abort_flag;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
@@ -159,7 +164,7 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
                     for (int kk = 0; kk < TK / 16; ++kk) {
                         const uint64_t o = static_cast<uint64_t>(2 * kk);
                         umma_bf16_pair(d_tmem, a_hi + o, b_hi + o, IDESC, (ks | kk) ? 1u : 0u);
-                        if (split) {
+                        if constexpr (split) {
                             umma_bf16_pair(d_tmem, a_hi + o, b_lo + o, IDESC, 1u);
                             umma_bf16_pair(d_tmem, a_lo + o, b_hi + o, IDESC, 1u);
                         }
@@ -205,7 +210,7 @@ merge_sweep_tensor_kernel(const __grid_constant__ CUtensorMap map_hi, const __gr
                 live_mask[h] = __ballot_sync(0xFFFFFFFFu, lv);
                 seed_mask[h] = two_sets ? __ballot_sync(0xFFFFFFFFu, lv && seed[gj] != 0) : 0u;
             }
-            if (!mbar_wait_idle(&sh->acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
+            if (!mbar_wait(&sh->acc_full[acc], acc_phase, abort_flag)) { ok = false; break; }
             tcgen05_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16) + acc * TN + half * (TN / 2);
             uint32_t ra[32], rb[32];
@@ -457,11 +462,13 @@ siso_status_t launch_pair_sweep_tensor(Cache *c, Scratch *scr, const float *X, i
     SISO_CUDA(cudaMemcpyAsync(pair_list, list.data(), sizeof(uint32_t) * list.size(), cudaMemcpyHostToDevice, s));
     const long long used = std::max<long long>(1, std::min<long long>(n_pairs, c->sm_count / 2));
     if (!c->merge_tensor_attr_set) {
-        SISO_CUDA(cudaFuncSetAttribute(tcm::merge_sweep_tensor_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, tcm::SMEM_BYTES));
+        SISO_CUDA(cudaFuncSetAttribute(tcm::merge_sweep_tensor_kernel<false>, cudaFuncAttributeMaxDynamicSharedMemorySize, tcm::SMEM_BYTES));
+        SISO_CUDA(cudaFuncSetAttribute(tcm::merge_sweep_tensor_kernel<true>, cudaFuncAttributeMaxDynamicSharedMemorySize, tcm::SMEM_BYTES));
         c->merge_tensor_attr_set = true;
     }
-    tcm::merge_sweep_tensor_kernel<<<static_cast<unsigned>(2 * used), tcm::THREADS, tcm::SMEM_BYTES, s>>>(
-        map_hi, map_lo, valid, seed, N, c->dim, pair_list, n_pairs, theta_c - margin, split,
+    auto kernel = split ? tcm::merge_sweep_tensor_kernel<true> : tcm::merge_sweep_tensor_kernel<false>;
+    kernel<<<static_cast<unsigned>(2 * used), tcm::THREADS, tcm::SMEM_BYTES, s>>>(
+        map_hi, map_lo, valid, seed, N, c->dim, pair_list, n_pairs, theta_c - margin,
         static_cast<MergeCtlView *>(ctl), static_cast<MergeCandidate *>(cand), max_cand, c->status);
     SISO_LAUNCHED(c);
     tcm::merge_verify_kernel<<<8 * c->sm_count, 256, 0, s>>>(static_cast<const MergeCtlView *>(ctl), X, c->dim, theta_c,

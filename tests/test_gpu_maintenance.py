@@ -13,6 +13,17 @@ siso = pytest.importorskip("paper_2508_18736_b200")
 VEC_TOL = {"f32": 1e-6, "bf16": 2.5e-4}       # max-abs on vector elements (1 ulp of bf16 at 1/sqrt(D) magnitudes)
 
 
+
+# the pairwise sweep of a merge: CUDA cores, or tensor cores as a filter (one bf16 product, or three bf16 parts) + exact check
+SWEEPS = [pytest.param((siso.PATH_SIMT, 1), id="cuda-cores"), pytest.param((siso.PATH_TENSOR, 1), id="tensor-one-part"),
+          pytest.param((siso.PATH_TENSOR, 3), id="tensor-three-parts")]
+
+
+def set_sweep(cache, sweep):
+    cache.set_option(siso.OPT_MERGE_PATH, sweep[0])
+    cache.set_option(siso.OPT_MERGE_SWEEP_PARTS, sweep[1])
+
+
 def state_np(cache):
     st = cache.export()
     torch.cuda.synchronize()
@@ -137,12 +148,12 @@ def test_update_counts_accesses_after_decay_reset():
 @pytest.mark.parametrize("dtype,mode,theta_c,weighted", [
     ("f32", "T", 0.90, True), ("f32", "P", 0.90, True), ("f32", "P", 0.86, False), ("bf16", "P", 0.90, True),
 ])
-@pytest.mark.parametrize("sweep", [siso.PATH_SIMT, siso.PATH_TENSOR])
+@pytest.mark.parametrize("sweep", SWEEPS)
 def test_self_merge_matches_oracle(dtype, mode, theta_c, weighted, sweep):
     w = W.config(3, n_centroids=1500, dim=136, n_clusters=90, mode=mode, sigma=0.06, dtype=dtype)
     sizes = np.random.default_rng(9).integers(1, 9, 1500).astype(np.float64)
     cache, ora = make_pair(w, capacity=1536, sizes=sizes)
-    cache.set_option(siso.OPT_MERGE_PATH, sweep)       # CUDA-core sweep, or tensor-core filter + exact check
+    set_sweep(cache, sweep)
     entry = ora.master.copy()
     flags = siso.MERGE_WEIGHTED_MEAN if weighted else siso.MERGE_SIZES_ONLY
     for rounds in range(40):
@@ -174,11 +185,42 @@ def test_self_merge_matches_oracle(dtype, mode, theta_c, weighted, sweep):
     cache.check_status()
 
 
-@pytest.mark.parametrize("sweep", [siso.PATH_SIMT, siso.PATH_TENSOR])
+@pytest.mark.parametrize("sweep", SWEEPS)
+def test_merge_keeps_pairs_whose_bf16_products_fall_below_the_threshold(sweep):
+    """Rows of +-1/sqrt(232): that magnitude loses 0.34 % when rounded to bf16 (nearly the worst case, 2^-8), so the
+    product of the ROUNDED rows of a planted pair lies 6e-3 below the exact similarity.  theta_C sits 1e-4 under the
+    exact similarity, so the pair merges (the oracle says so); a tensor-core filter must keep it for the exact check."""
+    N, D, flips = 4096, 232, 11
+    rng = np.random.default_rng(77)
+    m = np.float32(1.0 / np.sqrt(D))
+    rows = np.where(rng.random((N, D)) < 0.5, -m, m).astype(np.float32)
+    planted = 48
+    for p in range(planted):
+        a, b = 40 * p + 3, 40 * p + 29
+        rows[b] = rows[a]
+        rows[b, rng.choice(D, flips, replace=False)] *= -1
+    exact = float(rows[3].astype(np.float64) @ rows[29].astype(np.float64))
+    rounded = torch.from_numpy(rows[[3, 29]]).to(torch.bfloat16).to(torch.float64)
+    assert exact - float(rounded[0] @ rounded[1]) > 5e-3            # far outside a margin meant for fp32 rounding
+    theta_c = float(np.float32(exact - 1e-4))
+    cache = siso.SisoCache(N, D, "f32")
+    set_sweep(cache, sweep)
+    cache.insert(torch.from_numpy(rows).cuda())
+    ora = oracle.OracleCache(N, D, "f32")
+    ora.insert(rows)
+    mm, n = cache.merge(theta_c, siso.MERGE_WEIGHTED_MEAN)
+    o_mm, o_n = ora.merge(theta_c, True)
+    assert o_n == planted and n == o_n
+    assert (mm.cpu().numpy() == o_mm).all()
+    assert_state_equal(cache, ora, "f32", "planted pairs")
+    cache.check_status()
+
+
+@pytest.mark.parametrize("sweep", SWEEPS)
 def test_merge_extremes_holes_and_overflow(sweep):
     w = W.config(3, n_centroids=700, dim=64, n_clusters=30, mode="P")
     cache, ora = make_pair(w, capacity=1000)
-    cache.set_option(siso.OPT_MERGE_PATH, sweep)
+    set_sweep(cache, sweep)
     victims = cache.evict(50).cpu().numpy()
     assert (victims == ora.evict(50)).all()
     mm, n = cache.merge(1.0, siso.MERGE_WEIGHTED_MEAN)
@@ -199,7 +241,7 @@ def test_merge_extremes_holes_and_overflow(sweep):
 
 
 @pytest.mark.parametrize("dtype,weighted", [("f32", True), ("bf16", False)])
-@pytest.mark.parametrize("sweep", [siso.PATH_SIMT, siso.PATH_TENSOR])
+@pytest.mark.parametrize("sweep", SWEEPS)
 def test_two_set_merge_matches_oracle(dtype, weighted, sweep):
     """Algorithm 1 as printed: C_cur = the cache, C_repo = new rows; holes in the cache interleave the two."""
     w = W.config(3, n_centroids=1400, dim=136, n_clusters=80, mode="P", sigma=0.06, dtype=dtype)
@@ -209,7 +251,7 @@ def test_two_set_merge_matches_oracle(dtype, weighted, sweep):
     repo_sizes = rng.integers(1, 5, 600).astype(np.float64)
     cap = 1500
     cache = siso.SisoCache(cap, w.dim, dtype)
-    cache.set_option(siso.OPT_MERGE_PATH, sweep)
+    set_sweep(cache, sweep)
     ora = oracle.OracleCache(cap, w.dim, dtype)
     cache.insert(to_dev(cur, dtype), torch.from_numpy(cur_sizes))
     ora.insert(cur, sizes=cur_sizes)
