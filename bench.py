@@ -437,7 +437,14 @@ def small_batch_sweep(torch, cache, queries_dev, rows, dim, peaks, batches=(1, 8
         q = queries_dev[:b].contiguous()
         ms = _time_ms(torch, lambda: cache.lookup(q, 0.86, 1), steps, warm)
         gbs = rows * dim * 2 / ms / 1e6
-        out.append({"batch": b, "us": round(ms * 1e3, 2), "GB/s": round(gbs, 1), "frac": round(gbs / peaks["hbm_gbs"], 4)})
+        rec = {"batch": b, "us": round(ms * 1e3, 2), "GB/s": round(gbs, 1), "frac": round(gbs / peaks["hbm_gbs"], 4)}
+        if b >= 256:
+            # at 256 queries the sweep sits on the ridge (flop per centroid byte = 256): say where it stands against the
+            # tensor roof too; the binding roof is the larger of the two times
+            tf = 2.0 * b * rows * dim / ms / 1e9
+            rec["TFLOP/s"] = round(tf, 1)
+            rec["frac_tensor"] = round(tf / peaks["bf16_tflops"], 4)
+        out.append(rec)
     return out
 
 
