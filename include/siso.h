@@ -297,6 +297,10 @@ siso_status_t siso_select_evict_planned(const uint64_t *d_keys, int32_t n_lists,
  * All device pointers, no handle, current device, asynchronous on `stream`; the caller reads *d_count (one 8-byte copy)
  * to size the cold lookup.  SISO_ERR_INVALID_ARG on bad sizes or NULL pointers, nothing written. */
 double siso_tier_exit_sim(double sep_sim, double norm_slack);
+/* *h_max_dev = the largest | |v| - 1 | over the live entries, taken on the vectors that lookups read (fp64 sums, rounded
+ * up; +infinity if an entry holds a NaN; 0 for an empty cache): the smallest norm_slack that is true of the entries.
+ * Synchronises `stream`. */
+siso_status_t siso_norm_deviation(siso_cache_t *c, double *h_max_dev, void *stream);
 siso_status_t siso_tier_select(const uint64_t *d_hot_keys, int64_t n_queries, float exit_sim, const void *d_queries,
                                int64_t row_bytes, void *d_cold_queries, int32_t *d_rows, int64_t *d_count, void *stream);
 siso_status_t siso_tier_finish(const uint64_t *d_hot_keys, int64_t n_queries, float exit_sim, const uint64_t *d_cold_keys,

@@ -27,7 +27,7 @@ EXPORTS = ["siso_cache_create", "siso_cache_destroy", "siso_set_option", "siso_i
            "siso_route", "siso_evict_keys", "siso_select_evict", "siso_evict_slots", "siso_selftest_wait_timeout",
            "siso_measure_fp32_fma", "siso_pair_sweep_block", "siso_merge_resolve", "siso_merge_pack",
            "siso_merge_apply_shard", "siso_tier_build", "siso_tier_work_bytes", "siso_tier_lookup", "siso_free_slots",
-           "siso_shard_plan", "siso_route_planned", "siso_select_evict_planned"]
+           "siso_shard_plan", "siso_route_planned", "siso_select_evict_planned", "siso_norm_deviation"]
 
 
 class SisoError(RuntimeError):
@@ -89,6 +89,7 @@ def load_library(path: Optional[str] = None) -> ctypes.CDLL:
     L.siso_select_evict.argtypes = [vp, i32, i64, i64, vp, vp]
     L.siso_evict_slots.argtypes = [vp, vp, i64, i64, u32, vp]
     L.siso_free_slots.argtypes = [vp, vp, vp]
+    L.siso_norm_deviation.argtypes = [vp, ctypes.POINTER(ctypes.c_double), vp]
     L.siso_shard_plan.argtypes = [vp, i64, vp, i32, i32, vp, vp]
     L.siso_route_planned.argtypes = [vp, i64, vp, i64, i64, i64, vp, vp, vp, vp, vp]
     L.siso_select_evict_planned.argtypes = [vp, i32, i64, vp, vp, vp]
@@ -324,6 +325,12 @@ class SisoCache:
         v = victims.to(device=self._dev, dtype=torch.int64).contiguous()
         self._check(self._lib.siso_evict_slots(self._h, _ptr(v), v.numel(), int(slot_offset), flags, _stream(stream)),
                     "siso_evict_slots")
+
+    def norm_deviation(self, stream=None) -> float:
+        """Largest | |v| - 1 | over the live entries' lookup vectors (see siso_norm_deviation)."""
+        out = ctypes.c_double(0.0)
+        self._check(self._lib.siso_norm_deviation(self._h, ctypes.byref(out), _stream(stream)), "siso_norm_deviation")
+        return float(out.value)
 
     def free_slots(self, stream=None) -> torch.Tensor:
         """[1] int64 on the device: capacity - occupancy, without a host read (see siso_free_slots)."""

@@ -131,6 +131,31 @@ check_unit_rows_kernel(const T *__restrict__ rows, long long n, int D, const uin
     }
 }
 
+// the largest | |v| - 1 | over the live rows of the vectors that lookups read (fp64 sums), as the bit pattern of a
+// non-negative float (those order like unsigned integers); a row with a NaN counts as infinitely far
+template <typename T>
+__global__ void __launch_bounds__(256)
+norm_deviation_kernel(const T *__restrict__ rows, const uint8_t *__restrict__ valid, long long n, int D, unsigned int *out_bits) {
+    const int lane = threadIdx.x & 31;
+    const long long warps = static_cast<long long>(gridDim.x) * (blockDim.x >> 5);
+    for (long long r = static_cast<long long>(blockIdx.x) * (blockDim.x >> 5) + (threadIdx.x >> 5); r < n; r += warps) {
+        if (!valid[r]) continue;
+        double ss = 0.0;
+        for (int d = lane; d < D; d += 32) {
+            float v;
+            if constexpr (sizeof(T) == 2) v = __bfloat162float(rows[r * D + d]); else v = rows[r * D + d];
+            ss += static_cast<double>(v) * static_cast<double>(v);
+        }
+#pragma unroll
+        for (int o = 16; o >= 1; o >>= 1) ss += __shfl_xor_sync(0xFFFFFFFFu, ss, o);
+        if (lane == 0) {
+            const double dev = fabs(sqrt(ss) - 1.0);
+            const float up = dev == dev ? __double2float_ru(dev) : __int_as_float(0x7F800000);
+            atomicMax(out_bits, __float_as_uint(up));
+        }
+    }
+}
+
 // thresholds must be numbers; hit flags 0 or 1; slots of hits inside the cache
 __global__ void check_batch_args_kernel(const float *__restrict__ theta, const uint8_t *__restrict__ hit, const int32_t *__restrict__ idx,
                                         int idx_stride, long long n, long long capacity, int *status) {
@@ -478,6 +503,29 @@ siso_status_t siso_select_evict(const uint64_t *d_keys, int32_t n_lists, int64_t
     if (!d_victims || (n > 0 && !d_keys)) return SISO_ERR_INVALID_ARG;
     return launch_evict_select(reinterpret_cast<const unsigned long long *>(d_keys), n_lists, n, n_take,
                                reinterpret_cast<long long *>(d_victims), static_cast<cudaStream_t>(stream));
+}
+
+siso_status_t siso_norm_deviation(siso_cache_t *c, double *h_max_dev, void *stream) {
+    if (!c || !h_max_dev) return SISO_ERR_INVALID_ARG;
+    SISO_CUDA(cudaSetDevice(c->device));
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    Scratch scr;
+    SISO_TRY(scratch_reserve(c, 256, s, &scr));
+    unsigned int *bits = scr.take<unsigned int>(1);
+    SISO_CUDA(cudaMemsetAsync(bits, 0, sizeof(unsigned int), s));
+    const unsigned blocks = static_cast<unsigned>(std::min<int64_t>((c->capacity + 7) / 8, 8ll * c->sm_count));
+    if (c->dtype == SISO_F32)
+        norm_deviation_kernel<float><<<blocks, 256, 0, s>>>(static_cast<const float *>(c->vecs), c->valid, c->capacity, c->dim, bits);
+    else
+        norm_deviation_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>(static_cast<const __nv_bfloat16 *>(c->vecs), c->valid, c->capacity, c->dim, bits);
+    SISO_LAUNCHED(c);
+    unsigned int h = 0;
+    SISO_CUDA(cudaMemcpyAsync(&h, bits, sizeof(h), cudaMemcpyDeviceToHost, s));
+    SISO_CUDA(cudaStreamSynchronize(s));
+    float f;
+    memcpy(&f, &h, sizeof(f));
+    *h_max_dev = static_cast<double>(f);
+    return SISO_OK;
 }
 
 siso_status_t siso_free_slots(siso_cache_t *c, int64_t *d_free, void *stream) {

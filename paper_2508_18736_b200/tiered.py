@@ -28,8 +28,14 @@ class TieredCache:
         (bf16 rounding of unit vectors: about 1e-3).  The exit rule is only exact if the bound holds, and nothing in the
         cache's history guarantees it for good (a weighted merge recentres survivors, a two-set merge never compares
         the old entries with each other, later inserts and updates move vectors), so by default the build CHECKS it:
-        every hot/cold pair is swept (tensor cores + exact fp64 check) and a pair above sep_sim raises ValueError.
+        every hot/cold pair is swept (tensor cores + exact fp64 check) and a pair above sep_sim raises ValueError, and so
+        does an entry whose norm is further from 1 than norm_slack (the queries' norms stay the caller's promise).
         certify=False skips the check for a caller that has just established the bound some other way."""
+        if certify:
+            dev = cache.norm_deviation()
+            if not dev <= norm_slack:
+                raise ValueError(f"entries deviate from unit norm by up to {dev:.3g}, more than norm_slack = {norm_slack}: "
+                                 "the early exit would not be exact")
         occ = int(cache.stats()["occupancy"])
         hot_rows = max(0, min(int(hot_rows), occ))
         dev = cache._dev.index

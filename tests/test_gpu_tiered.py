@@ -59,6 +59,12 @@ def test_tiered_lookup_equals_whole_cache(dtype, n, n_clusters, dim, hot):
     sep = float(S.max()) + 1e-9
     assert sep <= theta_c + (4e-3 if dtype == "bf16" else 1e-6) and slack < (4e-3 if dtype == "bf16" else 1e-5)
 
+    # the library measures the entries' side of that bound itself, and refuses a slack the entries do not meet
+    ent = float(np.abs(np.linalg.norm(widen64(stored[live]), axis=1) - 1).max())
+    dev = cache.norm_deviation()
+    assert ent <= dev <= ent * (1 + 1e-6) + 1e-12
+    with pytest.raises(ValueError):
+        siso.TieredCache(cache, hot, sep, 0.5 * dev)
     tiers = siso.TieredCache(cache, hot, sep, slack)
     # hot tier = what FilteringCentroids keeps when told to leave `hot` entries
     cold = np.sort(ora.evict(occ - hot))
