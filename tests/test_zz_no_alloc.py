@@ -20,8 +20,8 @@ pytestmark = pytest.mark.gpu
 siso = pytest.importorskip("paper_2508_18736_b200")
 
 
-@pytest.mark.parametrize("dtype,dim", [("bf16", 768), ("f32", 384)])
-def test_no_alloc_lookup_matches_ordinary_lookup_twice_in_a_row(dtype, dim):
+@pytest.mark.parametrize("dtype,dim,shift", [("bf16", 768, 0), ("f32", 384, 0), ("bf16", 768, 4)])
+def test_no_alloc_lookup_matches_ordinary_lookup_twice_in_a_row(dtype, dim, shift):
     cfg = 2 if dtype == "bf16" else 1
     w = W.config(cfg, n_centroids=5003, n_queries=16, dim=dim, n_clusters=200, mode="P", dtype=dtype)
     cent, q_all = to_dev(w.centroids, dtype), to_dev(w.queries, dtype)
@@ -32,6 +32,11 @@ def test_no_alloc_lookup_matches_ordinary_lookup_twice_in_a_row(dtype, dim):
     st = cache.export()
     cache.import_(st["master"], st["size"], st["access"], st["last"], valid, 0)
     cache.set_lookup_path(siso.PATH_STREAM)
+    if shift:       # a matrix that does not start on a 16-byte boundary: the kernel's scalar loads instead of 128-bit ones
+        buf = torch.empty(cent.numel() + shift, dtype=cent.dtype, device="cuda")
+        buf[shift:].copy_(cent.reshape(-1))
+        cent = buf[shift:].view(cent.shape)
+        assert cent.data_ptr() % 16 != 0
     theta_all = torch.from_numpy(w.theta).cuda()
     tol = TOL[dtype]
     # two calls in a row: 8 queries with k = 4, then 5 other queries with k = 8 and a scalar threshold
