@@ -69,8 +69,8 @@ typedef enum { SISO_F32 = 0, SISO_BF16 = 1 } siso_dtype_t;
 #define SISO_OPT_STREAM_LIST 7          /* 0 (default): on a full cache the fused streaming step takes its victims from an
                                          * eviction-order list kept across batches (no grid-wide barrier); 1: never */
 #define SISO_OPT_MERGE_SWEEP_PARTS 8    /* tensor-core pairwise sweep over fp32 rows (MergeCentroids, clustering).  1 (default): the rows
-                                         * rounded to bf16 are multiplied once, as a filter whose margin (7.9e-3 + 1e-8 dim)
-                                         * bounds the rounding for rows of norm <= 1.002, and every pair above the filter is then
+                                         * rounded to bf16 are multiplied once, as a filter whose margin (8.1e-3 + 1e-8 dim)
+                                         * bounds the rounding for rows of norm <= 1.01, and every pair above the filter is then
                                          * decided by its exact fp32 similarity; 3: three products of bf16 parts reproduce the
                                          * fp32 product to 1e-4 before the same exact decision.  The results are the same. */
 #define SISO_OPT_CHECKED 9              /* 1: checked mode.  What the library otherwise takes on trust is verified on the device before

@@ -10,7 +10,7 @@
 // fp64 sweep; the tensor cores do the 2 N^2 D flops, the exact arithmetic touches the few candidates only.
 //
 // By default even less is asked of the tensor cores: the rows rounded to bf16 are multiplied ONCE (one MMA per 16
-// K-elements, half the operand bytes) and the filter margin is widened to the bound of that rounding (one_part_margin, 7.9e-3);
+// K-elements, half the operand bytes) and the filter margin is widened to the bound of that rounding (one_part_margin, 8.1e-3);
 // a few more pairs reach the exact check, the decisions stay the same.
 //
 // Kernel layout (CTA pairs, cta_group::2, as in the large-batch lookup): a cluster works on 256 rows i x 256 rows j
@@ -54,9 +54,9 @@ constexpr uint32_t SMEM_BYTES = RING_BYTES + 1024 + 4096;
 constexpr uint32_t TMEM_COLS = ACC_STAGES * TN;
 constexpr float FILTER_MARGIN = 1e-4f;             // three-part products (or rows that are bf16 values): left-out terms and fp32 sums
 // One-part filter on fp32 rows.  bf16 keeps 8 significant bits: with x^ = bf16(x), |x - x^| <= u |x| for u = 2^-8 (round
-// to nearest), so |x.y - x^.y^| <= (2u + u^2) |x| |y| = 7.86e-3 for norms up to 1.002; the fp32 accumulator is rounded
+// to nearest), so |x.y - x^.y^| <= (2u + u^2) |x| |y| = 7.99e-3 for norms up to 1.01 (what checked mode accepts); the fp32 accumulator is rounded
 // once per 16 K-elements (dim / 16 roundings of 2^-23 of a sum below 1).
-__host__ inline float one_part_margin(int dim) { return 7.9e-3f + 1.0e-8f * static_cast<float>(dim); }
+__host__ inline float one_part_margin(int dim) { return 8.1e-3f + 1.0e-8f * static_cast<float>(dim); }
 
 // D fp32, A and B bf16, K-major, N = 256, M = 256 (128 rows per CTA of the pair)
 constexpr uint32_t IDESC = (1u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(TN >> 3) << 17) |
