@@ -250,3 +250,48 @@ def test_sharded_merge_equals_one_cache(dtype, n, dim, shards, weighted, theta_c
             p.close()
     for p in parts:
         p.close()
+
+
+def test_one_rank_nccl_group_runs_the_real_collectives():
+    """A process group of ONE rank over NCCL on this GPU: the exchanges of the sharded operations then go through
+    all_gather_into_tensor / all_reduce of the real backend (a ring step with one rank is a copy), and the results must
+    equal the plain cache's bit for bit: lookup, streaming steps, a MergeCentroids pass."""
+    import socket
+    import torch.distributed as dist
+    if dist.is_initialized():
+        pytest.skip("a process group is already initialised in this process")
+    with socket.socket() as s:
+        s.bind(("127.0.0.1", 0))
+        port = s.getsockname()[1]
+    try:
+        dist.init_process_group("nccl", init_method=f"tcp://127.0.0.1:{port}", rank=0, world_size=1,
+                                device_id=torch.device("cuda", torch.cuda.current_device()))
+    except Exception as e:      # the environment, not the library under test: no NCCL group can be made on this box
+        pytest.skip(f"NCCL process group could not be created here: {e}")
+    try:
+        sp = W.StreamSpec(capacity=300, dim=128, n_queries=128 * 10, batch=128, n_clusters=1200, zipf_s=1.1, reshuffle_every=640,
+                          theta=0.80, mode="P", dtype="bf16", seed=63)
+        stream = W.QueryStream(sp)
+        one = siso.ShardedCache(300, 128, "bf16")
+        assert one.world == 1 and one.rank == 0
+        plain = siso.SisoCache(300, 128, "bf16")
+        for t in range(10):
+            q = to_dev(stream.batch(t)[0], "bf16")
+            a = one.stream_step(q, float(sp.theta))
+            b = plain.stream_step(q, float(sp.theta))
+            assert (a[0].to(torch.int32) == b[0][:, 0]).all().item() and (a[2] == b[2]).all().item()
+            assert (a[3].to(torch.int32) == b[3]).all().item() and (a[4].to(torch.int32) == b[4]).all().item()
+        q = to_dev(stream.batch(3)[0], "bf16")
+        i1, s1, h1 = one.lookup(q, 0.8, 4)
+        i2, s2, h2 = plain.lookup(q, 0.8, 4)
+        assert (i1.to(torch.int32) == i2).all().item() and (s1 == s2).all().item() and (h1 == h2).all().item()
+        mm1, n1 = one.merge(0.75, siso.MERGE_WEIGHTED_MEAN)
+        mm2, n2 = plain.merge(0.75, siso.MERGE_WEIGHTED_MEAN)
+        assert n1 == n2 and (mm1 == mm2[:300]).all().item()
+        x, y = one.local.export(), plain.export()
+        assert all((x[k] == y[k]).all().item() for k in ("valid", "size", "master", "vecs"))
+        assert plain.stats()["evictions"] > 0
+        one.close()
+        plain.close()
+    finally:
+        dist.destroy_process_group()
