@@ -389,7 +389,7 @@ def run_ours(args):
     if not args.no_cpu_baseline and world == 1:
         import oracle
         oracle.build()
-        n_sample = max(1, min(B, 4 * cores))
+        n_sample = max(1, min(B, 8 * cores))
         t0 = time.perf_counter()
         o_idx, o_sim, o_hit = oracle.lookup(w.centroids, w.queries[:n_sample], w.theta[:n_sample], k)
         t = time.perf_counter() - t0
