@@ -445,6 +445,74 @@ def test_fused_streaming_maintenance_equals_separate_kernels_bit_for_bit():
         c.close()
 
 
+@pytest.mark.parametrize("seed", [11, 12, 13, 14, 15, 16])
+def test_three_forms_of_the_streaming_step_agree_on_random_shapes(seed):
+    """The fused step with the eviction-order list kept across batches (default), the fused step without it and the
+    separate kernels, on a random capacity / dim / batch size / threshold, with evictions (with and without decay),
+    merges and plain lookups + updates thrown in between the batches: every output of every batch and the whole state
+    must agree bit for bit (each form is also compared with the oracle elsewhere; this guards their equivalence where
+    the oracle is too slow to follow)."""
+    rng = np.random.default_rng(seed)
+    dtype = "bf16" if rng.random() < 0.7 else "f32"
+    cap = int(rng.choice([300, 1000, 4096, 9000]))
+    dim = int(rng.choice([64, 128, 264, 768]))
+    batch = int(rng.choice([1, 7, 64, 200, 256]))
+    nb = int(rng.integers(80, 160))
+    theta = float(rng.choice([0.7, 0.8, 0.86, 0.9]))
+    ncl = max(8, int(cap * rng.choice([0.5, 1.5, 4.0])))
+    sp = W.StreamSpec(capacity=cap, dim=dim, n_queries=batch * nb, batch=batch, n_clusters=ncl, zipf_s=1.2,
+                      reshuffle_every=max(batch, batch * nb // 3), theta=theta, mode="P", dtype=dtype, seed=seed)
+    q_all = to_dev(W.QueryStream(sp).block(0, nb), dtype)
+    caches = []
+    for fused, list_off in ((1, 0), (1, 1), (0, 0)):
+        c = siso.SisoCache(cap, dim, dtype)
+        c.set_option(siso.OPT_STREAM_FUSED, fused)
+        c.set_option(siso.OPT_STREAM_LIST, list_off)
+        caches.append(c)
+    pre = int(cap * rng.choice([0.0, 0.6, 0.98]))
+    if pre:
+        fill_sp = W.StreamSpec(capacity=cap, dim=dim, n_queries=pre, batch=pre, n_clusters=ncl, theta=theta, mode="P", dtype=dtype,
+                               seed=seed + 100)
+        filler = to_dev(W.QueryStream(fill_sp).block(0, 1), dtype)[:pre]
+        for c in caches:
+            c.insert(filler)
+    other = rng.random(nb)
+    for t in range(nb):
+        q = q_all[t * batch:(t + 1) * batch]
+        outs = [[x.clone() for x in c.stream_step(q, theta)] for c in caches]
+        for o in outs[1:]:
+            assert all(torch.equal(x, y) for x, y in zip(outs[0], o)), f"batch {t}"
+        if other[t] < 0.04:
+            m, flags = int(rng.integers(1, 40)), (siso.EVICT_DECAY if rng.random() < 0.5 else 0)
+            vs = [c.evict(m, flags) for c in caches]
+            assert all(torch.equal(vs[0], v) for v in vs[1:]), f"evict after batch {t}"
+        elif other[t] < 0.06:
+            ms = []
+            for c in caches:
+                try:
+                    ms.append(c.merge(0.95, siso.MERGE_WEIGHTED_MEAN))
+                except siso.SisoError as e:          # more pairs than the candidate buffer holds: nothing is modified
+                    assert e.status == 5
+                    ms.append(None)
+            if any(m is None for m in ms):
+                assert all(m is None for m in ms), f"merge after batch {t}: overflow in some forms only"
+            else:
+                assert all(torch.equal(ms[0][0], m[0]) and ms[0][1] == m[1] for m in ms[1:]), f"merge after batch {t}"
+        elif other[t] < 0.10:
+            for c in caches:
+                i, _, h = c.lookup(q, theta, 1)
+                c.update(q, i, h)
+        if t % 40 == 39 or t == nb - 1:
+            sts = [state_np(c) for c in caches]
+            for s2 in sts[1:]:
+                for k in ("valid", "size", "access", "last", "master", "vecs"):
+                    assert (sts[0][k] == s2[k]).all(), f"{k} after batch {t}"
+    assert caches[0].stats() == caches[1].stats()
+    for c in caches:
+        c.check_status()
+        c.close()
+
+
 def test_streaming_eviction_is_exact_when_the_sample_misleads():
     """The fused step chooses its victims with the help of a strided sample of 256 entries.  Here exactly the
     sampled entries hold the smallest keys, so the sample says that hardly any entry is small; the selection
