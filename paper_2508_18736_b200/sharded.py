@@ -196,6 +196,8 @@ class ShardedCache:
         from .binding import combine_keys, route, select_evict_planned, shard_plan
         q = self.local._vec(queries, "queries")
         n = q.shape[0]
+        if n > self.total_rows:          # its misses could outnumber the slots of the whole cache (SISO_ERR_CAPACITY on one cache)
+            raise ValueError(f"a micro-batch of {n} rows does not fit a cache of {self.total_rows} entries")
         empty = self.hi == self.lo
         keys = self.local.lookup_keys(q, 1, slot_offset=self.lo)
         if empty:
