@@ -4,6 +4,7 @@
 //   n <= SMALL_N : one CTA, rank by counting over packed 64-bit (key, position) words
 //   otherwise    : least-significant-digit radix sort, 8 or 9 bits per pass (9 where that saves a pass: 17- and 18-bit
 //                  keys, e.g. the slots of a 65,536-entry cache, sort in two passes), three kernels per pass
+//                  (two up to 131,072 items: the scatter kernel then scans the small histogram itself)
 #include "common.cuh"
 
 namespace siso {
@@ -13,6 +14,7 @@ constexpr int RS_THREADS = 256;
 constexpr int RS_ITEMS = 4;                       // rounds per tile
 constexpr int RS_TILE = RS_THREADS * RS_ITEMS;    // items per CTA
 constexpr int RS_MAX_BINS = 512;                  // 9 bits
+constexpr int RS_FUSED_TILES = 128;               // up to here the scatter kernel scans the histogram itself
 
 __global__ void __launch_bounds__(1024)
 sort_small_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restrict__ vals, int n,
@@ -29,9 +31,11 @@ sort_small_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restrict_
     }
 }
 
-// pass 1: per-tile digit histogram, stored digit-major: hist[digit * n_tiles + tile]
+// pass 1: per-tile digit histogram, stored digit-major for the scan kernel, hist[digit * n_tiles + tile], or tile-major,
+// hist[tile * bins + digit], when the scatter kernel reads it raw (its threads then walk the tiles with coalesced loads)
 __global__ void __launch_bounds__(RS_THREADS)
-radix_hist_kernel(const uint32_t *__restrict__ keys, int64_t n, int shift, int bins, int n_tiles, uint32_t *__restrict__ hist) {
+radix_hist_kernel(const uint32_t *__restrict__ keys, int64_t n, int shift, int bins, int n_tiles, int tile_major,
+                  uint32_t *__restrict__ hist) {
     __shared__ uint32_t h[RS_MAX_BINS];
     const uint32_t mask = static_cast<uint32_t>(bins - 1);
     for (int d = threadIdx.x; d < bins; d += RS_THREADS) h[d] = 0;
@@ -43,7 +47,8 @@ radix_hist_kernel(const uint32_t *__restrict__ keys, int64_t n, int shift, int b
         if (i < n) atomicAdd(&h[(keys[i] >> shift) & mask], 1u);
     }
     __syncthreads();
-    for (int d = threadIdx.x; d < bins; d += RS_THREADS) hist[static_cast<int64_t>(d) * n_tiles + blockIdx.x] = h[d];
+    for (int d = threadIdx.x; d < bins; d += RS_THREADS)
+        hist[tile_major ? static_cast<int64_t>(blockIdx.x) * bins + d : static_cast<int64_t>(d) * n_tiles + blockIdx.x] = h[d];
 }
 
 // pass 2: exclusive scan of the histogram in place (one CTA; the array has bins * n_tiles entries).  A block of
@@ -101,13 +106,61 @@ __global__ void __launch_bounds__(1024) exclusive_scan_u32_kernel(uint32_t *__re
 // round the rank of an item among equal digits is (equal digits in earlier warps) + (in earlier lanes).
 __global__ void __launch_bounds__(RS_THREADS)
 radix_scatter_kernel(const uint32_t *__restrict__ keys, const uint32_t *__restrict__ vals, int64_t n, int shift, int bins,
-                     int n_tiles, const uint32_t *__restrict__ hist_scanned, uint32_t *__restrict__ keys_out,
+                     int n_tiles, const uint32_t *__restrict__ hist_scanned, int raw_hist, uint32_t *__restrict__ keys_out,
                      uint32_t *__restrict__ vals_out) {
     __shared__ uint32_t base_s[RS_MAX_BINS];
     __shared__ uint32_t cnt_s[RS_THREADS / 32][RS_MAX_BINS];
     const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5;
     const uint32_t mask = static_cast<uint32_t>(bins - 1);
-    for (int d = tid; d < bins; d += RS_THREADS) base_s[d] = hist_scanned[static_cast<int64_t>(d) * n_tiles + blockIdx.x];
+    if (!raw_hist) {
+        for (int d = tid; d < bins; d += RS_THREADS) base_s[d] = hist_scanned[static_cast<int64_t>(d) * n_tiles + blockIdx.x];
+    } else {
+        // few tiles: no scan kernel ran and the histogram is tile-major.  Every CTA works its bases out itself: thread t
+        // takes digits t and t + 256, sums each digit's counts over all tiles (and over the tiles before its own) with
+        // loads that are coalesced across the threads, and a block scan over the digit totals gives where each digit
+        // starts (digits t < 256 first, then t + 256).
+        __shared__ uint32_t warp_tot[2][RS_THREADS / 32];
+        uint32_t tot[2] = {0u, 0u}, before[2] = {0u, 0u};
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int d = tid + j * RS_THREADS;
+            if (d < bins) {
+                // 32 loads in flight at a time: the sums wait for L2 once per 32 tiles, not once per tile
+                for (int t0 = 0; t0 < n_tiles; t0 += 32) {
+                    uint32_t v[32];
+#pragma unroll
+                    for (int u = 0; u < 32; ++u) v[u] = t0 + u < n_tiles ? __ldg(hist_scanned + static_cast<int64_t>(t0 + u) * bins + d) : 0u;
+#pragma unroll
+                    for (int u = 0; u < 32; ++u) {
+                        tot[j] += v[u];
+                        before[j] += t0 + u < static_cast<int>(blockIdx.x) ? v[u] : 0u;
+                    }
+                }
+            }
+        }
+        uint32_t incl[2];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            uint32_t x = tot[j];
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t y = __shfl_up_sync(0xFFFFFFFFu, x, o);
+                if (lane >= o) x += y;
+            }
+            incl[j] = x;
+            if (lane == 31) warp_tot[j][warp] = x;
+        }
+        __syncthreads();
+        uint32_t lower_half = 0;                                   // all digits below 256
+        for (int w = 0; w < RS_THREADS / 32; ++w) lower_half += warp_tot[0][w];
+#pragma unroll
+        for (int j = 0; j < 2; ++j) {
+            const int d = tid + j * RS_THREADS;
+            uint32_t start = incl[j] - tot[j] + (j ? lower_half : 0u);
+            for (int w = 0; w < warp; ++w) start += warp_tot[j][w];
+            if (d < bins) base_s[d] = start + before[j];
+        }
+    }
     const int64_t base = static_cast<int64_t>(blockIdx.x) * RS_TILE;
     for (int r = 0; r < RS_ITEMS; ++r) {
         for (int d = tid; d < bins; d += RS_THREADS) {
@@ -170,11 +223,16 @@ siso_status_t launch_sort_pairs(Cache *c, Scratch *scr, uint32_t *keys, uint32_t
     const int bits = (key_bits + 8) / 9 < (key_bits + 7) / 8 ? 9 : 8;
     const int bins = 1 << bits;
     for (int shift = 0; shift < key_bits; shift += bits) {
-        radix_hist_kernel<<<n_tiles, RS_THREADS, 0, s>>>(ka, n, shift, bins, n_tiles, hist);
+        radix_hist_kernel<<<n_tiles, RS_THREADS, 0, s>>>(ka, n, shift, bins, n_tiles, n_tiles <= RS_FUSED_TILES ? 1 : 0, hist);
         SISO_LAUNCHED(c);
-        exclusive_scan_u32_kernel<<<1, 1024, 0, s>>>(hist, bins * static_cast<int64_t>(n_tiles));
-        SISO_LAUNCHED(c);
-        radix_scatter_kernel<<<n_tiles, RS_THREADS, 0, s>>>(ka, va, n, shift, bins, n_tiles, hist, kb, vb);
+        // up to 128 tiles (131,072 items) the scatter CTAs read the raw histogram themselves (256 KiB each, from L2):
+        // cheaper than a one-CTA scan kernel and the launch around it
+        const int raw_hist = n_tiles <= RS_FUSED_TILES ? 1 : 0;
+        if (!raw_hist) {
+            exclusive_scan_u32_kernel<<<1, 1024, 0, s>>>(hist, bins * static_cast<int64_t>(n_tiles));
+            SISO_LAUNCHED(c);
+        }
+        radix_scatter_kernel<<<n_tiles, RS_THREADS, 0, s>>>(ka, va, n, shift, bins, n_tiles, hist, raw_hist, kb, vb);
         SISO_LAUNCHED(c);
         uint32_t *t = ka; ka = kb; kb = t;
         t = va; va = vb; vb = t;
