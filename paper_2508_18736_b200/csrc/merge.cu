@@ -167,6 +167,7 @@ merge_resolve_kernel(MergeCtl *ctl, int64_t N, const uint8_t *__restrict__ valid
 // barrier per round.  A chain of k entries that each merge into the previous survivor needs k rounds; a round costs
 // a barrier plus a few memory round trips instead of one CTA's walk over all rows.
 namespace cgm = cooperative_groups;
+constexpr int RESOLVE_LOOKS = 32;
 __global__ void __launch_bounds__(256)
 merge_resolve_grid_kernel(MergeCtl *ctl, int64_t N, const uint8_t *__restrict__ valid, const uint8_t *__restrict__ seed,
                           const uint32_t *__restrict__ row_off, const uint32_t *__restrict__ row_count,
@@ -184,6 +185,11 @@ merge_resolve_grid_kernel(MergeCtl *ctl, int64_t N, const uint8_t *__restrict__ 
     grid.sync();
     for (int64_t round = 0; round <= N; ++round) {
         int left = 0;
+        // a row whose candidates are still undecided is looked at again a few times before the grid-wide barrier: the
+        // rows it waits for are being decided by other threads in this very round, and another look costs a memory
+        // round trip where a round costs a barrier as well (the outcome does not depend on who decides when)
+        for (int look = 0; look < RESOLVE_LOOKS; ++look) {
+        left = 0;
         for (int64_t i = first; i < N; i += stride) {
             if (state[i] != 0) continue;
             const uint32_t o = row_off[i], cnt = row_count[i];
@@ -214,6 +220,8 @@ merge_resolve_grid_kernel(MergeCtl *ctl, int64_t N, const uint8_t *__restrict__ 
             if (!ready) { ++left; continue; }
             if (best) { target[i] = key_slot(best) & 0x7FFFFFFF; state[i] = 2; }
             else state[i] = 1;
+        }
+        if (left == 0) break;
         }
 #pragma unroll
         for (int o = 16; o >= 1; o >>= 1) left += __shfl_xor_sync(0xFFFFFFFFu, left, o);
